@@ -385,9 +385,11 @@ def test_migrate_bytes_table_and_decode(kv_dtype):
     for s, d in zip(src_ids, dst_ids):
         assert np.array_equal(w.kv_pool[n_src + d], pool0[s])
         if sc0 is not None:
-            assert np.array_equal(w.kv_scales[n_src + d], sc0[s])
+            assert np.array_equal(w.kv_scales[n_src + d].view(np.uint32), sc0[s].view(np.uint32))
         moved[n_src + d] = True
     assert np.array_equal(w.kv_pool[~moved].view(np.uint8), pool0[~moved].view(np.uint8))
+    if sc0 is not None:
+        assert np.array_equal(w.kv_scales[~moved].view(np.uint32), sc0[~moved].view(np.uint32))
     # table: plain-python remap
     remap = {int(s): int(n_src + d) for s, d in zip(src_ids, dst_ids)}
     expect = np.array([[remap.get(int(e), int(e)) for e in row] for row in table0], dtype=np.int32)
