@@ -1,0 +1,203 @@
+/*
+ * splash_mla.h -- C ABI of the B200 (sm_100a) MLA decode library.
+ *
+ * One rank's attention shard under the paper's layouts, on one GPU:
+ *   - TP / DOP        : a head slice [head_begin, head_end) over each request's
+ *                       complete history (Sec. 3, "Computation" of DOP: every head
+ *                       attends over the complete history, outputs agree with TP up
+ *                       to floating-point reduction order);
+ *   - DP-attention    : a request slice (the caller passes only its requests), all
+ *                       heads;
+ *   - CP              : a KV token range per request (App. E, position-sharded CP),
+ *                       giving partial (O, LSE) that splash_lse_merge combines.
+ * The cache is the head-shared latent cache of absorbed MLA: one row of
+ * d_qk = d_c + d_r = 512 + 64 elements per token, the value being its first
+ * d_v = d_c = 512 elements (Sec. 3 "Cost": d_q = d_c + d_r, d_z = d_c; App. B
+ * dimensions).  splash_kv_page_migrate is the local part of a layout switch: the
+ * "discard" primitive's repack of kept blocks into the destination view (Sec. 3,
+ * Sec. 4.1 "Reuse"), after which every query must still read its complete history
+ * (Sec. 4.1 "Handoff").
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless stated otherwise.
+ *     The library allocates no device memory, never synchronises the host, enqueues
+ *     its kernels on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and returns.
+ *   - Return value: SPLASH_OK (0) or a negative splash_status.  On an error nothing
+ *     has been launched.  splash_last_error() gives a host string for the last
+ *     error of the calling thread.
+ *   - Empty work (no requests, an empty head slice, n = 0 pages) is a successful
+ *     no-op: idle ranks are legal (App. E: ranks that own no rows still take part).
+ */
+#ifndef SPLASH_MLA_H_
+#define SPLASH_MLA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SPLASH_API __attribute__((visibility("default")))
+#else
+#define SPLASH_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum splash_status {
+    SPLASH_OK = 0,
+    SPLASH_INVALID_ARG = -1,        /* null pointer, bad range, misalignment, short workspace */
+    SPLASH_UNSUPPORTED = -2,        /* dims / page size / dtype / head count not built */
+    SPLASH_UNSUPPORTED_DEVICE = -3, /* the current device is not compute capability 10.x */
+    SPLASH_CUDA_ERROR = -4,         /* a CUDA runtime / driver call failed */
+    SPLASH_DEVICE_TIMEOUT = -5      /* (status word only) a bounded device wait gave up */
+} splash_status;
+
+enum { SPLASH_KV_BF16 = 0, SPLASH_KV_E4M3_TOKEN_SCALE = 1 };
+
+/* shape.flags bits */
+enum {
+    /* Run the plain SIMT (fp32 CUDA-core) decode kernel instead of the tcgen05 one.
+     * A diagnostic path: same plan, same partial slots, same combine; slow. */
+    SPLASH_FLAG_SIMT = 1u
+};
+
+/*
+ * Shape of one decode call.  Strides are in ELEMENTS of the array they index.
+ *   q    : bf16,  element (i, g, d) at q  [i*q_stride_request   + g*q_stride_head   + d], d < d_qk
+ *   out  : fp32,  element (i, g, d) at out[i*out_stride_request + g*out_stride_head + d], d < d_v
+ *   lse  : fp32,  element (i, g)    at lse[i*lse_stride_request + g]
+ * g is the GLOBAL head id in [0, num_heads); a call touches only heads in
+ * [head_begin, head_end) and leaves every other element of out / lse untouched, so
+ * the slices of several calls can share one buffer.  A caller holding a compact
+ * per-rank q [N][H/T][d_q] passes num_heads = H/T and the slice [0, H/T).
+ */
+typedef struct splash_mla_shape {
+    uint32_t struct_size;        /* sizeof(splash_mla_shape), for versioning */
+    int32_t num_requests;        /* B >= 0; one query row per request (decode) */
+    int32_t num_heads;           /* H, 1..128 */
+    int32_t d_qk;                /* 576: [0,512) latent (also V), [512,576) rotary part */
+    int32_t d_v;                 /* 512 */
+    int32_t page_size;           /* 64 tokens */
+    int32_t num_pool_pages;      /* pages addressable from kv_pool (bounds the table's ids) */
+    int32_t block_table_stride;  /* entries per request row of block_table */
+    int32_t kv_dtype;            /* SPLASH_KV_BF16 or SPLASH_KV_E4M3_TOKEN_SCALE */
+    float softmax_scale;         /* multiplies q.k before the softmax (configs: 1/sqrt(192)) */
+    int64_t q_stride_request, q_stride_head;     /* multiples of 8 */
+    int64_t out_stride_request, out_stride_head; /* multiples of 4 */
+    int64_t lse_stride_request;
+    uint32_t flags;              /* SPLASH_FLAG_* bits, 0 for the default path */
+    uint32_t reserved;           /* must be 0 */
+} splash_mla_shape;
+
+/*
+ * Decode attention over a paged latent KV cache.
+ *
+ * For request i, head g in [head_begin, head_end) and token range
+ * R_i = [max(0, kv_begin[i]), min(seq_lens[i], kv_end[i])):
+ *     row_t  = kv_pool[block_table[i][t / 64]][t % 64][0..576)     (times kv_scales[..] for e4m3)
+ *     l_t    = softmax_scale * sum_{d<576} q[i][g][d] * row_t[d]
+ *     lse    = ln sum_{t in R_i} exp(l_t)                          (natural log, scale included)
+ *     out[d] = sum_{t in R_i} exp(l_t - lse) * row_t[d],  d < 512
+ * An empty R_i gives out = 0, lse = -inf.
+ *
+ *   q            bf16, 16-byte aligned
+ *   kv_pool      [num_pool_pages][64][576] bf16 (73,728 B / page) or e4m3 bytes
+ *                (36,864 B / page); 128-byte aligned
+ *   kv_scales    [num_pool_pages][64] fp32, one scale per token; required for e4m3,
+ *                NULL for bf16
+ *   block_table  [num_requests][block_table_stride] int32 page ids; only the entries
+ *                of pages that intersect R_i are read (others may hold anything)
+ *   seq_lens     [num_requests] int32
+ *   kv_begin,
+ *   kv_end       [num_requests] int32 each, or NULL for 0 / seq_lens[i]; need not be
+ *                page aligned
+ *   out, lse     fp32, 16-byte / 4-byte aligned
+ *   workspace    scratch of at least splash_mla_decode_workspace_bytes() bytes,
+ *                256-byte aligned; its contents on entry do not matter and two
+ *                calls that may overlap on the device need different workspaces
+ *
+ * Slots of a referenced page at or beyond seq_lens[i] and pages the table does not
+ * reference are never used: they may hold NaN / Inf patterns.  Slots below
+ * seq_lens[i] of a page that intersects R_i must hold finite values even if they lie
+ * outside R_i.  Results are bit-reproducible for a fixed call (same shape,
+ * lengths and ranges).
+ */
+SPLASH_API int splash_mla_decode(const splash_mla_shape *shape,
+                      const void *q, const void *kv_pool, const float *kv_scales,
+                      const int32_t *block_table, const int32_t *seq_lens,
+                      int32_t head_begin, int32_t head_end,
+                      const int32_t *kv_begin, const int32_t *kv_end,
+                      float *out, float *lse,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+/* Workspace size (host computation, no device access) for a call with this shape
+ * and head slice; depends only on the shape, the slice width and the device's SM
+ * count.  Returns 0 on invalid arguments. */
+SPLASH_API size_t splash_mla_decode_workspace_bytes(const splash_mla_shape *shape,
+                                         int32_t head_begin, int32_t head_end);
+
+/*
+ * Merge partial attention results over disjoint KV ranges (the CP combination step;
+ * also the reduction of the decode kernel's internal KV splits):
+ *     lse[r]    = ln sum_j exp(part_lse[j][r])
+ *     out[r][d] = sum_j exp(part_lse[j][r] - lse[r]) * part_out[j][r][d]
+ * Parts with lse = -inf contribute nothing (their out values are not read into the
+ * result); if all are -inf, out = 0 and lse = -inf.
+ *   part_out [num_parts][rows][d_v] fp32, part_lse [num_parts][rows] fp32,
+ *   out [rows][d_v], lse [rows]; all contiguous, 16-byte aligned; d_v a multiple of 4;
+ *   out / lse must not alias the parts.
+ */
+SPLASH_API int splash_lse_merge(int32_t num_parts, int64_t rows, int32_t d_v,
+                     const float *part_out, const float *part_lse,
+                     float *out, float *lse, void *stream);
+
+/*
+ * Copy a listed set of KV pages between two page pools in HBM and rewrite the
+ * block table: page src_page_ids[j] of src_pool is copied, byte for byte, to page
+ * dst_page_ids[j] of dst_pool (with its scale page when the scale pointers are
+ * given), and every block-table entry equal to src_id_base + src_page_ids[j]
+ * becomes dst_id_base + dst_page_ids[j].  Table ids are "arena-global": when both
+ * pools are sub-ranges of the allocation that decode receives as kv_pool, the bases
+ * are the pools' page offsets in it, so one table can name pages of both pools.
+ * Negative entries and entries naming other pages pass through.  Source pages are
+ * left intact (the caller retires them, Sec. 4.1 "Retire").
+ *
+ *   page_bytes       73,728 (bf16) or 36,864 (e4m3); a multiple of 16; pools 16-byte aligned
+ *   src/dst_scales   [pages][64] fp32 or both NULL
+ *   src/dst_page_ids [n] int32 device arrays; each duplicate-free, 0 <= id
+ *   max_page_id      exclusive upper bound on src_id_base + src_page_ids[j]
+ *   block_table      [num_table_entries] int32, rewritten in place
+ *   workspace        at least splash_kv_page_migrate_workspace_bytes(max_page_id) bytes
+ */
+SPLASH_API int splash_kv_page_migrate(const void *src_pool, const float *src_scales,
+                           void *dst_pool, float *dst_scales,
+                           int64_t page_bytes,
+                           const int32_t *src_page_ids, const int32_t *dst_page_ids, int64_t n,
+                           int32_t src_id_base, int32_t dst_id_base, int32_t max_page_id,
+                           int32_t *block_table, int64_t num_table_entries,
+                           void *workspace, size_t workspace_bytes, void *stream);
+
+SPLASH_API size_t splash_kv_page_migrate_workspace_bytes(int32_t max_page_id);
+
+/* Host-side helpers. */
+SPLASH_API const char *splash_status_string(int status);
+SPLASH_API const char *splash_last_error(void);
+SPLASH_API int splash_version(void);
+
+/* Number of kernels the last call of this thread enqueued (for launch accounting). */
+SPLASH_API int splash_last_launch_count(void);
+
+/*
+ * Read the device status word at the head of a decode workspace after the caller
+ * has synchronised the stream: SPLASH_OK, or SPLASH_DEVICE_TIMEOUT if a bounded wait
+ * inside a kernel gave up (the results of that call are then invalid).  Performs a
+ * blocking 16-byte device-to-host copy; not for the hot path.
+ */
+SPLASH_API int splash_workspace_status(const void *workspace, int32_t *detail /* host, [3], may be NULL */);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPLASH_MLA_H_ */

@@ -1,0 +1,254 @@
+"""ctypes binding of libsplash_mla.so: same names as the C ABI, argument
+marshalling only.  torch supplies device memory and streams; every step of the
+path runs in the library's CUDA kernels.  There is no fallback: if the shared
+library has not been built the import of its symbols fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsplash_mla.so")
+
+SPLASH_OK = 0
+SPLASH_INVALID_ARG = -1
+SPLASH_UNSUPPORTED = -2
+SPLASH_UNSUPPORTED_DEVICE = -3
+SPLASH_CUDA_ERROR = -4
+SPLASH_DEVICE_TIMEOUT = -5
+SPLASH_KV_BF16 = 0
+SPLASH_KV_E4M3_TOKEN_SCALE = 1
+SPLASH_FLAG_SIMT = 1
+
+D_QK, D_V, PAGE_SIZE = 576, 512, 64
+
+
+class SplashError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"splash status {status}: {message}")
+        self.status = status
+
+
+class MlaShape(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("num_requests", ctypes.c_int32),
+        ("num_heads", ctypes.c_int32),
+        ("d_qk", ctypes.c_int32),
+        ("d_v", ctypes.c_int32),
+        ("page_size", ctypes.c_int32),
+        ("num_pool_pages", ctypes.c_int32),
+        ("block_table_stride", ctypes.c_int32),
+        ("kv_dtype", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float),
+        ("q_stride_request", ctypes.c_int64),
+        ("q_stride_head", ctypes.c_int64),
+        ("out_stride_request", ctypes.c_int64),
+        ("out_stride_head", ctypes.c_int64),
+        ("lse_stride_request", ctypes.c_int64),
+        ("flags", ctypes.c_uint32),
+        ("reserved", ctypes.c_uint32),
+    ]
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load the shared library (raises if it has not been built)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2609_37626_b200.build` "
+            "(there is no CPU or eager fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    lib.splash_mla_decode.restype = ctypes.c_int
+    lib.splash_mla_decode.argtypes = [ctypes.POINTER(MlaShape), vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.splash_mla_decode_workspace_bytes.restype = sz
+    lib.splash_mla_decode_workspace_bytes.argtypes = [ctypes.POINTER(MlaShape), i32, i32]
+    lib.splash_lse_merge.restype = ctypes.c_int
+    lib.splash_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp]
+    lib.splash_kv_page_migrate.restype = ctypes.c_int
+    lib.splash_kv_page_migrate.argtypes = [vp, vp, vp, vp, i64, vp, vp, i64, i32, i32, i32, vp, i64, vp, sz, vp]
+    lib.splash_kv_page_migrate_workspace_bytes.restype = sz
+    lib.splash_kv_page_migrate_workspace_bytes.argtypes = [i32]
+    lib.splash_status_string.restype = ctypes.c_char_p
+    lib.splash_status_string.argtypes = [ctypes.c_int]
+    lib.splash_last_error.restype = ctypes.c_char_p
+    lib.splash_version.restype = ctypes.c_int
+    lib.splash_last_launch_count.restype = ctypes.c_int
+    lib.splash_workspace_status.restype = ctypes.c_int
+    lib.splash_workspace_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+    _lib = lib
+    return lib
+
+
+def _check(rc: int):
+    if rc != SPLASH_OK:
+        lib = load()
+        raise SplashError(rc, f"{lib.splash_status_string(rc).decode()}: {lib.splash_last_error().decode()}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def make_shape(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch.Tensor, out: torch.Tensor,
+               lse: torch.Tensor, softmax_scale: float, flags: int = 0) -> MlaShape:
+    B, H, dqk = q.shape
+    assert q.stride(2) == 1 and out.stride(2) == 1 and lse.stride(1) == 1
+    kv_dtype = SPLASH_KV_BF16 if kv_pool.dtype == torch.bfloat16 else SPLASH_KV_E4M3_TOKEN_SCALE
+    return MlaShape(
+        struct_size=ctypes.sizeof(MlaShape), num_requests=B, num_heads=H, d_qk=dqk, d_v=out.shape[2],
+        page_size=kv_pool.shape[1], num_pool_pages=kv_pool.shape[0],
+        block_table_stride=block_table.stride(0) if block_table.dim() == 2 and B > 0 else 0,
+        kv_dtype=kv_dtype, softmax_scale=float(softmax_scale),
+        q_stride_request=q.stride(0), q_stride_head=q.stride(1),
+        out_stride_request=out.stride(0), out_stride_head=out.stride(1),
+        lse_stride_request=lse.stride(0), flags=flags, reserved=0)
+
+
+def splash_mla_decode_workspace_bytes(shape: MlaShape, head_begin: int, head_end: int) -> int:
+    return int(load().splash_mla_decode_workspace_bytes(ctypes.byref(shape), head_begin, head_end))
+
+
+_workspaces = {}
+
+
+def _workspace(device: torch.device, nbytes: int, tag: str) -> torch.Tensor:
+    key = (device.index, tag)
+    ws = _workspaces.get(key)
+    if ws is None or ws.numel() < nbytes:
+        ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+        _workspaces[key] = ws
+    return ws
+
+
+def splash_mla_decode(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch.Tensor, seq_lens: torch.Tensor, *,
+                      softmax_scale: float, kv_scales: Optional[torch.Tensor] = None, head_begin: int = 0,
+                      head_end: Optional[int] = None, kv_begin: Optional[torch.Tensor] = None,
+                      kv_end: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                      lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                      stream: Optional[torch.cuda.Stream] = None, flags: int = 0):
+    """Decode attention of one shard; see ``splash_mla_decode`` in include/splash_mla.h.
+
+    q [B][H][576] bf16; kv_pool [P][64][576] bf16, or uint8 / float8_e4m3fn with
+    kv_scales [P][64] fp32; block_table [B][stride] int32; seq_lens, kv_begin, kv_end
+    [B] int32.  out [B][H][512] fp32 and lse [B][H] fp32 are allocated (uninitialised
+    outside the head slice) unless given.  Returns (out, lse).
+    """
+    lib = load()
+    assert q.is_cuda and q.dtype == torch.bfloat16
+    B, H, _ = q.shape
+    if head_end is None:
+        head_end = H
+    if out is None:
+        out = torch.empty((B, H, D_V), dtype=torch.float32, device=q.device)
+    if lse is None:
+        lse = torch.empty((B, H), dtype=torch.float32, device=q.device)
+    assert block_table.dtype == torch.int32 and seq_lens.dtype == torch.int32
+    shape = make_shape(q, kv_pool, block_table, out, lse, softmax_scale, flags)
+    if workspace is None:
+        need = splash_mla_decode_workspace_bytes(shape, head_begin, head_end)
+        workspace = _workspace(q.device, need, "decode")
+    rc = lib.splash_mla_decode(ctypes.byref(shape), _ptr(q), _ptr(kv_pool), _ptr(kv_scales), _ptr(block_table),
+                               _ptr(seq_lens), head_begin, head_end, _ptr(kv_begin), _ptr(kv_end),
+                               _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                               _stream_ptr(stream))
+    _check(rc)
+    return out, lse
+
+
+def splash_lse_merge(part_out: torch.Tensor, part_lse: torch.Tensor, out: Optional[torch.Tensor] = None,
+                     lse: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Merge [parts][rows][d_v] fp32 partial outputs by their [parts][rows] LSE."""
+    lib = load()
+    assert part_out.is_contiguous() and part_lse.is_contiguous()
+    parts, rows, d_v = part_out.shape
+    if out is None:
+        out = torch.empty((rows, d_v), dtype=torch.float32, device=part_out.device)
+    if lse is None:
+        lse = torch.empty((rows,), dtype=torch.float32, device=part_out.device)
+    _check(lib.splash_lse_merge(parts, rows, d_v, _ptr(part_out), _ptr(part_lse), _ptr(out), _ptr(lse),
+                                _stream_ptr(stream)))
+    return out, lse
+
+
+def splash_kv_page_migrate(src_pool: torch.Tensor, dst_pool: torch.Tensor, src_page_ids: torch.Tensor,
+                           dst_page_ids: torch.Tensor, block_table: torch.Tensor, *,
+                           src_scales: Optional[torch.Tensor] = None, dst_scales: Optional[torch.Tensor] = None,
+                           src_id_base: int = 0, dst_id_base: int = 0, max_page_id: Optional[int] = None,
+                           workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Copy listed pages pool -> pool and rewrite block_table in place."""
+    lib = load()
+    assert src_pool.is_contiguous() and dst_pool.is_contiguous() and block_table.is_contiguous()
+    assert src_page_ids.dtype == torch.int32 and dst_page_ids.dtype == torch.int32
+    page_bytes = src_pool.shape[1] * src_pool.shape[2] * src_pool.element_size()
+    n = src_page_ids.numel()
+    if max_page_id is None:
+        max_page_id = max(src_id_base + src_pool.shape[0], dst_id_base + dst_pool.shape[0])
+    if workspace is None:
+        workspace = _workspace(src_pool.device, int(lib.splash_kv_page_migrate_workspace_bytes(max_page_id)), "migrate")
+    _check(lib.splash_kv_page_migrate(_ptr(src_pool), _ptr(src_scales), _ptr(dst_pool), _ptr(dst_scales), page_bytes,
+                                      _ptr(src_page_ids), _ptr(dst_page_ids), n, src_id_base, dst_id_base,
+                                      max_page_id, _ptr(block_table), block_table.numel(), _ptr(workspace),
+                                      workspace.numel(), _stream_ptr(stream)))
+
+
+def splash_last_launch_count() -> int:
+    return int(load().splash_last_launch_count())
+
+
+def splash_version() -> int:
+    return int(load().splash_version())
+
+
+def splash_workspace_status(workspace: torch.Tensor):
+    detail = (ctypes.c_int32 * 3)()
+    rc = load().splash_workspace_status(_ptr(workspace), detail)
+    return rc, list(detail)
+
+
+def decode_workspace(device: torch.device) -> Optional[torch.Tensor]:
+    """The cached decode workspace of the last call on this device (for status reads)."""
+    return _workspaces.get((device.index, "decode"))
+
+
+# ---- host-buffer convenience path (end-to-end timing, small callers) --------------
+class DeviceWorkload:
+    """A workload's arrays resident on the device as torch tensors."""
+
+    def __init__(self, w, device="cuda"):
+        import numpy as np
+        dev = torch.device(device)
+        self.q = torch.from_numpy(w.q.view(np.int16)).to(dev).view(torch.bfloat16)
+        if w.kv_dtype == 0:
+            self.kv_pool = torch.from_numpy(w.kv_pool.view(np.int16)).to(dev).view(torch.bfloat16)
+            self.kv_scales = None
+        else:
+            self.kv_pool = torch.from_numpy(w.kv_pool).to(dev)
+            self.kv_scales = torch.from_numpy(w.kv_scales).to(dev)
+        self.block_table = torch.from_numpy(w.block_table).to(dev)
+        self.seq_lens = torch.from_numpy(w.seq_lens).to(dev)
+        self.kv_begin = None if w.kv_begin is None else torch.from_numpy(w.kv_begin).to(dev)
+        self.kv_end = None if w.kv_end is None else torch.from_numpy(w.kv_end).to(dev)
+        self.head_begin, self.head_end = w.head_begin, w.head_end
+        self.softmax_scale = w.softmax_scale
+
+    def decode(self, **kw):
+        args = dict(softmax_scale=self.softmax_scale, kv_scales=self.kv_scales, head_begin=self.head_begin,
+                    head_end=self.head_end, kv_begin=self.kv_begin, kv_end=self.kv_end)
+        args.update(kw)
+        return splash_mla_decode(self.q, self.kv_pool, self.block_table, self.seq_lens, **args)

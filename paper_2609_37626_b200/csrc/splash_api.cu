@@ -1,0 +1,262 @@
+// C ABI entry points: argument validation, workspace carving, kernel sequencing.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+
+#include "splash_common.cuh"
+
+namespace splash {
+
+namespace {
+thread_local std::string g_last_error;
+thread_local int g_launches = 0;
+
+struct DeviceInfo {
+    int device = -1;
+    int sm_count = 0;
+    int cc_major = 0;
+    bool ok = false;
+};
+
+// Properties of the current device (cached per device index).
+bool current_device_info(DeviceInfo &info) {
+    static DeviceInfo cache[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { set_error("cudaGetDevice failed"); return false; }
+    if (dev >= 0 && dev < 64 && cache[dev].ok) { info = cache[dev]; return true; }
+    DeviceInfo d;
+    d.device = dev;
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        set_error("cudaDeviceGetAttribute failed");
+        return false;
+    }
+    d.ok = true;
+    if (dev >= 0 && dev < 64) cache[dev] = d;
+    info = d;
+    return true;
+}
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int check_shape(const splash_mla_shape *s, int32_t head_begin, int32_t head_end) {
+    if (s == nullptr) { set_error("shape is NULL"); return SPLASH_INVALID_ARG; }
+    if (s->struct_size != sizeof(splash_mla_shape)) {
+        set_error("shape.struct_size is %u, this library expects %zu", s->struct_size, sizeof(splash_mla_shape));
+        return SPLASH_INVALID_ARG;
+    }
+    if (s->num_requests < 0) { set_error("num_requests < 0"); return SPLASH_INVALID_ARG; }
+    if (s->num_heads < 1 || s->num_heads > kMaxHeads) { set_error("num_heads must be in [1, 128]"); return SPLASH_UNSUPPORTED; }
+    if (s->d_qk != kDQK || s->d_v != kDV) { set_error("only d_qk = 576, d_v = 512 is built"); return SPLASH_UNSUPPORTED; }
+    if (s->page_size != kPage) { set_error("only page_size = 64 is built"); return SPLASH_UNSUPPORTED; }
+    if (s->kv_dtype != SPLASH_KV_BF16 && s->kv_dtype != SPLASH_KV_E4M3_TOKEN_SCALE) {
+        set_error("unknown kv_dtype %d", s->kv_dtype); return SPLASH_UNSUPPORTED;
+    }
+    if (head_begin < 0 || head_end > s->num_heads || head_begin > head_end) {
+        set_error("head slice [%d, %d) is not inside [0, %d)", head_begin, head_end, s->num_heads);
+        return SPLASH_INVALID_ARG;
+    }
+    if (s->num_pool_pages < 0 || s->block_table_stride < 0) { set_error("negative pool / table size"); return SPLASH_INVALID_ARG; }
+    if (s->q_stride_request % 8 || s->q_stride_head % 8 || s->q_stride_head < kDQK) {
+        set_error("q strides must be multiples of 8 elements and q_stride_head >= 576"); return SPLASH_INVALID_ARG;
+    }
+    if (s->out_stride_request % 4 || s->out_stride_head % 4 || s->out_stride_head < kDV) {
+        set_error("out strides must be multiples of 4 elements and out_stride_head >= 512"); return SPLASH_INVALID_ARG;
+    }
+    if (s->lse_stride_request < s->num_heads && s->num_requests > 1) { set_error("lse_stride_request < num_heads"); return SPLASH_INVALID_ARG; }
+    if (!(s->softmax_scale == s->softmax_scale)) { set_error("softmax_scale is NaN"); return SPLASH_INVALID_ARG; }
+    return SPLASH_OK;
+}
+
+// How one decode call is cut into CTAs.
+struct Tiling { int heads_per_group, num_groups, num_workers; };
+
+Tiling choose_tiling(const splash_mla_shape *s, int h, int sm_count, bool simt) {
+    Tiling t;
+    if (simt) {
+        t.heads_per_group = simt_heads_per_group();
+        t.num_groups = (h + t.heads_per_group - 1) / t.heads_per_group;
+        // two CTAs per SM's worth of KV workers in total, at least one
+        int w = (2 * sm_count) / t.num_groups;
+        t.num_workers = w > 0 ? w : 1;
+        return t;
+    }
+    umma_tiling(s->kv_dtype, h, sm_count, &t.heads_per_group, &t.num_groups, &t.num_workers);
+    return t;
+}
+
+}  // namespace
+
+void set_error(const char *fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_last_error = buf;
+}
+
+void count_launch(int n) { g_launches += n; }
+
+}  // namespace splash
+
+using namespace splash;
+
+extern "C" {
+
+size_t splash_mla_decode_workspace_bytes(const splash_mla_shape *shape, int32_t head_begin, int32_t head_end) {
+    if (check_shape(shape, head_begin, head_end) != SPLASH_OK) return 0;
+    DeviceInfo dev;
+    if (!current_device_info(dev)) return 0;
+    const int h = head_end - head_begin;
+    if (h == 0 || shape->num_requests == 0) return 256;
+    // the larger of the two kernels' needs, so one workspace serves both paths
+    size_t need = 0;
+    for (int simt = 0; simt < 2; ++simt) {
+        Tiling t = choose_tiling(shape, h, dev.sm_count, simt != 0);
+        PlanView v = make_plan_view(nullptr, shape->num_requests, t.num_workers, h);
+        if (v.bytes > need) need = v.bytes;
+    }
+    return align_up(need, 256);
+}
+
+int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *kv_pool, const float *kv_scales,
+                      const int32_t *block_table, const int32_t *seq_lens, int32_t head_begin, int32_t head_end,
+                      const int32_t *kv_begin, const int32_t *kv_end, float *out, float *lse,
+                      void *workspace, size_t workspace_bytes, void *stream_) {
+    g_launches = 0;
+    int rc = check_shape(shape, head_begin, head_end);
+    if (rc != SPLASH_OK) return rc;
+    const int B = shape->num_requests, h = head_end - head_begin;
+    if (B == 0 || h == 0) return SPLASH_OK;   // idle rank: nothing to do
+    if (!q || !kv_pool || !block_table || !seq_lens || !out || !lse || !workspace) {
+        set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG;
+    }
+    if (shape->kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE && !kv_scales) { set_error("kv_scales is NULL for e4m3 KV"); return SPLASH_INVALID_ARG; }
+    if (shape->kv_dtype == SPLASH_KV_BF16 && kv_scales) { set_error("kv_scales must be NULL for bf16 KV"); return SPLASH_INVALID_ARG; }
+    if (!aligned(q, 16) || !aligned(kv_pool, 128) || !aligned(out, 16) || !aligned(lse, 4) ||
+        !aligned(workspace, 256) || (kv_scales && !aligned(kv_scales, 16)) || !aligned(block_table, 4) ||
+        !aligned(seq_lens, 4)) {
+        set_error("misaligned pointer (q/out/kv_scales 16 B, kv_pool 128 B, workspace 256 B)"); return SPLASH_INVALID_ARG;
+    }
+    DeviceInfo dev;
+    if (!current_device_info(dev)) return SPLASH_CUDA_ERROR;
+    if (dev.cc_major != 10) { set_error("device compute capability %d.x is not 10.x", dev.cc_major); return SPLASH_UNSUPPORTED_DEVICE; }
+
+    const bool simt = (shape->flags & SPLASH_FLAG_SIMT) != 0;
+    Tiling t = choose_tiling(shape, h, dev.sm_count, simt);
+    PlanView v = make_plan_view(workspace, B, t.num_workers, h);
+    if (workspace_bytes < v.bytes) {
+        set_error("workspace has %zu bytes, %zu needed", workspace_bytes, v.bytes); return SPLASH_INVALID_ARG;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    DecodeParams p;
+    memset(&p, 0, sizeof p);
+    p.q = q; p.kv_pool = kv_pool; p.kv_scales = kv_scales; p.block_table = block_table; p.seq_lens = seq_lens;
+    p.out = out; p.lse = lse;
+    p.q_stride_request = shape->q_stride_request; p.q_stride_head = shape->q_stride_head;
+    p.out_stride_request = shape->out_stride_request; p.out_stride_head = shape->out_stride_head;
+    p.lse_stride_request = shape->lse_stride_request;
+    p.B = B; p.H = shape->num_heads; p.head_begin = head_begin; p.head_end = head_end;
+    p.table_stride = shape->block_table_stride; p.num_pool_pages = shape->num_pool_pages;
+    p.heads_per_group = t.heads_per_group; p.num_groups = t.num_groups; p.num_workers = t.num_workers;
+    p.softmax_scale = shape->softmax_scale;
+    p.tile_start = v.tile_start; p.req_lo = v.req_lo; p.req_hi = v.req_hi; p.worker_begin = v.worker_begin;
+    p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
+
+    cudaError_t e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
+                                v.cost_start, v.worker_begin, v.status, stream);
+    if (e == cudaSuccess) {
+        if (simt) e = launch_decode_simt(p, shape->kv_dtype, stream);
+        else e = launch_decode_umma(p, *shape, stream);
+    }
+    if (e == cudaSuccess) e = launch_split_combine(p, v.req_wfirst, v.req_wlast, stream);
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    return SPLASH_OK;
+}
+
+int splash_lse_merge(int32_t num_parts, int64_t rows, int32_t d_v, const float *part_out, const float *part_lse,
+                     float *out, float *lse, void *stream_) {
+    g_launches = 0;
+    if (num_parts < 0 || rows < 0 || d_v <= 0 || d_v % 4) { set_error("bad sizes (d_v must be a positive multiple of 4)"); return SPLASH_INVALID_ARG; }
+    if (rows == 0) return SPLASH_OK;
+    if (!out || !lse || (num_parts > 0 && (!part_out || !part_lse))) { set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG; }
+    if (!aligned(part_out, 16) || !aligned(out, 16) || !aligned(part_lse, 4) || !aligned(lse, 4)) {
+        set_error("misaligned pointer"); return SPLASH_INVALID_ARG;
+    }
+    if (rows > 0x7fffffffLL) { set_error("too many rows"); return SPLASH_INVALID_ARG; }
+    if (num_parts > 0) {
+        const char *po = reinterpret_cast<const char *>(part_out);
+        const char *oo = reinterpret_cast<const char *>(out);
+        size_t pbytes = (size_t)num_parts * rows * d_v * 4, obytes = (size_t)rows * d_v * 4;
+        if (oo < po + pbytes && po < oo + obytes) { set_error("out aliases part_out"); return SPLASH_INVALID_ARG; }
+    }
+    cudaError_t e = launch_lse_merge(num_parts, rows, d_v, part_out, part_lse, out, lse, static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    return SPLASH_OK;
+}
+
+size_t splash_kv_page_migrate_workspace_bytes(int32_t max_page_id) {
+    if (max_page_id < 0) return 0;
+    return align_up(sizeof(int32_t) * (size_t)max_page_id, 256) + 256;
+}
+
+int splash_kv_page_migrate(const void *src_pool, const float *src_scales, void *dst_pool, float *dst_scales,
+                           int64_t page_bytes, const int32_t *src_page_ids, const int32_t *dst_page_ids, int64_t n,
+                           int32_t src_id_base, int32_t dst_id_base, int32_t max_page_id,
+                           int32_t *block_table, int64_t num_table_entries,
+                           void *workspace, size_t workspace_bytes, void *stream_) {
+    g_launches = 0;
+    if (n < 0 || num_table_entries < 0 || page_bytes <= 0 || page_bytes % 16 || max_page_id < 0) {
+        set_error("bad sizes (page_bytes must be a positive multiple of 16)"); return SPLASH_INVALID_ARG;
+    }
+    if (n == 0) return SPLASH_OK;   // nothing moves, the table keeps every entry
+    if (!src_pool || !dst_pool || !src_page_ids || !dst_page_ids) { set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG; }
+    if ((src_scales == nullptr) != (dst_scales == nullptr)) { set_error("give both scale pools or neither"); return SPLASH_INVALID_ARG; }
+    if (num_table_entries > 0 && (!block_table || !workspace)) { set_error("block_table / workspace is NULL"); return SPLASH_INVALID_ARG; }
+    if (!aligned(src_pool, 16) || !aligned(dst_pool, 16) || !aligned(src_scales, 16) || !aligned(dst_scales, 16) ||
+        !aligned(workspace, 16)) {
+        set_error("misaligned pointer (pools, scales, workspace: 16 B)"); return SPLASH_INVALID_ARG;
+    }
+    if (num_table_entries > 0 && workspace_bytes < splash_kv_page_migrate_workspace_bytes(max_page_id)) {
+        set_error("workspace too small"); return SPLASH_INVALID_ARG;
+    }
+    if (n > 0x7fffffffLL) { set_error("too many pages"); return SPLASH_INVALID_ARG; }
+    cudaError_t e = launch_page_migrate(src_pool, src_scales, dst_pool, dst_scales, page_bytes, src_page_ids,
+                                        dst_page_ids, n, src_id_base, dst_id_base, max_page_id, block_table,
+                                        num_table_entries, static_cast<int32_t *>(workspace),
+                                        static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    return SPLASH_OK;
+}
+
+const char *splash_status_string(int status) {
+    switch (status) {
+        case SPLASH_OK: return "ok";
+        case SPLASH_INVALID_ARG: return "invalid argument";
+        case SPLASH_UNSUPPORTED: return "unsupported shape";
+        case SPLASH_UNSUPPORTED_DEVICE: return "unsupported device";
+        case SPLASH_CUDA_ERROR: return "CUDA error";
+        case SPLASH_DEVICE_TIMEOUT: return "device wait timed out";
+        default: return "unknown status";
+    }
+}
+
+const char *splash_last_error(void) { return g_last_error.c_str(); }
+
+int splash_version(void) { return 100; }
+
+int splash_last_launch_count(void) { return g_launches; }
+
+int splash_workspace_status(const void *workspace, int32_t *detail) {
+    if (!workspace) { set_error("workspace is NULL"); return SPLASH_INVALID_ARG; }
+    int32_t host[4] = {0, 0, 0, 0};
+    cudaError_t e = cudaMemcpy(host, workspace, sizeof host, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    if (detail) { detail[0] = host[1]; detail[1] = host[2]; detail[2] = host[3]; }
+    return host[0];
+}
+
+}  // extern "C"

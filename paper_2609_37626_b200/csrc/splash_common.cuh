@@ -1,0 +1,160 @@
+// Shared declarations of the MLA decode library: dimensions, the split-KV work
+// plan that the plan kernel writes into the caller's workspace, and host helpers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/splash_mla.h"
+
+namespace splash {
+
+constexpr int kDQK = 576;        // d_c + d_r (absorbed MLA row width)
+constexpr int kDV = 512;         // d_c (value width)
+constexpr int kDRope = 64;
+constexpr int kPage = 64;        // tokens per page
+constexpr int kMaxHeads = 128;
+
+// Cost, in page tiles, charged once per non-empty request when the plan balances
+// work over CTAs (query load + epilogue).
+constexpr int kRequestOverheadTiles = 4;
+
+// ---- workspace layout ------------------------------------------------------
+// [0, 64)                 status block (int32 x 16): [0] status, [1..3] detail
+// then int32 arrays       tile_start[B+1], req_lo[B], req_hi[B], req_wfirst[B],
+//                         req_wlast[B], cost_start[B+1], worker_begin[W+1]
+// then (256-B aligned)    partial_lse [2W][h] fp32
+// then (256-B aligned)    partial_out [2W][h][512] fp32
+struct PlanView {
+    int32_t *status;        // 16 ints
+    int32_t *tile_start;    // [B+1] exclusive prefix of per-request tile counts
+    int32_t *req_lo;        // [B] first token of the effective range
+    int32_t *req_hi;        // [B] one past the last token (>= lo; == lo when empty)
+    int32_t *req_wfirst;    // [B] first worker holding a piece of the request (-1 if empty)
+    int32_t *req_wlast;     // [B] last such worker
+    int32_t *cost_start;    // [B+1] exclusive prefix of per-request cost (tiles + overhead)
+    int32_t *worker_begin;  // [W+1] global tile index where each worker starts
+    float *partial_lse;     // [2W][h]
+    float *partial_out;     // [2W][h][512]
+    int32_t num_workers;    // W
+    int32_t h;              // width of the head slice
+    size_t bytes;           // total bytes needed
+};
+
+inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+inline __host__ PlanView make_plan_view(void *workspace, int B, int W, int h) {
+    PlanView v;
+    char *p = static_cast<char *>(workspace);
+    size_t off = 0;
+    v.status = reinterpret_cast<int32_t *>(p + off); off += 64;
+    v.tile_start = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(B + 1);
+    v.req_lo = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)B;
+    v.req_hi = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)B;
+    v.req_wfirst = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)B;
+    v.req_wlast = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)B;
+    v.cost_start = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(B + 1);
+    v.worker_begin = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
+    off = align_up(off, 256);
+    v.partial_lse = reinterpret_cast<float *>(p + off); off += sizeof(float) * (size_t)2 * W * h;
+    off = align_up(off, 256);
+    v.partial_out = reinterpret_cast<float *>(p + off); off += sizeof(float) * (size_t)2 * W * h * kDV;
+    v.num_workers = W;
+    v.h = h;
+    v.bytes = off;
+    return v;
+}
+
+// Arguments common to the decode kernels.
+struct DecodeParams {
+    const void *q;
+    const void *kv_pool;
+    const float *kv_scales;
+    const int32_t *block_table;
+    const int32_t *seq_lens;
+    float *out;
+    float *lse;
+    int64_t q_stride_request, q_stride_head;
+    int64_t out_stride_request, out_stride_head;
+    int64_t lse_stride_request;
+    int32_t B, H;
+    int32_t head_begin, head_end;
+    int32_t table_stride;
+    int32_t num_pool_pages;
+    int32_t heads_per_group;   // heads one CTA computes
+    int32_t num_groups;        // head groups per KV worker
+    float softmax_scale;
+    // plan (device pointers into the workspace)
+    const int32_t *tile_start, *req_lo, *req_hi, *worker_begin;
+    int32_t *status;
+    float *partial_lse, *partial_out;
+    int32_t num_workers;
+};
+
+// A worker's next piece of work: request, its relative tile range, where the
+// result goes.
+struct Segment {
+    int32_t request;
+    int32_t tile_begin, tile_end;   // page-tile indices relative to floor(lo/64)
+    int32_t lo, hi;                 // effective token range of the request
+    int32_t slot;                   // partial slot, or -1 when the piece is the whole request
+};
+
+// Iterates the segments of worker w in plan order.  Every thread of a CTA calls
+// it with the same arguments and gets the same answer.
+struct SegmentIter {
+    const int32_t *ts;
+    int32_t B, x, end, wb, i, w;
+    __device__ void init(const DecodeParams &p, int worker) {
+        ts = p.tile_start; B = p.B; w = worker;
+        wb = p.worker_begin[worker]; x = wb; end = p.worker_begin[worker + 1];
+        i = 0;
+        if (x < end) {   // request containing tile x: last i with ts[i] <= x and ts[i+1] > x
+            int lo = 0, hi = B;           // invariant: ts[lo] <= x < ts[hi]
+            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (ts[mid] <= x) lo = mid; else hi = mid; }
+            i = lo;
+        }
+    }
+    __device__ bool next(const DecodeParams &p, Segment &s) {
+        if (x >= end) return false;
+        while (ts[i + 1] <= x) ++i;                    // skip finished / empty requests
+        int rs = ts[i], re = ts[i + 1];
+        int seg_end = re < end ? re : end;
+        s.request = i;
+        s.tile_begin = x - rs;
+        s.tile_end = seg_end - rs;
+        s.lo = p.req_lo[i];
+        s.hi = p.req_hi[i];
+        bool full = (x == rs) && (seg_end == re);
+        s.slot = full ? -1 : 2 * w + (rs <= wb ? 0 : 1);
+        x = seg_end;
+        return true;
+    }
+};
+
+// ---- host helpers (splash_api.cu) -----------------------------------------
+void set_error(const char *fmt, ...);
+void count_launch(int n = 1);
+
+// kernels' host launchers
+cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
+                        int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
+                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *status,
+                        cudaStream_t stream);
+cudaError_t launch_decode_simt(const DecodeParams &p, int kv_dtype, cudaStream_t stream);
+int simt_heads_per_group();
+// tcgen05 kernel: how it cuts a head slice of width h into CTAs, and its launcher
+void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *num_groups, int *num_workers);
+cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream);
+cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
+                                 cudaStream_t stream);
+cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *part_out,
+                             const float *part_lse, float *out, float *lse, cudaStream_t stream);
+cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, void *dst_pool,
+                                float *dst_scales, int64_t page_bytes, const int32_t *src_ids,
+                                const int32_t *dst_ids, int64_t n, int32_t src_base, int32_t dst_base,
+                                int32_t max_page_id, int32_t *block_table, int64_t num_entries,
+                                int32_t *remap, cudaStream_t stream);
+
+}  // namespace splash

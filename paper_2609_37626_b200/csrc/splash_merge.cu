@@ -1,0 +1,109 @@
+// Log-sum-exp merges: the public CP merge (splash_lse_merge) and the reduction of
+// the decode kernels' split-KV partial slots.  Both compute, per row,
+//     L = ln sum_j exp(L_j),   O = sum_j exp(L_j - L) O_j,
+// parts with L_j = -inf contributing nothing.  Pure fp32, HBM-bound.
+#include "splash_common.cuh"
+
+namespace splash {
+
+namespace {
+
+constexpr int kMergeThreads = 128;
+
+// One CTA per row; each thread owns float4 columns tid, tid + 128, ...
+__global__ void __launch_bounds__(kMergeThreads)
+lse_merge_kernel(int num_parts, int64_t rows, int d_v, const float *__restrict__ part_out,
+                 const float *__restrict__ part_lse, float *__restrict__ out, float *__restrict__ lse) {
+    const int64_t r = blockIdx.x;
+    float m = -INFINITY;
+    for (int j = 0; j < num_parts; ++j) m = fmaxf(m, part_lse[(int64_t)j * rows + r]);
+    float4 *o4 = reinterpret_cast<float4 *>(out + r * d_v);
+    const int nvec = d_v / 4;
+    if (m == -INFINITY) {
+        for (int c = threadIdx.x; c < nvec; c += kMergeThreads) o4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (threadIdx.x == 0) lse[r] = -INFINITY;
+        return;
+    }
+    float Z = 0.f;
+    for (int j = 0; j < num_parts; ++j) {
+        float Lj = part_lse[(int64_t)j * rows + r];
+        if (Lj != -INFINITY) Z += expf(Lj - m);
+    }
+    const float L = m + logf(Z);
+    for (int c = threadIdx.x; c < nvec; c += kMergeThreads) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < num_parts; ++j) {
+            float Lj = part_lse[(int64_t)j * rows + r];
+            if (Lj == -INFINITY) continue;
+            float w = expf(Lj - L);
+            float4 v = reinterpret_cast<const float4 *>(part_out + ((int64_t)j * rows + r) * d_v)[c];
+            acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
+            acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+        }
+        o4[c] = acc;
+    }
+    if (threadIdx.x == 0) lse[r] = L;
+}
+
+// Grid B*h: block = request i, head k of the slice.  A request computed in one piece was
+// written by the decode kernel itself; an empty request gets (0, -inf) here; a split
+// request is merged from the slots of its workers in worker order.
+__global__ void __launch_bounds__(kMergeThreads)
+split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirst,
+                     const int32_t *__restrict__ req_wlast) {
+    const int h = p.head_end - p.head_begin;
+    const int k = blockIdx.x % h, i = blockIdx.x / h;
+    const int g = p.head_begin + k;
+    const int wf = req_wfirst[i], wl = req_wlast[i];
+    float4 *o4 = reinterpret_cast<float4 *>(p.out + (int64_t)i * p.out_stride_request + (int64_t)g * p.out_stride_head);
+    float *lse = p.lse + (int64_t)i * p.lse_stride_request + g;
+    const int c = threadIdx.x;             // 128 threads x float4 = 512 columns
+    if (wf < 0) {
+        o4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c == 0) *lse = -INFINITY;
+        return;
+    }
+    if (wf == wl) return;
+    const int rs = p.tile_start[i];
+    float m = -INFINITY;
+    for (int w = wf; w <= wl; ++w) {
+        int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
+        m = fmaxf(m, p.partial_lse[(int64_t)slot * h + k]);
+    }
+    float Z = 0.f;
+    for (int w = wf; w <= wl; ++w) {
+        int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
+        Z += expf(p.partial_lse[(int64_t)slot * h + k] - m);
+    }
+    const float L = m + logf(Z);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int w = wf; w <= wl; ++w) {
+        int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
+        int64_t row = (int64_t)slot * h + k;
+        float wgt = expf(p.partial_lse[row] - L);
+        float4 v = reinterpret_cast<const float4 *>(p.partial_out + row * kDV)[c];
+        acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
+        acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
+    }
+    o4[c] = acc;
+    if (c == 0) *lse = L;
+}
+
+}  // namespace
+
+cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *part_out,
+                             const float *part_lse, float *out, float *lse, cudaStream_t stream) {
+    lse_merge_kernel<<<(unsigned)rows, kMergeThreads, 0, stream>>>(num_parts, rows, d_v, part_out, part_lse, out, lse);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
+                                 cudaStream_t stream) {
+    dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * p.B));
+    split_combine_kernel<<<grid, kMergeThreads, 0, stream>>>(p, req_wfirst, req_wlast);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace splash

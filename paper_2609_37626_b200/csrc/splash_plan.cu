@@ -1,0 +1,117 @@
+// Split-KV work plan (device side, integer only, deterministic).
+//
+// The attention time of a decode step is set by the KV bytes read and the
+// contraction work, both linear in the context length (the paper's per-step cost
+// model, App. C: t_att = max{F_att / Phi_att, K_read / beta_KV}), so the plan
+// spreads page tiles -- not requests -- evenly over the CTAs: the global sequence of
+// (request, page tile) pairs is cut into `num_workers` contiguous runs of equal cost,
+// where a non-empty request costs its tile count plus a fixed overhead.  A run that
+// covers a whole request writes the final result; the (at most two) partial pieces
+// at the ends of a run go to per-worker partial slots and are combined afterwards.
+// The plan depends only on (seq_lens, kv ranges, shape), so a repeated call takes
+// the same split and is bit-reproducible.
+#include "splash_common.cuh"
+
+namespace splash {
+
+namespace {
+
+constexpr int kPlanThreads = 1024;
+
+__global__ void __launch_bounds__(kPlanThreads)
+plan_kernel(int B, int W, const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ kv_begin,
+            const int32_t *__restrict__ kv_end, int32_t *__restrict__ tile_start,
+            int32_t *__restrict__ req_lo, int32_t *__restrict__ req_hi,
+            int32_t *__restrict__ req_wfirst, int32_t *__restrict__ req_wlast,
+            int32_t *__restrict__ cost_start, int32_t *__restrict__ worker_begin, int32_t *__restrict__ status) {
+    __shared__ long long warp_tot_tiles[32], warp_tot_cost[32];
+    __shared__ long long carry_tiles, carry_cost;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (tid < 16) status[tid] = 0;
+    if (tid == 0) { carry_tiles = 0; carry_cost = 0; tile_start[0] = 0; cost_start[0] = 0; }
+    __syncthreads();
+
+    // pass 1: effective ranges, tile counts, exclusive prefixes of tiles and of cost
+    for (int base = 0; base < B; base += kPlanThreads) {
+        int i = base + tid;
+        long long n = 0;
+        if (i < B) {
+            int s = seq_lens[i];
+            int lo = kv_begin ? kv_begin[i] : 0;
+            int hi = kv_end ? kv_end[i] : s;
+            if (lo < 0) lo = 0;
+            if (hi > s) hi = s;
+            if (hi < lo) hi = lo;
+            req_lo[i] = lo; req_hi[i] = hi;
+            if (hi > lo) n = (hi + kPage - 1) / kPage - lo / kPage;
+        }
+        long long c = n > 0 ? n + kRequestOverheadTiles : 0;
+        long long sn = n, sc = c;
+        for (int o = 1; o < 32; o <<= 1) {
+            long long a = __shfl_up_sync(0xffffffffu, sn, o);
+            long long b = __shfl_up_sync(0xffffffffu, sc, o);
+            if (lane >= o) { sn += a; sc += b; }
+        }
+        if (lane == 31) { warp_tot_tiles[wid] = sn; warp_tot_cost[wid] = sc; }
+        __syncthreads();
+        long long offn = carry_tiles, offc = carry_cost;
+        for (int k = 0; k < wid; ++k) { offn += warp_tot_tiles[k]; offc += warp_tot_cost[k]; }
+        if (i < B) { tile_start[i + 1] = (int32_t)(offn + sn); cost_start[i + 1] = (int32_t)(offc + sc); }
+        __syncthreads();
+        if (tid == kPlanThreads - 1) { carry_tiles = offn + sn; carry_cost = offc + sc; }
+        __syncthreads();
+    }
+    const long long total_cost = carry_cost;
+    const int total_tiles = (int)carry_tiles;
+
+    // pass 2: worker w starts at cost floor(w * total_cost / W); the request whose
+    // cost interval [cost_start[i], cost_start[i+1]) holds that value is found by
+    // bisection, and a start that falls into the request's fixed overhead snaps to
+    // its first tile.
+    for (int w = tid; w <= W; w += kPlanThreads) {
+        int g = total_tiles;
+        if (w < W && total_cost > 0) {
+            long long target = (total_cost * w) / W;
+            int lo = 0, hi = B;   // invariant cost_start[lo] <= target < cost_start[hi]
+            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (cost_start[mid] <= target) lo = mid; else hi = mid; }
+            while (cost_start[lo + 1] <= target) ++lo;   // (defensive; bisection already lands on a non-empty request)
+            long long off = target - cost_start[lo] - kRequestOverheadTiles;
+            if (off < 0) off = 0;
+            g = tile_start[lo] + (int)off;
+        }
+        worker_begin[w] = g;
+    }
+    __threadfence_block();
+    __syncthreads();
+
+    // pass 3: first / last worker of every request
+    for (int i = tid; i < B; i += kPlanThreads) {
+        int rs = tile_start[i], re = tile_start[i + 1];
+        int wf = -1, wl = -1;
+        if (re > rs) {
+            // worker containing tile x: the w with worker_begin[w] <= x < worker_begin[w+1]
+            int lo = 0, hi = W;   // invariant worker_begin[lo] <= rs < worker_begin[hi]
+            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (worker_begin[mid] <= rs) lo = mid; else hi = mid; }
+            wf = lo;
+            int x = re - 1;
+            lo = 0; hi = W;
+            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (worker_begin[mid] <= x) lo = mid; else hi = mid; }
+            wl = lo;
+        }
+        req_wfirst[i] = wf; req_wlast[i] = wl;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
+                        int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
+                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *status,
+                        cudaStream_t stream) {
+    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.seq_lens, kv_begin, kv_end, tile_start,
+                                                req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace splash

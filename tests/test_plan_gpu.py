@@ -1,0 +1,61 @@
+"""The split-KV plan the device writes, against a plain-Python restatement: it must
+cover every (request, tile) exactly once, in order, and depend only on lengths."""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+def python_plan(lo, hi, W, overhead=4):
+    n = np.where(hi > lo, (hi + 63) // 64 - lo // 64, 0)
+    ts = np.concatenate([[0], np.cumsum(n)])
+    cost = np.where(n > 0, n + overhead, 0)
+    cs = np.concatenate([[0], np.cumsum(cost)])
+    total = int(cs[-1])
+    wb = []
+    for w in range(W + 1):
+        if w == W or total == 0:
+            wb.append(int(ts[-1])); continue
+        target = total * w // W
+        i = int(np.searchsorted(cs, target, side="right") - 1)
+        off = max(0, target - int(cs[i]) - overhead)
+        wb.append(int(ts[i]) + off)
+    return ts, np.array(wb)
+
+
+@pytest.mark.parametrize("seed,B", [(1, 1), (2, 7), (3, 64), (4, 512), (5, 2100)])
+def test_plan_matches_python_and_partitions_tiles(seed, B):
+    import ctypes
+    import torch
+    from paper_2609_37626_b200 import binding, workloads as W
+    rng = np.random.default_rng(seed)
+    lens = W.rollout_lengths(seed, B) // 8
+    lens[rng.integers(0, B, size=max(1, B // 10))] = 0
+    kb = rng.integers(-3, 50, size=B).astype(np.int32)
+    ke = (lens + rng.integers(-40, 5, size=B)).astype(np.int32)
+    w = W.make_workload("plan", seed, lens, H=16, poison=False)
+    dw = binding.DeviceWorkload(w)
+    dw.decode(kv_begin=torch.from_numpy(kb).cuda(), kv_end=torch.from_numpy(ke).cuda(), flags=1)
+    torch.cuda.synchronize()
+    ws = binding.decode_workspace(torch.device("cuda", 0)).cpu().numpy()
+    sm = torch.cuda.get_device_properties(0).multi_processor_count
+    Wn = (2 * sm) // 2         # SIMT path: 16 heads = 2 groups of 8 -> 2*SMs/2 workers
+    ints = ws.view(np.int32)
+    off = 16
+    ts = ints[off:off + B + 1]; off += B + 1
+    lo = ints[off:off + B]; off += B
+    hi = ints[off:off + B]; off += B
+    wf = ints[off:off + B]; off += B
+    wl = ints[off:off + B]; off += B
+    cs = ints[off:off + B + 1]; off += B + 1
+    wb = ints[off:off + Wn + 1]
+    elo = np.maximum(kb, 0); ehi = np.maximum(np.minimum(ke, lens), elo)
+    assert np.array_equal(lo, elo) and np.array_equal(hi, ehi)
+    pts, pwb = python_plan(elo.astype(np.int64), ehi.astype(np.int64), Wn)
+    assert np.array_equal(ts, pts) and np.array_equal(wb, pwb)
+    assert wb[0] == 0 and wb[-1] == ts[-1] and np.all(np.diff(wb) >= 0)
+    for i in range(B):
+        if ts[i + 1] == ts[i]:
+            assert wf[i] == -1
+        else:
+            assert wb[wf[i]] <= ts[i] < wb[wf[i] + 1] and wb[wl[i]] <= ts[i + 1] - 1 < wb[wl[i] + 1]
