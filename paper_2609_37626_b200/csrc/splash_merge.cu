@@ -64,20 +64,25 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
         return;
     }
     if (wf == wl) return;
+    // workers between the first and the last may own no tiles at all (their start
+    // snapped to the same tile as their successor's): they wrote no slot
     const int rs = p.tile_start[i];
     float m = -INFINITY;
     for (int w = wf; w <= wl; ++w) {
+        if (p.worker_begin[w + 1] <= p.worker_begin[w]) continue;
         int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
         m = fmaxf(m, p.partial_lse[(int64_t)slot * h + k]);
     }
     float Z = 0.f;
     for (int w = wf; w <= wl; ++w) {
+        if (p.worker_begin[w + 1] <= p.worker_begin[w]) continue;
         int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
         Z += expf(p.partial_lse[(int64_t)slot * h + k] - m);
     }
     const float L = m + logf(Z);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int w = wf; w <= wl; ++w) {
+        if (p.worker_begin[w + 1] <= p.worker_begin[w]) continue;
         int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
         int64_t row = (int64_t)slot * h + k;
         float wgt = expf(p.partial_lse[row] - L);
