@@ -1,12 +1,646 @@
-// placeholder until the tcgen05 kernel lands
+// tcgen05 / TMA decode kernel for sm_100a.
+//
+// One CTA per (KV worker, head group).  A head group is N = 16, 32 or 64 query heads
+// of one request; the CTA streams the request's pages through shared memory and keeps
+// the transposed problem in tensor memory ("tokens on M"):
+//
+//     S^T [64 tokens x N heads]  = K_tile [64 x 576]   * Q^T [576 x N]      (M = 64)
+//     O^T [512 dv    x N heads] += V_tile^T [512 x 64] * P^T [64 x N]       (4 x M = 128)
+//
+// so a 16-head TP/DOP slice costs a 16-wide MMA instead of a padded 64/128-row one,
+// and both contractions read the SAME shared-memory tile: V is the first 512 columns
+// of the K rows (the latent), taken as an MN-major operand, so every KV byte crosses
+// HBM once per head group.
+//
+// Warp roles (192 threads):
+//   warp 0     TMA producer: block-table driven page gathers into a ring of stages
+//              (nine 64x64-element boxes per page, 128-byte swizzle), and the query
+//              rows of each segment.  Page tails and unaligned KV ranges are handled
+//              by shifting the box in the token dimension so that out-of-range tokens
+//              fall outside the page and are zero-filled by the TMA unit.
+//   warp 1     MMA issuer (one thread): QK^T of tile i+1 is issued before P.V of
+//              tile i, so the tensor pipe works while the softmax warps handle tile i.
+//   warps 2-5  online softmax over tokens (= TMEM lanes): per-head maxima by a
+//              warp-shuffle reduce-scatter plus a small shared-memory exchange, lazy
+//              rescaling of O^T (only when a maximum grows by more than 2^8), P written
+//              to shared memory as the K-major B operand, epilogue.
+//
+// Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA records
+// SPLASH_DEVICE_TIMEOUT in the workspace status block, raises a CTA-wide abort flag,
+// lets copies in flight land, frees its tensor memory and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
 #include "splash_common.cuh"
+
 namespace splash {
-void umma_tiling(int, int h, int sm_count, int *hpg, int *ng, int *nw) {
-    *hpg = h <= 16 ? 16 : (h <= 32 ? 32 : 64);
-    *ng = (h + *hpg - 1) / *hpg;
-    *nw = sm_count / *ng > 0 ? sm_count / *ng : 1;
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kNumSoftmaxThreads = 128;
+constexpr int kChunks = 9;                         // 576 / 64-element (128 B) chunks
+constexpr uint32_t kSlabBytes = 64 * 128;          // one chunk of one page: 64 tokens x 128 B
+constexpr uint32_t kStageBytes = kChunks * kSlabBytes;   // 73,728
+constexpr int kStages = 2;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;          // log2 units
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+enum BarrierId {
+    kBarKvFull = 0,                    // [kStages]
+    kBarKvEmpty = kBarKvFull + kStages,
+    kBarQFull = kBarKvEmpty + kStages,
+    kBarQEmpty,
+    kBarSFull,                         // [2]
+    kBarSEmpty = kBarSFull + 2,        // [2]
+    kBarPFull = kBarSEmpty + 2,
+    kBarPEmpty,
+    kBarOFull,
+    kBarOEmpty,
+    kNumBarriers
+};
+
+template <int N>
+struct Layout {
+    static constexpr uint32_t kQBytes = N * kDQK * 2;
+    static constexpr uint32_t kPBytes = N * 128;             // N rows (heads) x 64 tokens bf16
+    static constexpr uint32_t kOffKv = 0;
+    static constexpr uint32_t kOffQ = kOffKv + kStages * kStageBytes;
+    static constexpr uint32_t kOffP = kOffQ + kQBytes;
+    static constexpr uint32_t kOffRed = kOffP + kPBytes;     // float [N][4]
+    static constexpr uint32_t kOffM = kOffRed + N * 16;      // float [N] running max, log2 domain
+    static constexpr uint32_t kOffAlpha = kOffM + N * 4;     // float [N]
+    static constexpr uint32_t kOffL = kOffAlpha + N * 4;     // float [N]
+    static constexpr uint32_t kOffBar = kOffL + N * 4;       // uint64 [kNumBarriers]
+    static constexpr uint32_t kOffMisc = kOffBar + kNumBarriers * 8;   // u32: tmem base, abort, rescale flag
+    static constexpr uint32_t kBytes = kOffMisc + 16;
+    // tensor memory columns
+    static constexpr uint32_t kColO = 0;                     // 4 blocks x N columns
+    static constexpr uint32_t kColS = 4 * N;                 // 2 buffers x N columns
+    static_assert(kColS + 2 * N <= 512, "tensor memory overflow");
+    static_assert(kBytes <= 232448, "shared memory overflow");
+    static_assert(kOffQ % 1024 == 0 && kOffP % 1024 == 0 && (N * 128) % 1024 == 0, "swizzle atoms need 1024-byte alignment");
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
-cudaError_t launch_decode_umma(const DecodeParams &, const splash_mla_shape &, cudaStream_t) {
-    return cudaErrorNotSupported;
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+struct Ctx {
+    volatile uint32_t *abort_flag;   // shared
+    int32_t *status;                 // global, 16 ints
+};
+
+// Bounded wait.  Returns false if the CTA is aborting (this wait or another one timed out).
+__device__ __noinline__ bool mbar_wait_slow(const Ctx &ctx, uint32_t bar, uint32_t parity, int bar_id) {
+    const unsigned long long start = global_timer_ns();
+    for (;;) {
+        for (int k = 0; k < 256; ++k)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*ctx.abort_flag) return false;
+        if (global_timer_ns() - start > kWaitLimitNs) {
+            *ctx.abort_flag = 1;
+            if (atomicCAS(ctx.status, 0, (int)SPLASH_DEVICE_TIMEOUT) == 0) {
+                ctx.status[1] = (int)blockIdx.x;
+                ctx.status[2] = bar_id;
+                ctx.status[3] = (int)threadIdx.x;
+            }
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(const Ctx &ctx, uint32_t bar, uint32_t parity, int bar_id) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(ctx, bar, parity, bar_id);
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// 16 consecutive fp32 columns of this warp's 32 lanes
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+          "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+          "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+          "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+          "r"(__float_as_uint(v[15])) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor: fp32 accumulate, bf16 x bf16.
+__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+// Reduce-scatter over the 32 lanes of a warp: on return lane L holds, in v[0 .. max(1, N/32)),
+// the reduction over all lanes of the entries it owns (N = 64: heads 2L, 2L+1; N = 32: head L;
+// N = 16: head L >> 1, both lanes of a pair holding it).
+template <int CNT, int MASK, bool IS_MAX>
+struct ReduceScatter {
+    template <int N>
+    static __device__ __forceinline__ void run(float (&v)[N], int lane) {
+        if constexpr (MASK >= 1) {
+            if constexpr (CNT > 1) {
+                constexpr int kHalf = CNT / 2;
+                const bool upper = (lane & MASK) != 0;
+#pragma unroll
+                for (int i = 0; i < kHalf; ++i) {
+                    float keep = upper ? v[i + kHalf] : v[i];
+                    float send = upper ? v[i] : v[i + kHalf];
+                    float recv = __shfl_xor_sync(0xffffffffu, send, MASK);
+                    v[i] = IS_MAX ? fmaxf(keep, recv) : keep + recv;
+                }
+                ReduceScatter<kHalf, MASK / 2, IS_MAX>::run(v, lane);
+            } else {
+                float recv = __shfl_xor_sync(0xffffffffu, v[0], MASK);
+                v[0] = IS_MAX ? fmaxf(v[0], recv) : v[0] + recv;
+                ReduceScatter<1, MASK / 2, IS_MAX>::run(v, lane);
+            }
+        }
+    }
+};
+
+template <int N>
+__device__ __forceinline__ int owned_head(int lane, int i) {
+    if (N >= 32) return lane * (N / 32) + i;
+    return lane >> 1;     // N == 16
+}
+
+// Valid rows of a tile after the token shift: page-relative tokens [a, b) land in rows
+// [r_lo, r_hi) of the 64-row box when the box starts at token tok0.
+struct TileGeom { int tok0, r_lo, r_hi; };
+__device__ __forceinline__ TileGeom tile_geom(int lo, int hi, int t0) {
+    int a = max(lo, t0) - t0;
+    int b = min(hi, t0 + kPage) - t0;
+    TileGeom g;
+    if (b < kPage) { g.tok0 = b - kPage; g.r_lo = kPage - b + a; g.r_hi = kPage; }   // end cut: align the end to the box end
+    else { g.tok0 = a; g.r_lo = 0; g.r_hi = kPage - a; }                              // front cut (or none)
+    return g;
+}
+
+// ---------------------------------------------------------------- the kernel
+template <int N>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmap_kv,
+                   const __grid_constant__ CUtensorMap tmap_q) {
+    using L = Layout<N>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int worker = blockIdx.x / p.num_groups;
+    const int group = blockIdx.x % p.num_groups;
+    const int head0 = p.head_begin + group * N;
+    const int h = p.head_end - p.head_begin;
+
+    volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + L::kOffMisc);
+    Ctx ctx{misc + 1, p.status};
+    auto bar = [&](int id) -> uint32_t { return sbase + L::kOffBar + 8u * (uint32_t)id; };
+
+    if ((sbase & 1023u) != 0) {      // swizzle atoms need a 1024-byte aligned window
+        if (tid == 0 && atomicCAS(p.status, 0, (int)SPLASH_CUDA_ERROR) == 0) { p.status[1] = (int)blockIdx.x; p.status[2] = -100; }
+        return;
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), 1); }
+        mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), 1); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxThreads); }
+        mbar_init(bar(kBarPFull), kNumSoftmaxThreads); mbar_init(bar(kBarPEmpty), 1);
+        mbar_init(bar(kBarOFull), 1); mbar_init(bar(kBarOEmpty), kNumSoftmaxThreads);
+        misc[1] = 0; misc[2] = 0; misc[3] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + L::kOffMisc), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = misc[0];
+
+    SegmentIter it;
+    it.init(p, worker);
+    Segment seg;
+
+    if (warp == 0) {
+        // ===================================================== TMA producer
+        uint32_t kv_it = 0, seg_it = 0;
+        bool ok = true;
+        while (ok && it.next(p, seg)) {
+            if (lane == 0) {
+                ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
+                if (ok) {
+                    mbar_expect_tx(bar(kBarQFull), L::kQBytes);
+                    for (int c = 0; c < kChunks; ++c)
+                        tma_load_3d(sbase + L::kOffQ + c * (N * 128), &tmap_q, bar(kBarQFull), c * 64, head0, seg.request);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            const int first_page = seg.lo / kPage;
+            const int32_t *table = p.block_table + (int64_t)seg.request * p.table_stride;
+            int entry = 0;
+            for (int tile = seg.tile_begin; ok && tile < seg.tile_end; ++tile) {
+                const int rel = tile - seg.tile_begin;
+                if ((rel & 31) == 0) {
+                    int idx = tile + lane;
+                    entry = idx < seg.tile_end ? table[first_page + idx] : 0;
+                }
+                const int page = __shfl_sync(0xffffffffu, entry, rel & 31);
+                if (lane == 0) {
+                    const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
+                    ok = mbar_wait(ctx, bar(kBarKvEmpty + stage), ph ^ 1, kBarKvEmpty + stage);
+                    if (ok) {
+                        const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
+                        mbar_expect_tx(bar(kBarKvFull + stage), kStageBytes);
+                        const uint32_t dst = sbase + L::kOffKv + stage * kStageBytes;
+                        for (int c = 0; c < kChunks; ++c)
+                            tma_load_3d(dst + c * kSlabBytes, &tmap_kv, bar(kBarKvFull + stage), c * 64, g.tok0, page);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                ++kv_it;
+            }
+            ++seg_it;
+        }
+    } else if (warp == 1) {
+        // ===================================================== MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t kIdescQK = make_idesc(64, N, 0, 0);
+            constexpr uint32_t kIdescPV = make_idesc(128, N, 1, 0);
+            uint32_t kv_it = 0, s_it = 0, p_it = 0, seg_it = 0;
+            bool ok = true;
+            // S^T of the tile with global index kv: 36 MMAs of K = 16
+            auto issue_qk = [&](uint32_t kv, uint32_t sidx) -> bool {
+                const uint32_t stage = kv % kStages, ph = (kv / kStages) & 1, b = sidx & 1;
+                if (!mbar_wait(ctx, bar(kBarKvFull + stage), ph, kBarKvFull + stage)) return false;
+                if (!mbar_wait(ctx, bar(kBarSEmpty + b), ((sidx >> 1) & 1) ^ 1, kBarSEmpty + b)) return false;
+                tcgen05_fence_after();
+                const uint32_t a0 = sbase + L::kOffKv + stage * kStageBytes;
+                const uint32_t b0 = sbase + L::kOffQ;
+                const uint32_t d = tmem_base + L::kColS + b * N;
+#pragma unroll
+                for (int c = 0; c < kChunks; ++c) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        uint64_t da = make_desc(a0 + c * kSlabBytes + k * 32, 16, 1024);
+                        uint64_t db = make_desc(b0 + c * (N * 128) + k * 32, 16, 1024);
+                        umma_bf16(d, da, db, kIdescQK, (c | k) != 0);
+                    }
+                }
+                umma_commit(bar(kBarSFull + b));
+                return true;
+            };
+            while (ok && it.next(p, seg)) {
+                const int ntiles = seg.tile_end - seg.tile_begin;
+                ok = mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
+                if (!ok) break;
+                ok = issue_qk(kv_it, s_it);
+                if (ok && ntiles == 1) umma_commit(bar(kBarQEmpty));
+                for (int i = 0; ok && i < ntiles; ++i) {
+                    if (i + 1 < ntiles) {
+                        ok = issue_qk(kv_it + i + 1, s_it + i + 1);
+                        if (!ok) break;
+                        if (i + 2 == ntiles) umma_commit(bar(kBarQEmpty));
+                    }
+                    ok = mbar_wait(ctx, bar(kBarPFull), p_it & 1, kBarPFull);
+                    if (!ok) break;
+                    if (i == 0) {
+                        ok = mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty);
+                        if (!ok) break;
+                    }
+                    tcgen05_fence_after();
+                    const uint32_t stage = (kv_it + i) % kStages;
+                    const uint32_t v0 = sbase + L::kOffKv + stage * kStageBytes;
+                    const uint32_t p0 = sbase + L::kOffP;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            // A = V^T block j: 128 dv (two 64-element chunks, LBO apart) x 16 tokens (SBO per 8)
+                            uint64_t da = make_desc(v0 + (2 * j) * kSlabBytes + k * 2048, kSlabBytes, 1024);
+                            uint64_t db = make_desc(p0 + k * 32, 16, 1024);
+                            umma_bf16(tmem_base + L::kColO + j * N, da, db, kIdescPV, (i | k) != 0);
+                        }
+                    }
+                    umma_commit(bar(kBarKvEmpty + stage));
+                    umma_commit(bar(kBarPEmpty));
+                    if (i + 1 == ntiles) umma_commit(bar(kBarOFull));
+                    ++p_it;
+                }
+                kv_it += ntiles; s_it += ntiles;
+                ++seg_it;
+            }
+        }
+    } else {
+        // ===================================================== softmax + epilogue warps
+        const int q4 = warp & 3;                       // TMEM lane quadrant of this warp
+        const int st = (warp - 2) * 32 + lane;         // 0..127
+        const int row = 16 * q4 + lane;                // token row of the S^T tile (lanes < 16)
+        const uint32_t lane_addr = (uint32_t)(32 * q4) << 16;
+        float *red = reinterpret_cast<float *>(smem + L::kOffRed);
+        float *m_s = reinterpret_cast<float *>(smem + L::kOffM);
+        float *alpha_s = reinterpret_cast<float *>(smem + L::kOffAlpha);
+        float *l_s = reinterpret_cast<float *>(smem + L::kOffL);
+        const float scale_log2 = p.softmax_scale * kLog2e;
+        constexpr int kOwn = N >= 32 ? N / 32 : 1;
+        uint32_t s_it = 0, p_it = 0, seg_it = 0;
+        bool ok = true;
+        while (ok && it.next(p, seg)) {
+            if (st < N) m_s[st] = -INFINITY;
+            float l_local[N];
+#pragma unroll
+            for (int n = 0; n < N; ++n) l_local[n] = 0.f;
+            softmax_bar_sync();
+            const int first_page = seg.lo / kPage;
+            const int ntiles = seg.tile_end - seg.tile_begin;
+            for (int i = 0; ok && i < ntiles; ++i) {
+                const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + seg.tile_begin + i) * kPage);
+                const bool valid = lane < 16 && row >= g.r_lo && row < g.r_hi;
+                const uint32_t b = s_it & 1;
+                ok = mbar_wait(ctx, bar(kBarSFull + b), (s_it >> 1) & 1, kBarSFull + b);
+                if (!ok) break;
+                tcgen05_fence_after();
+                float s[N];
+#pragma unroll
+                for (int c = 0; c < N / 16; ++c)
+                    tmem_ld16(tmem_base + lane_addr + L::kColS + b * N + c * 16, *reinterpret_cast<float(*)[16]>(&s[c * 16]));
+                tmem_wait_ld();
+                tcgen05_fence_before();
+                mbar_arrive(bar(kBarSEmpty + b));
+                float mx[N];
+#pragma unroll
+                for (int n = 0; n < N; ++n) { s[n] = valid ? s[n] * scale_log2 : -INFINITY; mx[n] = s[n]; }
+                ReduceScatter<N, 16, true>::run(mx, lane);
+                if (N >= 32 || (lane & 1) == 0) {
+#pragma unroll
+                    for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + (warp - 2)] = mx[k];
+                }
+                if (st == 0) misc[2 + (i & 1)] = 0;      // this tile's "some maximum grew" flag
+                softmax_bar_sync();
+                if (st < N) {
+                    float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
+                    float mt = fmaxf(fmaxf(r4.x, r4.y), fmaxf(r4.z, r4.w));
+                    float m_old = m_s[st];
+                    float al = 1.f;
+                    if (mt > m_old + kRescaleThreshold) {        // also taken when m_old = -inf
+                        al = (m_old == -INFINITY) ? 0.f : fast_exp2(m_old - mt);
+                        m_s[st] = mt;
+                        misc[2 + (i & 1)] = 1;
+                    }
+                    alpha_s[st] = al;
+                }
+                softmax_bar_sync();
+                const bool rescale = misc[2 + (i & 1)] != 0;
+                if (rescale) {
+#pragma unroll
+                    for (int n = 0; n < N; ++n) l_local[n] *= alpha_s[n];
+                }
+#pragma unroll
+                for (int n = 0; n < N; ++n) {
+                    s[n] = fast_exp2(s[n] - m_s[n]);
+                    l_local[n] += s[n];
+                }
+                // P.V of the previous tile must be done with the P buffer and with O^T
+                ok = mbar_wait(ctx, bar(kBarPEmpty), (p_it & 1) ^ 1, kBarPEmpty);
+                if (!ok) break;
+                tcgen05_fence_after();
+                if (rescale && i > 0) {
+#pragma unroll 1
+                    for (int c = 0; c < 4 * N / 16; ++c) {
+                        float o[16];
+                        const uint32_t addr = tmem_base + lane_addr + L::kColO + c * 16;
+                        tmem_ld16(addr, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) o[k] *= alpha_s[(c * 16 + k) % N];
+                        tmem_st16(addr, o);
+                    }
+                    tmem_wait_st();
+                }
+                if (lane < 16) {
+                    // P^T as the K-major, 128-byte-swizzled B operand: row = head, 64 tokens per row
+                    uint8_t *pb = smem + L::kOffP;
+                    const uint32_t chunk = (uint32_t)row >> 3, within = ((uint32_t)row & 7) * 2;
+#pragma unroll
+                    for (int n = 0; n < N; ++n) {
+                        __nv_bfloat16 v = __float2bfloat16_rn(s[n]);
+                        *reinterpret_cast<__nv_bfloat16 *>(pb + n * 128 + ((chunk ^ (uint32_t)(n & 7)) << 4) + within) = v;
+                    }
+                }
+                fence_proxy_async();
+                tcgen05_fence_before();
+                mbar_arrive(bar(kBarPFull));
+                ++s_it; ++p_it;
+            }
+            if (!ok) break;
+            // ---- row sums over all 128 lanes' partial sums
+            ReduceScatter<N, 16, false>::run(l_local, lane);
+            if (N >= 32 || (lane & 1) == 0) {
+#pragma unroll
+                for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + (warp - 2)] = l_local[k];
+            }
+            softmax_bar_sync();
+            if (st < N) {
+                float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
+                float l = (r4.x + r4.y) + (r4.z + r4.w);
+                l_s[st] = 1.f / l;
+                const int gh = head0 + st;
+                if (gh < p.head_end) {
+                    float lse = (m_s[st] + log2f(l)) * kLn2;
+                    if (seg.slot < 0) p.lse[(int64_t)seg.request * p.lse_stride_request + gh] = lse;
+                    else p.partial_lse[(int64_t)seg.slot * h + (gh - p.head_begin)] = lse;
+                }
+            }
+            softmax_bar_sync();
+            // ---- epilogue: O^T block j holds dv = 128 j + TMEM lane, one column per head
+            ok = mbar_wait(ctx, bar(kBarOFull), seg_it & 1, kBarOFull);
+            if (!ok) break;
+            tcgen05_fence_after();
+            float *obase;
+            int64_t ostride;
+            if (seg.slot < 0) {
+                obase = p.out + (int64_t)seg.request * p.out_stride_request + (int64_t)head0 * p.out_stride_head;
+                ostride = p.out_stride_head;
+            } else {
+                obase = p.partial_out + ((int64_t)seg.slot * h + (head0 - p.head_begin)) * kDV;
+                ostride = kDV;
+            }
+            const int nvalid = min(N, p.head_end - head0);
+#pragma unroll 1
+            for (int j = 0; j < 4; ++j) {
+                const int dv = 128 * j + 32 * q4 + lane;
+#pragma unroll
+                for (int c = 0; c < N / 16; ++c) {
+                    float o[16];
+                    tmem_ld16(tmem_base + lane_addr + L::kColO + j * N + c * 16, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const int n = c * 16 + k;
+                        if (n < nvalid) obase[(int64_t)n * ostride + dv] = o[k] * l_s[n];
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            mbar_arrive(bar(kBarOEmpty));
+            ++seg_it;
+        }
+    }
+
+    // ---- teardown
+    if (*ctx.abort_flag) {
+        // let bulk copies that were already issued land before the CTA's shared memory goes away
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+bool make_map_3d(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
+                 uint64_t stride2_bytes, uint32_t box0, uint32_t box1) {
+    EncodeTiledFn fn = encode_tiled();
+    if (!fn) { set_error("cuTensorMapEncodeTiled is not available"); return false; }
+    cuuint64_t dims[3] = {d0, d1, d2};
+    cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
+    cuuint32_t box[3] = {box0, box1, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r); return false; }
+    return true;
+}
+
+template <int N>
+cudaError_t launch_n(const DecodeParams &p, const CUtensorMap &mkv, const CUtensorMap &mq, cudaStream_t stream) {
+    const int smem = (int)Layout<N>::kBytes;
+    cudaError_t e = cudaFuncSetAttribute(decode_umma_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    decode_umma_kernel<N><<<(unsigned)(p.num_workers * p.num_groups), kThreads, smem, stream>>>(p, mkv, mq);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *num_groups, int *num_workers) {
+    (void)kv_dtype;
+    const int n = h <= 16 ? 16 : (h <= 32 ? 32 : 64);
+    *heads_per_group = n;
+    *num_groups = (h + n - 1) / n;
+    const int w = sm_count / *num_groups;
+    *num_workers = w > 0 ? w : 1;
+}
+
+cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream) {
+    if (shape.kv_dtype != SPLASH_KV_BF16) return cudaErrorNotSupported;
+    alignas(64) CUtensorMap mkv, mq;
+    const int n = p.heads_per_group;
+    if (!make_map_3d(&mkv, p.kv_pool, kDQK, kPage, (uint64_t)(p.num_pool_pages > 0 ? p.num_pool_pages : 1),
+                     (uint64_t)kDQK * 2, (uint64_t)kPage * kDQK * 2, 64, 64))
+        return cudaErrorInvalidValue;
+    if (!make_map_3d(&mq, p.q, kDQK, (uint64_t)p.H, (uint64_t)p.B, (uint64_t)p.q_stride_head * 2,
+                     (uint64_t)(p.B > 1 ? p.q_stride_request : p.q_stride_head * p.H) * 2, 64, (uint32_t)n))
+        return cudaErrorInvalidValue;
+    switch (n) {
+        case 16: return launch_n<16>(p, mkv, mq, stream);
+        case 32: return launch_n<32>(p, mkv, mq, stream);
+        case 64: return launch_n<64>(p, mkv, mq, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
 }  // namespace splash
