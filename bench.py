@@ -1,0 +1,438 @@
+#!/usr/bin/env python
+"""Benchmark of the MLA decode hot path (one attention layer-call over a paged latent
+KV cache) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
+
+A step is one ``splash_mla_decode`` call (work plan, page gather, QK^T, online softmax,
+P.V, epilogue, split-KV combine) over one synthetic batch.  The default workload is the
+DP-attention request slice (64 requests, contexts U[1024, 8192], 128 heads, bf16 KV);
+``--workload`` picks another configuration, and the default run also reports the other
+configurations (head slice at 32K, CP ranges + LSE merge, fp8 rollout + page migration)
+under ``"workloads"``.  Rank 0 prints ONE JSON line.
+
+Timing: CUDA events on the launching stream around every step, L2 flushed between
+steps by writing a 256 MiB buffer outside the timed intervals, and every workload's KV
+is larger than the 126 MB L2 anyway.  ``value`` is requests decoded per second for one
+layer-call with inputs resident in HBM; ``e2e`` repeats it with the step's inputs
+(q, block table, lengths) copied from pinned host memory and out / lse copied back
+inside the timed region (the KV pool itself is serving state that lives in HBM).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_37626_b200 import workloads as W  # noqa: E402
+
+METRIC = "mla_decode_tokens_per_s_per_gpu"
+UNIT = "tokens/s"
+WORKLOAD_IDS = {"c1": 1, "c2": 2, "c3": 3, "c4": 4, "c5": 5}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return dict(FALLBACK_PEAKS)
+
+
+def load_traffic():
+    """Per-launch DRAM traffic of the decode kernel from committed ncu summaries."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(path):
+        return json.load(open(path))
+    return {}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while running."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        # "under load": samples at or above the median of the upper half
+        load = sorted(sm)[len(sm) // 2:]
+        return {"sm_mhz": float(np.median(load)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def pairs_sample(w, budget_macs: float, seed: int = 0):
+    """A bounded random sample of (request, head) pairs for the oracle."""
+    rng = np.random.default_rng(seed)
+    heads = np.arange(w.head_begin, w.head_end)
+    all_pairs = [(i, g) for i in range(w.B) for g in heads]
+    order = rng.permutation(len(all_pairs))
+    lens = w.seq_lens.astype(np.int64)
+    picked, macs = [], 0.0
+    for k in order:
+        i, g = all_pairs[k]
+        picked.append((i, g))
+        macs += float(lens[i]) * (W.D_QK + W.D_V)
+        if macs >= budget_macs:
+            break
+    return np.array(picked, dtype=np.int32), macs, len(all_pairs)
+
+
+def time_oracle(w, seconds_target: float = 12.0):
+    """Times the oracle, as it stands, on a bounded sample of the workload."""
+    import oracle
+    threads = oracle.num_threads()
+    # probe rate with a small sample, then size the main sample
+    probe, macs0, total_pairs = pairs_sample(w, 2e8 * threads, seed=1)
+    t0 = time.perf_counter()
+    oracle.mla_decode(w.q, w.kv_pool, w.block_table, w.seq_lens, softmax_scale=w.softmax_scale,
+                      kv_scales=w.kv_scales, kv_begin=w.kv_begin, kv_end=w.kv_end, pairs=probe)
+    rate = macs0 / max(time.perf_counter() - t0, 1e-6)
+    sample, macs, _ = pairs_sample(w, rate * seconds_target, seed=2)
+    t0 = time.perf_counter()
+    oracle.mla_decode(w.q, w.kv_pool, w.block_table, w.seq_lens, softmax_scale=w.softmax_scale,
+                      kv_scales=w.kv_scales, kv_begin=w.kv_begin, kv_end=w.kv_end, pairs=sample)
+    dt = time.perf_counter() - t0
+    total_macs = float(w.total_tokens()) * (W.D_QK + W.D_V) * (w.head_end - w.head_begin)
+    full_time = dt * total_macs / macs
+    return {"value": w.B / full_time, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{len(sample)} of {total_pairs} (request, head) pairs, {dt:.1f} s of CPU work, "
+                      f"scaled to the whole batch by multiply-accumulates"}, dt
+
+
+# --------------------------------------------------------------------------- GPU side
+class GpuBench:
+    def __init__(self, device):
+        import torch
+        from paper_2609_37626_b200 import binding
+        self.torch, self.binding, self.device = torch, binding, device
+        binding.load()
+        self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+
+    def flush_l2(self):
+        self.flush_buf.fill_(1)
+
+    def timed(self, fn, steps, warmup):
+        torch = self.torch
+        for _ in range(warmup):
+            self.flush_l2(); fn()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(steps):
+            self.flush_l2()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record()
+            b.synchronize()
+            times.append(a.elapsed_time(b))
+        return np.array(times)
+
+    def decode_workload(self, w, steps, warmup, peaks, traffic_table, name):
+        torch, binding = self.torch, self.binding
+        dw = binding.DeviceWorkload(w, self.device)
+        out = torch.empty((w.B, w.H, W.D_V), dtype=torch.float32, device=self.device)
+        lse = torch.empty((w.B, w.H), dtype=torch.float32, device=self.device)
+        step = lambda: dw.decode(out=out, lse=lse)
+        ms = self.timed(step, steps, warmup)
+        launches = binding.splash_last_launch_count()
+        # kernel-level durations (events recorded by the library around each kernel)
+        binding.splash_set_kernel_timing(True)
+        kt = []
+        for _ in range(steps):
+            self.flush_l2(); step()
+            kt.append(binding.splash_get_kernel_timing())
+        binding.splash_set_kernel_timing(False)
+        kt = np.array(kt)
+        ws = binding.decode_workspace(torch.device(self.device))
+        rc, detail = binding.splash_workspace_status(ws)
+        if rc != 0:
+            raise RuntimeError(f"device status {rc} {detail}")
+        dec_ms = float(kt[:, 1].mean())
+        alg_bytes, alg_flops = w.algorithmic_bytes(), w.algorithmic_flops()
+        t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+        fp8 = w.kv_dtype == 1
+        t_tensor = alg_flops / (peaks["bf16_tflops"] * 1e12)
+        if t_hbm >= t_tensor:
+            roof = {"bound": "hbm", "achieved": alg_bytes / (dec_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        else:
+            roof = {"bound": "tensor", "achieved": alg_flops / (dec_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
+                    "unit": "TFLOP/s"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["traffic"] = traffic_table.get(name)
+        roof.update({"kernel": "decode_umma_kernel", "kernel_ms": dec_ms, "peak_source": peaks["source"],
+                     "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
+                     "roofline_ms": max(t_hbm, t_tensor) * 1e3,
+                     "achieved_gbs": alg_bytes / (dec_ms * 1e-3) / 1e9,
+                     "achieved_tflops": alg_flops / (dec_ms * 1e-3) / 1e12,
+                     "plan_ms": float(kt[:, 0].mean()), "combine_ms": float(kt[:, 2].mean()),
+                     "note": "fp8 KV: tensor peak taken at the bf16 rate" if fp8 else None})
+        res = {"ms_per_step": float(ms.mean()), "ms_p50": float(np.median(ms)), "ms_p95": float(np.percentile(ms, 95)),
+               "tokens_per_s": w.B / (ms.mean() * 1e-3), "tokens_per_s_78_layers": w.B / (ms.mean() * 1e-3) / 78,
+               "launches_per_step": launches, "roofline": roof,
+               "frac_of_roofline_whole_call": max(t_hbm, t_tensor) * 1e3 / float(np.median(ms)),
+               "tokens": w.total_tokens(), "requests": w.B, "heads": w.head_end - w.head_begin}
+        return res, dw, out, lse
+
+    def e2e(self, w, dw, steps, warmup):
+        """Same call with the step's inputs coming from pinned host memory and the
+        results going back to it inside the timed region."""
+        torch, binding = self.torch, self.binding
+        hq = torch.from_numpy(w.q.view(np.int16)).pin_memory()
+        ht = torch.from_numpy(w.block_table).pin_memory()
+        hs = torch.from_numpy(w.seq_lens).pin_memory()
+        dq = torch.empty_like(dw.q); dt_ = torch.empty_like(dw.block_table); ds = torch.empty_like(dw.seq_lens)
+        out = torch.empty((w.B, w.H, W.D_V), dtype=torch.float32, device=self.device)
+        lse = torch.empty((w.B, w.H), dtype=torch.float32, device=self.device)
+        hb, he = w.head_begin, w.head_end
+        ho = torch.empty((w.B, he - hb, W.D_V), dtype=torch.float32).pin_memory()
+        hl = torch.empty((w.B, he - hb), dtype=torch.float32).pin_memory()
+
+        def step():
+            dq.view(torch.int16).copy_(hq, non_blocking=True)
+            dt_.copy_(ht, non_blocking=True); ds.copy_(hs, non_blocking=True)
+            binding.splash_mla_decode(dq, dw.kv_pool, dt_, ds, softmax_scale=w.softmax_scale, kv_scales=dw.kv_scales,
+                                      head_begin=hb, head_end=he, kv_begin=dw.kv_begin, kv_end=dw.kv_end,
+                                      out=out, lse=lse)
+            ho.copy_(out[:, hb:he], non_blocking=True); hl.copy_(lse[:, hb:he], non_blocking=True)
+
+        ms = self.timed(step, steps, warmup)
+        h2d = hq.numel() * 2 + ht.numel() * 4 + hs.numel() * 4
+        d2h = ho.numel() * 4 + hl.numel() * 4
+        return {"value": w.B / (ms.mean() * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                "d2h_bytes_per_step": int(d2h), "ms_per_step": float(ms.mean())}
+
+    def cp_workload(self, w, steps, warmup):
+        """CP: 8 contiguous KV ranges, each a partial (O, LSE) call, then splash_lse_merge."""
+        torch, binding = self.torch, self.binding
+        dw = binding.DeviceWorkload(w, self.device)
+        ranges = [(torch.from_numpy(a).to(self.device), torch.from_numpy(b).to(self.device))
+                  for a, b in W.cp_ranges(w.seq_lens, 8)]
+        po = torch.empty((8, w.B, w.H, W.D_V), dtype=torch.float32, device=self.device)
+        pl = torch.empty((8, w.B, w.H), dtype=torch.float32, device=self.device)
+        mo = torch.empty((w.B * w.H, W.D_V), dtype=torch.float32, device=self.device)
+        ml = torch.empty((w.B * w.H,), dtype=torch.float32, device=self.device)
+
+        def step():
+            for j, (a, b) in enumerate(ranges):
+                dw.decode(out=po[j], lse=pl[j], kv_begin=a, kv_end=b)
+            binding.splash_lse_merge(po.view(8, -1, W.D_V), pl.view(8, -1), out=mo, lse=ml)
+
+        ms = self.timed(step, steps, warmup)
+        merge = self.timed(lambda: binding.splash_lse_merge(po.view(8, -1, W.D_V), pl.view(8, -1), out=mo, lse=ml),
+                           steps, warmup)
+        return {"ms_8_ranges_plus_merge": float(ms.mean()), "ms_merge": float(merge.mean()),
+                "launches_per_step": 8 * 3 + 1}
+
+    def migrate_workload(self, w, dw, steps, warmup, peaks):
+        torch, binding = self.torch, self.binding
+        # the workload was built with a second pool of ceil(0.3 * used pages) pages appended
+        total = w.num_pool_pages
+        extra_pages = int(np.ceil(len(w.used_pages) * 0.3))
+        n_src = total - extra_pages
+        src, dst = W.migration_plan(W.BASE_SEED + 55, w.used_pages, extra_pages, 0.3)
+        dsrc, ddst = torch.from_numpy(src).to(self.device), torch.from_numpy(dst).to(self.device)
+        table0 = dw.block_table.clone()
+
+        def step():
+            dw.block_table.copy_(table0)
+            binding.splash_kv_page_migrate(dw.kv_pool[:n_src], dw.kv_pool[n_src:], dsrc, ddst, dw.block_table,
+                                           src_scales=dw.kv_scales[:n_src], dst_scales=dw.kv_scales[n_src:],
+                                           src_id_base=0, dst_id_base=n_src, max_page_id=total)
+
+        ms = self.timed(step, steps, warmup)
+        page_bytes = 64 * 576 + 256
+        moved = 2.0 * len(src) * page_bytes
+        dw.block_table.copy_(table0)
+        return {"ms_per_call": float(ms.mean()), "pages": int(len(src)), "bytes_read_plus_written": moved,
+                "achieved_gbs": moved / (ms.mean() * 1e-3) / 1e9, "frac_of_hbm_peak": moved / (ms.mean() * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                "note": "includes the block-table restore copy issued before each call"}
+
+
+def run_reference(args, rank):
+    """The oracle as the reference arm: each step is a bounded sample of the workload."""
+    if rank != 0:
+        return
+    w = W.config(WORKLOAD_IDS[args.workload])
+    per_step = max(2.0, min(20.0, 150.0 / max(args.steps + args.warmup, 1)))
+    vals, cores, sample = [], None, None
+    for k in range(args.warmup + args.steps):
+        res, _ = time_oracle(w, seconds_target=per_step)
+        if k >= args.warmup:
+            vals.append(res["value"])
+        cores, sample = res["cores"], res["sample"]
+    v = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": w.B / v * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": W.CONFIG_NAMES[WORKLOAD_IDS[args.workload] - 1], "requests": w.B,
+                       "heads": w.head_end - w.head_begin, "tokens": w.total_tokens()},
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", choices=sorted(WORKLOAD_IDS), default="c2")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only-main", action="store_true", help="skip the other configurations")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(device))
+    peaks = load_peaks()
+    traffic = load_traffic()
+    gb = GpuBench(device)
+
+    # every rank owns its own batch (request slices are independent: weak scaling, no collective)
+    idx = WORKLOAD_IDS[args.workload]
+    t_gen = time.time()
+    w = W.config(idx) if world == 1 else W.config(idx)
+    if world > 1:
+        w = W.make_workload(w.name, W.BASE_SEED + idx + 100 * rank, w.seq_lens, H=w.H, head_begin=w.head_begin,
+                            head_end=w.head_end, kv_dtype=w.kv_dtype)
+    gen_s = time.time() - t_gen
+
+    sampler = ClockSampler(local_rank)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    main_res, dw, out, lse = gb.decode_workload(w, args.steps, args.warmup, peaks, traffic, args.workload)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    e2e = gb.e2e(w, dw, args.steps, args.warmup)
+
+    ms = main_res["ms_per_step"]
+    e2e_ms = e2e["ms_per_step"]
+    if world > 1:
+        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_ms = float(t[0]), float(t[1])
+    value = world * w.B / (ms * 1e-3)
+    e2e_value = world * w.B / (e2e_ms * 1e-3)
+
+    extra = {}
+    cpu = None
+    if rank == 0 and world == 1:
+        if not args.no_cpu_baseline:
+            cpu, _ = time_oracle(w)
+        if not args.only_main:
+            del dw, out, lse
+            torch.cuda.empty_cache()
+            for name in ("c3", "c4", "c5"):
+                if name == args.workload:
+                    continue
+                try:
+                    if name == "c5":
+                        wx = W.config(5, extra_pool_factor=0.3)
+                    else:
+                        wx = W.config(WORKLOAD_IDS[name])
+                    r, dwx, ox, lx = gb.decode_workload(wx, args.steps, args.warmup, peaks, traffic, name)
+                    if name == "c4":
+                        del dwx
+                        r["cp"] = gb.cp_workload(wx, max(5, args.steps // 2), args.warmup)
+                    if name == "c5":
+                        r["page_migrate"] = gb.migrate_workload(wx, dwx, max(5, args.steps // 2), args.warmup, peaks)
+                    extra[name] = r
+                    del wx, ox, lx
+                    dwx = None
+                    torch.cuda.empty_cache()
+                except Exception as exc:  # report, do not hide
+                    extra[name] = {"error": repr(exc)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": W.CONFIG_NAMES[idx - 1], "requests_per_gpu": w.B, "heads": w.head_end - w.head_begin,
+                       "tokens_per_gpu": w.total_tokens(), "kv_dtype": "bf16" if w.kv_dtype == 0 else "e4m3+token scale",
+                       "page_size": 64, "l2": "256 MiB flush write between steps; KV larger than L2",
+                       "parallelism": f"dp{world} (request slices, no collective)"},
+            "ms_p50": main_res["ms_p50"], "ms_p95": main_res["ms_p95"],
+            "tokens_per_s_78_layers": value / 78,
+            "roofline": main_res["roofline"],
+            "cpu_baseline": cpu,
+            "e2e": {k: (e2e_value if k == "value" else v) for k, v in e2e.items()},
+            "gpu_launches": int(main_res["launches_per_step"]) * args.steps,
+            "clocks": clocks,
+            "workloads": extra,
+            "input_generation_s": gen_s,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -190,6 +190,17 @@ SPLASH_API int splash_version(void);
 SPLASH_API int splash_last_launch_count(void);
 
 /*
+ * Per-kernel timing of splash_mla_decode, for benchmarks.  While enabled (per host
+ * thread), every decode call records CUDA events on its stream around its three
+ * kernels (plan, decode, split combine); the events are created on first use.
+ * splash_get_kernel_timing() synchronises on the last call's final event and returns
+ * the three durations in milliseconds (host pointers, each may be NULL).  Off by
+ * default; enabling it adds four event records per call and nothing else.
+ */
+SPLASH_API int splash_set_kernel_timing(int enable);
+SPLASH_API int splash_get_kernel_timing(float *plan_ms, float *decode_ms, float *combine_ms);
+
+/*
  * Read the device status word at the head of a decode workspace after the caller
  * has synchronised the stream: SPLASH_OK, or SPLASH_DEVICE_TIMEOUT if a bounded wait
  * inside a kernel gave up (the results of that call are then invalid).  Performs a

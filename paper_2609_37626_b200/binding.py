@@ -84,6 +84,10 @@ def load() -> ctypes.CDLL:
     lib.splash_last_error.restype = ctypes.c_char_p
     lib.splash_version.restype = ctypes.c_int
     lib.splash_last_launch_count.restype = ctypes.c_int
+    lib.splash_set_kernel_timing.restype = ctypes.c_int
+    lib.splash_set_kernel_timing.argtypes = [ctypes.c_int]
+    lib.splash_get_kernel_timing.restype = ctypes.c_int
+    lib.splash_get_kernel_timing.argtypes = [ctypes.POINTER(ctypes.c_float)] * 3
     lib.splash_workspace_status.restype = ctypes.c_int
     lib.splash_workspace_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
     _lib = lib
@@ -213,6 +217,17 @@ def splash_last_launch_count() -> int:
 
 def splash_version() -> int:
     return int(load().splash_version())
+
+
+def splash_set_kernel_timing(enable: bool):
+    _check(load().splash_set_kernel_timing(1 if enable else 0))
+
+
+def splash_get_kernel_timing():
+    """(plan_ms, decode_ms, combine_ms) of the last timed decode call."""
+    a, b, c = ctypes.c_float(), ctypes.c_float(), ctypes.c_float()
+    _check(load().splash_get_kernel_timing(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)))
+    return a.value, b.value, c.value
 
 
 def splash_workspace_status(workspace: torch.Tensor):

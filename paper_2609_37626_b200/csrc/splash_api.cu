@@ -11,6 +11,18 @@ namespace splash {
 namespace {
 thread_local std::string g_last_error;
 thread_local int g_launches = 0;
+thread_local bool g_timing = false;
+thread_local cudaEvent_t g_events[4] = {nullptr, nullptr, nullptr, nullptr};
+thread_local bool g_events_recorded = false;
+
+cudaError_t record_timing_event(int k, cudaStream_t stream) {
+    if (!g_timing) return cudaSuccess;
+    if (g_events[k] == nullptr) {
+        cudaError_t e = cudaEventCreate(&g_events[k]);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaEventRecord(g_events[k], stream);
+}
 
 struct DeviceInfo {
     int device = -1;
@@ -166,13 +178,19 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     p.tile_start = v.tile_start; p.req_lo = v.req_lo; p.req_hi = v.req_hi; p.worker_begin = v.worker_begin;
     p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
 
-    cudaError_t e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
-                                v.cost_start, v.worker_begin, v.status, stream);
+    cudaError_t e = record_timing_event(0, stream);
+    if (e == cudaSuccess)
+        e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
+                        v.cost_start, v.worker_begin, v.status, stream);
+    if (e == cudaSuccess) e = record_timing_event(1, stream);
     if (e == cudaSuccess) {
         if (simt) e = launch_decode_simt(p, shape->kv_dtype, stream);
         else e = launch_decode_umma(p, *shape, stream);
     }
+    if (e == cudaSuccess) e = record_timing_event(2, stream);
     if (e == cudaSuccess) e = launch_split_combine(p, v.req_wfirst, v.req_wlast, stream);
+    if (e == cudaSuccess) e = record_timing_event(3, stream);
+    if (e == cudaSuccess && g_timing) g_events_recorded = true;
     if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
     return SPLASH_OK;
 }
@@ -249,6 +267,24 @@ const char *splash_last_error(void) { return g_last_error.c_str(); }
 int splash_version(void) { return 100; }
 
 int splash_last_launch_count(void) { return g_launches; }
+
+int splash_set_kernel_timing(int enable) {
+    g_timing = enable != 0;
+    if (!g_timing) g_events_recorded = false;
+    return SPLASH_OK;
+}
+
+int splash_get_kernel_timing(float *plan_ms, float *decode_ms, float *combine_ms) {
+    if (!g_events_recorded) { set_error("no timed decode call on this thread"); return SPLASH_INVALID_ARG; }
+    cudaError_t e = cudaEventSynchronize(g_events[3]);
+    float ms[3] = {0.f, 0.f, 0.f};
+    for (int k = 0; k < 3 && e == cudaSuccess; ++k) e = cudaEventElapsedTime(&ms[k], g_events[k], g_events[k + 1]);
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    if (plan_ms) *plan_ms = ms[0];
+    if (decode_ms) *decode_ms = ms[1];
+    if (combine_ms) *combine_ms = ms[2];
+    return SPLASH_OK;
+}
 
 int splash_workspace_status(const void *workspace, int32_t *detail) {
     if (!workspace) { set_error("workspace is NULL"); return SPLASH_INVALID_ARG; }
