@@ -201,6 +201,14 @@ SPLASH_API int splash_set_kernel_timing(int enable);
 SPLASH_API int splash_get_kernel_timing(float *plan_ms, float *decode_ms, float *combine_ms);
 
 /*
+ * Diagnostics: give the decode kernel a device buffer of 64 x 8 int64 into which CTA 0
+ * writes SM-clock timestamps of its pipeline events for its first 64 tiles (event
+ * order: stage free, TMA issued, tile landed, QK^T issued, S ready, P written, P seen,
+ * P.V issued).  NULL (the default) switches it off.  Per host thread.
+ */
+SPLASH_API int splash_debug_set_trace(void *device_buffer);
+
+/*
  * Read the device status word at the head of a decode workspace after the caller
  * has synchronised the stream: SPLASH_OK, or SPLASH_DEVICE_TIMEOUT if a bounded wait
  * inside a kernel gave up (the results of that call are then invalid).  Performs a

@@ -219,6 +219,12 @@ def splash_version() -> int:
     return int(load().splash_version())
 
 
+def splash_debug_set_trace(buf: Optional[torch.Tensor]):
+    lib = load()
+    lib.splash_debug_set_trace.argtypes = [ctypes.c_void_p]
+    lib.splash_debug_set_trace(_ptr(buf))
+
+
 def splash_set_kernel_timing(enable: bool):
     _check(load().splash_set_kernel_timing(1 if enable else 0))
 

@@ -12,6 +12,7 @@ namespace {
 thread_local std::string g_last_error;
 thread_local int g_launches = 0;
 thread_local bool g_timing = false;
+thread_local long long *g_trace = nullptr;
 thread_local cudaEvent_t g_events[4] = {nullptr, nullptr, nullptr, nullptr};
 thread_local bool g_events_recorded = false;
 
@@ -156,7 +157,8 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     if (!current_device_info(dev)) return SPLASH_CUDA_ERROR;
     if (dev.cc_major != 10) { set_error("device compute capability %d.x is not 10.x", dev.cc_major); return SPLASH_UNSUPPORTED_DEVICE; }
 
-    const bool simt = (shape->flags & SPLASH_FLAG_SIMT) != 0;
+    // e4m3 KV runs on the SIMT kernel until the fp8 tensor-core path is in place
+    const bool simt = (shape->flags & SPLASH_FLAG_SIMT) != 0 || shape->kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE;
     Tiling t = choose_tiling(shape, h, dev.sm_count, simt);
     PlanView v = make_plan_view(workspace, B, t.num_workers, h);
     if (workspace_bytes < v.bytes) {
@@ -177,6 +179,7 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     p.softmax_scale = shape->softmax_scale;
     p.tile_start = v.tile_start; p.req_lo = v.req_lo; p.req_hi = v.req_hi; p.worker_begin = v.worker_begin;
     p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
+    p.trace = g_trace;
 
     cudaError_t e = record_timing_event(0, stream);
     if (e == cudaSuccess)
@@ -267,6 +270,11 @@ const char *splash_last_error(void) { return g_last_error.c_str(); }
 int splash_version(void) { return 100; }
 
 int splash_last_launch_count(void) { return g_launches; }
+
+int splash_debug_set_trace(void *device_buffer) {
+    g_trace = static_cast<long long *>(device_buffer);
+    return SPLASH_OK;
+}
 
 int splash_set_kernel_timing(int enable) {
     g_timing = enable != 0;

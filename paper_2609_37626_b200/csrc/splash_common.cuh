@@ -90,6 +90,7 @@ struct DecodeParams {
     int32_t *status;
     float *partial_lse, *partial_out;
     int32_t num_workers;
+    long long *trace;          // optional device buffer for pipeline timestamps (diagnostics), or NULL
 };
 
 // A worker's next piece of work: request, its relative tile range, where the

@@ -12,15 +12,20 @@
 // of the K rows (the latent), taken as an MN-major operand, so every KV byte crosses
 // HBM once per head group.
 //
-// Warp roles (192 threads):
+// Warp roles (288 threads):
 //   warp 0     TMA producer: block-table driven page gathers into a ring of stages
 //              (nine 64x64-element boxes per page, 128-byte swizzle), and the query
 //              rows of each segment.  Page tails and unaligned KV ranges are handled
 //              by shifting the box in the token dimension so that out-of-range tokens
 //              fall outside the page and are zero-filled by the TMA unit.
-//   warp 1     MMA issuer (one thread): QK^T of tile i+1 is issued before P.V of
-//              tile i, so the tensor pipe works while the softmax warps handle tile i.
-//   warps 2-5  online softmax over tokens (= TMEM lanes): per-head maxima by a
+//   warps 1-4  MMA issuers (one thread each).  One thread sustains only one tcgen05.mma
+//              per ~65 cycles whatever the shape, far below the pipe's rate for these
+//              small-N MMAs, so the work is spread: every issuer owns one of the
+//              independent S^T partial accumulators and one of the four dv blocks of
+//              O^T, runs its own ready-driven loop over the barriers and commits its
+//              own MMAs (the consumer barriers count one arrival per issuer).  QK^T of
+//              tile i+1 is issued while the softmax warps handle tile i.
+//   warps 5-8  online softmax over tokens (= TMEM lanes): per-head maxima by a
 //              warp-shuffle reduce-scatter plus a small shared-memory exchange, lazy
 //              rescaling of O^T (only when a maximum grows by more than 2^8), P written
 //              to shared memory as the K-major B operand, epilogue.
@@ -37,7 +42,8 @@ namespace splash {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 288;                      // 9 warps: producer, 4 MMA issuers, 4 softmax
+constexpr int kMmaWarps = 4;
 constexpr int kNumSoftmaxThreads = 128;
 constexpr int kChunks = 9;                         // 576 / 64-element (128 B) chunks
 constexpr uint32_t kSlabBytes = 64 * 128;          // one chunk of one page: 64 tokens x 128 B
@@ -78,8 +84,11 @@ struct Layout {
     static constexpr uint32_t kBytes = kOffMisc + 16;
     // tensor memory columns
     static constexpr uint32_t kColO = 0;                     // 4 blocks x N columns
-    static constexpr uint32_t kColS = 4 * N;                 // 2 buffers x N columns
-    static_assert(kColS + 2 * N <= 512, "tensor memory overflow");
+    // S^T is accumulated in kAcc independent partial sums (summed by the softmax warps): a
+    // chain of 36 small MMAs into ONE accumulator runs at the MMA latency, not its rate.
+    static constexpr int kAcc = N >= 64 ? 2 : 4;             // = number of issuers that take part in QK^T
+    static constexpr uint32_t kColS = 4 * N;                 // 2 buffers x kAcc x N columns
+    static_assert(kColS + 2 * kAcc * N <= 512, "tensor memory overflow");
     static_assert(kBytes <= 232448, "shared memory overflow");
     static_assert(kOffQ % 1024 == 0 && kOffP % 1024 == 0 && (N * 128) % 1024 == 0, "swizzle atoms need 1024-byte alignment");
 };
@@ -143,6 +152,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -272,11 +287,11 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
         return;
     }
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), 1); }
-        mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), 1);
-        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), 1); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxThreads); }
-        mbar_init(bar(kBarPFull), kNumSoftmaxThreads); mbar_init(bar(kBarPEmpty), 1);
-        mbar_init(bar(kBarOFull), 1); mbar_init(bar(kBarOEmpty), kNumSoftmaxThreads);
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kMmaWarps); }
+        mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), L::kAcc);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), L::kAcc); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxThreads); }
+        mbar_init(bar(kBarPFull), kNumSoftmaxThreads); mbar_init(bar(kBarPEmpty), kMmaWarps);
+        mbar_init(bar(kBarOFull), kMmaWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxThreads);
         misc[1] = 0; misc[2] = 0; misc[3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -292,6 +307,10 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
     SegmentIter it;
     it.init(p, worker);
     Segment seg;
+    long long *const trace = blockIdx.x == 0 ? p.trace : nullptr;
+    auto mark = [&](uint32_t tile, int ev) {
+        if (trace != nullptr && tile < 64) trace[tile * 8 + ev] = clock64();
+    };
 
     if (warp == 0) {
         // ===================================================== TMA producer
@@ -302,8 +321,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
                 if (ok) {
                     mbar_expect_tx(bar(kBarQFull), L::kQBytes);
-                    for (int c = 0; c < kChunks; ++c)
-                        tma_load_3d(sbase + L::kOffQ + c * (N * 128), &tmap_q, bar(kBarQFull), c * 64, head0, seg.request);
+                    tma_load_4d(sbase + L::kOffQ, &tmap_q, bar(kBarQFull), 0, head0, 0, seg.request);
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -320,12 +338,14 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 if (lane == 0) {
                     const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
                     ok = mbar_wait(ctx, bar(kBarKvEmpty + stage), ph ^ 1, kBarKvEmpty + stage);
+                    mark(kv_it, 0);
                     if (ok) {
                         const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
                         mbar_expect_tx(bar(kBarKvFull + stage), kStageBytes);
                         const uint32_t dst = sbase + L::kOffKv + stage * kStageBytes;
-                        for (int c = 0; c < kChunks; ++c)
-                            tma_load_3d(dst + c * kSlabBytes, &tmap_kv, bar(kBarKvFull + stage), c * 64, g.tok0, page);
+                        // one box = the whole page: (64 elements, 64 tokens, 9 chunks) -> [chunk][token][128 B]
+                        tma_load_4d(dst, &tmap_kv, bar(kBarKvFull + stage), 0, g.tok0, 0, page);
+                        mark(kv_it, 1);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -333,79 +353,103 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             }
             ++seg_it;
         }
-    } else if (warp == 1) {
-        // ===================================================== MMA issuer
+    } else if (warp <= kMmaWarps) {
+        // ===================================================== MMA issuers
         if (lane == 0) {
+            const int mw = warp - 1;                 // issuer index: S^T accumulator mw, dv block mw
+            const bool does_qk = mw < L::kAcc;
             constexpr uint32_t kIdescQK = make_idesc(64, N, 0, 0);
             constexpr uint32_t kIdescPV = make_idesc(128, N, 1, 0);
             uint32_t kv_it = 0, s_it = 0, p_it = 0, seg_it = 0;
             bool ok = true;
-            // S^T of the tile with global index kv: 36 MMAs of K = 16
-            auto issue_qk = [&](uint32_t kv, uint32_t sidx) -> bool {
-                const uint32_t stage = kv % kStages, ph = (kv / kStages) & 1, b = sidx & 1;
-                if (!mbar_wait(ctx, bar(kBarKvFull + stage), ph, kBarKvFull + stage)) return false;
-                if (!mbar_wait(ctx, bar(kBarSEmpty + b), ((sidx >> 1) & 1) ^ 1, kBarSEmpty + b)) return false;
+            // This issuer's share of S^T for the tile with global index kv: the K = 16 steps
+            // idx = mw, mw + kAcc, ... of the 36, into partial accumulator mw.
+            auto issue_qk = [&](uint32_t kv, uint32_t sidx) {
+                const uint32_t stage = kv % kStages, b = sidx & 1;
+                if (mw == 0) mark(kv, 2);
                 tcgen05_fence_after();
                 const uint32_t a0 = sbase + L::kOffKv + stage * kStageBytes;
                 const uint32_t b0 = sbase + L::kOffQ;
-                const uint32_t d = tmem_base + L::kColS + b * N;
+                const uint32_t d = tmem_base + L::kColS + (b * L::kAcc + mw) * N;
 #pragma unroll
-                for (int c = 0; c < kChunks; ++c) {
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        uint64_t da = make_desc(a0 + c * kSlabBytes + k * 32, 16, 1024);
-                        uint64_t db = make_desc(b0 + c * (N * 128) + k * 32, 16, 1024);
-                        umma_bf16(d, da, db, kIdescQK, (c | k) != 0);
-                    }
+                for (int t = 0; t < 36 / L::kAcc; ++t) {
+                    const int idx = t * L::kAcc + mw, c = idx >> 2, k = idx & 3;
+                    uint64_t da = make_desc(a0 + c * kSlabBytes + k * 32, 16, 1024);
+                    uint64_t db = make_desc(b0 + c * (N * 128) + k * 32, 16, 1024);
+                    umma_bf16(d, da, db, kIdescQK, t != 0);
                 }
                 umma_commit(bar(kBarSFull + b));
-                return true;
+                if (mw == 0) mark(kv, 3);
+            };
+            // O^T block mw += V^T block mw (128 dv x 64 tokens) * P^T, four K = 16 steps.
+            auto issue_pv = [&](uint32_t stage, bool first_tile) {
+                tcgen05_fence_after();
+                const uint32_t v0 = sbase + L::kOffKv + stage * kStageBytes + (2 * mw) * kSlabBytes;
+                const uint32_t p0 = sbase + L::kOffP;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    // A: two 64-element chunks (LBO apart) x 16 tokens (SBO per 8 tokens), MN-major
+                    uint64_t da = make_desc(v0 + k * 2048, kSlabBytes, 1024);
+                    uint64_t db = make_desc(p0 + k * 32, 16, 1024);
+                    umma_bf16(tmem_base + L::kColO + mw * N, da, db, kIdescPV, (!first_tile) || k != 0);
+                }
             };
             while (ok && it.next(p, seg)) {
                 const int ntiles = seg.tile_end - seg.tile_begin;
-                ok = mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
-                if (!ok) break;
-                ok = issue_qk(kv_it, s_it);
-                if (ok && ntiles == 1) umma_commit(bar(kBarQEmpty));
-                for (int i = 0; ok && i < ntiles; ++i) {
-                    if (i + 1 < ntiles) {
-                        ok = issue_qk(kv_it + i + 1, s_it + i + 1);
-                        if (!ok) break;
-                        if (i + 2 == ntiles) umma_commit(bar(kBarQEmpty));
-                    }
-                    ok = mbar_wait(ctx, bar(kBarPFull), p_it & 1, kBarPFull);
+                if (does_qk) {
+                    ok = mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
                     if (!ok) break;
-                    if (i == 0) {
-                        ok = mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty);
-                        if (!ok) break;
+                }
+                // Issue whatever is ready: P.V of tile pv_i (frees a stage) or QK^T of tile qk_i
+                // (at most one tile ahead of the softmax: two S buffers).
+                int qk_i = does_qk ? 0 : ntiles, pv_i = 0;
+                unsigned long long idle_since = 0;
+                while (pv_i < ntiles) {
+                    bool progressed = false;
+                    if ((qk_i > pv_i) && mbar_try_wait(bar(kBarPFull), (p_it + pv_i) & 1)) {
+                        if (pv_i == 0 && !mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty)) { ok = false; break; }
+                        if (mw == 0) mark(kv_it + pv_i, 6);
+                        const uint32_t stage = (kv_it + pv_i) % kStages;
+                        issue_pv(stage, pv_i == 0);
+                        umma_commit(bar(kBarKvEmpty + stage));
+                        umma_commit(bar(kBarPEmpty));
+                        if (pv_i + 1 == ntiles) umma_commit(bar(kBarOFull));
+                        if (mw == 0) mark(kv_it + pv_i, 7);
+                        ++pv_i;
+                        progressed = true;
                     }
-                    tcgen05_fence_after();
-                    const uint32_t stage = (kv_it + i) % kStages;
-                    const uint32_t v0 = sbase + L::kOffKv + stage * kStageBytes;
-                    const uint32_t p0 = sbase + L::kOffP;
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            // A = V^T block j: 128 dv (two 64-element chunks, LBO apart) x 16 tokens (SBO per 8)
-                            uint64_t da = make_desc(v0 + (2 * j) * kSlabBytes + k * 2048, kSlabBytes, 1024);
-                            uint64_t db = make_desc(p0 + k * 32, 16, 1024);
-                            umma_bf16(tmem_base + L::kColO + j * N, da, db, kIdescPV, (i | k) != 0);
+                    if (does_qk && qk_i < ntiles && qk_i < pv_i + 2) {
+                        const uint32_t kv = kv_it + qk_i, sidx = s_it + qk_i;
+                        if (mbar_try_wait(bar(kBarKvFull + kv % kStages), (kv / kStages) & 1) &&
+                            mbar_try_wait(bar(kBarSEmpty + (sidx & 1)), ((sidx >> 1) & 1) ^ 1)) {
+                            issue_qk(kv, sidx);
+                            ++qk_i;
+                            if (qk_i == ntiles) umma_commit(bar(kBarQEmpty));
+                            progressed = true;
                         }
                     }
-                    umma_commit(bar(kBarKvEmpty + stage));
-                    umma_commit(bar(kBarPEmpty));
-                    if (i + 1 == ntiles) umma_commit(bar(kBarOFull));
-                    ++p_it;
+                    if (progressed) { idle_since = 0; continue; }
+                    if (*ctx.abort_flag) { ok = false; break; }
+                    const unsigned long long now = global_timer_ns();
+                    if (idle_since == 0) idle_since = now;
+                    else if (now - idle_since > kWaitLimitNs) {
+                        *ctx.abort_flag = 1;
+                        if (atomicCAS(ctx.status, 0, (int)SPLASH_DEVICE_TIMEOUT) == 0) {
+                            ctx.status[1] = (int)blockIdx.x; ctx.status[2] = 100 + (qk_i > pv_i ? kBarPFull : kBarKvFull);
+                            ctx.status[3] = pv_i;
+                        }
+                        ok = false; break;
+                    }
                 }
-                kv_it += ntiles; s_it += ntiles;
+                kv_it += ntiles; s_it += ntiles; p_it += ntiles;
                 ++seg_it;
             }
         }
     } else {
         // ===================================================== softmax + epilogue warps
         const int q4 = warp & 3;                       // TMEM lane quadrant of this warp
-        const int st = (warp - 2) * 32 + lane;         // 0..127
+        const int sw = warp - 1 - kMmaWarps;           // softmax warp 0..3
+        const int st = sw * 32 + lane;                 // 0..127
         const int row = 16 * q4 + lane;                // token row of the S^T tile (lanes < 16)
         const uint32_t lane_addr = (uint32_t)(32 * q4) << 16;
         float *red = reinterpret_cast<float *>(smem + L::kOffRed);
@@ -418,9 +462,9 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
         bool ok = true;
         while (ok && it.next(p, seg)) {
             if (st < N) m_s[st] = -INFINITY;
-            float l_local[N];
+            float l_own[kOwn];            // running sums of the heads this lane owns (this warp's 16 tokens)
 #pragma unroll
-            for (int n = 0; n < N; ++n) l_local[n] = 0.f;
+            for (int k = 0; k < kOwn; ++k) l_own[k] = 0.f;
             softmax_bar_sync();
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;
@@ -430,11 +474,25 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 const uint32_t b = s_it & 1;
                 ok = mbar_wait(ctx, bar(kBarSFull + b), (s_it >> 1) & 1, kBarSFull + b);
                 if (!ok) break;
+                if (st == 0) mark(s_it, 4);
                 tcgen05_fence_after();
                 float s[N];
+                {
+                    const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (L::kAcc * N);
 #pragma unroll
-                for (int c = 0; c < N / 16; ++c)
-                    tmem_ld16(tmem_base + lane_addr + L::kColS + b * N + c * 16, *reinterpret_cast<float(*)[16]>(&s[c * 16]));
+                    for (int c = 0; c < N / 16; ++c)
+                        tmem_ld16(sb + c * 16, *reinterpret_cast<float(*)[16]>(&s[c * 16]));
+#pragma unroll
+                    for (int a = 1; a < L::kAcc; ++a) {
+                        float part[N];
+#pragma unroll
+                        for (int c = 0; c < N / 16; ++c)
+                            tmem_ld16(sb + a * N + c * 16, *reinterpret_cast<float(*)[16]>(&part[c * 16]));
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int n = 0; n < N; ++n) s[n] += part[n];
+                    }
+                }
                 tmem_wait_ld();
                 tcgen05_fence_before();
                 mbar_arrive(bar(kBarSEmpty + b));
@@ -444,7 +502,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 ReduceScatter<N, 16, true>::run(mx, lane);
                 if (N >= 32 || (lane & 1) == 0) {
 #pragma unroll
-                    for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + (warp - 2)] = mx[k];
+                    for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + sw] = mx[k];
                 }
                 if (st == 0) misc[2 + (i & 1)] = 0;      // this tile's "some maximum grew" flag
                 softmax_bar_sync();
@@ -464,13 +522,13 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 const bool rescale = misc[2 + (i & 1)] != 0;
                 if (rescale) {
 #pragma unroll
-                    for (int n = 0; n < N; ++n) l_local[n] *= alpha_s[n];
+                    for (int k = 0; k < kOwn; ++k) l_own[k] *= alpha_s[owned_head<N>(lane, k)];
                 }
 #pragma unroll
-                for (int n = 0; n < N; ++n) {
-                    s[n] = fast_exp2(s[n] - m_s[n]);
-                    l_local[n] += s[n];
-                }
+                for (int n = 0; n < N; ++n) { s[n] = fast_exp2(s[n] - m_s[n]); mx[n] = s[n]; }
+                ReduceScatter<N, 16, false>::run(mx, lane);      // per-head sums over this warp's tokens
+#pragma unroll
+                for (int k = 0; k < kOwn; ++k) l_own[k] += mx[k];
                 // P.V of the previous tile must be done with the P buffer and with O^T
                 ok = mbar_wait(ctx, bar(kBarPEmpty), (p_it & 1) ^ 1, kBarPEmpty);
                 if (!ok) break;
@@ -500,15 +558,15 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 }
                 fence_proxy_async();
                 tcgen05_fence_before();
+                if (st == 0) mark(s_it, 5);
                 mbar_arrive(bar(kBarPFull));
                 ++s_it; ++p_it;
             }
             if (!ok) break;
             // ---- row sums over all 128 lanes' partial sums
-            ReduceScatter<N, 16, false>::run(l_local, lane);
             if (N >= 32 || (lane & 1) == 0) {
 #pragma unroll
-                for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + (warp - 2)] = l_local[k];
+                for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + sw] = l_own[k];
             }
             softmax_bar_sync();
             if (st < N) {
@@ -589,15 +647,18 @@ EncodeTiledFn encode_tiled() {
     return fn;
 }
 
-bool make_map_3d(CUtensorMap *map, const void *base, uint64_t d0, uint64_t d1, uint64_t d2, uint64_t stride1_bytes,
-                 uint64_t stride2_bytes, uint32_t box0, uint32_t box1) {
+// 4-D map (64 elements, rows, 9 chunks, outer): a 576-wide row is seen as 9 chunks of
+// 64 elements, so one box of (64, box_rows, 9, 1) lands in shared memory as
+// [chunk][row][128 B], each chunk slab in the 128-byte swizzle the MMA descriptors expect.
+bool make_map_4d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t outer, uint64_t row_stride_bytes,
+                 uint64_t outer_stride_bytes, uint32_t box_rows) {
     EncodeTiledFn fn = encode_tiled();
     if (!fn) { set_error("cuTensorMapEncodeTiled is not available"); return false; }
-    cuuint64_t dims[3] = {d0, d1, d2};
-    cuuint64_t strides[2] = {stride1_bytes, stride2_bytes};
-    cuuint32_t box[3] = {box0, box1, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+    cuuint64_t dims[4] = {64, rows, kChunks, outer};
+    cuuint64_t strides[3] = {row_stride_bytes, 128, outer_stride_bytes};
+    cuuint32_t box[4] = {64, box_rows, kChunks, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r); return false; }
@@ -629,11 +690,11 @@ cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &sh
     if (shape.kv_dtype != SPLASH_KV_BF16) return cudaErrorNotSupported;
     alignas(64) CUtensorMap mkv, mq;
     const int n = p.heads_per_group;
-    if (!make_map_3d(&mkv, p.kv_pool, kDQK, kPage, (uint64_t)(p.num_pool_pages > 0 ? p.num_pool_pages : 1),
-                     (uint64_t)kDQK * 2, (uint64_t)kPage * kDQK * 2, 64, 64))
+    if (!make_map_4d(&mkv, p.kv_pool, kPage, (uint64_t)(p.num_pool_pages > 0 ? p.num_pool_pages : 1),
+                     (uint64_t)kDQK * 2, (uint64_t)kPage * kDQK * 2, 64))
         return cudaErrorInvalidValue;
-    if (!make_map_3d(&mq, p.q, kDQK, (uint64_t)p.H, (uint64_t)p.B, (uint64_t)p.q_stride_head * 2,
-                     (uint64_t)(p.B > 1 ? p.q_stride_request : p.q_stride_head * p.H) * 2, 64, (uint32_t)n))
+    if (!make_map_4d(&mq, p.q, (uint64_t)p.H, (uint64_t)p.B, (uint64_t)p.q_stride_head * 2,
+                     (uint64_t)(p.B > 1 ? p.q_stride_request : p.q_stride_head * p.H) * 2, (uint32_t)n))
         return cudaErrorInvalidValue;
     switch (n) {
         case 16: return launch_n<16>(p, mkv, mq, stream);
