@@ -181,6 +181,42 @@ SPLASH_API int splash_kv_page_migrate(const void *src_pool, const float *src_sca
 
 SPLASH_API size_t splash_kv_page_migrate_workspace_bytes(int32_t max_page_id);
 
+/*
+ * splash_kv_page_migrate without a workspace argument and without any allocation.
+ * (The paper has no counterpart for this entry point; it exists for the library's
+ * callers.)
+ *
+ * Who needs it: code that moves pages from a place where it may not allocate or
+ * free device memory -- a serving loop that has already handed the whole HBM budget to
+ * its KV pool and keeps no allocator of its own, a plugin or callback that runs under
+ * a host framework's memory manager and must not call cudaMalloc behind its back, a
+ * latency-critical path where an allocation (which can synchronise the device) is
+ * not acceptable.  Such a caller has nowhere to get the remap table that
+ * splash_kv_page_migrate wants as `workspace`.
+ *
+ * Here the table is a fixed array inside the library's own device image:
+ * SPLASH_STATIC_MIGRATE_MAX_PAGE_ID (262,144) int32 entries = 1 MiB, present on every
+ * GPU that loads the library for as long as the process lives.  Arguments, results and
+ * error codes are those of splash_kv_page_migrate; in addition max_page_id above the
+ * limit is rejected with SPLASH_INVALID_ARG and nothing is launched.  The function
+ * calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   - The first call on each device looks up the array's device address (a host-side
+ *     query, no allocation); make that first call outside any stream capture.
+ *   - All calls on a device share the one table, and it keeps the previous call's
+ *     contents: each call first resets the entries [0, max_page_id) on `stream`.  Two
+ *     calls that can overlap on the GPU (different streams, no ordering between them)
+ *     race on it -- order them, or give one of them its own workspace through
+ *     splash_kv_page_migrate.
+ */
+#define SPLASH_STATIC_MIGRATE_MAX_PAGE_ID (1 << 18)
+SPLASH_API int splash_kv_page_migrate_static(const void *src_pool, const float *src_scales,
+                                             void *dst_pool, float *dst_scales,
+                                             int64_t page_bytes,
+                                             const int32_t *src_page_ids, const int32_t *dst_page_ids, int64_t n,
+                                             int32_t src_id_base, int32_t dst_id_base, int32_t max_page_id,
+                                             int32_t *block_table, int64_t num_table_entries, void *stream);
+
 /* Host-side helpers. */
 SPLASH_API const char *splash_status_string(int status);
 SPLASH_API const char *splash_last_error(void);

@@ -77,6 +77,8 @@ def load() -> ctypes.CDLL:
     lib.splash_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp]
     lib.splash_kv_page_migrate.restype = ctypes.c_int
     lib.splash_kv_page_migrate.argtypes = [vp, vp, vp, vp, i64, vp, vp, i64, i32, i32, i32, vp, i64, vp, sz, vp]
+    lib.splash_kv_page_migrate_static.restype = ctypes.c_int
+    lib.splash_kv_page_migrate_static.argtypes = [vp, vp, vp, vp, i64, vp, vp, i64, i32, i32, i32, vp, i64, vp]
     lib.splash_kv_page_migrate_workspace_bytes.restype = sz
     lib.splash_kv_page_migrate_workspace_bytes.argtypes = [i32]
     lib.splash_status_string.restype = ctypes.c_char_p
@@ -209,6 +211,28 @@ def splash_kv_page_migrate(src_pool: torch.Tensor, dst_pool: torch.Tensor, src_p
                                       _ptr(src_page_ids), _ptr(dst_page_ids), n, src_id_base, dst_id_base,
                                       max_page_id, _ptr(block_table), block_table.numel(), _ptr(workspace),
                                       workspace.numel(), _stream_ptr(stream)))
+
+
+def splash_kv_page_migrate_static(src_pool: torch.Tensor, dst_pool: torch.Tensor, src_page_ids: torch.Tensor,
+                                  dst_page_ids: torch.Tensor, block_table: torch.Tensor, *,
+                                  src_scales: Optional[torch.Tensor] = None,
+                                  dst_scales: Optional[torch.Tensor] = None, src_id_base: int = 0,
+                                  dst_id_base: int = 0, max_page_id: Optional[int] = None,
+                                  stream: Optional[torch.cuda.Stream] = None):
+    """Page migration for callers that cannot allocate device memory: same effect as
+    splash_kv_page_migrate, but the remap table is the library's built-in 1 MiB device
+    array, so this wrapper passes no workspace and creates no tensor.  Page ids must stay
+    below 262,144; calls that could overlap on the GPU must be ordered by the caller."""
+    lib = load()
+    assert src_pool.is_contiguous() and dst_pool.is_contiguous() and block_table.is_contiguous()
+    assert src_page_ids.dtype == torch.int32 and dst_page_ids.dtype == torch.int32
+    page_bytes = src_pool.shape[1] * src_pool.shape[2] * src_pool.element_size()
+    if max_page_id is None:
+        max_page_id = max(src_id_base + src_pool.shape[0], dst_id_base + dst_pool.shape[0])
+    _check(lib.splash_kv_page_migrate_static(_ptr(src_pool), _ptr(src_scales), _ptr(dst_pool), _ptr(dst_scales),
+                                             page_bytes, _ptr(src_page_ids), _ptr(dst_page_ids),
+                                             src_page_ids.numel(), src_id_base, dst_id_base, max_page_id,
+                                             _ptr(block_table), block_table.numel(), _stream_ptr(stream)))
 
 
 def splash_last_launch_count() -> int:

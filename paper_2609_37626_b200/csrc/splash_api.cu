@@ -253,6 +253,37 @@ int splash_kv_page_migrate(const void *src_pool, const float *src_scales, void *
     return SPLASH_OK;
 }
 
+int splash_kv_page_migrate_static(const void *src_pool, const float *src_scales, void *dst_pool, float *dst_scales,
+                                  int64_t page_bytes, const int32_t *src_page_ids, const int32_t *dst_page_ids,
+                                  int64_t n, int32_t src_id_base, int32_t dst_id_base, int32_t max_page_id,
+                                  int32_t *block_table, int64_t num_table_entries, void *stream_) {
+    g_launches = 0;
+    if (max_page_id > kStaticMigrateMaxPageId) {
+        set_error("max_page_id %d exceeds the built-in remap table of %d entries; use splash_kv_page_migrate "
+                  "with a caller-provided workspace", max_page_id, kStaticMigrateMaxPageId);
+        return SPLASH_INVALID_ARG;
+    }
+    if (n < 0 || num_table_entries < 0 || page_bytes <= 0 || page_bytes % 16 || max_page_id < 0) {
+        set_error("bad sizes (page_bytes must be a positive multiple of 16)"); return SPLASH_INVALID_ARG;
+    }
+    if (n == 0) return SPLASH_OK;
+    if (!src_pool || !dst_pool || !src_page_ids || !dst_page_ids) { set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG; }
+    if ((src_scales == nullptr) != (dst_scales == nullptr)) { set_error("give both scale pools or neither"); return SPLASH_INVALID_ARG; }
+    if (num_table_entries > 0 && !block_table) { set_error("block_table is NULL"); return SPLASH_INVALID_ARG; }
+    if (!aligned(src_pool, 16) || !aligned(dst_pool, 16) || !aligned(src_scales, 16) || !aligned(dst_scales, 16)) {
+        set_error("misaligned pointer (pools, scales: 16 B)"); return SPLASH_INVALID_ARG;
+    }
+    if (n > 0x7fffffffLL) { set_error("too many pages"); return SPLASH_INVALID_ARG; }
+    int32_t *remap = nullptr;
+    cudaError_t e = static_remap_address(&remap);      // first call on a device looks the symbol up
+    if (e != cudaSuccess) { set_error("cudaGetSymbolAddress failed: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    e = launch_page_migrate(src_pool, src_scales, dst_pool, dst_scales, page_bytes, src_page_ids, dst_page_ids, n,
+                            src_id_base, dst_id_base, max_page_id, block_table, num_table_entries, remap,
+                            static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    return SPLASH_OK;
+}
+
 const char *splash_status_string(int status) {
     switch (status) {
         case SPLASH_OK: return "ok";

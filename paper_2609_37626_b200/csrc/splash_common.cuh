@@ -15,6 +15,8 @@ constexpr int kDV = 512;         // d_c (value width)
 constexpr int kDRope = 64;
 constexpr int kPage = 64;        // tokens per page
 constexpr int kMaxHeads = 128;
+// largest page id (exclusive) the allocation-free migrate entry point can remap: 1 MiB of table
+constexpr int kStaticMigrateMaxPageId = 1 << 18;
 
 // Cost, in page tiles, charged once per non-empty request when the plan balances
 // work over CTAs (query load + epilogue).
@@ -157,5 +159,7 @@ cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, v
                                 const int32_t *dst_ids, int64_t n, int32_t src_base, int32_t dst_base,
                                 int32_t max_page_id, int32_t *block_table, int64_t num_entries,
                                 int32_t *remap, cudaStream_t stream);
+
+cudaError_t static_remap_address(int32_t **ptr);
 
 }  // namespace splash

@@ -63,7 +63,30 @@ page_copy_kernel(const uint4 *__restrict__ src_pool, uint4 *__restrict__ dst_poo
         dst_scales[d * (kPage * 4 / 16) + threadIdx.x] = __ldg(src_scales + s * (kPage * 4 / 16) + threadIdx.x);
 }
 
+// Remap table of the allocation-free entry point: lives in the library's device image,
+// one copy on every GPU that loads it, until the process exits.
+static __device__ __align__(256) int32_t g_static_remap[kStaticMigrateMaxPageId];
+
 }  // namespace
+
+// Device address of g_static_remap on the current device.  In host code the array's
+// name only stands for the symbol; the address a kernel can use comes from
+// cudaGetSymbolAddress, looked up once per device with that device current.
+cudaError_t static_remap_address(int32_t **ptr) {
+    static int32_t *cache[64] = {nullptr};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (cache[dev] == nullptr) {
+        void *addr = nullptr;
+        e = cudaGetSymbolAddress(&addr, g_static_remap);
+        if (e != cudaSuccess) return e;
+        cache[dev] = static_cast<int32_t *>(addr);
+    }
+    *ptr = cache[dev];
+    return cudaSuccess;
+}
 
 cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, void *dst_pool,
                                 float *dst_scales, int64_t page_bytes, const int32_t *src_ids,
