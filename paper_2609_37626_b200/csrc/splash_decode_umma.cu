@@ -86,6 +86,10 @@ struct Layout {
     static constexpr uint32_t kColO = 0;                     // 4 blocks x N columns
     // S^T is accumulated in kAcc independent partial sums (summed by the softmax warps): a
     // chain of 36 small MMAs into ONE accumulator runs at the MMA latency, not its rate.
+    // 64-head groups compute S = Q K^T with the heads on the MMA's M (a softmax row lives in
+    // one thread: no shuffles, no exchange); narrower groups compute S^T with the tokens on M
+    // so that a 16- or 32-head slice is not padded to 64 rows.
+    static constexpr bool kHeadsOnM = N == 64;
     static constexpr int kAcc = N >= 64 ? 2 : 4;             // = number of issuers that take part in QK^T
     static constexpr uint32_t kColS = 4 * N;                 // 2 buffers x kAcc x N columns
     static_assert(kColS + 2 * kAcc * N <= 512, "tensor memory overflow");
@@ -195,10 +199,46 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) 
           "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
           "r"(__float_as_uint(v[15])) : "memory");
 }
+// 16 TMEM lanes x 64 fp32 columns in the MMA accumulator fragment layout: thread T of the
+// warp gets, for k = 0..7, v[4k+0..1] = (lane T/4,     columns 8k + 2(T%4), +1) and
+//                          v[4k+2..3] = (lane T/4 + 8, the same two columns).
+__device__ __forceinline__ void tmem_ld_16x256b_x8(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// bar.sync among the 128 softmax threads that also ORs a predicate over them
+__device__ __forceinline__ bool softmax_bar_or(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"(pred ? 1u : 0u) : "memory");
+    return out != 0;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -358,7 +398,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
         if (lane == 0) {
             const int mw = warp - 1;                 // issuer index: S^T accumulator mw, dv block mw
             const bool does_qk = mw < L::kAcc;
-            constexpr uint32_t kIdescQK = make_idesc(64, N, 0, 0);
+            constexpr uint32_t kIdescQK = L::kHeadsOnM ? make_idesc(64, 64, 0, 0) : make_idesc(64, N, 0, 0);
             constexpr uint32_t kIdescPV = make_idesc(128, N, 1, 0);
             uint32_t kv_it = 0, s_it = 0, p_it = 0, seg_it = 0;
             bool ok = true;
@@ -374,9 +414,10 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
 #pragma unroll
                 for (int t = 0; t < 36 / L::kAcc; ++t) {
                     const int idx = t * L::kAcc + mw, c = idx >> 2, k = idx & 3;
-                    uint64_t da = make_desc(a0 + c * kSlabBytes + k * 32, 16, 1024);
-                    uint64_t db = make_desc(b0 + c * (N * 128) + k * 32, 16, 1024);
-                    umma_bf16(d, da, db, kIdescQK, t != 0);
+                    uint64_t dk = make_desc(a0 + c * kSlabBytes + k * 32, 16, 1024);      // K tile rows = tokens
+                    uint64_t dq = make_desc(b0 + c * (N * 128) + k * 32, 16, 1024);       // Q rows = heads
+                    if constexpr (L::kHeadsOnM) umma_bf16(d, dq, dk, kIdescQK, t != 0);   // S  [heads x tokens]
+                    else umma_bf16(d, dk, dq, kIdescQK, t != 0);                          // S^T [tokens x heads]
                 }
                 umma_commit(bar(kBarSFull + b));
                 if (mw == 0) mark(kv, 3);
@@ -462,6 +503,9 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
         bool ok = true;
         while (ok && it.next(p, seg)) {
             if (st < N) m_s[st] = -INFINITY;
+            // heads-on-M: this thread's two heads (reference maxima; partial row sums over its tokens)
+            const int hA = 16 * q4 + (lane >> 2);
+            float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;
             float l_own[kOwn];            // running sums of the heads this lane owns (this warp's 16 tokens)
 #pragma unroll
             for (int k = 0; k < kOwn; ++k) l_own[k] = 0.f;
@@ -476,6 +520,86 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 if (!ok) break;
                 if (st == 0) mark(s_it, 4);
                 tcgen05_fence_after();
+                if constexpr (L::kHeadsOnM) {
+                // ---- heads on M.  S [64 heads x 64 tokens] sits in 16 lanes per TMEM quadrant; the
+                // fragment load spreads those over all 32 threads: this thread holds heads
+                // hA = 16 q4 + lane/4 and hB = hA + 8, tokens 8k + 2(lane%4) + {0,1}, k = 0..7.
+                float s[32];
+                {
+                    const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (L::kAcc * N);
+                    tmem_ld_16x256b_x8(sb, s);
+#pragma unroll
+                    for (int a = 1; a < L::kAcc; ++a) {
+                        float part[32];
+                        tmem_ld_16x256b_x8(sb + a * N, part);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int n = 0; n < 32; ++n) s[n] += part[n];
+                    }
+                }
+                tmem_wait_ld();
+                tcgen05_fence_before();
+                mbar_arrive(bar(kBarSEmpty + b));
+                const int tq = lane & 3;
+                float mtA = -INFINITY, mtB = -INFINITY;
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int t = 8 * k + 2 * tq + e;
+                        const bool v = t >= g.r_lo && t < g.r_hi;
+                        s[4 * k + e] = v ? s[4 * k + e] * scale_log2 : -INFINITY;
+                        s[4 * k + 2 + e] = v ? s[4 * k + 2 + e] * scale_log2 : -INFINITY;
+                        mtA = fmaxf(mtA, s[4 * k + e]);
+                        mtB = fmaxf(mtB, s[4 * k + 2 + e]);
+                    }
+                }
+                mtA = fmaxf(mtA, __shfl_xor_sync(0xffffffffu, mtA, 1)); mtB = fmaxf(mtB, __shfl_xor_sync(0xffffffffu, mtB, 1));
+                mtA = fmaxf(mtA, __shfl_xor_sync(0xffffffffu, mtA, 2)); mtB = fmaxf(mtB, __shfl_xor_sync(0xffffffffu, mtB, 2));
+                // the four threads of a head take the same decision from the same numbers
+                bool grew = false;
+                float alA = 1.f, alB = 1.f;
+                if (mtA > mA + kRescaleThreshold) { alA = (mA == -INFINITY) ? 0.f : fast_exp2(mA - mtA); mA = mtA; lA *= alA; grew = true; }
+                if (mtB > mB + kRescaleThreshold) { alB = (mB == -INFINITY) ? 0.f : fast_exp2(mB - mtB); mB = mtB; lB *= alB; grew = true; }
+                if (tq == 0) { alpha_s[hA] = alA; alpha_s[hA + 8] = alB; }
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        s[4 * k + e] = fast_exp2(s[4 * k + e] - mA); lA += s[4 * k + e];
+                        s[4 * k + 2 + e] = fast_exp2(s[4 * k + 2 + e] - mB); lB += s[4 * k + 2 + e];
+                    }
+                }
+                const bool rescale = softmax_bar_or(grew);
+                // P.V of the previous tile must be done with the P buffer and with O^T
+                ok = mbar_wait(ctx, bar(kBarPEmpty), (p_it & 1) ^ 1, kBarPEmpty);
+                if (!ok) break;
+                tcgen05_fence_after();
+                if (rescale && i > 0) {
+#pragma unroll 1
+                    for (int c = 0; c < 4 * N / 16; ++c) {
+                        float o[16];
+                        const uint32_t addr = tmem_base + lane_addr + L::kColO + c * 16;
+                        tmem_ld16(addr, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) o[k] *= alpha_s[(c * 16 + k) % N];
+                        tmem_st16(addr, o);
+                    }
+                    tmem_wait_st();
+                }
+                {
+                    // P as the K-major, 128-byte-swizzled B operand of P.V: row = head, chunk k = tokens 8k..8k+7
+                    uint8_t *pA = smem + L::kOffP + hA * 128 + tq * 4;
+                    uint8_t *pB = pA + 8 * 128;                       // head hA + 8: same (h & 7)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint32_t off = (uint32_t)(k ^ (hA & 7)) << 4;
+                        *reinterpret_cast<uint32_t *>(pA + off) = pack_bf16x2(s[4 * k + 0], s[4 * k + 1]);
+                        *reinterpret_cast<uint32_t *>(pB + off) = pack_bf16x2(s[4 * k + 2], s[4 * k + 3]);
+                    }
+                }
+                } else {
                 float s[N];
                 {
                     const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (L::kAcc * N);
@@ -556,6 +680,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                         *reinterpret_cast<__nv_bfloat16 *>(pb + n * 128 + ((chunk ^ (uint32_t)(n & 7)) << 4) + within) = v;
                     }
                 }
+                }
                 fence_proxy_async();
                 tcgen05_fence_before();
                 if (st == 0) mark(s_it, 5);
@@ -563,21 +688,40 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 ++s_it; ++p_it;
             }
             if (!ok) break;
-            // ---- row sums over all 128 lanes' partial sums
-            if (N >= 32 || (lane & 1) == 0) {
+            if constexpr (L::kHeadsOnM) {
+                lA += __shfl_xor_sync(0xffffffffu, lA, 1); lB += __shfl_xor_sync(0xffffffffu, lB, 1);
+                lA += __shfl_xor_sync(0xffffffffu, lA, 2); lB += __shfl_xor_sync(0xffffffffu, lB, 2);
+                if ((lane & 3) == 0) {
 #pragma unroll
-                for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + sw] = l_own[k];
-            }
-            softmax_bar_sync();
-            if (st < N) {
-                float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
-                float l = (r4.x + r4.y) + (r4.z + r4.w);
-                l_s[st] = 1.f / l;
-                const int gh = head0 + st;
-                if (gh < p.head_end) {
-                    float lse = (m_s[st] + log2f(l)) * kLn2;
-                    if (seg.slot < 0) p.lse[(int64_t)seg.request * p.lse_stride_request + gh] = lse;
-                    else p.partial_lse[(int64_t)seg.slot * h + (gh - p.head_begin)] = lse;
+                    for (int e = 0; e < 2; ++e) {
+                        const int hh = hA + 8 * e;
+                        const float l = e ? lB : lA, m = e ? mB : mA;
+                        l_s[hh] = 1.f / l;
+                        const int gh = head0 + hh;
+                        if (gh < p.head_end) {
+                            float lse = (m + log2f(l)) * kLn2;
+                            if (seg.slot < 0) p.lse[(int64_t)seg.request * p.lse_stride_request + gh] = lse;
+                            else p.partial_lse[(int64_t)seg.slot * h + (gh - p.head_begin)] = lse;
+                        }
+                    }
+                }
+            } else {
+                // ---- row sums over all 128 lanes' partial sums
+                if (N >= 32 || (lane & 1) == 0) {
+#pragma unroll
+                    for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + sw] = l_own[k];
+                }
+                softmax_bar_sync();
+                if (st < N) {
+                    float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
+                    float l = (r4.x + r4.y) + (r4.z + r4.w);
+                    l_s[st] = 1.f / l;
+                    const int gh = head0 + st;
+                    if (gh < p.head_end) {
+                        float lse = (m_s[st] + log2f(l)) * kLn2;
+                        if (seg.slot < 0) p.lse[(int64_t)seg.request * p.lse_stride_request + gh] = lse;
+                        else p.partial_lse[(int64_t)seg.slot * h + (gh - p.head_begin)] = lse;
+                    }
                 }
             }
             softmax_bar_sync();
