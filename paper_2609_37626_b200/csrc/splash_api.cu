@@ -157,8 +157,7 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     if (!current_device_info(dev)) return SPLASH_CUDA_ERROR;
     if (dev.cc_major != 10) { set_error("device compute capability %d.x is not 10.x", dev.cc_major); return SPLASH_UNSUPPORTED_DEVICE; }
 
-    // e4m3 KV runs on the SIMT kernel until the fp8 tensor-core path is in place
-    const bool simt = (shape->flags & SPLASH_FLAG_SIMT) != 0 || shape->kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE;
+    const bool simt = (shape->flags & SPLASH_FLAG_SIMT) != 0;
     Tiling t = choose_tiling(shape, h, dev.sm_count, simt);
     PlanView v = make_plan_view(workspace, B, t.num_workers, h);
     if (workspace_bytes < v.bytes) {

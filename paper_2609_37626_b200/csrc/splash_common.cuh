@@ -150,6 +150,7 @@ int simt_heads_per_group();
 // tcgen05 kernel: how it cuts a head slice of width h into CTAs, and its launcher
 void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *num_groups, int *num_workers);
 cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream);
+cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
                                  cudaStream_t stream);
 cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *part_out,

@@ -33,14 +33,13 @@
 // Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA records
 // SPLASH_DEVICE_TIMEOUT in the workspace status block, raises a CTA-wide abort flag,
 // lets copies in flight land, frees its tensor memory and returns.
-#include <cuda.h>
-#include <cuda_bf16.h>
-
-#include "splash_common.cuh"
+#include "splash_umma.cuh"
 
 namespace splash {
 
 namespace {
+
+using namespace umma;
 
 constexpr int kThreads = 288;                      // 9 warps: producer, 4 MMA issuers, 4 softmax
 constexpr int kMmaWarps = 4;
@@ -49,10 +48,7 @@ constexpr int kChunks = 9;                         // 576 / 64-element (128 B) c
 constexpr uint32_t kSlabBytes = 64 * 128;          // one chunk of one page: 64 tokens x 128 B
 constexpr uint32_t kStageBytes = kChunks * kSlabBytes;   // 73,728
 constexpr int kStages = 2;
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 enum BarrierId {
     kBarKvFull = 0,                    // [kStages]
@@ -90,173 +86,15 @@ struct Layout {
     // one thread: no shuffles, no exchange); narrower groups compute S^T with the tokens on M
     // so that a 16- or 32-head slice is not padded to 64 rows.
     static constexpr bool kHeadsOnM = N == 64;
-    static constexpr int kAcc = N >= 64 ? 2 : 4;             // = number of issuers that take part in QK^T
-    static constexpr uint32_t kColS = 4 * N;                 // 2 buffers x kAcc x N columns
-    static_assert(kColS + 2 * kAcc * N <= 512, "tensor memory overflow");
+    static constexpr int kAcc = 4;                           // = number of issuers that take part in QK^T
+    // two S buffers let QK^T run a tile ahead of the softmax; the 64-head kernel has tensor
+    // memory for one only (O^T 256 columns + 4 partials x 64)
+    static constexpr int kSBufs = N >= 64 ? 1 : 2;
+    static constexpr uint32_t kColS = 4 * N;                 // kSBufs buffers x kAcc x N columns
+    static_assert(kColS + kSBufs * kAcc * N <= 512, "tensor memory overflow");
     static_assert(kBytes <= 232448, "shared memory overflow");
     static_assert(kOffQ % 1024 == 0 && kOffP % 1024 == 0 && (N * 128) % 1024 == 0, "swizzle atoms need 1024-byte alignment");
 };
-
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    return done != 0;
-}
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-struct Ctx {
-    volatile uint32_t *abort_flag;   // shared
-    int32_t *status;                 // global, 16 ints
-};
-
-// Bounded wait.  Returns false if the CTA is aborting (this wait or another one timed out).
-__device__ __noinline__ bool mbar_wait_slow(const Ctx &ctx, uint32_t bar, uint32_t parity, int bar_id) {
-    const unsigned long long start = global_timer_ns();
-    for (;;) {
-        for (int k = 0; k < 256; ++k)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*ctx.abort_flag) return false;
-        if (global_timer_ns() - start > kWaitLimitNs) {
-            *ctx.abort_flag = 1;
-            if (atomicCAS(ctx.status, 0, (int)SPLASH_DEVICE_TIMEOUT) == 0) {
-                ctx.status[1] = (int)blockIdx.x;
-                ctx.status[2] = bar_id;
-                ctx.status[3] = (int)threadIdx.x;
-            }
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ bool mbar_wait(const Ctx &ctx, uint32_t bar, uint32_t parity, int bar_id) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(ctx, bar, parity, bar_id);
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-
-__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-// 16 consecutive fp32 columns of this warp's 32 lanes
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr) : "memory");
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
-          "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
-          "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
-          "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
-          "r"(__float_as_uint(v[15])) : "memory");
-}
-// 16 TMEM lanes x 64 fp32 columns in the MMA accumulator fragment layout: thread T of the
-// warp gets, for k = 0..7, v[4k+0..1] = (lane T/4,     columns 8k + 2(T%4), +1) and
-//                          v[4k+2..3] = (lane T/4 + 8, the same two columns).
-__device__ __forceinline__ void tmem_ld_16x256b_x8(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void softmax_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-// bar.sync among the 128 softmax threads that also ORs a predicate over them
-__device__ __forceinline__ bool softmax_bar_or(bool pred) {
-    uint32_t out;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, 128, q;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(out) : "r"(pred ? 1u : 0u) : "memory");
-    return out != 0;
-}
-
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-
-__device__ __forceinline__ float fast_exp2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
-           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
-}
-
-// Instruction descriptor: fp32 accumulate, bf16 x bf16.
-__host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, int b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
-           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
 
 // Reduce-scatter over the 32 lanes of a warp: on return lane L holds, in v[0 .. max(1, N/32)),
 // the reduction over all lanes of the entries it owns (N = 64: heads 2L, 2L+1; N = 32: head L;
@@ -292,18 +130,6 @@ __device__ __forceinline__ int owned_head(int lane, int i) {
     return lane >> 1;     // N == 16
 }
 
-// Valid rows of a tile after the token shift: page-relative tokens [a, b) land in rows
-// [r_lo, r_hi) of the 64-row box when the box starts at token tok0.
-struct TileGeom { int tok0, r_lo, r_hi; };
-__device__ __forceinline__ TileGeom tile_geom(int lo, int hi, int t0) {
-    int a = max(lo, t0) - t0;
-    int b = min(hi, t0 + kPage) - t0;
-    TileGeom g;
-    if (b < kPage) { g.tok0 = b - kPage; g.r_lo = kPage - b + a; g.r_hi = kPage; }   // end cut: align the end to the box end
-    else { g.tok0 = a; g.r_lo = 0; g.r_hi = kPage - a; }                              // front cut (or none)
-    return g;
-}
-
 // ---------------------------------------------------------------- the kernel
 template <int N>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -329,8 +155,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kMmaWarps); }
         mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), L::kAcc);
-        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), L::kAcc); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxThreads); }
-        mbar_init(bar(kBarPFull), kNumSoftmaxThreads); mbar_init(bar(kBarPEmpty), kMmaWarps);
+        for (int b = 0; b < L::kSBufs; ++b) { mbar_init(bar(kBarSFull + b), L::kAcc); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxThreads); }
+        mbar_init(bar(kBarPFull), kNumSoftmaxThreads); mbar_init(bar(kBarPEmpty), 1);   // (PEmpty unused)
         mbar_init(bar(kBarOFull), kMmaWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxThreads);
         misc[1] = 0; misc[2] = 0; misc[3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -405,7 +231,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             // This issuer's share of S^T for the tile with global index kv: the K = 16 steps
             // idx = mw, mw + kAcc, ... of the 36, into partial accumulator mw.
             auto issue_qk = [&](uint32_t kv, uint32_t sidx) {
-                const uint32_t stage = kv % kStages, b = sidx & 1;
+                const uint32_t stage = kv % kStages, b = sidx % L::kSBufs;
                 if (mw == 0) mark(kv, 2);
                 tcgen05_fence_after();
                 const uint32_t a0 = sbase + L::kOffKv + stage * kStageBytes;
@@ -447,13 +273,12 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 unsigned long long idle_since = 0;
                 while (pv_i < ntiles) {
                     bool progressed = false;
-                    if ((qk_i > pv_i) && mbar_try_wait(bar(kBarPFull), (p_it + pv_i) & 1)) {
+                    if ((qk_i > pv_i) && mbar_test_wait(bar(kBarPFull), (p_it + pv_i) & 1)) {
                         if (pv_i == 0 && !mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty)) { ok = false; break; }
                         if (mw == 0) mark(kv_it + pv_i, 6);
                         const uint32_t stage = (kv_it + pv_i) % kStages;
                         issue_pv(stage, pv_i == 0);
-                        umma_commit(bar(kBarKvEmpty + stage));
-                        umma_commit(bar(kBarPEmpty));
+                        umma_commit(bar(kBarKvEmpty + stage));   // P.V done: stage free, P buffer free, O^T updated
                         if (pv_i + 1 == ntiles) umma_commit(bar(kBarOFull));
                         if (mw == 0) mark(kv_it + pv_i, 7);
                         ++pv_i;
@@ -461,8 +286,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                     }
                     if (does_qk && qk_i < ntiles && qk_i < pv_i + 2) {
                         const uint32_t kv = kv_it + qk_i, sidx = s_it + qk_i;
-                        if (mbar_try_wait(bar(kBarKvFull + kv % kStages), (kv / kStages) & 1) &&
-                            mbar_try_wait(bar(kBarSEmpty + (sidx & 1)), ((sidx >> 1) & 1) ^ 1)) {
+                        if (mbar_test_wait(bar(kBarKvFull + kv % kStages), (kv / kStages) & 1) &&
+                            mbar_test_wait(bar(kBarSEmpty + sidx % L::kSBufs), ((sidx / L::kSBufs) & 1) ^ 1)) {
                             issue_qk(kv, sidx);
                             ++qk_i;
                             if (qk_i == ntiles) umma_commit(bar(kBarQEmpty));
@@ -515,8 +340,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             for (int i = 0; ok && i < ntiles; ++i) {
                 const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + seg.tile_begin + i) * kPage);
                 const bool valid = lane < 16 && row >= g.r_lo && row < g.r_hi;
-                const uint32_t b = s_it & 1;
-                ok = mbar_wait(ctx, bar(kBarSFull + b), (s_it >> 1) & 1, kBarSFull + b);
+                const uint32_t b = s_it % L::kSBufs;
+                ok = mbar_wait(ctx, bar(kBarSFull + b), (s_it / L::kSBufs) & 1, kBarSFull + b);
                 if (!ok) break;
                 if (st == 0) mark(s_it, 4);
                 tcgen05_fence_after();
@@ -572,8 +397,11 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 }
                 const bool rescale = softmax_bar_or(grew);
                 // P.V of the previous tile must be done with the P buffer and with O^T
-                ok = mbar_wait(ctx, bar(kBarPEmpty), (p_it & 1) ^ 1, kBarPEmpty);
-                if (!ok) break;
+                if (s_it > 0) {
+                    const uint32_t prev = s_it - 1;
+                    ok = mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
+                    if (!ok) break;
+                }
                 tcgen05_fence_after();
                 if (rescale && i > 0) {
 #pragma unroll 1
@@ -654,8 +482,11 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
 #pragma unroll
                 for (int k = 0; k < kOwn; ++k) l_own[k] += mx[k];
                 // P.V of the previous tile must be done with the P buffer and with O^T
-                ok = mbar_wait(ctx, bar(kBarPEmpty), (p_it & 1) ^ 1, kBarPEmpty);
-                if (!ok) break;
+                if (s_it > 0) {
+                    const uint32_t prev = s_it - 1;
+                    ok = mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
+                    if (!ok) break;
+                }
                 tcgen05_fence_after();
                 if (rescale && i > 0) {
 #pragma unroll 1
@@ -775,40 +606,6 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled() {
-    static EncodeTiledFn fn = nullptr;
-    if (fn == nullptr) {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
-    return fn;
-}
-
-// 4-D map (64 elements, rows, 9 chunks, outer): a 576-wide row is seen as 9 chunks of
-// 64 elements, so one box of (64, box_rows, 9, 1) lands in shared memory as
-// [chunk][row][128 B], each chunk slab in the 128-byte swizzle the MMA descriptors expect.
-bool make_map_4d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t outer, uint64_t row_stride_bytes,
-                 uint64_t outer_stride_bytes, uint32_t box_rows) {
-    EncodeTiledFn fn = encode_tiled();
-    if (!fn) { set_error("cuTensorMapEncodeTiled is not available"); return false; }
-    cuuint64_t dims[4] = {64, rows, kChunks, outer};
-    cuuint64_t strides[3] = {row_stride_bytes, 128, outer_stride_bytes};
-    cuuint32_t box[4] = {64, box_rows, kChunks, 1};
-    cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled failed with CUresult %d", (int)r); return false; }
-    return true;
-}
-
 template <int N>
 cudaError_t launch_n(const DecodeParams &p, const CUtensorMap &mkv, const CUtensorMap &mq, cudaStream_t stream) {
     const int smem = (int)Layout<N>::kBytes;
@@ -822,8 +619,8 @@ cudaError_t launch_n(const DecodeParams &p, const CUtensorMap &mkv, const CUtens
 }  // namespace
 
 void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *num_groups, int *num_workers) {
-    (void)kv_dtype;
-    const int n = h <= 16 ? 16 : (h <= 32 ? 32 : 64);
+    // e4m3 KV always runs 64-head groups (narrower slices pad their group with zero heads)
+    const int n = kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE ? 64 : (h <= 16 ? 16 : (h <= 32 ? 32 : 64));
     *heads_per_group = n;
     *num_groups = (h + n - 1) / n;
     const int w = sm_count / *num_groups;
@@ -831,13 +628,15 @@ void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *n
 }
 
 cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream) {
-    if (shape.kv_dtype != SPLASH_KV_BF16) return cudaErrorNotSupported;
+    if (shape.kv_dtype != SPLASH_KV_BF16) return launch_decode_umma_fp8(p, stream);
     alignas(64) CUtensorMap mkv, mq;
     const int n = p.heads_per_group;
-    if (!make_map_4d(&mkv, p.kv_pool, kPage, (uint64_t)(p.num_pool_pages > 0 ? p.num_pool_pages : 1),
-                     (uint64_t)kDQK * 2, (uint64_t)kPage * kDQK * 2, 64))
+    if (!make_map_4d(&mkv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, p.kv_pool, kPage,
+                     (uint64_t)(p.num_pool_pages > 0 ? p.num_pool_pages : 1), (uint64_t)kDQK * 2, 128,
+                     (uint64_t)kPage * kDQK * 2, 64))
         return cudaErrorInvalidValue;
-    if (!make_map_4d(&mq, p.q, (uint64_t)p.H, (uint64_t)p.B, (uint64_t)p.q_stride_head * 2,
+    if (!make_map_4d(&mq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, p.q, (uint64_t)p.H,
+                     (uint64_t)p.B, (uint64_t)p.q_stride_head * 2, 128,
                      (uint64_t)(p.B > 1 ? p.q_stride_request : p.q_stride_head * p.H) * 2, (uint32_t)n))
         return cudaErrorInvalidValue;
     switch (n) {
