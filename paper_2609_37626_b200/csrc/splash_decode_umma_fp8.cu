@@ -62,7 +62,8 @@ constexpr uint32_t kOffScale = kOffPLo + kN * 64;          // float [kStages][64
 constexpr uint32_t kOffQs = kOffScale + kStages * kScaleBytes;   // float [64] query scales
 constexpr uint32_t kOffAlpha = kOffQs + kN * 4;
 constexpr uint32_t kOffL = kOffAlpha + kN * 4;
-constexpr uint32_t kOffBar = kOffL + kN * 4;
+constexpr uint32_t kOffTok = kOffL + kN * 4;                // float2 [2][64]: (log2 scale_t, 1 / scale_t) of a tile
+constexpr uint32_t kOffBar = kOffTok + 2 * 64 * 8;
 constexpr uint32_t kOffMisc = (kOffBar + kNumBarriers * 8 + 15) / 16 * 16;
 constexpr uint32_t kSmemBytes = kOffMisc + 32;
 static_assert(kSmemBytes <= 232448, "shared memory overflow");
@@ -111,6 +112,14 @@ __device__ __forceinline__ float fast_rcp(float x) {
     return y;
 }
 
+// Split x >= 0 into hi + lo with hi carrying 4 significant bits (an e4m3 value when it is in
+// e4m3's normal range): Veltkamp's splitting with 2^20 + 1, all in the fp32 pipe.
+__device__ __forceinline__ void split4(float x, float &hi, float &lo) {
+    const float c = x * 1048577.0f;
+    hi = c - (c - x);
+    lo = x - hi;
+}
+
 // byte offset of (row, byte column) inside a [rows][64 B] slab in the 64-byte swizzle
 __device__ __forceinline__ uint32_t sw64(uint32_t row, uint32_t col_byte) {
     return row * 64 + ((((col_byte >> 4) ^ (row >> 1)) & 3) << 4) + (col_byte & 15);
@@ -155,6 +164,10 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
     SegmentIter it;
     it.init(p, worker);
     Segment seg;
+    long long *const trace = blockIdx.x == 0 ? p.trace : nullptr;
+    auto mark = [&](uint32_t tile, int ev) {
+        if (trace != nullptr && tile < 64) trace[tile * 8 + ev] = clock64();
+    };
 
     if (warp == 0) {
         // ===================================================== TMA producer (pages + their scale pages)
@@ -174,6 +187,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 if (lane == 0) {
                     const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
                     ok = mbar_wait(ctx, bar(kBarKvEmpty + stage), ph ^ 1, kBarKvEmpty + stage);
+                    mark(kv_it, 0);
                     if (ok) {
                         const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
                         // a page id outside the pool reads as zeros through the tensor map; its
@@ -184,6 +198,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                         if (in_pool)
                             bulk_load(sbase + kOffScale + stage * kScaleBytes, p.kv_scales + (int64_t)page * kPage,
                                       kScaleBytes, bar(kBarKvFull + stage));
+                        mark(kv_it, 1);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -201,6 +216,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
             // 18 K = 32 steps x (q hi, q lo) = 36 MMAs per tile; this issuer takes every fourth
             auto issue_qk = [&](uint32_t kv) {
                 const uint32_t stage = kv % kStages;
+                if (mw == 0) mark(kv, 2);
                 tcgen05_fence_after();
                 const uint32_t k0 = sbase + kOffKv + stage * kStageBytes;
                 const uint32_t d = tmem_base + kColS + mw * kN;
@@ -213,6 +229,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     umma_e4m3(d, dq, dk, kIdescQK, t != 0);
                 }
                 umma_commit(bar(kBarSFull));
+                if (mw == 0) mark(kv, 3);
             };
             // O^T block mw += V^T (128 dv x 64 tokens) * (P hi + P lo): 2 K = 32 steps x 2 terms
             auto issue_pv = [&](uint32_t stage, bool first_tile) {
@@ -241,9 +258,11 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     if (qk_i > pv_i && mbar_test_wait(bar(kBarPFull), (kv_it + pv_i) & 1)) {
                         if (pv_i == 0 && !mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty)) { ok = false; break; }
                         const uint32_t stage = (kv_it + pv_i) % kStages;
+                        if (mw == 0) mark(kv_it + pv_i, 6);
                         issue_pv(stage, pv_i == 0);
                         umma_commit(bar(kBarKvEmpty + stage));   // P.V done: stage free, P buffers free, O^T updated
                         if (pv_i + 1 == ntiles) umma_commit(bar(kBarOFull));
+                        if (mw == 0) mark(kv_it + pv_i, 7);
                         ++pv_i;
                         progressed = true;
                     }
@@ -349,6 +368,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 const uint32_t stage = s_it % kStages;
                 ok = mbar_wait(ctx, bar(kBarSFull), s_it & 1, kBarSFull);
                 if (!ok) break;
+                if (st == 0) mark(s_it, 4);
                 // the scale page rode on the stage's own barrier, long complete by now
                 ok = mbar_wait(ctx, bar(kBarKvFull + stage), (s_it / kStages) & 1, kBarKvFull + stage);
                 if (!ok) break;
@@ -369,19 +389,27 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 tmem_wait_ld();
                 tcgen05_fence_before();
                 mbar_arrive(bar(kBarSEmpty));
-                // y = log2-domain logit + log2(token scale); rts = 1 / token scale
+                // per-token tables of this tile, one token per thread: (log2 scale_t, 1 / scale_t)
+                float2 *tok = reinterpret_cast<float2 *>(smem + kOffTok) + (s_it & 1) * 64;
                 const float *sc = scale_s + stage * 64 + g.tok0;
-                float rts[16];
+                if (st < 64) {
+                    const bool v = st >= g.r_lo && st < g.r_hi;
+                    const float ts = v ? sc[st] : 1.0f;
+                    tok[st] = make_float2(fast_log2(ts), fast_rcp(ts));
+                }
+                softmax_bar_sync();
+                // y = log2-domain logit + log2(token scale)
                 float mtA = -INFINITY, mtB = -INFINITY;
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
+                    const int r0 = 8 * k + 2 * tq;
+                    const float4 t2 = *reinterpret_cast<const float4 *>(&tok[r0]);     // (lg, rts) of r0 and r0 + 1
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
-                        const int r = 8 * k + 2 * tq + e;
+                        const int r = r0 + e;
                         const bool v = r >= g.r_lo && r < g.r_hi;
                         const float ts = v ? sc[r] : 1.0f;
-                        const float lg = fast_log2(ts);
-                        rts[2 * k + e] = fast_rcp(ts);
+                        const float lg = e ? t2.z : t2.x;
                         const float yA = v ? fmaf(s[4 * k + e], cqA * ts, lg) : -INFINITY;
                         const float yB = v ? fmaf(s[4 * k + 2 + e], cqB * ts, lg) : -INFINITY;
                         s[4 * k + e] = yA; s[4 * k + 2 + e] = yB;
@@ -399,15 +427,16 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 uint16_t phiA[8], ploA[8], phiB[8], ploB[8];
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
+                    const float4 t2 = *reinterpret_cast<const float4 *>(&tok[8 * k + 2 * tq]);
                     const float a0 = fast_exp2(s[4 * k + 0] + offA), a1 = fast_exp2(s[4 * k + 1] + offA);
                     const float b0 = fast_exp2(s[4 * k + 2] + offB), b1 = fast_exp2(s[4 * k + 3] + offB);
-                    lA = fmaf(a0, rts[2 * k], lA); lA = fmaf(a1, rts[2 * k + 1], lA);
-                    lB = fmaf(b0, rts[2 * k], lB); lB = fmaf(b1, rts[2 * k + 1], lB);
-                    phiA[k] = to_e4m3x2(a0, a1);
-                    phiB[k] = to_e4m3x2(b0, b1);
-                    const float2 ba = from_e4m3x2(phiA[k]), bb = from_e4m3x2(phiB[k]);
-                    ploA[k] = to_e4m3x2(a0 - ba.x, a1 - ba.y);
-                    ploB[k] = to_e4m3x2(b0 - bb.x, b1 - bb.y);
+                    lA = fmaf(a0, t2.y, lA); lA = fmaf(a1, t2.w, lA);
+                    lB = fmaf(b0, t2.y, lB); lB = fmaf(b1, t2.w, lB);
+                    float h0, h1, r0, r1;
+                    split4(a0, h0, r0); split4(a1, h1, r1);
+                    phiA[k] = to_e4m3x2(h0, h1); ploA[k] = to_e4m3x2(r0, r1);
+                    split4(b0, h0, r0); split4(b1, h1, r1);
+                    phiB[k] = to_e4m3x2(h0, h1); ploB[k] = to_e4m3x2(r0, r1);
                 }
                 const bool rescale = softmax_bar_or(grew);
                 // P.V of the previous tile must be done with the P buffers and with O^T
@@ -444,6 +473,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 }
                 fence_proxy_async();
                 tcgen05_fence_before();
+                if (st == 0) mark(s_it, 5);
                 mbar_arrive(bar(kBarPFull));
                 ++s_it;
             }
