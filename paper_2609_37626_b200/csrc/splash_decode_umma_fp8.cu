@@ -26,16 +26,16 @@ namespace {
 
 using namespace umma;
 
-constexpr int kThreads = 288;                      // producer, 4 MMA issuers, 4 softmax warps
-constexpr int kMmaWarps = 4;
-constexpr int kNumSoftmaxThreads = 128;
+constexpr int kThreads = 416;                      // 13 warps: producer, 2 QK issuers, 2 PV issuers, 8 softmax
+constexpr int kQkWarps = 2;                        // = partial accumulators of S
+constexpr int kPvWarps = 2;                        // each owns two of the four dv blocks of O^T
+constexpr int kNumSoftmaxThreads = 256;            // two warps per TMEM lane quadrant, 32 tokens of a tile each
 constexpr int kN = 64;                             // heads per CTA
 constexpr int kChunks = 9;                         // 576 / 64-element (64 B) chunks
 constexpr uint32_t kSlab = 64 * 64;                // one chunk of one page: 64 tokens x 64 B
 constexpr uint32_t kStageBytes = kChunks * kSlab;  // 36,864
 constexpr uint32_t kScaleBytes = 256;              // 64 fp32 token scales of a page
-constexpr int kStages = 4;
-constexpr int kAcc = 4;                            // partial accumulators of S = QK issuers
+constexpr int kStages = 3;
 constexpr float kTau = 4.0f;                       // lazy rescale threshold, log2 units
 constexpr float kLift = 4.0f;                      // weights are stored as 2^(y - m + kLift) <= 2^8
 
@@ -44,9 +44,9 @@ enum BarrierId {
     kBarKvEmpty = kBarKvFull + kStages,
     kBarQFull = kBarKvEmpty + kStages,
     kBarQEmpty,
-    kBarSFull,
-    kBarSEmpty,
-    kBarPFull,
+    kBarSFull,                    // [2]
+    kBarSEmpty = kBarSFull + 2,   // [2]
+    kBarPFull = kBarSEmpty + 2,
     kBarOFull,
     kBarOEmpty,
     kNumBarriers
@@ -57,18 +57,19 @@ constexpr uint32_t kOffKv = 0;
 constexpr uint32_t kOffQHi = kOffKv + kStages * kStageBytes;
 constexpr uint32_t kOffQLo = kOffQHi + kN * kDQK;
 constexpr uint32_t kOffPHi = kOffQLo + kN * kDQK;
-constexpr uint32_t kOffPLo = kOffPHi + kN * 64;
-constexpr uint32_t kOffScale = kOffPLo + kN * 64;          // float [kStages][64]
+constexpr uint32_t kOffPLo = kOffPHi + 2 * kN * 64;         // P hi and P lo are double buffered (tile parity)
+constexpr uint32_t kOffScale = kOffPLo + 2 * kN * 64;      // float [kStages][64]
 constexpr uint32_t kOffQs = kOffScale + kStages * kScaleBytes;   // float [64] query scales
 constexpr uint32_t kOffAlpha = kOffQs + kN * 4;
 constexpr uint32_t kOffL = kOffAlpha + kN * 4;
-constexpr uint32_t kOffTok = kOffL + kN * 4;                // float2 [2][64]: (log2 scale_t, 1 / scale_t) of a tile
-constexpr uint32_t kOffBar = kOffTok + 2 * 64 * 8;
+constexpr uint32_t kOffTok = kOffL + kN * 4;                // float2 [64]: (log2 scale_t, 1 / scale_t) of the tile
+constexpr uint32_t kOffXch = kOffTok + 64 * 8;              // float [64][2]: per-head exchange between token halves
+constexpr uint32_t kOffBar = kOffXch + kN * 8;
 constexpr uint32_t kOffMisc = (kOffBar + kNumBarriers * 8 + 15) / 16 * 16;
 constexpr uint32_t kSmemBytes = kOffMisc + 32;
 static_assert(kSmemBytes <= 232448, "shared memory overflow");
 static_assert(kOffQHi % 512 == 0 && kOffQLo % 512 == 0 && kOffPHi % 512 == 0 && kOffPLo % 512 == 0, "alignment");
-// tensor memory: O^T 4 blocks x 64 columns, then 4 partial S accumulators x 64 columns
+// tensor memory: O^T 4 blocks x 64 columns, then 2 S buffers x 2 partial accumulators x 64 columns
 constexpr uint32_t kColO = 0, kColS = 256;
 
 __host__ __device__ constexpr uint32_t make_idesc_e4m3(int M, int N, int a_mn_major) {
@@ -144,11 +145,11 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
         return;
     }
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kMmaWarps); }
-        mbar_init(bar(kBarQFull), kNumSoftmaxThreads); mbar_init(bar(kBarQEmpty), kAcc);
-        mbar_init(bar(kBarSFull), kAcc); mbar_init(bar(kBarSEmpty), kNumSoftmaxThreads);
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kPvWarps); }
+        mbar_init(bar(kBarQFull), kNumSoftmaxThreads); mbar_init(bar(kBarQEmpty), kQkWarps);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxThreads); }
         mbar_init(bar(kBarPFull), kNumSoftmaxThreads);
-        mbar_init(bar(kBarOFull), kMmaWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxThreads);
+        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxThreads);
         misc[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -205,124 +206,113 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 ++kv_it;
             }
         }
-    } else if (warp <= kMmaWarps) {
-        // ===================================================== MMA issuers
+    } else if (warp <= kQkWarps) {
+        // ===================================================== QK^T issuers: S = (q hi + q lo) K^T
         if (lane == 0) {
-            const int mw = warp - 1;                 // partial accumulator mw of S, dv block mw of O^T
+            const int a = warp - 1;                  // partial accumulator a
             constexpr uint32_t kIdescQK = make_idesc_e4m3(64, 64, 0);
-            constexpr uint32_t kIdescPV = make_idesc_e4m3(128, 64, 1);
-            uint32_t kv_it = 0, seg_it = 0;
+            uint32_t kv = 0, seg_it = 0;
             bool ok = true;
-            // 18 K = 32 steps x (q hi, q lo) = 36 MMAs per tile; this issuer takes every fourth
-            auto issue_qk = [&](uint32_t kv) {
-                const uint32_t stage = kv % kStages;
-                if (mw == 0) mark(kv, 2);
-                tcgen05_fence_after();
-                const uint32_t k0 = sbase + kOffKv + stage * kStageBytes;
-                const uint32_t d = tmem_base + kColS + mw * kN;
-#pragma unroll
-                for (int t = 0; t < 36 / kAcc; ++t) {
-                    const int idx = t * kAcc + mw, hl = idx / 18, ks = idx % 18, c = ks >> 1, k = ks & 1;
-                    const uint32_t q0 = sbase + (hl ? kOffQLo : kOffQHi);
-                    uint64_t dq = make_desc_sw64(q0 + c * kSlab + k * 32, 16, 512);     // A: 64 heads x 32
-                    uint64_t dk = make_desc_sw64(k0 + c * kSlab + k * 32, 16, 512);     // B: 64 tokens x 32
-                    umma_e4m3(d, dq, dk, kIdescQK, t != 0);
-                }
-                umma_commit(bar(kBarSFull));
-                if (mw == 0) mark(kv, 3);
-            };
-            // O^T block mw += V^T (128 dv x 64 tokens) * (P hi + P lo): 2 K = 32 steps x 2 terms
-            auto issue_pv = [&](uint32_t stage, bool first_tile) {
-                tcgen05_fence_after();
-                const uint32_t v0 = sbase + kOffKv + stage * kStageBytes + (2 * mw) * kSlab;
-#pragma unroll
-                for (int hl = 0; hl < 2; ++hl) {
-#pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-                        // A: two 64-element chunks (LBO apart) x 32 tokens (SBO per 8 tokens), MN-major
-                        uint64_t da = make_desc_sw64(v0 + k * 2048, kSlab, 512);
-                        uint64_t db = make_desc_sw64(sbase + (hl ? kOffPLo : kOffPHi) + k * 32, 16, 512);
-                        umma_e4m3(tmem_base + kColO + mw * kN, da, db, kIdescPV, (!first_tile) || (hl | k) != 0);
-                    }
-                }
-            };
             while (ok && it.next(p, seg)) {
                 const int ntiles = seg.tile_end - seg.tile_begin;
                 ok = mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
-                if (!ok) break;
-                int qk_i = 0, pv_i = 0;
-                unsigned long long idle_since = 0;
-                uint32_t spins = 0;
-                while (pv_i < ntiles) {
-                    bool progressed = false;
-                    if (qk_i > pv_i && mbar_test_wait(bar(kBarPFull), (kv_it + pv_i) & 1)) {
-                        if (pv_i == 0 && !mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty)) { ok = false; break; }
-                        const uint32_t stage = (kv_it + pv_i) % kStages;
-                        if (mw == 0) mark(kv_it + pv_i, 6);
-                        issue_pv(stage, pv_i == 0);
-                        umma_commit(bar(kBarKvEmpty + stage));   // P.V done: stage free, P buffers free, O^T updated
-                        if (pv_i + 1 == ntiles) umma_commit(bar(kBarOFull));
-                        if (mw == 0) mark(kv_it + pv_i, 7);
-                        ++pv_i;
-                        progressed = true;
+                for (int i = 0; ok && i < ntiles; ++i, ++kv) {
+                    const uint32_t stage = kv % kStages, b = kv & 1;
+                    ok = mbar_wait(ctx, bar(kBarKvFull + stage), (kv / kStages) & 1, kBarKvFull + stage) &&
+                         mbar_wait(ctx, bar(kBarSEmpty + b), ((kv >> 1) & 1) ^ 1, kBarSEmpty + b);
+                    if (!ok) break;
+                    if (a == 0) mark(kv, 2);
+                    tcgen05_fence_after();
+                    const uint32_t k0 = sbase + kOffKv + stage * kStageBytes;
+                    const uint32_t d = tmem_base + kColS + (b * kQkWarps + a) * kN;
+                    // 18 K = 32 steps x (q hi, q lo) = 36 MMAs per tile; this issuer takes every second
+#pragma unroll
+                    for (int t = 0; t < 36 / kQkWarps; ++t) {
+                        const int idx = t * kQkWarps + a, hl = idx / 18, ks = idx % 18, c = ks >> 1, k = ks & 1;
+                        const uint32_t q0 = sbase + (hl ? kOffQLo : kOffQHi);
+                        uint64_t dq = make_desc_sw64(q0 + c * kSlab + k * 32, 16, 512);     // A: 64 heads x 32
+                        uint64_t dk = make_desc_sw64(k0 + c * kSlab + k * 32, 16, 512);     // B: 64 tokens x 32
+                        umma_e4m3(d, dq, dk, kIdescQK, t != 0);
                     }
-                    if (qk_i < ntiles && qk_i < pv_i + 2) {
-                        const uint32_t kv = kv_it + qk_i;
-                        if (mbar_test_wait(bar(kBarKvFull + kv % kStages), (kv / kStages) & 1) &&
-                            mbar_test_wait(bar(kBarSEmpty), (kv & 1) ^ 1)) {
-                            issue_qk(kv);
-                            ++qk_i;
-                            if (qk_i == ntiles) umma_commit(bar(kBarQEmpty));
-                            progressed = true;
-                        }
-                    }
-                    if (progressed) { idle_since = 0; spins = 0; continue; }
-                    if ((++spins & 1023u) != 0) continue;
-                    if (*ctx.abort_flag) { ok = false; break; }
-                    const unsigned long long now = global_timer_ns();
-                    if (idle_since == 0) idle_since = now;
-                    else if (now - idle_since > kWaitLimitNs) {
-                        *ctx.abort_flag = 1;
-                        if (atomicCAS(ctx.status, 0, (int)SPLASH_DEVICE_TIMEOUT) == 0) {
-                            ctx.status[1] = (int)blockIdx.x; ctx.status[2] = 100 + (qk_i > pv_i ? kBarPFull : kBarKvFull);
-                            ctx.status[3] = pv_i;
-                        }
-                        ok = false; break;
-                    }
+                    umma_commit(bar(kBarSFull + b));
+                    if (a == 0) mark(kv, 3);
                 }
-                kv_it += ntiles;
+                if (ok) umma_commit(bar(kBarQEmpty));
+                ++seg_it;
+            }
+        }
+    } else if (warp <= kQkWarps + kPvWarps) {
+        // ===================================================== P.V issuers: O^T += V^T (P hi + P lo)^T
+        if (lane == 0) {
+            const int pj = warp - 1 - kQkWarps;      // dv blocks 2 pj and 2 pj + 1
+            constexpr uint32_t kIdescPV = make_idesc_e4m3(128, 64, 1);
+            uint32_t kv = 0, seg_it = 0;
+            bool ok = true;
+            while (ok && it.next(p, seg)) {
+                const int ntiles = seg.tile_end - seg.tile_begin;
+                for (int i = 0; ok && i < ntiles; ++i, ++kv) {
+                    const uint32_t stage = kv % kStages;
+                    ok = mbar_wait(ctx, bar(kBarPFull), kv & 1, kBarPFull);
+                    if (ok && i == 0) ok = mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty);
+                    if (!ok) break;
+                    if (pj == 0) mark(kv, 6);
+                    tcgen05_fence_after();
+                    const uint32_t v0 = sbase + kOffKv + stage * kStageBytes;
+#pragma unroll
+                    for (int hl = 0; hl < 2; ++hl) {
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                            for (int jj = 0; jj < 2; ++jj) {
+                                const int j = 2 * pj + jj;
+                                // A: two 64-element chunks (LBO apart) x 32 tokens (SBO per 8 tokens), MN-major
+                                uint64_t da = make_desc_sw64(v0 + (2 * j) * kSlab + k * 2048, kSlab, 512);
+                                uint64_t db = make_desc_sw64(sbase + (hl ? kOffPLo : kOffPHi) + (kv & 1) * (kN * 64) + k * 32, 16, 512);
+                                umma_e4m3(tmem_base + kColO + j * kN, da, db, kIdescPV, (i != 0) || (hl | k) != 0);
+                            }
+                        }
+                    }
+                    umma_commit(bar(kBarKvEmpty + stage));   // P.V done: stage free, P buffers free, O^T updated
+                    if (i + 1 == ntiles) umma_commit(bar(kBarOFull));
+                    if (pj == 0) mark(kv, 7);
+                }
                 ++seg_it;
             }
         }
     } else {
         // ===================================================== softmax + epilogue warps
+        const int sw = warp - 1 - kQkWarps - kPvWarps;  // 0..7
         const int q4 = warp & 3;                       // TMEM lane quadrant of this warp
-        const int st = (warp - 1 - kMmaWarps) * 32 + lane;   // 0..127
+        const int hf = sw >> 2;                        // which 32 tokens of a tile this warp handles
+        const int st = sw * 32 + lane;                 // 0..255
         const uint32_t lane_addr = (uint32_t)(32 * q4) << 16;
         const int hA = 16 * q4 + (lane >> 2);          // this thread's heads: hA and hA + 8
-        const int tq = lane & 3;                       // its tokens: 8k + 2 tq + {0, 1}
+        const int tq = lane & 3;                       // its tokens: 32 hf + 8k + 2 tq + {0, 1}, k = 0..3
         float *qs_s = reinterpret_cast<float *>(smem + kOffQs);
         float *alpha_s = reinterpret_cast<float *>(smem + kOffAlpha);
         float *l_s = reinterpret_cast<float *>(smem + kOffL);
+        float *xch = reinterpret_cast<float *>(smem + kOffXch);
+        float2 *tok = reinterpret_cast<float2 *>(smem + kOffTok);
         const float *scale_s = reinterpret_cast<const float *>(smem + kOffScale);
         const float scale_log2 = p.softmax_scale * kLog2e;
         uint32_t s_it = 0, seg_it = 0;
+        // A failed (timed-out) wait only clears `ok`; the role keeps walking its tiles so that every
+        // thread still meets the named barriers -- once the CTA aborts, waits return at once.
         bool ok = true;
-        while (ok && it.next(p, seg)) {
-            // ---- query rows -> e4m3 hi + lo, one scale per head; two threads per head
-            ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
-            if (!ok) break;
+        while (it.next(p, seg)) {
+            // ---- query rows -> e4m3 hi + lo, one scale per head; four threads per head
+            ok &= mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
             {
-                const int hd = st >> 1, half = st & 1;
+                const int hd = st >> 2, part = st & 3;
                 const int gh = head0 + hd;
                 const bool live = gh < p.head_end;
                 const uint4 *src = reinterpret_cast<const uint4 *>(
                     static_cast<const __nv_bfloat16 *>(p.q) + (int64_t)seg.request * p.q_stride_request +
-                    (int64_t)(live ? gh : p.head_begin) * p.q_stride_head + half * 288);
+                    (int64_t)(live ? gh : p.head_begin) * p.q_stride_head + part * 144);
                 float amax = 0.f;
                 if (live) {
-#pragma unroll 4
-                    for (int v = 0; v < 36; ++v) {
+#pragma unroll 6
+                    for (int v = 0; v < 18; ++v) {
                         uint4 x = __ldg(src + v);
                         const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
@@ -333,11 +323,12 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     }
                 }
                 amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
                 const float qs = amax > 0.f ? amax * (1.0f / 448.0f) : 1.0f;
                 const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
-                if (half == 0) qs_s[hd] = qs;
+                if (part == 0) qs_s[hd] = qs;
 #pragma unroll 2
-                for (int v = 0; v < 36; ++v) {
+                for (int v = 0; v < 18; ++v) {
                     uint4 x = live ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
                     const uint32_t w[4] = {x.x, x.y, x.z, x.w};
                     uint16_t hi[4], lo[4];
@@ -348,7 +339,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                         const float2 back = from_e4m3x2(hi[k]);
                         lo[k] = to_e4m3x2(e0 - back.x, e1 - back.y);
                     }
-                    const uint32_t d = (uint32_t)(half * 288 + v * 8);
+                    const uint32_t d = (uint32_t)(part * 144 + v * 8);
                     const uint32_t off = (d >> 6) * kSlab + sw64((uint32_t)hd, d & 63);
                     *reinterpret_cast<uint2 *>(smem + kOffQHi + off) =
                         make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
@@ -358,51 +349,44 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 fence_proxy_async();
                 mbar_arrive(bar(kBarQFull));
             }
-            softmax_bar_sync();                            // qs_s visible to everyone
+            named_bar_sync<1, kNumSoftmaxThreads>();       // qs_s visible to everyone
             const float cqA = scale_log2 * qs_s[hA], cqB = scale_log2 * qs_s[hA + 8];
             float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;
-            for (int i = 0; ok && i < ntiles; ++i) {
+            for (int i = 0; i < ntiles; ++i) {
                 const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + seg.tile_begin + i) * kPage);
-                const uint32_t stage = s_it % kStages;
-                ok = mbar_wait(ctx, bar(kBarSFull), s_it & 1, kBarSFull);
-                if (!ok) break;
+                const uint32_t stage = s_it % kStages, b = s_it & 1;
+                ok &= mbar_wait(ctx, bar(kBarSFull + b), (s_it >> 1) & 1, kBarSFull + b);
                 if (st == 0) mark(s_it, 4);
                 // the scale page rode on the stage's own barrier, long complete by now
-                ok = mbar_wait(ctx, bar(kBarKvFull + stage), (s_it / kStages) & 1, kBarKvFull + stage);
-                if (!ok) break;
+                ok &= mbar_wait(ctx, bar(kBarKvFull + stage), (s_it / kStages) & 1, kBarKvFull + stage);
                 tcgen05_fence_after();
-                float s[32];
+                float s[16];
                 {
-                    const uint32_t sb = tmem_base + lane_addr + kColS;
-                    tmem_ld_16x256b_x8(sb, s);
+                    float part[16];
+                    const uint32_t sb = tmem_base + lane_addr + kColS + (b * kQkWarps) * kN + 32 * hf;
+                    tmem_ld_16x256b_x4(sb, s);
+                    tmem_ld_16x256b_x4(sb + kN, part);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int a = 1; a < kAcc; ++a) {
-                        float part[32];
-                        tmem_ld_16x256b_x8(sb + a * kN, part);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int n = 0; n < 32; ++n) s[n] += part[n];
-                    }
+                    for (int n = 0; n < 16; ++n) s[n] += part[n];
                 }
-                tmem_wait_ld();
                 tcgen05_fence_before();
-                mbar_arrive(bar(kBarSEmpty));
-                // per-token tables of this tile, one token per thread: (log2 scale_t, 1 / scale_t)
-                float2 *tok = reinterpret_cast<float2 *>(smem + kOffTok) + (s_it & 1) * 64;
+                mbar_arrive(bar(kBarSEmpty + b));
+                // per-token table of this tile, one token per thread: (log2 scale_t, 1 / scale_t)
                 const float *sc = scale_s + stage * 64 + g.tok0;
                 if (st < 64) {
                     const bool v = st >= g.r_lo && st < g.r_hi;
                     const float ts = v ? sc[st] : 1.0f;
                     tok[st] = make_float2(fast_log2(ts), fast_rcp(ts));
                 }
-                softmax_bar_sync();
+                named_bar_sync<1, kNumSoftmaxThreads>();
                 // y = log2-domain logit + log2(token scale)
                 float mtA = -INFINITY, mtB = -INFINITY;
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int r0 = 8 * k + 2 * tq;
+                for (int k = 0; k < 4; ++k) {
+                    const int r0 = 32 * hf + 8 * k + 2 * tq;
                     const float4 t2 = *reinterpret_cast<const float4 *>(&tok[r0]);     // (lg, rts) of r0 and r0 + 1
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
@@ -418,16 +402,25 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 }
                 mtA = fmaxf(mtA, __shfl_xor_sync(0xffffffffu, mtA, 1)); mtB = fmaxf(mtB, __shfl_xor_sync(0xffffffffu, mtB, 1));
                 mtA = fmaxf(mtA, __shfl_xor_sync(0xffffffffu, mtA, 2)); mtB = fmaxf(mtB, __shfl_xor_sync(0xffffffffu, mtB, 2));
+                // combine with the warp that holds the other 32 tokens of these heads
+                if (tq == 0) { xch[2 * hA + hf] = mtA; xch[2 * (hA + 8) + hf] = mtB; }
+                named_bar_sync_dyn<64>(2 + q4);
+                {
+                    const float2 xa = *reinterpret_cast<const float2 *>(&xch[2 * hA]);
+                    const float2 xb = *reinterpret_cast<const float2 *>(&xch[2 * (hA + 8)]);
+                    mtA = fmaxf(xa.x, xa.y); mtB = fmaxf(xb.x, xb.y);
+                }
+                // all eight threads of a head take the same decision from the same numbers
                 bool grew = false;
                 float alA = 1.f, alB = 1.f;
                 if (mtA > mA + kTau) { alA = (mA == -INFINITY) ? 0.f : fast_exp2(mA - mtA); mA = mtA; lA *= alA; grew = true; }
                 if (mtB > mB + kTau) { alB = (mB == -INFINITY) ? 0.f : fast_exp2(mB - mtB); mB = mtB; lB *= alB; grew = true; }
-                if (tq == 0) { alpha_s[hA] = alA; alpha_s[hA + 8] = alB; }
+                if (tq == 0 && hf == 0) { alpha_s[hA] = alA; alpha_s[hA + 8] = alB; }
                 const float offA = kLift - mA, offB = kLift - mB;
-                uint16_t phiA[8], ploA[8], phiB[8], ploB[8];
+                uint16_t phiA[4], ploA[4], phiB[4], ploB[4];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const float4 t2 = *reinterpret_cast<const float4 *>(&tok[8 * k + 2 * tq]);
+                for (int k = 0; k < 4; ++k) {
+                    const float4 t2 = *reinterpret_cast<const float4 *>(&tok[32 * hf + 8 * k + 2 * tq]);
                     const float a0 = fast_exp2(s[4 * k + 0] + offA), a1 = fast_exp2(s[4 * k + 1] + offA);
                     const float b0 = fast_exp2(s[4 * k + 2] + offB), b1 = fast_exp2(s[4 * k + 3] + offB);
                     lA = fmaf(a0, t2.y, lA); lA = fmaf(a1, t2.w, lA);
@@ -438,19 +431,24 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     split4(b0, h0, r0); split4(b1, h1, r1);
                     phiB[k] = to_e4m3x2(h0, h1); ploB[k] = to_e4m3x2(r0, r1);
                 }
-                const bool rescale = softmax_bar_or(grew);
-                // P.V of the previous tile must be done with the P buffers and with O^T
-                if (s_it > 0) {
+                const bool rescale = named_bar_or<1, kNumSoftmaxThreads>(grew);
+                // the P.V that read this P buffer (two tiles back) must be done; a rescale of O^T also
+                // needs the previous tile's P.V
+                if (s_it > 1) {
+                    const uint32_t prev = s_it - 2;
+                    ok &= mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
+                }
+                if (rescale && i > 0) {
                     const uint32_t prev = s_it - 1;
-                    ok = mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
-                    if (!ok) break;
+                    ok &= mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
                 }
                 tcgen05_fence_after();
                 if (rescale && i > 0) {
+                    // this warp rescales columns [128 hf, 128 hf + 128) of its quadrant's O^T lanes
 #pragma unroll 1
-                    for (int c = 0; c < 4 * kN / 16; ++c) {
+                    for (int c = 0; c < 8; ++c) {
                         float o[16];
-                        const uint32_t addr = tmem_base + lane_addr + kColO + c * 16;
+                        const uint32_t addr = tmem_base + lane_addr + kColO + 128 * hf + c * 16;
                         tmem_ld16(addr, o);
                         tmem_wait_ld();
 #pragma unroll
@@ -462,8 +460,8 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 {
                     // P hi / lo as K-major, 64-byte-swizzled B operands: row = head, byte = token
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const uint32_t offA_ = sw64((uint32_t)hA, (uint32_t)(8 * k + 2 * tq));
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t offA_ = (s_it & 1) * (kN * 64) + sw64((uint32_t)hA, (uint32_t)(32 * hf + 8 * k + 2 * tq));
                         const uint32_t offB_ = offA_ + 8 * 64;           // head hA + 8: same swizzle phase
                         *reinterpret_cast<uint16_t *>(smem + kOffPHi + offA_) = phiA[k];
                         *reinterpret_cast<uint16_t *>(smem + kOffPLo + offA_) = ploA[k];
@@ -477,14 +475,16 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 mbar_arrive(bar(kBarPFull));
                 ++s_it;
             }
-            if (!ok) break;
+            // ---- row sums: the 4 threads of a row, then the two token halves
             lA += __shfl_xor_sync(0xffffffffu, lA, 1); lB += __shfl_xor_sync(0xffffffffu, lB, 1);
             lA += __shfl_xor_sync(0xffffffffu, lA, 2); lB += __shfl_xor_sync(0xffffffffu, lB, 2);
-            if (tq == 0) {
+            if (tq == 0) { xch[2 * hA + hf] = lA; xch[2 * (hA + 8) + hf] = lB; }
+            named_bar_sync_dyn<64>(2 + q4);
+            if (tq == 0 && hf == 0) {
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int hh = hA + 8 * e;
-                    const float l = e ? lB : lA, m = e ? mB : mA;
+                    const float l = xch[2 * hh] + xch[2 * hh + 1], m = e ? mB : mA;
                     l_s[hh] = 1.f / l;
                     const int gh = head0 + hh;
                     if (gh < p.head_end) {
@@ -494,10 +494,10 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     }
                 }
             }
-            softmax_bar_sync();
-            // ---- epilogue: O^T block j holds dv = 128 j + TMEM lane, one column per head
-            ok = mbar_wait(ctx, bar(kBarOFull), seg_it & 1, kBarOFull);
-            if (!ok) break;
+            named_bar_sync<1, kNumSoftmaxThreads>();
+            // ---- epilogue: O^T block j holds dv = 128 j + TMEM lane, one column per head;
+            // this warp takes blocks 2 hf and 2 hf + 1 of its quadrant's lanes
+            ok &= mbar_wait(ctx, bar(kBarOFull), seg_it & 1, kBarOFull);
             tcgen05_fence_after();
             float *obase;
             int64_t ostride;
@@ -510,7 +510,8 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
             }
             const int nvalid = min(kN, p.head_end - head0);
 #pragma unroll 1
-            for (int j = 0; j < 4; ++j) {
+            for (int jj = 0; jj < 2; ++jj) {
+                const int j = 2 * hf + jj;
                 const int dv = 128 * j + 32 * q4 + lane;
 #pragma unroll
                 for (int c = 0; c < kN / 16; ++c) {

@@ -58,6 +58,7 @@ struct Ctx {
 
 // Bounded wait.  Returns false if the CTA is aborting (this wait or another one timed out).
 static __device__ __noinline__ bool mbar_wait_slow(const Ctx &ctx, uint32_t bar, uint32_t parity, int bar_id) {
+    if (*ctx.abort_flag) return false;            // once the CTA is aborting no wait blocks any more
     const unsigned long long start = global_timer_ns();
     for (;;) {
         for (int k = 0; k < 256; ++k)
@@ -144,6 +145,20 @@ __device__ __forceinline__ void tmem_ld_16x256b_x8(uint32_t taddr, float (&v)[32
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// Same fragment layout, 32 columns: v[4k+0..1] = (lane T/4, columns 8k + 2(T%4), +1),
+// v[4k+2..3] = (lane T/4 + 8, same columns), k = 0..3.
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -159,6 +174,28 @@ __device__ __forceinline__ bool softmax_bar_or(bool pred) {
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(out) : "r"(pred ? 1u : 0u) : "memory");
     return out != 0;
+}
+
+// named barriers with a compile-time id and thread count
+template <int ID, int COUNT>
+__device__ __forceinline__ void named_bar_sync() {
+    asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(COUNT) : "memory");
+}
+template <int ID, int COUNT>
+__device__ __forceinline__ bool named_bar_or(bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, %2, %3, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"(pred ? 1u : 0u), "n"(ID), "n"(COUNT) : "memory");
+    return out != 0;
+}
+// named barrier whose id is a run-time value (one of several equivalent barriers)
+template <int COUNT>
+__device__ __forceinline__ void named_bar_sync_dyn(int id) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "n"(COUNT) : "memory");
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
