@@ -18,9 +18,11 @@ constexpr int kMaxHeads = 128;
 // largest page id (exclusive) the allocation-free migrate entry point can remap: 1 MiB of table
 constexpr int kStaticMigrateMaxPageId = 1 << 18;
 
-// Cost, in page tiles, charged once per non-empty request when the plan balances
-// work over CTAs (query load + epilogue).
-constexpr int kRequestOverheadTiles = 4;
+// Cost, in page tiles, charged once per non-empty request when the plan balances work
+// over CTAs (query operands, pipeline refill, epilogue): measured per kernel, passed to the
+// plan kernel at launch.
+constexpr int kRequestOverheadTilesDefault = 4;
+constexpr int kRequestOverheadTilesFp8 = 6;
 
 // ---- workspace layout ------------------------------------------------------
 // [0, 64)                 status block (int32 x 16): [0] status, [1..3] detail
@@ -92,6 +94,7 @@ struct DecodeParams {
     int32_t *status;
     float *partial_lse, *partial_out;
     int32_t num_workers;
+    int32_t request_overhead_tiles;   // per-request cost the plan adds to the tile count
     long long *trace;          // optional device buffer for pipeline timestamps (diagnostics), or NULL
 };
 

@@ -44,6 +44,7 @@ using namespace umma;
 constexpr int kThreads = 288;                      // 9 warps: producer, 4 MMA issuers, 4 softmax
 constexpr int kMmaWarps = 4;
 constexpr int kNumSoftmaxThreads = 128;
+constexpr int kNumSoftmaxWarps = 4;                // barriers fed by the softmax role count one arrival per warp
 constexpr int kChunks = 9;                         // 576 / 64-element (128 B) chunks
 constexpr uint32_t kSlabBytes = 64 * 128;          // one chunk of one page: 64 tokens x 128 B
 constexpr uint32_t kStageBytes = kChunks * kSlabBytes;   // 73,728
@@ -155,9 +156,9 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kMmaWarps); }
         mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), L::kAcc);
-        for (int b = 0; b < L::kSBufs; ++b) { mbar_init(bar(kBarSFull + b), L::kAcc); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxThreads); }
-        mbar_init(bar(kBarPFull), kNumSoftmaxThreads); mbar_init(bar(kBarPEmpty), 1);   // (PEmpty unused)
-        mbar_init(bar(kBarOFull), kMmaWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxThreads);
+        for (int b = 0; b < L::kSBufs; ++b) { mbar_init(bar(kBarSFull + b), L::kAcc); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxWarps); }
+        mbar_init(bar(kBarPFull), kNumSoftmaxWarps); mbar_init(bar(kBarPEmpty), 1);   // (PEmpty unused)
+        mbar_init(bar(kBarOFull), kMmaWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxWarps);
         misc[1] = 0; misc[2] = 0; misc[3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -364,7 +365,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 }
                 tmem_wait_ld();
                 tcgen05_fence_before();
-                mbar_arrive(bar(kBarSEmpty + b));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarSEmpty + b));
                 const int tq = lane & 3;
                 float mtA = -INFINITY, mtB = -INFINITY;
 #pragma unroll
@@ -447,7 +449,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 }
                 tmem_wait_ld();
                 tcgen05_fence_before();
-                mbar_arrive(bar(kBarSEmpty + b));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarSEmpty + b));
                 float mx[N];
 #pragma unroll
                 for (int n = 0; n < N; ++n) { s[n] = valid ? s[n] * scale_log2 : -INFINITY; mx[n] = s[n]; }
@@ -515,7 +518,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 fence_proxy_async();
                 tcgen05_fence_before();
                 if (st == 0) mark(s_it, 5);
-                mbar_arrive(bar(kBarPFull));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarPFull));
                 ++s_it; ++p_it;
             }
             if (!ok) break;
@@ -586,7 +590,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 }
             }
             tcgen05_fence_before();
-            mbar_arrive(bar(kBarOEmpty));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarOEmpty));
             ++seg_it;
         }
     }

@@ -26,10 +26,12 @@ namespace {
 
 using namespace umma;
 
-constexpr int kThreads = 416;                      // 13 warps: producer, 2 QK issuers, 2 PV issuers, 8 softmax
+constexpr int kThreads = 544;                      // 17 warps: producer, 2 QK issuers, 2 PV issuers, 8 softmax, 4 query converters
+constexpr int kNumConvertWarps = 4;
 constexpr int kQkWarps = 2;                        // = partial accumulators of S
 constexpr int kPvWarps = 2;                        // each owns two of the four dv blocks of O^T
 constexpr int kNumSoftmaxThreads = 256;            // two warps per TMEM lane quadrant, 32 tokens of a tile each
+constexpr int kNumSoftmaxWarps = kNumSoftmaxThreads / 32;   // barriers fed by the softmax role count one arrival per warp
 constexpr int kN = 64;                             // heads per CTA
 constexpr int kChunks = 9;                         // 576 / 64-element (64 B) chunks
 constexpr uint32_t kSlab = 64 * 64;                // one chunk of one page: 64 tokens x 64 B
@@ -59,8 +61,8 @@ constexpr uint32_t kOffQLo = kOffQHi + kN * kDQK;
 constexpr uint32_t kOffPHi = kOffQLo + kN * kDQK;
 constexpr uint32_t kOffPLo = kOffPHi + 2 * kN * 64;         // P hi and P lo are double buffered (tile parity)
 constexpr uint32_t kOffScale = kOffPLo + 2 * kN * 64;      // float [kStages][64]
-constexpr uint32_t kOffQs = kOffScale + kStages * kScaleBytes;   // float [64] query scales
-constexpr uint32_t kOffAlpha = kOffQs + kN * 4;
+constexpr uint32_t kOffQs = kOffScale + kStages * kScaleBytes;   // float [4][64] query scales, by segment & 3
+constexpr uint32_t kOffAlpha = kOffQs + 4 * kN * 4;         // (four deep: the converters run ahead of the softmax warps)
 constexpr uint32_t kOffL = kOffAlpha + kN * 4;
 constexpr uint32_t kOffTok = kOffL + kN * 4;                // float2 [64]: (log2 scale_t, 1 / scale_t) of the tile
 constexpr uint32_t kOffXch = kOffTok + 64 * 8;              // float [64][2]: per-head exchange between token halves
@@ -146,10 +148,10 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
     }
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kPvWarps); }
-        mbar_init(bar(kBarQFull), kNumSoftmaxThreads); mbar_init(bar(kBarQEmpty), kQkWarps);
-        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxThreads); }
-        mbar_init(bar(kBarPFull), kNumSoftmaxThreads);
-        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxThreads);
+        mbar_init(bar(kBarQFull), kNumConvertWarps); mbar_init(bar(kBarQEmpty), kQkWarps);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxWarps); }
+        mbar_init(bar(kBarPFull), kNumSoftmaxWarps);
+        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxWarps);
         misc[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -161,6 +163,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = misc[0];
+    const long long t_start = clock64();
 
     SegmentIter it;
     it.init(p, worker);
@@ -279,6 +282,67 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 ++seg_it;
             }
         }
+    } else if (warp >= 1 + kQkWarps + kPvWarps + kNumSoftmaxWarps) {
+        // ===================================================== query converters
+        // bf16 query rows -> e4m3 hi + lo operands with one scale per head, two threads per head.
+        // They run a segment ahead of the softmax warps: the operands of the next request are
+        // rebuilt as soon as the last QK^T of the current one has been issued and retired.
+        const int ct = (warp - (1 + kQkWarps + kPvWarps + kNumSoftmaxWarps)) * 32 + lane;   // 0..127
+        float *qs_s = reinterpret_cast<float *>(smem + kOffQs);
+        uint32_t seg_it = 0;
+        bool ok = true;
+        while (ok && it.next(p, seg)) {
+            ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
+            if (!ok) break;
+            {
+                const int hd = ct >> 1, part = ct & 1;
+                const int gh = head0 + hd;
+                const bool live = gh < p.head_end;
+                const uint4 *src = reinterpret_cast<const uint4 *>(
+                    static_cast<const __nv_bfloat16 *>(p.q) + (int64_t)seg.request * p.q_stride_request +
+                    (int64_t)(live ? gh : p.head_begin) * p.q_stride_head + part * 288);
+                float amax = 0.f;
+                if (live) {
+#pragma unroll 6
+                    for (int v = 0; v < 36; ++v) {
+                        uint4 x = __ldg(src + v);
+                        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            amax = fmaxf(amax, fabsf(__uint_as_float(w[k] << 16)));
+                            amax = fmaxf(amax, fabsf(__uint_as_float(w[k] & 0xffff0000u)));
+                        }
+                    }
+                }
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                const float qs = amax > 0.f ? amax * (1.0f / 448.0f) : 1.0f;
+                const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
+                if (part == 0) qs_s[(seg_it & 3) * kN + hd] = qs;
+#pragma unroll 2
+                for (int v = 0; v < 36; ++v) {
+                    uint4 x = live ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
+                    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+                    uint16_t hi[4], lo[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float e0 = __uint_as_float(w[k] << 16) * inv, e1 = __uint_as_float(w[k] & 0xffff0000u) * inv;
+                        hi[k] = to_e4m3x2(e0, e1);
+                        const float2 back = from_e4m3x2(hi[k]);
+                        lo[k] = to_e4m3x2(e0 - back.x, e1 - back.y);
+                    }
+                    const uint32_t d = (uint32_t)(part * 288 + v * 8);
+                    const uint32_t off = (d >> 6) * kSlab + sw64((uint32_t)hd, d & 63);
+                    *reinterpret_cast<uint2 *>(smem + kOffQHi + off) =
+                        make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
+                    *reinterpret_cast<uint2 *>(smem + kOffQLo + off) =
+                        make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarQFull));
+            }
+            ++seg_it;
+        }
     } else {
         // ===================================================== softmax + epilogue warps
         const int sw = warp - 1 - kQkWarps - kPvWarps;  // 0..7
@@ -300,57 +364,9 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
         // thread still meets the named barriers -- once the CTA aborts, waits return at once.
         bool ok = true;
         while (it.next(p, seg)) {
-            // ---- query rows -> e4m3 hi + lo, one scale per head; four threads per head
-            ok &= mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
-            {
-                const int hd = st >> 2, part = st & 3;
-                const int gh = head0 + hd;
-                const bool live = gh < p.head_end;
-                const uint4 *src = reinterpret_cast<const uint4 *>(
-                    static_cast<const __nv_bfloat16 *>(p.q) + (int64_t)seg.request * p.q_stride_request +
-                    (int64_t)(live ? gh : p.head_begin) * p.q_stride_head + part * 144);
-                float amax = 0.f;
-                if (live) {
-#pragma unroll 6
-                    for (int v = 0; v < 18; ++v) {
-                        uint4 x = __ldg(src + v);
-                        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            amax = fmaxf(amax, fabsf(__uint_as_float(w[k] << 16)));
-                            amax = fmaxf(amax, fabsf(__uint_as_float(w[k] & 0xffff0000u)));
-                        }
-                    }
-                }
-                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-                const float qs = amax > 0.f ? amax * (1.0f / 448.0f) : 1.0f;
-                const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
-                if (part == 0) qs_s[hd] = qs;
-#pragma unroll 2
-                for (int v = 0; v < 18; ++v) {
-                    uint4 x = live ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
-                    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-                    uint16_t hi[4], lo[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float e0 = __uint_as_float(w[k] << 16) * inv, e1 = __uint_as_float(w[k] & 0xffff0000u) * inv;
-                        hi[k] = to_e4m3x2(e0, e1);
-                        const float2 back = from_e4m3x2(hi[k]);
-                        lo[k] = to_e4m3x2(e0 - back.x, e1 - back.y);
-                    }
-                    const uint32_t d = (uint32_t)(part * 144 + v * 8);
-                    const uint32_t off = (d >> 6) * kSlab + sw64((uint32_t)hd, d & 63);
-                    *reinterpret_cast<uint2 *>(smem + kOffQHi + off) =
-                        make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
-                    *reinterpret_cast<uint2 *>(smem + kOffQLo + off) =
-                        make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
-                }
-                fence_proxy_async();
-                mbar_arrive(bar(kBarQFull));
-            }
-            named_bar_sync<1, kNumSoftmaxThreads>();       // qs_s visible to everyone
-            const float cqA = scale_log2 * qs_s[hA], cqB = scale_log2 * qs_s[hA + 8];
+            // the converter warps have written this segment's query operands and scales
+            ok &= mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
+            const float cqA = scale_log2 * qs_s[(seg_it & 3) * kN + hA], cqB = scale_log2 * qs_s[(seg_it & 3) * kN + hA + 8];
             float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;
@@ -373,7 +389,8 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     for (int n = 0; n < 16; ++n) s[n] += part[n];
                 }
                 tcgen05_fence_before();
-                mbar_arrive(bar(kBarSEmpty + b));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarSEmpty + b));
                 // per-token table of this tile, one token per thread: (log2 scale_t, 1 / scale_t)
                 const float *sc = scale_s + stage * 64 + g.tok0;
                 if (st < 64) {
@@ -472,7 +489,8 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 fence_proxy_async();
                 tcgen05_fence_before();
                 if (st == 0) mark(s_it, 5);
-                mbar_arrive(bar(kBarPFull));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarPFull));
                 ++s_it;
             }
             // ---- row sums: the 4 threads of a row, then the two token halves
@@ -526,12 +544,14 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 }
             }
             tcgen05_fence_before();
-            mbar_arrive(bar(kBarOEmpty));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarOEmpty));
             ++seg_it;
         }
     }
 
     // ---- teardown
+    if (p.trace != nullptr && tid == 0) p.trace[512 + blockIdx.x] = clock64() - t_start;   // per-CTA cycles
     if (*ctx.abort_flag) {
         const unsigned long long t0 = global_timer_ns();
         while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }

@@ -19,7 +19,7 @@ namespace {
 constexpr int kPlanThreads = 1024;
 
 __global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(int B, int W, const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ kv_begin,
+plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ kv_begin,
             const int32_t *__restrict__ kv_end, int32_t *__restrict__ tile_start,
             int32_t *__restrict__ req_lo, int32_t *__restrict__ req_hi,
             int32_t *__restrict__ req_wfirst, int32_t *__restrict__ req_wlast,
@@ -45,7 +45,7 @@ plan_kernel(int B, int W, const int32_t *__restrict__ seq_lens, const int32_t *_
             req_lo[i] = lo; req_hi[i] = hi;
             if (hi > lo) n = (hi + kPage - 1) / kPage - lo / kPage;
         }
-        long long c = n > 0 ? n + kRequestOverheadTiles : 0;
+        long long c = n > 0 ? n + overhead : 0;
         long long sn = n, sc = c;
         for (int o = 1; o < 32; o <<= 1) {
             long long a = __shfl_up_sync(0xffffffffu, sn, o);
@@ -75,7 +75,7 @@ plan_kernel(int B, int W, const int32_t *__restrict__ seq_lens, const int32_t *_
             int lo = 0, hi = B;   // invariant cost_start[lo] <= target < cost_start[hi]
             while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (cost_start[mid] <= target) lo = mid; else hi = mid; }
             while (cost_start[lo + 1] <= target) ++lo;   // (defensive; bisection already lands on a non-empty request)
-            long long off = target - cost_start[lo] - kRequestOverheadTiles;
+            long long off = target - cost_start[lo] - overhead;
             if (off < 0) off = 0;
             g = tile_start[lo] + (int)off;
         }
@@ -108,7 +108,7 @@ cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const in
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *status,
                         cudaStream_t stream) {
-    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.seq_lens, kv_begin, kv_end, tile_start,
+    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.seq_lens, kv_begin, kv_end, tile_start,
                                                 req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, status);
     count_launch();
     return cudaGetLastError();
