@@ -139,6 +139,26 @@ struct SegmentIter {
     }
 };
 
+// ---- programmatic dependent launch ---------------------------------------------
+// The three kernels of a decode call are chained with programmatic stream serialisation:
+// a dependent kernel may be scheduled while its predecessor is still running, does its
+// own set-up (barriers, tensor memory), and blocks in grid_dependency_wait() before it
+// touches anything the predecessor wrote.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- host helpers (splash_api.cu) -----------------------------------------
 void set_error(const char *fmt, ...);
 void count_launch(int n = 1);

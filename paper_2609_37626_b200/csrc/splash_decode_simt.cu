@@ -44,6 +44,7 @@ decode_simt_kernel(const DecodeParams p) {
     const int head0 = p.head_begin + group * kSimtHeads;       // first global head of this CTA
     const int h = p.head_end - p.head_begin;
 
+    grid_dependency_wait();       // the plan kernel's output is read from here on
     SegmentIter it;
     it.init(p, worker);
     Segment seg;
@@ -192,14 +193,14 @@ cudaError_t launch_decode_simt(const DecodeParams &p, int kv_dtype, cudaStream_t
     if (kv_dtype == 0) {
         e = cudaFuncSetAttribute(decode_simt_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        decode_simt_kernel<0><<<grid, kSimtThreads, smem, stream>>>(p);
+        e = launch_dependent(decode_simt_kernel<0>, grid, dim3(kSimtThreads), smem, stream, p);
     } else {
         e = cudaFuncSetAttribute(decode_simt_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        decode_simt_kernel<1><<<grid, kSimtThreads, smem, stream>>>(p);
+        e = launch_dependent(decode_simt_kernel<1>, grid, dim3(kSimtThreads), smem, stream, p);
     }
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 int simt_heads_per_group() { return kSimtHeads; }

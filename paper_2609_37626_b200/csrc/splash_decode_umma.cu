@@ -170,6 +170,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = misc[0];
+    grid_dependency_wait();       // the plan kernel's output is read from here on
 
     SegmentIter it;
     it.init(p, worker);
@@ -616,9 +617,10 @@ cudaError_t launch_n(const DecodeParams &p, const CUtensorMap &mkv, const CUtens
     const int smem = (int)Layout<N>::kBytes;
     cudaError_t e = cudaFuncSetAttribute(decode_umma_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    decode_umma_kernel<N><<<(unsigned)(p.num_workers * p.num_groups), kThreads, smem, stream>>>(p, mkv, mq);
+    e = launch_dependent(decode_umma_kernel<N>, dim3((unsigned)(p.num_workers * p.num_groups)), dim3(kThreads), (size_t)smem,
+                         stream, p, mkv, mq);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace

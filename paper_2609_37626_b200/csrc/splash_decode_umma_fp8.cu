@@ -163,6 +163,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = misc[0];
+    grid_dependency_wait();       // the plan kernel's output is read from here on
     const long long t_start = clock64();
 
     SegmentIter it;
@@ -574,9 +575,10 @@ cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream) {
         return cudaErrorInvalidValue;
     cudaError_t e = cudaFuncSetAttribute(decode_umma_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    decode_umma_fp8_kernel<<<(unsigned)(p.num_workers * p.num_groups), kThreads, kSmemBytes, stream>>>(p, mkv);
+    e = launch_dependent(decode_umma_fp8_kernel, dim3((unsigned)(p.num_workers * p.num_groups)), dim3(kThreads),
+                         (size_t)kSmemBytes, stream, p, mkv);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace splash

@@ -47,13 +47,21 @@ lse_merge_kernel(int num_parts, int64_t rows, int d_v, const float *__restrict__
 
 // Grid B*h: block = request i, head k of the slice.  A request computed in one piece was
 // written by the decode kernel itself; an empty request gets (0, -inf) here; a split
-// request is merged from the slots of its workers in worker order.
+// request is merged from the slots of its workers in worker order.  The weights are
+// computed once per block (thread j takes worker wf + j), then every thread streams its
+// float4 column over the parts with several loads in flight.
+constexpr int kMaxParts = 512;     // >= number of workers of any launch (one per SM at most)
+
 __global__ void __launch_bounds__(kMergeThreads)
 split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirst,
                      const int32_t *__restrict__ req_wlast) {
+    __shared__ float w_s[kMaxParts];
+    __shared__ int slot_s[kMaxParts];
+    __shared__ float red_s[kMergeThreads / 32];
     const int h = p.head_end - p.head_begin;
     const int k = blockIdx.x % h, i = blockIdx.x / h;
     const int g = p.head_begin + k;
+    grid_dependency_wait();       // the decode kernel's partial slots (and the plan) are read from here on
     const int wf = req_wfirst[i], wl = req_wlast[i];
     float4 *o4 = reinterpret_cast<float4 *>(p.out + (int64_t)i * p.out_stride_request + (int64_t)g * p.out_stride_head);
     float *lse = p.lse + (int64_t)i * p.lse_stride_request + g;
@@ -64,31 +72,53 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
         return;
     }
     if (wf == wl) return;
-    // workers between the first and the last may own no tiles at all (their start
-    // snapped to the same tile as their successor's): they wrote no slot
+    // workers between the first and the last may own no tiles at all (their start snapped to
+    // the same tile as their successor's): they wrote no slot and get weight 0
     const int rs = p.tile_start[i];
+    const int nparts = wl - wf + 1;
     float m = -INFINITY;
-    for (int w = wf; w <= wl; ++w) {
-        if (p.worker_begin[w + 1] <= p.worker_begin[w]) continue;
-        int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
-        m = fmaxf(m, p.partial_lse[(int64_t)slot * h + k]);
+    for (int j = c; j < nparts; j += kMergeThreads) {
+        const int w = wf + j;
+        const bool live = p.worker_begin[w + 1] > p.worker_begin[w];
+        const int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
+        const float L = live ? p.partial_lse[(int64_t)slot * h + k] : -INFINITY;
+        slot_s[j] = slot;
+        w_s[j] = L;
+        m = fmaxf(m, L);
     }
+    for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((c & 31) == 0) red_s[c >> 5] = m;
+    __syncthreads();
+    m = fmaxf(fmaxf(red_s[0], red_s[1]), fmaxf(red_s[2], red_s[3]));
+    for (int j = c; j < nparts; j += kMergeThreads) w_s[j] = expf(w_s[j] - m);     // 0 for dead workers
+    __syncthreads();
     float Z = 0.f;
-    for (int w = wf; w <= wl; ++w) {
-        if (p.worker_begin[w + 1] <= p.worker_begin[w]) continue;
-        int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
-        Z += expf(p.partial_lse[(int64_t)slot * h + k] - m);
-    }
+    for (int j = 0; j < nparts; ++j) Z += w_s[j];          // same order in every thread: one value of Z
     const float L = m + logf(Z);
+    const float inv_z = 1.f / Z;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int w = wf; w <= wl; ++w) {
-        if (p.worker_begin[w + 1] <= p.worker_begin[w]) continue;
-        int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
-        int64_t row = (int64_t)slot * h + k;
-        float wgt = expf(p.partial_lse[row] - L);
-        float4 v = reinterpret_cast<const float4 *>(p.partial_out + row * kDV)[c];
-        acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
-        acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
+    int j = 0;
+    for (; j + 4 <= nparts; j += 4) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            v[u] = reinterpret_cast<const float4 *>(p.partial_out + ((int64_t)slot_s[j + u] * h + k) * kDV)[c];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float wgt = w_s[j + u] * inv_z;
+            if (wgt != 0.f) {          // a dead worker's slot holds stale bytes
+                acc.x = fmaf(wgt, v[u].x, acc.x); acc.y = fmaf(wgt, v[u].y, acc.y);
+                acc.z = fmaf(wgt, v[u].z, acc.z); acc.w = fmaf(wgt, v[u].w, acc.w);
+            }
+        }
+    }
+    for (; j < nparts; ++j) {
+        const float wgt = w_s[j] * inv_z;
+        if (wgt != 0.f) {
+            float4 v = reinterpret_cast<const float4 *>(p.partial_out + ((int64_t)slot_s[j] * h + k) * kDV)[c];
+            acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
+            acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
+        }
     }
     o4[c] = acc;
     if (c == 0) *lse = L;
@@ -106,9 +136,9 @@ cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *
 cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
                                  cudaStream_t stream) {
     dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * p.B));
-    split_combine_kernel<<<grid, kMergeThreads, 0, stream>>>(p, req_wfirst, req_wlast);
+    cudaError_t e = launch_dependent(split_combine_kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace splash

@@ -17,16 +17,25 @@ namespace splash {
 namespace {
 
 constexpr int kPlanThreads = 1024;
+constexpr int kPlanSmemRequests = 4096;
+constexpr int kPlanSmemWorkers = 512;
 
 __global__ void __launch_bounds__(kPlanThreads)
 plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ kv_begin,
-            const int32_t *__restrict__ kv_end, int32_t *__restrict__ tile_start,
+            const int32_t *__restrict__ kv_end, int32_t *tile_start,
             int32_t *__restrict__ req_lo, int32_t *__restrict__ req_hi,
             int32_t *__restrict__ req_wfirst, int32_t *__restrict__ req_wlast,
-            int32_t *__restrict__ cost_start, int32_t *__restrict__ worker_begin, int32_t *__restrict__ status) {
+            int32_t *cost_start, int32_t *worker_begin, int32_t *__restrict__ status) {
     __shared__ long long warp_tot_tiles[32], warp_tot_cost[32];
     __shared__ long long carry_tiles, carry_cost;
+    // The bisections below chase a dozen dependent loads each; for the usual sizes the
+    // prefix arrays live in shared memory while the plan is built and are copied out at the end.
+    __shared__ int32_t s_tile[kPlanSmemRequests + 1], s_cost[kPlanSmemRequests + 1], s_wbeg[kPlanSmemWorkers + 1];
+    const bool staged = B <= kPlanSmemRequests && W <= kPlanSmemWorkers;
+    int32_t *const g_tile_start = tile_start, *const g_cost_start = cost_start, *const g_worker_begin = worker_begin;
+    if (staged) { tile_start = s_tile; cost_start = s_cost; worker_begin = s_wbeg; }
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    grid_launch_dependents();     // the decode kernel may start its set-up now; it waits for this grid before reading the plan
     if (tid < 16) status[tid] = 0;
     if (tid == 0) { carry_tiles = 0; carry_cost = 0; tile_start[0] = 0; cost_start[0] = 0; }
     __syncthreads();
@@ -99,6 +108,10 @@ plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, co
             wl = lo;
         }
         req_wfirst[i] = wf; req_wlast[i] = wl;
+    }
+    if (staged) {
+        for (int i = tid; i <= B; i += kPlanThreads) { g_tile_start[i] = s_tile[i]; g_cost_start[i] = s_cost[i]; }
+        for (int w = tid; w <= W; w += kPlanThreads) g_worker_begin[w] = s_wbeg[w];
     }
 }
 
