@@ -185,14 +185,14 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     cudaError_t e = record_timing_event(0, stream);
     if (e == cudaSuccess)
         e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
-                        v.cost_start, v.worker_begin, v.status, stream);
+                        v.cost_start, v.worker_begin, v.split_list, v.status, stream);
     if (e == cudaSuccess) e = record_timing_event(1, stream);
     if (e == cudaSuccess) {
         if (simt) e = launch_decode_simt(p, shape->kv_dtype, stream);
         else e = launch_decode_umma(p, *shape, stream);
     }
     if (e == cudaSuccess) e = record_timing_event(2, stream);
-    if (e == cudaSuccess) e = launch_split_combine(p, v.req_wfirst, v.req_wlast, stream);
+    if (e == cudaSuccess) e = launch_split_combine(p, v.req_wfirst, v.req_wlast, v.split_list, stream);
     if (e == cudaSuccess) e = record_timing_event(3, stream);
     if (e == cudaSuccess && g_timing) g_events_recorded = true;
     if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }

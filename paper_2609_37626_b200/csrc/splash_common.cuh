@@ -27,7 +27,8 @@ constexpr int kRequestOverheadTilesFp8 = 6;
 // ---- workspace layout ------------------------------------------------------
 // [0, 64)                 status block (int32 x 16): [0] status, [1..3] detail
 // then int32 arrays       tile_start[B+1], req_lo[B], req_hi[B], req_wfirst[B],
-//                         req_wlast[B], cost_start[B+1], worker_begin[W+1]
+//                         req_wlast[B], cost_start[B+1], worker_begin[W+1], split_list[W+1]
+//                         (status[8] = number of entries of split_list)
 // then (256-B aligned)    partial_lse [2W][h] fp32
 // then (256-B aligned)    partial_out [2W][h][512] fp32
 struct PlanView {
@@ -39,6 +40,7 @@ struct PlanView {
     int32_t *req_wlast;     // [B] last such worker
     int32_t *cost_start;    // [B+1] exclusive prefix of per-request cost (tiles + overhead)
     int32_t *worker_begin;  // [W+1] global tile index where each worker starts
+    int32_t *split_list;    // [W+1] requests computed in more than one piece (count in status[8])
     float *partial_lse;     // [2W][h]
     float *partial_out;     // [2W][h][512]
     int32_t num_workers;    // W
@@ -60,6 +62,7 @@ inline __host__ PlanView make_plan_view(void *workspace, int B, int W, int h) {
     v.req_wlast = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)B;
     v.cost_start = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(B + 1);
     v.worker_begin = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
+    v.split_list = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
     off = align_up(off, 256);
     v.partial_lse = reinterpret_cast<float *>(p + off); off += sizeof(float) * (size_t)2 * W * h;
     off = align_up(off, 256);
@@ -139,6 +142,23 @@ struct SegmentIter {
     }
 };
 
+// Requests whose effective KV range is empty belong to no segment: O = 0, LSE = -inf is
+// written by the decode CTA (worker, head group) with worker == request mod num_workers,
+// for its own heads.  Called by all threads of the CTA once its segments are done.
+__device__ __forceinline__ void fill_empty_requests(const DecodeParams &p, int worker, int head0, int heads_per_group,
+                                                    int tid, int nthreads) {
+    const int nheads = min(heads_per_group, p.head_end - head0);
+    for (int i = worker; i < p.B; i += p.num_workers) {
+        if (p.tile_start[i + 1] != p.tile_start[i]) continue;
+        for (int idx = tid; idx < nheads * (kDV / 4); idx += nthreads) {
+            const int hh = idx / (kDV / 4), c = idx % (kDV / 4);
+            reinterpret_cast<float4 *>(p.out + (int64_t)i * p.out_stride_request + (int64_t)(head0 + hh) * p.out_stride_head)[c] =
+                make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int hh = tid; hh < nheads; hh += nthreads) p.lse[(int64_t)i * p.lse_stride_request + head0 + hh] = -INFINITY;
+    }
+}
+
 // ---- programmatic dependent launch ---------------------------------------------
 // The three kernels of a decode call are chained with programmatic stream serialisation:
 // a dependent kernel may be scheduled while its predecessor is still running, does its
@@ -166,8 +186,8 @@ void count_launch(int n = 1);
 // kernels' host launchers
 cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
-                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *status,
-                        cudaStream_t stream);
+                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
+                        int32_t *status, cudaStream_t stream);
 cudaError_t launch_decode_simt(const DecodeParams &p, int kv_dtype, cudaStream_t stream);
 int simt_heads_per_group();
 // tcgen05 kernel: how it cuts a head slice of width h into CTAs, and its launcher
@@ -175,7 +195,7 @@ void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *n
 cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream);
 cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
-                                 cudaStream_t stream);
+                                 const int32_t *split_list, cudaStream_t stream);
 cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *part_out,
                              const float *part_lse, float *out, float *lse, cudaStream_t stream);
 cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, void *dst_pool,

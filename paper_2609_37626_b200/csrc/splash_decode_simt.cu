@@ -182,6 +182,7 @@ decode_simt_kernel(const DecodeParams p) {
         }
         __syncthreads();
     }
+    fill_empty_requests(p, worker, head0, kSimtHeads, tid, kSimtThreads);
 }
 
 }  // namespace

@@ -597,6 +597,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
         }
     }
 
+    fill_empty_requests(p, worker, head0, N, tid, kThreads);
+
     // ---- teardown
     if (*ctx.abort_flag) {
         // let bulk copies that were already issued land before the CTA's shared memory goes away

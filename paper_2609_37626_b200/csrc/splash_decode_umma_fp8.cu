@@ -551,6 +551,8 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
         }
     }
 
+    fill_empty_requests(p, worker, head0, kN, tid, kThreads);
+
     // ---- teardown
     if (p.trace != nullptr && tid == 0) p.trace[512 + blockIdx.x] = clock64() - t_start;   // per-CTA cycles
     if (*ctx.abort_flag) {

@@ -45,33 +45,29 @@ lse_merge_kernel(int num_parts, int64_t rows, int d_v, const float *__restrict__
     if (threadIdx.x == 0) lse[r] = L;
 }
 
-// Grid B*h: block = request i, head k of the slice.  A request computed in one piece was
-// written by the decode kernel itself; an empty request gets (0, -inf) here; a split
-// request is merged from the slots of its workers in worker order.  The weights are
+// Grid W*h: block = (entry of the plan's list of split requests, head k of the slice).  A
+// request computed in one piece and an empty one were written by the decode kernel itself; a
+// split request is merged from the slots of its workers in worker order.  The weights are
 // computed once per block (thread j takes worker wf + j), then every thread streams its
 // float4 column over the parts with several loads in flight.
 constexpr int kMaxParts = 512;     // >= number of workers of any launch (one per SM at most)
 
 __global__ void __launch_bounds__(kMergeThreads)
 split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirst,
-                     const int32_t *__restrict__ req_wlast) {
+                     const int32_t *__restrict__ req_wlast, const int32_t *__restrict__ split_list) {
     __shared__ float w_s[kMaxParts];
     __shared__ int slot_s[kMaxParts];
     __shared__ float red_s[kMergeThreads / 32];
     const int h = p.head_end - p.head_begin;
-    const int k = blockIdx.x % h, i = blockIdx.x / h;
+    const int k = blockIdx.x % h, entry = blockIdx.x / h;
     const int g = p.head_begin + k;
     grid_dependency_wait();       // the decode kernel's partial slots (and the plan) are read from here on
+    if (entry >= p.status[8]) return;
+    const int i = split_list[entry];
     const int wf = req_wfirst[i], wl = req_wlast[i];
     float4 *o4 = reinterpret_cast<float4 *>(p.out + (int64_t)i * p.out_stride_request + (int64_t)g * p.out_stride_head);
     float *lse = p.lse + (int64_t)i * p.lse_stride_request + g;
     const int c = threadIdx.x;             // 128 threads x float4 = 512 columns
-    if (wf < 0) {
-        o4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (c == 0) *lse = -INFINITY;
-        return;
-    }
-    if (wf == wl) return;
     // workers between the first and the last may own no tiles at all (their start snapped to
     // the same tile as their successor's): they wrote no slot and get weight 0
     const int rs = p.tile_start[i];
@@ -134,9 +130,11 @@ cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *
 }
 
 cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
-                                 cudaStream_t stream) {
-    dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * p.B));
-    cudaError_t e = launch_dependent(split_combine_kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast);
+                                 const int32_t *split_list, cudaStream_t stream) {
+    // at most one request straddles each boundary between consecutive workers
+    const int max_split = p.num_workers < p.B ? p.num_workers : p.B;
+    dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * max_split));
+    cudaError_t e = launch_dependent(split_combine_kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_list);
     count_launch();
     return e;
 }

@@ -25,9 +25,10 @@ plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, co
             const int32_t *__restrict__ kv_end, int32_t *tile_start,
             int32_t *__restrict__ req_lo, int32_t *__restrict__ req_hi,
             int32_t *__restrict__ req_wfirst, int32_t *__restrict__ req_wlast,
-            int32_t *cost_start, int32_t *worker_begin, int32_t *__restrict__ status) {
+            int32_t *cost_start, int32_t *worker_begin, int32_t *__restrict__ split_list, int32_t *__restrict__ status) {
     __shared__ long long warp_tot_tiles[32], warp_tot_cost[32];
     __shared__ long long carry_tiles, carry_cost;
+    __shared__ int n_split;
     // The bisections below chase a dozen dependent loads each; for the usual sizes the
     // prefix arrays live in shared memory while the plan is built and are copied out at the end.
     __shared__ int32_t s_tile[kPlanSmemRequests + 1], s_cost[kPlanSmemRequests + 1], s_wbeg[kPlanSmemWorkers + 1];
@@ -37,7 +38,7 @@ plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, co
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     grid_launch_dependents();     // the decode kernel may start its set-up now; it waits for this grid before reading the plan
     if (tid < 16) status[tid] = 0;
-    if (tid == 0) { carry_tiles = 0; carry_cost = 0; tile_start[0] = 0; cost_start[0] = 0; }
+    if (tid == 0) { carry_tiles = 0; carry_cost = 0; tile_start[0] = 0; cost_start[0] = 0; n_split = 0; }
     __syncthreads();
 
     // pass 1: effective ranges, tile counts, exclusive prefixes of tiles and of cost
@@ -108,7 +109,12 @@ plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, co
             wl = lo;
         }
         req_wfirst[i] = wf; req_wlast[i] = wl;
+        // requests cut into several pieces are listed for the combine kernel (at most W - 1 of them;
+        // the list order varies from run to run, the results do not depend on it)
+        if (wf != wl) split_list[atomicAdd(&n_split, 1)] = i;
     }
+    __syncthreads();
+    if (tid == 0) status[8] = n_split;
     if (staged) {
         for (int i = tid; i <= B; i += kPlanThreads) { g_tile_start[i] = s_tile[i]; g_cost_start[i] = s_cost[i]; }
         for (int w = tid; w <= W; w += kPlanThreads) g_worker_begin[w] = s_wbeg[w];
@@ -119,10 +125,10 @@ plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, co
 
 cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
-                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *status,
-                        cudaStream_t stream) {
+                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
+                        int32_t *status, cudaStream_t stream) {
     plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.seq_lens, kv_begin, kv_end, tile_start,
-                                                req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, status);
+                                                req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, split_list, status);
     count_launch();
     return cudaGetLastError();
 }
