@@ -39,7 +39,7 @@ constexpr uint32_t kStageBytes = kChunks * kSlab;  // 36,864
 constexpr uint32_t kScaleBytes = 256;              // 64 fp32 token scales of a page
 constexpr int kStages = 3;
 constexpr float kTau = 4.0f;                       // lazy rescale threshold, log2 units
-constexpr float kLift = 4.0f;                      // weights are stored as 2^(y - m + kLift) <= 2^8
+constexpr float kLift = 4.75f;                     // weights are stored as 2^(y - m + kLift) <= 2^8.75 = 431 < 448
 
 enum BarrierId {
     kBarKvFull = 0,
@@ -74,9 +74,10 @@ static_assert(kOffQHi % 512 == 0 && kOffQLo % 512 == 0 && kOffPHi % 512 == 0 && 
 // tensor memory: O^T 4 blocks x 64 columns, then 2 S buffers x 2 partial accumulators x 64 columns
 constexpr uint32_t kColO = 0, kColS = 256;
 
-__host__ __device__ constexpr uint32_t make_idesc_e4m3(int M, int N, int a_mn_major) {
-    // fp32 accumulate (bit 4), A and B formats E4M3 (= 0)
-    return (1u << 4) | ((uint32_t)a_mn_major << 15) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+__host__ __device__ constexpr uint32_t make_idesc_e4m3(int M, int N, int a_mn_major, int b_e5m2 = 0) {
+    // fp32 accumulate (bit 4), A format E4M3 (= 0), B format E4M3 (= 0) or E5M2 (= 1, bits 10..12)
+    return (1u << 4) | ((uint32_t)b_e5m2 << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_e4m3(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -96,6 +97,11 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
 __device__ __forceinline__ uint16_t to_e4m3x2(float lo, float hi) {
     uint16_t r;
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint16_t to_e5m2x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
     return r;
 }
 __device__ __forceinline__ float2 from_e4m3x2(uint16_t v) {
@@ -249,7 +255,9 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
         // ===================================================== P.V issuers: O^T += V^T (P hi + P lo)^T
         if (lane == 0) {
             const int pj = warp - 1 - kQkWarps;      // dv blocks 2 pj and 2 pj + 1
-            constexpr uint32_t kIdescPV = make_idesc_e4m3(128, 64, 1);
+            // the low-order term of P is stored as e5m2: residuals of weights that fall into e4m3's
+            // subnormal range (the long tail of a long context) keep three significant bits there
+            constexpr uint32_t kIdescPV = make_idesc_e4m3(128, 64, 1), kIdescPVLo = make_idesc_e4m3(128, 64, 1, 1);
             uint32_t kv = 0, seg_it = 0;
             bool ok = true;
             while (ok && it.next(p, seg)) {
@@ -272,7 +280,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                                 // A: two 64-element chunks (LBO apart) x 32 tokens (SBO per 8 tokens), MN-major
                                 uint64_t da = make_desc_sw64(v0 + (2 * j) * kSlab + k * 2048, kSlab, 512);
                                 uint64_t db = make_desc_sw64(sbase + (hl ? kOffPLo : kOffPHi) + (kv & 1) * (kN * 64) + k * 32, 16, 512);
-                                umma_e4m3(tmem_base + kColO + j * kN, da, db, kIdescPV, (i != 0) || (hl | k) != 0);
+                                umma_e4m3(tmem_base + kColO + j * kN, da, db, hl ? kIdescPVLo : kIdescPV, (i != 0) || (hl | k) != 0);
                             }
                         }
                     }
@@ -443,11 +451,12 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     const float b0 = fast_exp2(s[4 * k + 2] + offB), b1 = fast_exp2(s[4 * k + 3] + offB);
                     lA = fmaf(a0, t2.y, lA); lA = fmaf(a1, t2.w, lA);
                     lB = fmaf(b0, t2.y, lB); lB = fmaf(b1, t2.w, lB);
-                    float h0, h1, r0, r1;
-                    split4(a0, h0, r0); split4(a1, h1, r1);
-                    phiA[k] = to_e4m3x2(h0, h1); ploA[k] = to_e4m3x2(r0, r1);
-                    split4(b0, h0, r0); split4(b1, h1, r1);
-                    phiB[k] = to_e4m3x2(h0, h1); ploB[k] = to_e4m3x2(r0, r1);
+                    // hi = the e4m3 value nearest to the weight, lo = what is left, kept as e5m2
+                    phiA[k] = to_e4m3x2(a0, a1);
+                    phiB[k] = to_e4m3x2(b0, b1);
+                    const float2 ba = from_e4m3x2(phiA[k]), bb = from_e4m3x2(phiB[k]);
+                    ploA[k] = to_e5m2x2(a0 - ba.x, a1 - ba.y);
+                    ploB[k] = to_e5m2x2(b0 - bb.x, b1 - bb.y);
                 }
                 const bool rescale = named_bar_or<1, kNumSoftmaxThreads>(grew);
                 // the P.V that read this P buffer (two tiles back) must be done; a rescale of O^T also
