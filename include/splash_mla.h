@@ -240,8 +240,7 @@ SPLASH_API int splash_get_kernel_timing(float *plan_ms, float *decode_ms, float 
  * Diagnostics: give the decode kernel a device buffer of 64 x 8 + 512 int64 into which
  * CTA 0 writes SM-clock timestamps of its pipeline events for its first 64 tiles (event
  * order: stage free, TMA issued, tile landed, QK^T issued, S ready, P written, P seen,
- * P.V issued); the e4m3 kernel also writes every CTA's total cycle count at
- * [512 + CTA index].  NULL (the default) switches it off.  Per host thread.
+ * P.V issued); every CTA also writes its total cycle count at [512 + CTA index].  NULL (the default) switches it off.  Per host thread.
  */
 SPLASH_API int splash_debug_set_trace(void *device_buffer);
 

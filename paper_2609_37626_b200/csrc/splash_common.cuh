@@ -179,6 +179,15 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Function attributes are per device: true the first time a launcher runs on the current device.
+inline bool first_use_on_device(bool (&seen)[64]) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+    if (seen[dev]) return false;
+    seen[dev] = true;
+    return true;
+}
+
 // ---- host helpers (splash_api.cu) -----------------------------------------
 void set_error(const char *fmt, ...);
 void count_launch(int n = 1);

@@ -171,6 +171,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
     tcgen05_fence_after();
     const uint32_t tmem_base = misc[0];
     grid_dependency_wait();       // the plan kernel's output is read from here on
+    const long long t_start = clock64();
 
     SegmentIter it;
     it.init(p, worker);
@@ -598,6 +599,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
     }
 
     fill_empty_requests(p, worker, head0, N, tid, kThreads);
+    if (p.trace != nullptr && tid == 0) p.trace[512 + blockIdx.x] = clock64() - t_start;   // per-CTA cycles
 
     // ---- teardown
     if (*ctx.abort_flag) {
@@ -617,8 +619,12 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
 template <int N>
 cudaError_t launch_n(const DecodeParams &p, const CUtensorMap &mkv, const CUtensorMap &mq, cudaStream_t stream) {
     const int smem = (int)Layout<N>::kBytes;
-    cudaError_t e = cudaFuncSetAttribute(decode_umma_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
+    static bool configured[64] = {};      // (per device attribute; set again if it was lost to another device)
+    cudaError_t e = cudaSuccess;
+    if (first_use_on_device(configured)) {
+        e = cudaFuncSetAttribute(decode_umma_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+    }
     e = launch_dependent(decode_umma_kernel<N>, dim3((unsigned)(p.num_workers * p.num_groups)), dim3(kThreads), (size_t)smem,
                          stream, p, mkv, mq);
     count_launch();

@@ -584,8 +584,12 @@ cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream) {
                      (uint64_t)(p.num_pool_pages > 0 ? p.num_pool_pages : 1), (uint64_t)kDQK, 64,
                      (uint64_t)kPage * kDQK, 64))
         return cudaErrorInvalidValue;
-    cudaError_t e = cudaFuncSetAttribute(decode_umma_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
+    static bool configured[64] = {};
+    cudaError_t e = cudaSuccess;
+    if (first_use_on_device(configured)) {
+        e = cudaFuncSetAttribute(decode_umma_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+    }
     e = launch_dependent(decode_umma_fp8_kernel, dim3((unsigned)(p.num_workers * p.num_groups)), dim3(kThreads),
                          (size_t)kSmemBytes, stream, p, mkv);
     count_launch();

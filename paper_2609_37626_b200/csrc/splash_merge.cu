@@ -134,6 +134,10 @@ cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirs
     // at most one request straddles each boundary between consecutive workers
     const int max_split = p.num_workers < p.B ? p.num_workers : p.B;
     dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * max_split));
+    static bool configured[64] = {};
+    if (first_use_on_device(configured)) {   // keep the decode kernel's shared-memory carve-out
+        cudaFuncSetAttribute(split_combine_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    }
     cudaError_t e = launch_dependent(split_combine_kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_list);
     count_launch();
     return e;

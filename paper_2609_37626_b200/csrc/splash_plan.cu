@@ -127,6 +127,11 @@ cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const in
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
                         int32_t *status, cudaStream_t stream) {
+    // same shared-memory carve-out as the decode kernel that follows: no reconfiguration between them
+    static bool configured[64] = {};
+    if (first_use_on_device(configured)) {
+        cudaFuncSetAttribute(plan_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    }
     plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.seq_lens, kv_begin, kv_end, tile_start,
                                                 req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, split_list, status);
     count_launch();
