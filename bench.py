@@ -33,7 +33,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2609_37626_b200 import workloads as W  # noqa: E402
+from paper_2609_37626_b200 import sharding, workloads as W  # noqa: E402
 
 METRIC = "mla_decode_tokens_per_s_per_gpu"
 UNIT = "tokens/s"
@@ -374,12 +374,9 @@ def main():
 
     ms = main_res["ms_per_step"]
     e2e_ms = e2e["ms_per_step"]
-    if world > 1:
-        t = torch.tensor([ms, e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_ms = float(t[0]), float(t[1])
-    value = world * w.B / (ms * 1e-3)
-    e2e_value = world * w.B / (e2e_ms * 1e-3)
+    ms, e2e_ms = sharding.max_over_ranks([ms, e2e_ms], device=device)
+    value = sharding.weak_scaling_value(w.B, world, ms)
+    e2e_value = sharding.weak_scaling_value(w.B, world, e2e_ms)
 
     extra = {}
     cpu = None

@@ -164,6 +164,32 @@ def test_fp8_extreme_rows(flags):
     compare(out, lse, *ref, kv_dtype=1, what="fp8 extremes")
 
 
+def test_many_empty_requests_among_live_ones(flags):
+    """Idle shards inside a batch: every other request has an empty range (or no tokens);
+    they get O = 0, LSE = -inf from the decode CTAs, the live ones are unaffected."""
+    import torch
+    rng = np.random.default_rng(77)
+    B = 200
+    lens = rng.integers(0, 400, size=B).astype(np.int32)
+    lens[::7] = 0
+    w = W.make_workload("empties", 820, lens, H=32)
+    kb = np.zeros(B, np.int32); ke = lens.copy()
+    kb[1::2] = lens[1::2]            # empty range for every other request
+    ref = oracle_run(w, kv_begin=kb, kv_end=ke)
+    out, lse = gpu_run(w, flags=flags, sentinel=3.0, kv_begin=torch.from_numpy(kb).cuda(), kv_end=torch.from_numpy(ke).cuda())
+    compare(out, lse, *ref, kv_dtype=0, what="empties")
+    assert np.all(out[1::2] == 0) and np.all(np.isneginf(lse[1::2]))
+
+
+@pytest.mark.parametrize("kv_dtype", [0, 1])
+def test_wide_slices_are_deterministic_too(kv_dtype):
+    w = W.make_workload("det128", 830 + kv_dtype, [3000, 40, 900, 64, 2000], H=128, kv_dtype=kv_dtype)
+    a = gpu_run(w)
+    b = gpu_run(w)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    compare(a[0], a[1], *oracle_run(w), kv_dtype=kv_dtype, what="det128")
+
+
 def test_run_to_run_determinism(flags):
     import torch
     w = W.make_workload("det", 800, [5000, 100, 2500], H=16)
