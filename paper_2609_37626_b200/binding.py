@@ -23,6 +23,7 @@ SPLASH_DEVICE_TIMEOUT = -5
 SPLASH_KV_BF16 = 0
 SPLASH_KV_E4M3_TOKEN_SCALE = 1
 SPLASH_FLAG_SIMT = 1
+SPLASH_FLAG_NO_PAIR = 2
 
 D_QK, D_V, PAGE_SIZE = 576, 512, 64
 

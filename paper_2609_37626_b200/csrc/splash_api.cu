@@ -179,8 +179,10 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     p.tile_start = v.tile_start; p.req_lo = v.req_lo; p.req_hi = v.req_hi; p.worker_begin = v.worker_begin;
     p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
     p.trace = g_trace;
-    p.request_overhead_tiles = (!simt && shape->kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE) ? kRequestOverheadTilesFp8
-                                                                                        : kRequestOverheadTilesDefault;
+    p.request_overhead_tiles = kRequestOverheadTilesDefault;
+    if (!simt && shape->kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE)
+        p.request_overhead_tiles = (t.num_groups == 2 && !(shape->flags & SPLASH_FLAG_NO_PAIR)) ? kRequestOverheadTilesFp8Pair
+                                                                                                 : kRequestOverheadTilesFp8;
 
     cudaError_t e = record_timing_event(0, stream);
     if (e == cudaSuccess)

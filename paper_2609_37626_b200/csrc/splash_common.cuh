@@ -23,6 +23,7 @@ constexpr int kStaticMigrateMaxPageId = 1 << 18;
 // plan kernel at launch.
 constexpr int kRequestOverheadTilesDefault = 4;
 constexpr int kRequestOverheadTilesFp8 = 6;
+constexpr int kRequestOverheadTilesFp8Pair = 12;   // CTA-pair kernel: tiles are cheaper, the per-request work is not
 
 // ---- workspace layout ------------------------------------------------------
 // [0, 64)                 status block (int32 x 16): [0] status, [1..3] detail
@@ -203,6 +204,7 @@ int simt_heads_per_group();
 void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *num_groups, int *num_workers);
 cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream);
 cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream);
+cudaError_t launch_decode_umma_fp8_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
                                  const int32_t *split_list, cudaStream_t stream);
 cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *part_out,

@@ -643,7 +643,11 @@ void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *n
 }
 
 cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream) {
-    if (shape.kv_dtype != SPLASH_KV_BF16) return launch_decode_umma_fp8(p, stream);
+    if (shape.kv_dtype != SPLASH_KV_BF16) {
+        // slices of more than 64 heads run on CTA pairs (cta_group::2) unless the caller opts out
+        if (p.num_groups == 2 && !(shape.flags & SPLASH_FLAG_NO_PAIR)) return launch_decode_umma_fp8_pair(p, stream);
+        return launch_decode_umma_fp8(p, stream);
+    }
     alignas(64) CUtensorMap mkv, mq;
     const int n = p.heads_per_group;
     if (!make_map_4d(&mkv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, p.kv_pool, kPage,

@@ -16,9 +16,7 @@
 // Four e4m3 products per bf16-precision product pair cost the tensor pipe the same time as
 // the bf16 kernel (fp8 MMAs run at twice the rate), which is why the roofline of this
 // workload is taken at the bf16 rate.
-#include <cuda_fp16.h>
-
-#include "splash_umma.cuh"
+#include "splash_fp8.cuh"
 
 namespace splash {
 
@@ -46,6 +44,7 @@ enum BarrierId {
     kBarKvEmpty = kBarKvFull + kStages,
     kBarQFull = kBarKvEmpty + kStages,
     kBarQEmpty,
+    kBarQsRead,                   // the softmax warps have picked up the request's query scales
     kBarSFull,                    // [2]
     kBarSEmpty = kBarSFull + 2,   // [2]
     kBarPFull = kBarSEmpty + 2,
@@ -74,66 +73,6 @@ static_assert(kOffQHi % 512 == 0 && kOffQLo % 512 == 0 && kOffPHi % 512 == 0 && 
 // tensor memory: O^T 4 blocks x 64 columns, then 2 S buffers x 2 partial accumulators x 64 columns
 constexpr uint32_t kColO = 0, kColS = 256;
 
-__host__ __device__ constexpr uint32_t make_idesc_e4m3(int M, int N, int a_mn_major, int b_e5m2 = 0) {
-    // fp32 accumulate (bit 4), A format E4M3 (= 0), B format E4M3 (= 0) or E5M2 (= 1, bits 10..12)
-    return (1u << 4) | ((uint32_t)b_e5m2 << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)(N >> 3) << 17) |
-           ((uint32_t)(M >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_e4m3(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-// two floats -> two e4m3 bytes (first argument in the low byte), round to nearest, saturating
-__device__ __forceinline__ uint16_t to_e4m3x2(float lo, float hi) {
-    uint16_t r;
-    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-__device__ __forceinline__ uint16_t to_e5m2x2(float lo, float hi) {
-    uint16_t r;
-    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-    return r;
-}
-__device__ __forceinline__ float2 from_e4m3x2(uint16_t v) {
-    uint32_t h2;
-    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(v));
-    __half2 h = *reinterpret_cast<__half2 *>(&h2);
-    return __half22float2(h);
-}
-__device__ __forceinline__ float fast_log2(float x) {
-    float y;
-    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float fast_rcp(float x) {
-    float y;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// Split x >= 0 into hi + lo with hi carrying 4 significant bits (an e4m3 value when it is in
-// e4m3's normal range): Veltkamp's splitting with 2^20 + 1, all in the fp32 pipe.
-__device__ __forceinline__ void split4(float x, float &hi, float &lo) {
-    const float c = x * 1048577.0f;
-    hi = c - (c - x);
-    lo = x - hi;
-}
-
-// byte offset of (row, byte column) inside a [rows][64 B] slab in the 64-byte swizzle
-__device__ __forceinline__ uint32_t sw64(uint32_t row, uint32_t col_byte) {
-    return row * 64 + ((((col_byte >> 4) ^ (row >> 1)) & 3) << 4) + (col_byte & 15);
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmap_kv) {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -155,6 +94,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kPvWarps); }
         mbar_init(bar(kBarQFull), kNumConvertWarps); mbar_init(bar(kBarQEmpty), kQkWarps);
+        mbar_init(bar(kBarQsRead), kNumSoftmaxWarps);
         for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxWarps); }
         mbar_init(bar(kBarPFull), kNumSoftmaxWarps);
         mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxWarps);
@@ -348,7 +288,13 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 }
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarQFull));
+                // The softmax warps wait on QFull by phase parity, so QFull must never complete two
+                // phases ahead of them: hold this request's arrival until they have entered the previous one.
+                if (lane == 0) {
+                    if (seg_it > 0) ok = mbar_wait(ctx, bar(kBarQsRead), (seg_it - 1) & 1, kBarQsRead);
+                    mbar_arrive(bar(kBarQFull));
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             }
             ++seg_it;
         }
@@ -376,6 +322,8 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
             // the converter warps have written this segment's query operands and scales
             ok &= mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
             const float cqA = scale_log2 * qs_s[(seg_it & 3) * kN + hA], cqB = scale_log2 * qs_s[(seg_it & 3) * kN + hA + 8];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarQsRead));
             float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;

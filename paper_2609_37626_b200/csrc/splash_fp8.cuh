@@ -1,0 +1,73 @@
+// Building blocks shared by the e4m3 decode kernels: 8-bit MMA issue, conversions, swizzle.
+#pragma once
+
+#include <cuda_fp16.h>
+
+#include "splash_umma.cuh"
+
+namespace splash {
+namespace umma {
+
+__host__ __device__ constexpr uint32_t make_idesc_e4m3(int M, int N, int a_mn_major, int b_e5m2 = 0, int b_mn_major = 0,
+                                                        int a_e5m2 = 0) {
+    // fp32 accumulate (bit 4); A / B formats E4M3 (= 0) or E5M2 (= 1) in bits 7..9 / 10..12
+    return (1u << 4) | ((uint32_t)a_e5m2 << 7) | ((uint32_t)b_e5m2 << 10) | ((uint32_t)a_mn_major << 15) |
+           ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_e4m3(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// two floats -> two e4m3 bytes (first argument in the low byte), round to nearest, saturating
+__device__ __forceinline__ uint16_t to_e4m3x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint16_t to_e5m2x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ float2 from_e4m3x2(uint16_t v) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(v));
+    __half2 h = *reinterpret_cast<__half2 *>(&h2);
+    return __half22float2(h);
+}
+__device__ __forceinline__ float fast_log2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float fast_rcp(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Split x >= 0 into hi + lo with hi carrying 4 significant bits (an e4m3 value when it is in
+// e4m3's normal range): Veltkamp's splitting with 2^20 + 1, all in the fp32 pipe.
+__device__ __forceinline__ void split4(float x, float &hi, float &lo) {
+    const float c = x * 1048577.0f;
+    hi = c - (c - x);
+    lo = x - hi;
+}
+
+// byte offset of (row, byte column) inside a [rows][64 B] slab in the 64-byte swizzle
+__device__ __forceinline__ uint32_t sw64(uint32_t row, uint32_t col_byte) {
+    return row * 64 + ((((col_byte >> 4) ^ (row >> 1)) & 3) << 4) + (col_byte & 15);
+}
+
+}  // namespace umma
+}  // namespace splash

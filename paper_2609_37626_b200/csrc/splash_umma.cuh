@@ -262,12 +262,12 @@ inline EncodeTiledFn encode_tiled() {
 // elements, 64 B for 8-bit ones).
 inline bool make_map_4d(CUtensorMap *map, CUtensorMapDataType dtype, CUtensorMapSwizzle swizzle, const void *base,
                         uint64_t rows, uint64_t outer, uint64_t row_stride_bytes, uint64_t chunk_stride_bytes,
-                        uint64_t outer_stride_bytes, uint32_t box_rows) {
+                        uint64_t outer_stride_bytes, uint32_t box_rows, uint32_t box_chunks = 9) {
     EncodeTiledFn fn = encode_tiled();
     if (!fn) { set_error("cuTensorMapEncodeTiled is not available"); return false; }
     cuuint64_t dims[4] = {64, rows, 9, outer};
     cuuint64_t strides[3] = {row_stride_bytes, chunk_stride_bytes, outer_stride_bytes};
-    cuuint32_t box[4] = {64, box_rows, 9, 1};
+    cuuint32_t box[4] = {64, box_rows, box_chunks, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, dtype, 4, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

@@ -164,6 +164,33 @@ def test_fp8_extreme_rows(flags):
     compare(out, lse, *ref, kv_dtype=1, what="fp8 extremes")
 
 
+# Slices of more than 64 heads over an e4m3 cache run on CTA pairs (one page per CTA, two pages per
+# step); flag 2 selects two independent 64-head CTAs instead.  Lengths cover a lone ragged page, odd
+# and even page counts, requests that several workers split, and many short requests per worker.
+@pytest.mark.parametrize("no_pair", [0, 2], ids=["pair", "single"])
+@pytest.mark.parametrize("H,lens", [
+    (128, [1]), (128, [63, 64, 65, 128, 129]), (128, [200, 5000, 1, 777, 12345]), (80, [333, 64, 4097]),
+    (72, [130] * 40), (128, list(range(1, 400, 7))), (128, [40000]),
+])
+def test_fp8_wide_head_slices(no_pair, H, lens):
+    w = W.make_workload("fp8w", 720 + H + len(lens), lens, H=H, kv_dtype=1)
+    ref = oracle_run(w)
+    out, lse = gpu_run(w, flags=no_pair)
+    compare(out, lse, *ref, kv_dtype=1, what="fp8 wide")
+
+
+@pytest.mark.parametrize("no_pair", [0, 2], ids=["pair", "single"])
+def test_fp8_wide_slice_of_a_wider_layer_and_kv_ranges(no_pair):
+    import torch
+    kb = np.array([100, 0, 64, 128], dtype=np.int32); ke = np.array([899, 70, 2500, 129], dtype=np.int32)
+    w = W.make_workload("fp8ws", 731, [900, 70, 3000, 129], H=128, kv_dtype=1, head_begin=16, head_end=112)
+    ref = oracle_run(w, kv_begin=kb, kv_end=ke)
+    out, lse = gpu_run(w, flags=no_pair, sentinel=5.0,
+                       kv_begin=torch.from_numpy(kb).cuda(), kv_end=torch.from_numpy(ke).cuda())
+    assert (out[:, :16] == 5.0).all() and (out[:, 112:] == 5.0).all()
+    compare(out, lse, *ref, kv_dtype=1, rows=[(i, g) for i in range(4) for g in range(16, 112)], what="fp8 wide slice")
+
+
 def test_many_empty_requests_among_live_ones(flags):
     """Idle shards inside a batch: every other request has an empty range (or no tokens);
     they get O = 0, LSE = -inf from the decode CTAs, the live ones are unaffected."""
