@@ -61,8 +61,8 @@ enum {
     /* Run the plain SIMT (fp32 CUDA-core) decode kernel instead of the tcgen05 one.
      * A diagnostic path: same plan, same partial slots, same combine; slow. */
     SPLASH_FLAG_SIMT = 1u,
-    /* e4m3 KV, slices of 65..128 heads: use two independent 64-head CTAs per KV worker instead
-     * of a CTA pair issuing cta_group::2 MMAs.  A diagnostic path. */
+    /* slices of 65..128 heads: use two independent 64-head CTAs per KV worker instead of a CTA
+     * pair issuing cta_group::2 MMAs.  A diagnostic path. */
     SPLASH_FLAG_NO_PAIR = 2u
 };
 

@@ -180,9 +180,11 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
     p.trace = g_trace;
     p.request_overhead_tiles = kRequestOverheadTilesDefault;
+    const bool pair = !simt && t.num_groups == 2 && t.heads_per_group == 64 && !(shape->flags & SPLASH_FLAG_NO_PAIR);
     if (!simt && shape->kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE)
-        p.request_overhead_tiles = (t.num_groups == 2 && !(shape->flags & SPLASH_FLAG_NO_PAIR)) ? kRequestOverheadTilesFp8Pair
-                                                                                                 : kRequestOverheadTilesFp8;
+        p.request_overhead_tiles = pair ? kRequestOverheadTilesFp8Pair : kRequestOverheadTilesFp8;
+    else if (pair)
+        p.request_overhead_tiles = kRequestOverheadTilesPair;
 
     cudaError_t e = record_timing_event(0, stream);
     if (e == cudaSuccess)

@@ -23,6 +23,7 @@ constexpr int kStaticMigrateMaxPageId = 1 << 18;
 // plan kernel at launch.
 constexpr int kRequestOverheadTilesDefault = 4;
 constexpr int kRequestOverheadTilesFp8 = 6;
+constexpr int kRequestOverheadTilesPair = 8;       // bf16 CTA-pair kernel
 constexpr int kRequestOverheadTilesFp8Pair = 12;   // CTA-pair kernel: tiles are cheaper, the per-request work is not
 
 // ---- workspace layout ------------------------------------------------------
@@ -205,6 +206,7 @@ void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *n
 cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream);
 cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_decode_umma_fp8_pair(const DecodeParams &p, cudaStream_t stream);
+cudaError_t launch_decode_umma_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
                                  const int32_t *split_list, cudaStream_t stream);
 cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *part_out,

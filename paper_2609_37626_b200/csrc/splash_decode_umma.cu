@@ -648,6 +648,7 @@ cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &sh
         if (p.num_groups == 2 && !(shape.flags & SPLASH_FLAG_NO_PAIR)) return launch_decode_umma_fp8_pair(p, stream);
         return launch_decode_umma_fp8(p, stream);
     }
+    if (p.num_groups == 2 && p.heads_per_group == 64 && !(shape.flags & SPLASH_FLAG_NO_PAIR)) return launch_decode_umma_pair(p, stream);
     alignas(64) CUtensorMap mkv, mq;
     const int n = p.heads_per_group;
     if (!make_map_4d(&mkv, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, p.kv_pool, kPage,

@@ -29,6 +29,7 @@
 // per barrier kind forwards the completed phase across the cluster, so that no softmax warp
 // pays for a cluster-scope release.  TMA loads of the peer complete on the leader's barriers.
 #include "splash_fp8.cuh"
+#include "splash_pair.cuh"
 
 namespace splash {
 
@@ -50,8 +51,9 @@ constexpr uint32_t kPageBytes = 9 * kSlab;          // 36,864
 constexpr uint32_t kPeerBytes = 4 * kSlab;          // the peer page's chunks this CTA multiplies: 16,384
 constexpr uint32_t kScaleBytes = 256;
 constexpr int kStages = 3;
-constexpr float kTau = 4.0f;
-constexpr float kLift = 4.75f;
+constexpr int kPrefetchAhead = 4;                    // supertiles between the L2 prefetch of a page and its use
+constexpr float kTau = 6.0f;
+constexpr float kLift = 2.75f;
 
 enum BarrierId {
     kBarKFull = 0,                        // [3] leader: both CTAs' pages landed (tx bytes of both)
@@ -90,57 +92,6 @@ static_assert(kOffQHi % 1024 == 0 && kOffP % 1024 == 0 && kOffTok % 16 == 0 && k
 // tensor memory: O two halves of dv x 128 columns, then 2 S buffers x 2 partials x 64 columns
 constexpr uint32_t kColO = 0, kColS = 256;
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// address of the same shared-memory offset in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// cluster-scope acquire for barriers the peer CTA arrives on
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    return done != 0;
-}
-static __device__ __noinline__ bool mbar_wait_cluster(const Ctx &ctx, uint32_t bar, uint32_t parity, int bar_id) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    if (*ctx.abort_flag) return false;
-    const unsigned long long start = global_timer_ns();
-    for (;;) {
-        for (int k = 0; k < 256; ++k)
-            if (mbar_try_wait_cluster(bar, parity)) return true;
-        if (*ctx.abort_flag) return false;
-        if (global_timer_ns() - start > kWaitLimitNs) {
-            *ctx.abort_flag = 1;
-            if (atomicCAS(ctx.status, 0, (int)SPLASH_DEVICE_TIMEOUT) == 0) {
-                ctx.status[1] = (int)blockIdx.x; ctx.status[2] = 200 + bar_id; ctx.status[3] = (int)threadIdx.x;
-            }
-            return false;
-        }
-    }
-}
-// TMA load whose completion bytes go to a barrier of the pair's leader CTA
-__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int c0, int c1,
-                                                 int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(leader_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
 __device__ __forceinline__ void umma_e4m3_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -148,19 +99,6 @@ __device__ __forceinline__ void umma_e4m3_pair(uint32_t d_tmem, uint64_t a_desc,
         "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// commit: arrive on the barrier at this offset in BOTH CTAs once all MMAs issued so far have retired
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((uint16_t)3) : "memory");
-}
-// 32 consecutive fp32 columns of this warp's 32 lanes
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-    tmem_ld16(taddr, *reinterpret_cast<float(*)[16]>(&v[0]));
-    tmem_ld16(taddr + 16, *reinterpret_cast<float(*)[16]>(&v[16]));
-}
-
-struct PairGeom { TileGeom a, b; bool has_b; };
-
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmap_page,
                             const __grid_constant__ CUtensorMap tmap_pair) {
@@ -258,6 +196,14 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                             const uint32_t sdst = sbase + kOffScale + stage * 2 * kScaleBytes;
                             if (in_a) bulk_load(sdst, p.kv_scales + (int64_t)page_a * kPage, kScaleBytes, bar(kBarScFull + stage));
                             if (in_b) bulk_load(sdst + kScaleBytes, p.kv_scales + (int64_t)page_b * kPage, kScaleBytes, bar(kBarScFull + stage));
+                            // A stage is held from its load until P.V has read it, about three supertiles, so the
+                            // load of supertile s + 3 starts only when the issuers are about to need it: have its
+                            // page in L2 by then.
+                            const int tf = ta + 2 * kPrefetchAhead + (int)rank;
+                            if (tf < seg.tile_end) {
+                                const int page_f = table[first_page + tf];
+                                if (page_f >= 0 && page_f < p.num_pool_pages) tma_prefetch_4d(&tmap_page, 0, 0, 0, page_f);
+                            }
                         }
                     } else {
                         ok = mbar_wait(ctx, bar(kBarQkDone + stage), ph, kBarQkDone + stage);

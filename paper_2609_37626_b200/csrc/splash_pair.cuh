@@ -1,0 +1,81 @@
+// Building blocks of the CTA-pair (tcgen05 cta_group::2) decode kernels: cluster addressing,
+// barrier arrivals and waits across the pair, TMA loads that complete on the leader's barrier.
+#pragma once
+
+#include "splash_umma.cuh"
+
+namespace splash {
+namespace umma {
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// cluster-scope acquire for barriers the peer CTA arrives on
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+static __device__ __noinline__ bool mbar_wait_cluster(const Ctx &ctx, uint32_t bar, uint32_t parity, int bar_id) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if (*ctx.abort_flag) return false;
+    const unsigned long long start = global_timer_ns();
+    for (;;) {
+        for (int k = 0; k < 256; ++k)
+            if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (*ctx.abort_flag) return false;
+        if (global_timer_ns() - start > kWaitLimitNs) {
+            *ctx.abort_flag = 1;
+            if (atomicCAS(ctx.status, 0, (int)SPLASH_DEVICE_TIMEOUT) == 0) {
+                ctx.status[1] = (int)blockIdx.x; ctx.status[2] = 200 + bar_id; ctx.status[3] = (int)threadIdx.x;
+            }
+            return false;
+        }
+    }
+}
+// TMA load whose completion bytes go to a barrier of the pair's leader CTA
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int c0, int c1,
+                                                 int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(leader_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+// pull a box into L2 ahead of the load that will need it
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap *map, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global [%0, {%1, %2, %3, %4}];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+// commit: arrive on the barrier at this offset in BOTH CTAs once all MMAs issued so far have retired
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+// 32 consecutive fp32 columns of this warp's 32 lanes
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    tmem_ld16(taddr, *reinterpret_cast<float(*)[16]>(&v[0]));
+    tmem_ld16(taddr + 16, *reinterpret_cast<float(*)[16]>(&v[16]));
+}
+
+// Page tiles of the two CTAs of a pair for one step, after the token shift.
+struct PairGeom { TileGeom a, b; bool has_b; };
+
+}  // namespace umma
+}  // namespace splash
