@@ -23,11 +23,10 @@
 // first half of N) and lane 64 + h (second half).
 //
 // Roles per CTA (576 threads): K-page + scale producer, 2 QK^T issuers and 2 P.V issuers
-// (leader CTA; in the peer CTA these four warps forward barrier arrivals to the leader), 8
-// softmax warps, 4 query converters, 1 producer of the peer chunks.  Barriers that the issuers
-// wait on live in the leader.  Warps of the peer arrive on their own CTA's copy; one thread
-// per barrier kind forwards the completed phase across the cluster, so that no softmax warp
-// pays for a cluster-scope release.  TMA loads of the peer complete on the leader's barriers.
+// (leader CTA only), 8 softmax warps, 4 query converters, 1 producer of the peer chunks.
+// Barriers that the issuers wait on live in the leader; the peer's warps arrive on them across
+// the cluster (relaxed arrivals: what they announce is already in place on the peer's SM), and
+// TMA loads of the peer complete on them too.
 #include "splash_fp8.cuh"
 #include "splash_pair.cuh"
 
@@ -62,7 +61,8 @@ enum BarrierId {
     kBarStageEmpty = kBarVFull + kStages, // [3] P.V of the stage retired (multicast commit): stage, its scales and
                                           //     the P buffer are free, O is up to date
     kBarScFull = kBarStageEmpty + kStages,// [3] local: scale pages of the stage landed
-    kBarQFull = kBarScFull + kStages,     // query operands written (leader: of both CTAs)
+    kBarQFull = kBarScFull + kStages,     // leader: query operands of both CTAs written
+    kBarQLocal,                           // local: this CTA's query scales written
     kBarQEmpty,                           // last QK^T of the request retired (multicast commit)
     kBarQsRead,                           // local: the softmax warps have picked up the request's query scales
     kBarSFull,                            // [2] S buffer written (multicast commit)
@@ -114,23 +114,26 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
     Ctx ctx{misc + 1, p.status};
     auto bar = [&](int id) -> uint32_t { return sbase + kOffBar + 8u * (uint32_t)id; };
     auto leader_bar = [&](int id) -> uint32_t { return map_to_cta(sbase + kOffBar + 8u * (uint32_t)id, 0); };
+    // one arrival of a warp of either CTA on a barrier that lives in the leader
+    auto arrive_on_leader = [&](int id) {
+        if (rank == 0) mbar_arrive(bar(id));
+        else mbar_arrive_cluster_relaxed(leader_bar(id));
+    };
 
     if (tid == 0) {
-        // barriers the leader's issuers wait on count this CTA's warps, plus, in the leader, the
-        // one forwarded arrival that stands for the peer's warps
-        const uint32_t fwd = rank == 0 ? 1u : 0u;
+        // barriers the leader's issuers wait on count the warps of both CTAs (the peer's copies are unused)
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(kBarKFull + s), 1); mbar_init(bar(kBarQkDone + s), kQkWarps);
             mbar_init(bar(kBarVFull + s), 1); mbar_init(bar(kBarStageEmpty + s), kPvWarps);
             mbar_init(bar(kBarScFull + s), 1);
         }
-        mbar_init(bar(kBarQFull), kConvertWarps + fwd); mbar_init(bar(kBarQEmpty), kQkWarps);
+        mbar_init(bar(kBarQFull), 2 * kConvertWarps); mbar_init(bar(kBarQLocal), kConvertWarps); mbar_init(bar(kBarQEmpty), kQkWarps);
         mbar_init(bar(kBarQsRead), kSoftmaxWarps);
         for (int b = 0; b < 2; ++b) {
-            mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kSoftmaxWarps + fwd);
-            mbar_init(bar(kBarPFull + b), kSoftmaxWarps + fwd);
+            mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), 2 * kSoftmaxWarps);
+            mbar_init(bar(kBarPFull + b), 2 * kSoftmaxWarps);
         }
-        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kSoftmaxWarps + fwd);
+        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), 2 * kSoftmaxWarps);
         misc[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -145,6 +148,7 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
     const uint32_t tmem_base = misc[0];
     grid_dependency_wait();                               // the plan kernel's output is read from here on
     const long long t_start = clock64();
+    const unsigned long long ns_start = global_timer_ns();
 
     SegmentIter it;
     it.init(p, worker);
@@ -292,32 +296,8 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                 ++seg_it;
             }
         }
-    } else if (warp >= kWarpQk && warp < kWarpPv + kPvWarps) {
-        // ===================================================== peer CTA: forward completed phases to the leader
-        // one thread per barrier kind waits for its own CTA's warps and arrives once on the leader's barrier
-        if (lane == 0) {
-            const int kind = warp - kWarpQk;              // 0: S read, 1: P written, 2: query written, 3: O drained
-            uint32_t st_it = 0, seg_it = 0;
-            bool ok = true;
-            while (ok && it.next(p, seg)) {
-                const int nsuper = (seg.tile_end - seg.tile_begin + 1) >> 1;
-                if (kind == 2) {
-                    ok = mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
-                    if (ok) mbar_arrive_cluster(leader_bar(kBarQFull));
-                } else if (kind < 2) {
-                    const int id = kind == 0 ? kBarSEmpty : kBarPFull;
-                    for (int s = 0; ok && s < nsuper; ++s, ++st_it) {
-                        const uint32_t b = st_it & 1;
-                        ok = mbar_wait(ctx, bar(id + b), (st_it >> 1) & 1, id + b);
-                        if (ok) mbar_arrive_cluster(leader_bar(id + b));
-                    }
-                } else {
-                    ok = mbar_wait(ctx, bar(kBarOEmpty), seg_it & 1, kBarOEmpty);
-                    if (ok) mbar_arrive_cluster(leader_bar(kBarOEmpty));
-                }
-                ++seg_it;
-            }
-        }
+    } else if (warp >= kWarpQk && warp < kWarpSoftmax) {
+        // the issuer warps of the peer CTA have nothing to do
     } else if (warp >= kWarpConvert && warp < kWarpConvert + kConvertWarps) {
         // ===================================================== query converters (this CTA's 64 heads)
         const int ct = (warp - kWarpConvert) * 32 + lane;   // 0..127
@@ -384,11 +364,11 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                 }
                 fence_proxy_async();
                 __syncwarp();
-                // The softmax warps wait on QFull by phase parity, so it must never complete two phases
+                // The softmax warps wait on QLocal by phase parity, so it must never complete two phases
                 // ahead of them: hold this request's arrival until they have entered the previous one.
                 if (lane == 0) {
                     if (seg_it > 0) ok = mbar_wait(ctx, bar(kBarQsRead), (seg_it - 1) & 1, kBarQsRead);
-                    mbar_arrive(bar(kBarQFull));
+                    mbar_arrive(bar(kBarQLocal)); arrive_on_leader(kBarQFull);
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             }
@@ -422,7 +402,7 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
         // thread still meets the named barriers -- once the CTA aborts, waits return at once.
         bool ok = true;
         while (it.next(p, seg)) {
-            ok &= mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
+            ok &= mbar_wait(ctx, bar(kBarQLocal), seg_it & 1, kBarQLocal);
             const float cq = scale_log2 * qs_s[(seg_it & 3) * kN + hd];
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarQsRead));
@@ -454,7 +434,7 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                 }
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarSEmpty + b));
+                if (lane == 0) arrive_on_leader(kBarSEmpty + b);
                 const uint32_t valid = __ballot_sync(0xffffffffu, 32 * cf + lane >= geo.r_lo && 32 * cf + lane < geo.r_hi);
                 float mt = -INFINITY;
                 if (valid == 0xffffffffu) {
@@ -538,7 +518,7 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                 fence_proxy_async();
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPFull + b));
+                if (lane == 0) arrive_on_leader(kBarPFull + b);
             }
             // ---- row sums of the 4 threads of a head
             xch[hd * 4 + slot4] = l;
@@ -594,13 +574,16 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
             }
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarOEmpty));
+            if (lane == 0) arrive_on_leader(kBarOEmpty);
             ++seg_it;
         }
     }
 
     fill_empty_requests(p, worker, head0, kN, tid, kThreads);
-    if (p.trace != nullptr && tid == 0) p.trace[512 + blockIdx.x] = clock64() - t_start;   // per-CTA cycles
+    if (p.trace != nullptr && tid == 0) {   // per-CTA cycles and nanoseconds
+        p.trace[512 + blockIdx.x] = clock64() - t_start;
+        if (blockIdx.x < 256) p.trace[768 + blockIdx.x] = (long long)(global_timer_ns() - ns_start);
+    }
 
     // ---- teardown: nobody leaves while its partner may still touch its shared memory or barriers
     if (*ctx.abort_flag) {

@@ -21,11 +21,10 @@
 // lane 64 + h (second half).
 //
 // Roles per CTA (512 threads): page + query producer, 4 QK^T issuers and 2 P.V issuers
-// (leader CTA; in the peer CTA three of these warps forward barrier arrivals to the
-// leader), 8 softmax warps, 1 producer of the peer chunks.  Barriers that the issuers wait
-// on live in the leader.  Warps of the peer arrive on their own CTA's copy; one thread per
-// barrier kind forwards the completed phase across the cluster, so that no softmax warp pays
-// for a cluster-scope release.  TMA loads of the peer complete on the leader's barriers.
+// (leader CTA only), 8 softmax warps, 1 producer of the peer chunks.  Barriers that the
+// issuers wait on live in the leader; the peer's warps arrive on them across the cluster
+// (relaxed arrivals: what they announce is already in place on the peer's SM), and TMA loads
+// of the peer complete on them too.
 #include "splash_pair.cuh"
 
 namespace splash {
@@ -106,21 +105,24 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
     Ctx ctx{misc + 1, p.status};
     auto bar = [&](int id) -> uint32_t { return sbase + kOffBar + 8u * (uint32_t)id; };
     auto leader_bar = [&](int id) -> uint32_t { return map_to_cta(sbase + kOffBar + 8u * (uint32_t)id, 0); };
+    // one arrival of a warp of either CTA on a barrier that lives in the leader
+    auto arrive_on_leader = [&](int id) {
+        if (rank == 0) mbar_arrive(bar(id));
+        else mbar_arrive_cluster_relaxed(leader_bar(id));
+    };
 
     if (tid == 0) {
-        // barriers the leader's issuers wait on count this CTA's warps, plus, in the leader, the
-        // one forwarded arrival that stands for the peer's warps
-        const uint32_t fwd = rank == 0 ? 1u : 0u;
+        // barriers the leader's issuers wait on count the warps of both CTAs (the peer's copies are unused)
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(kBarKFull + s), 1); mbar_init(bar(kBarQkDone + s), kQkWarps);
             mbar_init(bar(kBarVFull + s), 1); mbar_init(bar(kBarStageEmpty + s), kPvWarps);
         }
         mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), kQkWarps);
         for (int b = 0; b < 2; ++b) {
-            mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kSoftmaxWarps + fwd);
-            mbar_init(bar(kBarPFull + b), kSoftmaxWarps + fwd);
+            mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), 2 * kSoftmaxWarps);
+            mbar_init(bar(kBarPFull + b), 2 * kSoftmaxWarps);
         }
-        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kSoftmaxWarps + fwd);
+        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), 2 * kSoftmaxWarps);
         misc[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -135,6 +137,7 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
     const uint32_t tmem_base = misc[0];
     grid_dependency_wait();                               // the plan kernel's output is read from here on
     const long long t_start = clock64();
+    const unsigned long long ns_start = global_timer_ns();
 
     SegmentIter it;
     it.init(p, worker);
@@ -267,27 +270,7 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
             }
         }
     } else if (warp >= kWarpQk && warp < kWarpSoftmax) {
-        // ===================================================== peer CTA: forward completed phases to the leader
-        // one thread per barrier kind waits for its own CTA's warps and arrives once on the leader's barrier
-        const int kind = warp - kWarpQk;                  // 0: S read, 1: P written, 2: O drained
-        if (lane == 0 && kind < 3) {
-            uint32_t kv_it = 0, seg_it = 0;
-            bool ok = true;
-            while (ok && it.next(p, seg)) {
-                if (kind < 2) {
-                    const int id = kind == 0 ? kBarSEmpty : kBarPFull;
-                    for (int tile = seg.tile_begin; ok && tile < seg.tile_end; ++tile, ++kv_it) {
-                        const uint32_t b = kv_it & 1;
-                        ok = mbar_wait(ctx, bar(id + b), (kv_it >> 1) & 1, id + b);
-                        if (ok) mbar_arrive_cluster(leader_bar(id + b));
-                    }
-                } else {
-                    ok = mbar_wait(ctx, bar(kBarOEmpty), seg_it & 1, kBarOEmpty);
-                    if (ok) mbar_arrive_cluster(leader_bar(kBarOEmpty));
-                }
-                ++seg_it;
-            }
-        }
+        // the issuer warps of the peer CTA have nothing to do
     } else {
         // ===================================================== softmax + epilogue warps
         // S partial layout per CTA: TMEM lane L < 64 = head L, tokens of half-page 0 in 32 columns;
@@ -332,7 +315,7 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                 }
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarSEmpty + b));
+                if (lane == 0) arrive_on_leader(kBarSEmpty + b);
                 // rows outside [r_lo, r_hi) are zero fill or tokens outside the request's range
                 if (row0 < geo.r_lo || row0 + 16 > geo.r_hi) {
 #pragma unroll
@@ -392,7 +375,7 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                 fence_proxy_async();
                 tcgen05_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPFull + b));
+                if (lane == 0) arrive_on_leader(kBarPFull + b);
             }
             // ---- row sums of the 4 threads of a head
             xch[hd * 4 + slot4] = l;
@@ -447,13 +430,16 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
             }
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarOEmpty));
+            if (lane == 0) arrive_on_leader(kBarOEmpty);
             ++seg_it;
         }
     }
 
     fill_empty_requests(p, worker, head0, kN, tid, kThreads);
-    if (p.trace != nullptr && tid == 0) p.trace[512 + blockIdx.x] = clock64() - t_start;   // per-CTA cycles
+    if (p.trace != nullptr && tid == 0) {   // per-CTA cycles and nanoseconds
+        p.trace[512 + blockIdx.x] = clock64() - t_start;
+        if (blockIdx.x < 256) p.trace[768 + blockIdx.x] = (long long)(global_timer_ns() - ns_start);
+    }
 
     // ---- teardown: nobody leaves while its partner may still touch its shared memory or barriers
     if (*ctx.abort_flag) {

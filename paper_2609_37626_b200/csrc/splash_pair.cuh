@@ -24,6 +24,15 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Arrival on a barrier of the other CTA that carries no data with it: a release at cluster scope
+// stalls the arriving thread for ~300 cycles and takes ~500 to land, the relaxed form ~20 and
+// ~200.  It is used where what the arrival announces is already in place on this SM when it is
+// sent -- shared-memory writes followed by fence.proxy.async, tensor-memory reads followed by
+// tcgen05.wait::ld -- and is consumed on this SM, by MMAs that the pair's leader issues only
+// after it has seen the arrival.
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // cluster-scope acquire for barriers the peer CTA arrives on
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
     uint32_t done;
