@@ -17,6 +17,9 @@
 // retired they are overwritten with the peer half-page's chunks 4 n + 2 r, 4 n + 2 r + 1.
 // The MMAs over half-page g then start at slot 4 n + 2 g in both CTAs.  That second load
 // (L2 hits: the peer has just read the page) hides behind the softmax of the tile.
+// P of a tile is written in two [64 heads x 32 tokens] halves: the first into the stage's rope
+// chunk slot, which nothing reads after QK^T (that is what makes room for a fourth stage), the
+// second into a small buffer of its own.
 // Accumulators: CTA r holds its 64 heads; a head's row is TMEM lane h (first half of N) and
 // lane 64 + h (second half).
 //
@@ -47,16 +50,16 @@ constexpr uint32_t kStageBytes = 9 * kSlab;         // 36,864
 constexpr uint32_t kPeerBytes = 4 * kSlab;          // the peer half-page's chunks this CTA multiplies: 16,384
 constexpr uint32_t kQSlab = kN * 128;               // one chunk of the query rows: 64 heads x 128 B
 constexpr uint32_t kQBytes = 9 * kQSlab;            // 73,728
-constexpr uint32_t kPBytes = kN * 128;              // 64 heads x 64 tokens bf16
-constexpr int kStages = 3;
+constexpr uint32_t kPHalfBytes = kN * 64;           // P of one half-page: 64 heads x 32 tokens bf16
+constexpr int kStages = 4;
 constexpr int kPrefetchAhead = 4;                   // tiles between the L2 prefetch of a page and its use
 constexpr float kTau = 8.0f;                        // O is rescaled only when a row maximum grows by more than 2^8
 
 enum BarrierId {
-    kBarKFull = 0,                        // [3] leader: both half-pages landed (tx bytes of both CTAs)
-    kBarQkDone = kBarKFull + kStages,     // [3] QK^T of the stage retired (multicast commit): peer chunks may land
-    kBarVFull = kBarQkDone + kStages,     // [3] leader: both CTAs' peer chunks landed
-    kBarStageEmpty = kBarVFull + kStages, // [3] P.V of the stage retired (multicast commit): stage and P buffer
+    kBarKFull = 0,                        // [4] leader: both half-pages landed (tx bytes of both CTAs)
+    kBarQkDone = kBarKFull + kStages,     // [4] QK^T of the stage retired (multicast commit): peer chunks may land
+    kBarVFull = kBarQkDone + kStages,     // [4] leader: both CTAs' peer chunks landed
+    kBarStageEmpty = kBarVFull + kStages, // [4] P.V of the stage retired (multicast commit): stage and P buffers
                                           //     are free, O is up to date
     kBarQFull = kBarStageEmpty + kStages, // leader: query rows of both CTAs landed
     kBarQEmpty,                           // last QK^T of the request retired (multicast commit)
@@ -68,17 +71,17 @@ enum BarrierId {
     kNumBarriers
 };
 
-constexpr uint32_t kOffK = 0;                                   // [3 stages] 9 chunk slots of 32 tokens
+constexpr uint32_t kOffK = 0;                                   // [4 stages] 9 chunk slots of 32 tokens
 constexpr uint32_t kOffQ = kOffK + kStages * kStageBytes;       // 9 chunks x 64 heads x 128 B
-constexpr uint32_t kOffP = kOffQ + kQBytes;                     // [2 buffers] 64 heads x 128 B
-constexpr uint32_t kOffAlpha = kOffP + 2 * kPBytes;             // float [64]
+constexpr uint32_t kOffP1 = kOffQ + kQBytes;                    // [2 buffers] P of half-page 1: 64 heads x 64 B
+constexpr uint32_t kOffAlpha = kOffP1 + 2 * kPHalfBytes;            // float [64]
 constexpr uint32_t kOffL = kOffAlpha + kN * 4;                  // float [64]
 constexpr uint32_t kOffXch = kOffL + kN * 4;                    // float [64][4]
 constexpr uint32_t kOffBar = kOffXch + kN * 16;
 constexpr uint32_t kOffMisc = (kOffBar + kNumBarriers * 8 + 15) / 16 * 16;
 constexpr uint32_t kSmemBytes = kOffMisc + 32;
 static_assert(kSmemBytes <= 232448, "shared memory overflow");
-static_assert(kOffQ % 1024 == 0 && kOffP % 1024 == 0 && kSlab % 1024 == 0, "swizzle atoms need 1024-byte alignment");
+static_assert(kOffQ % 1024 == 0 && kOffP1 % 1024 == 0 && kSlab % 1024 == 0, "swizzle atoms need 1024-byte alignment");
 // tensor memory: O two halves of dv x 128 columns, then 2 S buffers x 4 partials x 32 columns
 constexpr uint32_t kColO = 0, kColS = 256;
 
@@ -253,13 +256,14 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                     if (!ok) break;
                     tcgen05_fence_after();
                     const uint32_t k0 = sbase + kOffK + stage * kStageBytes;
-                    const uint32_t p0 = sbase + kOffP + pb * kPBytes;
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        // 16 tokens of half-page g.  A: P rows (heads), 32 bytes of the 128-byte row;
+                        // 16 tokens of half-page g.  A: P rows (heads), 32 bytes of the 64-byte row (g = 0: in the
+                        // stage's rope slot, g = 1: in its own buffer);
                         // B: slots 4n + 2g, + 1 (two 64-wide dv chunks, LBO apart), 16 token rows, MN-major
                         const int g = j >> 1;
-                        uint64_t da = make_desc(p0 + j * 32, 16, 1024);
+                        const uint32_t p0 = g == 0 ? k0 + 8 * kSlab : sbase + kOffP1 + pb * kPHalfBytes;
+                        uint64_t da = make_desc_sw64(p0 + (j & 1) * 32, 16, 512);
                         uint64_t db = make_desc(k0 + (4 * n + 2 * g) * kSlab + (j & 1) * 2048, kSlab, 1024);
                         umma_bf16_pair(tmem_base + kColO + n * 128, da, db, kIdescPV, (tile != seg.tile_begin) || j != 0);
                     }
@@ -344,7 +348,7 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                     pk[j >> 1] = pack_bf16x2(u0, u1);
                 }
                 const bool rescale = named_bar_or<1, kSoftmaxWarps * 32>(grew);
-                // P.V of the tile that last used this P buffer (two back) must be done; a rescale
+                // P.V of the tile that last used the P buffer of half-page 1 (two back) must be done; a rescale
                 // of O also needs the previous tile's P.V
                 if (kv_it > 1) ok &= mbar_wait(ctx, bar(kBarStageEmpty + (kv_it - 2) % kStages), ((kv_it - 2) / kStages) & 1, kBarStageEmpty);
                 if (rescale && tile != seg.tile_begin) {
@@ -366,11 +370,10 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                     tmem_wait_st();
                 }
                 {
-                    // P: K-major, 128-byte swizzle; row = head, 32 bytes at token row0: two 16-byte chunks
-                    uint8_t *prow = smem + kOffP + b * kPBytes + hd * 128;
-                    const uint32_t ci = (uint32_t)(row0 >> 3);
-                    *reinterpret_cast<uint4 *>(prow + (((ci) ^ (uint32_t)(hd & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                    *reinterpret_cast<uint4 *>(prow + (((ci + 1) ^ (uint32_t)(hd & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    // P of this half-page: K-major, 64-byte swizzle; row = head, bytes [32 cf, 32 cf + 32)
+                    uint8_t *ph = g == 0 ? smem + kOffK + (kv_it % kStages) * kStageBytes + 8 * kSlab : smem + kOffP1 + b * kPHalfBytes;
+                    *reinterpret_cast<uint4 *>(ph + sw64((uint32_t)hd, (uint32_t)(32 * cf))) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4 *>(ph + sw64((uint32_t)hd, (uint32_t)(32 * cf + 16))) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                 }
                 fence_proxy_async();
                 tcgen05_fence_before();

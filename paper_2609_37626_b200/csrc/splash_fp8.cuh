@@ -64,10 +64,5 @@ __device__ __forceinline__ void split4(float x, float &hi, float &lo) {
     lo = x - hi;
 }
 
-// byte offset of (row, byte column) inside a [rows][64 B] slab in the 64-byte swizzle
-__device__ __forceinline__ uint32_t sw64(uint32_t row, uint32_t col_byte) {
-    return row * 64 + ((((col_byte >> 4) ^ (row >> 1)) & 3) << 4) + (col_byte & 15);
-}
-
 }  // namespace umma
 }  // namespace splash

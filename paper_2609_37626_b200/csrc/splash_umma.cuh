@@ -221,6 +221,11 @@ __device__ __forceinline__ uint64_t make_desc_sw64(uint32_t saddr, uint32_t lbo_
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (4ull << 61);
 }
 
+// byte offset of (row, byte column) inside a [rows][64 B] slab in the 64-byte swizzle
+__device__ __forceinline__ uint32_t sw64(uint32_t row, uint32_t col_byte) {
+    return row * 64 + ((((col_byte >> 4) ^ (row >> 1)) & 3) << 4) + (col_byte & 15);
+}
+
 // Instruction descriptor: fp32 accumulate, bf16 x bf16.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, int b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
