@@ -24,7 +24,7 @@ constexpr int kStaticMigrateMaxPageId = 1 << 18;
 constexpr int kRequestOverheadTilesDefault = 4;
 constexpr int kRequestOverheadTilesFp8 = 6;
 constexpr int kRequestOverheadTilesPair = 8;       // bf16 CTA-pair kernel
-constexpr int kRequestOverheadTilesFp8Pair = 12;   // CTA-pair kernel: tiles are cheaper, the per-request work is not
+constexpr int kRequestOverheadTilesFp8Pair = 14;   // CTA-pair kernel: tiles are cheaper, the per-request work is not
 
 // ---- workspace layout ------------------------------------------------------
 // [0, 64)                 status block (int32 x 16): [0] status, [1..3] detail

@@ -645,7 +645,10 @@ void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *n
 cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream) {
     if (shape.kv_dtype != SPLASH_KV_BF16) {
         // slices of more than 64 heads run on CTA pairs (cta_group::2) unless the caller opts out
-        if (p.num_groups == 2 && !(shape.flags & SPLASH_FLAG_NO_PAIR)) return launch_decode_umma_fp8_pair(p, stream);
+        if (p.num_groups == 2 && !(shape.flags & SPLASH_FLAG_NO_PAIR)) {
+            const cudaError_t e = launch_decode_umma_fp8_pair(p, stream);
+            if (e != cudaErrorNotSupported) return e;      // output rows not 16-byte aligned: no TMA stores
+        }
         return launch_decode_umma_fp8(p, stream);
     }
     if (p.num_groups == 2 && p.heads_per_group == 64 && !(shape.flags & SPLASH_FLAG_NO_PAIR)) return launch_decode_umma_pair(p, stream);

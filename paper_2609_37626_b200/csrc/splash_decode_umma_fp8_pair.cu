@@ -101,7 +101,8 @@ __device__ __forceinline__ void umma_e4m3_pair(uint32_t d_tmem, uint64_t a_desc,
 }
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmap_page,
-                            const __grid_constant__ CUtensorMap tmap_pair) {
+                            const __grid_constant__ CUtensorMap tmap_pair, const __grid_constant__ CUtensorMap tmap_out,
+                            const __grid_constant__ CUtensorMap tmap_part) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -540,43 +541,46 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
             // take one n each.
             ok &= mbar_wait(ctx, bar(kBarOFull), seg_it & 1, kBarOFull);
             tcgen05_fence_after();
-            // Read in the accumulator fragment layout (16 lanes at a time: thread T gets rows T/4 and
-            // T/4 + 8, two columns of every eight), so that a store instruction writes whole 32-byte
-            // sectors: 8 rows x 4 lanes x 8 bytes.
+            // Every warp drains its [32 heads x 128 dv] block in four rounds of 32 columns through a
+            // 4 KB tile of the P buffers (idle now: the last P.V has retired): a thread writes its row
+            // in the 128-byte swizzle (conflict-free), one TMA store moves the tile out in whole lines
+            // and clips the rows past the head slice.
             {
-                float *obase;
-                int64_t ostride;
-                if (seg.slot < 0) {
-                    obase = p.out + (int64_t)seg.request * p.out_stride_request + (int64_t)head0 * p.out_stride_head;
-                    ostride = p.out_stride_head;
-                } else {
-                    obase = p.partial_out + ((int64_t)seg.slot * h + (head0 - p.head_begin)) * kDV;
-                    ostride = kDV;
-                }
                 const int n = cf;
-                const int dv0 = 256 * n + 128 * pg + 2 * (lane & 3);
-                const int nvalid = min(kN, p.head_end - head0);
+                const int dv0 = 256 * n + 128 * pg;
+                const int row0 = 32 * (q4 & 1);
+                uint8_t *stg = smem + kOffP + sw * 4096;
+                const float inv_l = l_s[hd];
+                const bool final_out = seg.slot < 0;
+                const CUtensorMap *omap = final_out ? &tmap_out : &tmap_part;
+                const int rowc = final_out ? head0 + row0 : head0 - p.head_begin + row0;
+                const int outer = final_out ? seg.request : seg.slot;
 #pragma unroll 1
-                for (int hc = 0; hc < 4; ++hc) {
-                    const int half = hc >> 1, c = hc & 1;
-                    const int hA = 32 * (q4 & 1) + 16 * half + (lane >> 2), hB = hA + 8;
+                for (int c = 0; c < 4; ++c) {
                     float o[32];
-                    tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * q4 + 16 * half) << 16) + kColO + n * 128 + c * 64, o);
-                    const float iA = l_s[hA], iB = l_s[hB];
-                    float *rowA = obase + (int64_t)hA * ostride + dv0 + c * 64, *rowB = obase + (int64_t)hB * ostride + dv0 + c * 64;
+                    tmem_ld32(tmem_base + lane_addr + kColO + n * 128 + c * 32, o);
                     tmem_wait_ld();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        if (hA < nvalid) *reinterpret_cast<float2 *>(rowA + 8 * k) = make_float2(o[4 * k] * iA, o[4 * k + 1] * iA);
-                        if (hB < nvalid) *reinterpret_cast<float2 *>(rowB + 8 * k) = make_float2(o[4 * k + 2] * iB, o[4 * k + 3] * iB);
+                    if (c > 0) {                          // the previous round's store has read the tile
+                        if (lane == 0) bulk_wait_group_read();
+                        __syncwarp();
                     }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        *reinterpret_cast<float4 *>(stg + lane * 128 + ((i ^ (lane & 7)) << 4)) =
+                            make_float4(o[4 * i] * inv_l, o[4 * i + 1] * inv_l, o[4 * i + 2] * inv_l, o[4 * i + 3] * inv_l);
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) { tma_store_3d(omap, smem_u32(stg), dv0 + 32 * c, rowc, outer); bulk_commit_group(); }
                 }
+                if (lane == 0) bulk_wait_group_read();    // the tile goes back to being a P buffer
+                __syncwarp();
             }
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) arrive_on_leader(kBarOEmpty);
             ++seg_it;
         }
+        if (lane == 0) bulk_wait_group();                 // this warp's output stores have completed
     }
 
     fill_empty_requests(p, worker, head0, kN, tid, kThreads);
@@ -610,6 +614,16 @@ cudaError_t launch_decode_umma_fp8_pair(const DecodeParams &p, cudaStream_t stre
     if (!make_map_4d(&mpair, CU_TENSOR_MAP_DATA_TYPE_UINT8, CU_TENSOR_MAP_SWIZZLE_64B, p.kv_pool, kPage, pages,
                      (uint64_t)kDQK, 64, (uint64_t)kPage * kDQK, 64, 2))
         return cudaErrorInvalidValue;
+    // output maps: (512 dv, heads below head_end, requests) over `out`, (512, h, partial slots) over the workspace
+    alignas(64) CUtensorMap mout, mpart;
+    if (p.out_stride_head % 4 || p.out_stride_request % 4) return cudaErrorNotSupported;   // rows must start on 16-byte boundaries
+    const uint64_t hbytes = (uint64_t)p.out_stride_head * 4;
+    if (!make_store_map_3d(&mout, p.out, kDV, (uint64_t)p.head_end, (uint64_t)p.B, hbytes,
+                           p.B > 1 ? (uint64_t)p.out_stride_request * 4 : hbytes * (uint64_t)p.head_end, 32))
+        return cudaErrorNotSupported;
+    const uint64_t h = (uint64_t)(p.head_end - p.head_begin);
+    if (!make_store_map_3d(&mpart, p.partial_out, kDV, h, (uint64_t)2 * p.num_workers, (uint64_t)kDV * 4, h * kDV * 4, 32))
+        return cudaErrorInvalidValue;
     static bool configured[64] = {};
     cudaError_t e = cudaSuccess;
     if (first_use_on_device(configured)) {
@@ -623,7 +637,7 @@ cudaError_t launch_decode_umma_fp8_pair(const DecodeParams &p, cudaStream_t stre
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, decode_umma_fp8_pair_kernel, p, mpage, mpair);
+    e = cudaLaunchKernelEx(&cfg, decode_umma_fp8_pair_kernel, p, mpage, mpair, mout, mpart);
     count_launch();
     return e;
 }
