@@ -207,7 +207,12 @@ class GpuBench:
                     "unit": "TFLOP/s"}
         roof["frac"] = roof["achieved"] / roof["peak"]
         roof["traffic"] = traffic_table.get(name)
-        roof.update({"kernel": "decode_umma_kernel", "kernel_ms": dec_ms, "peak_source": peaks["source"],
+        hs = w.head_end - w.head_begin
+        if hs > 64:     # slices of more than 64 heads run on CTA pairs
+            kernel = "decode_umma_fp8_pair_kernel" if fp8 else "decode_umma_pair_kernel"
+        else:
+            kernel = "decode_umma_fp8_kernel" if fp8 else "decode_umma_kernel<%d>" % (16 if hs <= 16 else 32 if hs <= 32 else 64)
+        roof.update({"kernel": kernel, "kernel_ms": dec_ms, "peak_source": peaks["source"],
                      "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
                      "roofline_ms": max(t_hbm, t_tensor) * 1e3,
                      "achieved_gbs": alg_bytes / (dec_ms * 1e-3) / 1e9,
