@@ -336,14 +336,15 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                 const float qs = amax > 0.f ? amax * (1.0f / 448.0f) : 1.0f;
                 const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
                 if (part == 0) qs_s[(seg_it & 3) * kN + hd] = qs;
-                // the operand buffers are free once the last QK^T of the previous request has retired
-                ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
-                if (!ok) break;
-#pragma unroll 1
-                for (int v0 = 0; v0 < 36; v0 += 9) {
-                    uint4 x[9];
+                // second pass in four batches of nine 16-byte loads, a batch ahead: the first batch is in
+                // flight while this warp waits for the operand buffers, which are free once the last
+                // QK^T of the previous request has retired
+                uint4 xa[9], xb[9];
+                auto load_batch = [&](uint4 (&x)[9], int v0) {
 #pragma unroll
                     for (int i = 0; i < 9; ++i) x[i] = live ? __ldg(src + v0 + i) : make_uint4(0u, 0u, 0u, 0u);
+                };
+                auto convert_batch = [&](const uint4 (&x)[9], int v0) {
 #pragma unroll
                     for (int i = 0; i < 9; ++i) {
                         const uint32_t w[4] = {x[i].x, x[i].y, x[i].z, x[i].w};
@@ -362,7 +363,14 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                         *reinterpret_cast<uint2 *>(smem + kOffQLo + off) =
                             make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
                     }
-                }
+                };
+                load_batch(xa, 0);
+                ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
+                if (!ok) break;
+                load_batch(xb, 9);  convert_batch(xa, 0);
+                load_batch(xa, 18); convert_batch(xb, 9);
+                load_batch(xb, 27); convert_batch(xa, 18);
+                convert_batch(xb, 27);
                 fence_proxy_async();
                 __syncwarp();
                 // The softmax warps wait on QLocal by phase parity, so it must never complete two phases
