@@ -43,7 +43,6 @@ using namespace umma;
 
 constexpr int kThreads = 288;                      // 9 warps: producer, 4 MMA issuers, 4 softmax
 constexpr int kMmaWarps = 4;
-constexpr int kNumSoftmaxThreads = 128;
 constexpr int kNumSoftmaxWarps = 4;                // barriers fed by the softmax role count one arrival per warp
 constexpr int kChunks = 9;                         // 576 / 64-element (128 B) chunks
 constexpr uint32_t kSlabBytes = 64 * 128;          // one chunk of one page: 64 tokens x 128 B
@@ -328,8 +327,10 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
         const float scale_log2 = p.softmax_scale * kLog2e;
         constexpr int kOwn = N >= 32 ? N / 32 : 1;
         uint32_t s_it = 0, p_it = 0, seg_it = 0;
+        // A failed (timed-out) wait only clears `ok`: the role keeps walking its tiles so that every thread still
+        // meets the named barriers -- once the CTA aborts, waits return at once.
         bool ok = true;
-        while (ok && it.next(p, seg)) {
+        while (it.next(p, seg)) {
             if (st < N) m_s[st] = -INFINITY;
             // heads-on-M: this thread's two heads (reference maxima; partial row sums over its tokens)
             const int hA = 16 * q4 + (lane >> 2);
@@ -340,12 +341,11 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             softmax_bar_sync();
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;
-            for (int i = 0; ok && i < ntiles; ++i) {
+            for (int i = 0; i < ntiles; ++i) {
                 const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + seg.tile_begin + i) * kPage);
                 const bool valid = lane < 16 && row >= g.r_lo && row < g.r_hi;
                 const uint32_t b = s_it % L::kSBufs;
-                ok = mbar_wait(ctx, bar(kBarSFull + b), (s_it / L::kSBufs) & 1, kBarSFull + b);
-                if (!ok) break;
+                ok &= mbar_wait(ctx, bar(kBarSFull + b), (s_it / L::kSBufs) & 1, kBarSFull + b);
                 if (st == 0) mark(s_it, 4);
                 tcgen05_fence_after();
                 if constexpr (L::kHeadsOnM) {
@@ -403,8 +403,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 // P.V of the previous tile must be done with the P buffer and with O^T
                 if (s_it > 0) {
                     const uint32_t prev = s_it - 1;
-                    ok = mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
-                    if (!ok) break;
+                    ok &= mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
                 }
                 tcgen05_fence_after();
                 if (rescale && i > 0) {
@@ -489,8 +488,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 // P.V of the previous tile must be done with the P buffer and with O^T
                 if (s_it > 0) {
                     const uint32_t prev = s_it - 1;
-                    ok = mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
-                    if (!ok) break;
+                    ok &= mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
                 }
                 tcgen05_fence_after();
                 if (rescale && i > 0) {
@@ -524,7 +522,6 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 if (lane == 0) mbar_arrive(bar(kBarPFull));
                 ++s_it; ++p_it;
             }
-            if (!ok) break;
             if constexpr (L::kHeadsOnM) {
                 lA += __shfl_xor_sync(0xffffffffu, lA, 1); lB += __shfl_xor_sync(0xffffffffu, lB, 1);
                 lA += __shfl_xor_sync(0xffffffffu, lA, 2); lB += __shfl_xor_sync(0xffffffffu, lB, 2);
@@ -563,8 +560,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             }
             softmax_bar_sync();
             // ---- epilogue: O^T block j holds dv = 128 j + TMEM lane, one column per head
-            ok = mbar_wait(ctx, bar(kBarOFull), seg_it & 1, kBarOFull);
-            if (!ok) break;
+            ok &= mbar_wait(ctx, bar(kBarOFull), seg_it & 1, kBarOFull);
             tcgen05_fence_after();
             float *obase;
             int64_t ostride;
