@@ -36,6 +36,7 @@ def _load():
         lib.oracle_e4m3_to_double.restype = ctypes.c_double
         lib.oracle_e4m3_to_double.argtypes = [ctypes.c_uint8]
         lib.oracle_mla_decode.restype = ctypes.c_int
+        lib.oracle_mla_decode_rows.restype = ctypes.c_int
         lib.oracle_lse_merge.restype = ctypes.c_int
         lib.oracle_kv_page_migrate.restype = ctypes.c_int
         _lib = lib
@@ -123,6 +124,54 @@ def mla_decode(q, kv_pool, block_table, seq_lens, *, softmax_scale, kv_scales=No
         _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double))
     if rc != 0:
         raise ValueError(f"oracle_mla_decode rejected its arguments (rc={rc})")
+    return out, lse
+
+
+def mla_decode_rows(q, kv_pool, block_table, seq_lens, *, softmax_scale, kv_scales=None,
+                    head_begin=0, head_end=None, kv_begin=None, kv_end=None, page_size=64, d_v=512):
+    """Attention for R causal query rows per request (see oracle_mla_decode_rows).
+
+    q [B][H][R][d_qk] uint16 (bf16 bits); the R rows are the request's newest tokens.
+    Returns (out [B][H][R][d_v] float64, lse [B][H][R] float64), NaN outside the head slice.
+    """
+    lib = _load()
+    assert q.dtype == np.uint16 and q.ndim == 4 and q.flags.c_contiguous
+    B, H, R, d_qk = q.shape
+    if kv_pool.dtype == np.uint16:
+        kv_dtype = 0
+        assert kv_scales is None
+    elif kv_pool.dtype == np.uint8:
+        kv_dtype = 1
+        assert kv_scales is not None and kv_scales.dtype == np.float32
+        kv_scales = np.ascontiguousarray(kv_scales)
+    else:
+        raise TypeError("kv_pool must be uint16 (bf16 bits) or uint8 (e4m3 codes)")
+    kv_pool = np.ascontiguousarray(kv_pool)
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+    if block_table.ndim == 1:
+        block_table = block_table.reshape(B, -1) if B else block_table.reshape(0, 1)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    if head_end is None:
+        head_end = H
+    if kv_begin is not None:
+        kv_begin = np.ascontiguousarray(kv_begin, dtype=np.int32)
+    if kv_end is not None:
+        kv_end = np.ascontiguousarray(kv_end, dtype=np.int32)
+    out = np.full((B, H, R, d_v), np.nan, dtype=np.float64)
+    lse = np.full((B, H, R), np.nan, dtype=np.float64)
+    rc = lib.oracle_mla_decode_rows(
+        ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(R), ctypes.c_int(d_qk), ctypes.c_int(d_v),
+        ctypes.c_int(page_size),
+        _ptr(q, ctypes.c_uint16), ctypes.c_int64(H * R * d_qk), ctypes.c_int64(R * d_qk),
+        kv_pool.ctypes.data_as(ctypes.c_void_p), ctypes.c_int(kv_dtype), _ptr(kv_scales, ctypes.c_float),
+        _ptr(block_table, ctypes.c_int32), ctypes.c_int64(block_table.shape[1]),
+        _ptr(seq_lens, ctypes.c_int32),
+        ctypes.c_int(head_begin), ctypes.c_int(head_end),
+        _ptr(kv_begin, ctypes.c_int32), _ptr(kv_end, ctypes.c_int32),
+        ctypes.c_double(float(softmax_scale)),
+        _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"oracle_mla_decode_rows rejected its arguments (rc={rc})")
     return out, lse
 
 

@@ -142,6 +142,79 @@ int oracle_mla_decode(int B, int H, int d_qk, int d_v, int page_size,
 }
 
 /*
+ * Attention for R query rows per request (a short prefill chunk or a multi-token
+ * decode step: the batch entry of a request carries q_i > 1 rows, Sec. 4.1).  The R
+ * rows are the request's R newest tokens, already in the cache; row r sits at position
+ * seq_len - R + r and attends causally, i.e. over the tokens
+ *     [max(0, kv_begin), min(kv_end, seq_len - (R - 1 - r))),
+ * with the same formula as oracle_mla_decode for each row on its own:
+ *     l_t = scale * q_r . row_t,  lse = ln sum_t exp(l_t),  out = sum_t exp(l_t - lse) row_t[0..d_v).
+ * A row whose range is empty gives out = 0, lse = -inf.
+ *
+ *   q    [B][H][R][d_qk] bf16 bits: element (i, g, r, d) at i*q_stride_b + g*q_stride_h + r*d_qk + d
+ *   out  [B][H][R][d_v] double, lse [B][H][R] double (dense)
+ */
+int oracle_mla_decode_rows(int B, int H, int R, int d_qk, int d_v, int page_size,
+                           const uint16_t *q, int64_t q_stride_b, int64_t q_stride_h,
+                           const void *kv_pool, int kv_dtype, const float *kv_scales,
+                           const int32_t *block_table, int64_t table_stride,
+                           const int32_t *seq_lens,
+                           int head_begin, int head_end,
+                           const int32_t *kv_begin, const int32_t *kv_end,
+                           double softmax_scale,
+                           double *out, double *lse) {
+    int h = head_end - head_begin;
+    if (h < 0 || head_begin < 0 || head_end > H || R < 1) return -1;
+    int64_t total = (int64_t)B * h * R;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t job = 0; job < total; ++job) {
+        int r = (int)(job % R);
+        int g = head_begin + (int)((job / R) % h);
+        int i = (int)(job / ((int64_t)R * h));
+
+        int s = seq_lens[i];
+        int lo = kv_begin ? kv_begin[i] : 0;
+        int hi = kv_end ? kv_end[i] : s;
+        int causal_end = s - (R - 1 - r);          /* one past the row's own position */
+        if (lo < 0) lo = 0;
+        if (hi > causal_end) hi = causal_end;
+        int n = hi > lo ? hi - lo : 0;
+
+        double *o = out + (((int64_t)i * H + g) * R + r) * d_v;
+        double *L = lse + ((int64_t)i * H + g) * R + r;
+        for (int d = 0; d < d_v; ++d) o[d] = 0.0;
+        if (n == 0) { *L = -INFINITY; continue; }
+
+        const uint16_t *qrow = q + i * q_stride_b + g * q_stride_h + (int64_t)r * d_qk;
+        double *logit = (double *)malloc(sizeof(double) * (size_t)n);
+        double m = -INFINITY;
+        for (int t = lo; t < hi; ++t) {
+            int64_t page = block_table[i * table_stride + t / page_size];
+            int slot = t % page_size;
+            double acc = 0.0;
+            for (int d = 0; d < d_qk; ++d)
+                acc += bf16_to_double(qrow[d]) *
+                       kv_elem(kv_pool, kv_dtype, kv_scales, page, slot, d, d_qk, page_size);
+            logit[t - lo] = softmax_scale * acc;
+            if (logit[t - lo] > m) m = logit[t - lo];
+        }
+        double Z = 0.0;
+        for (int t = 0; t < n; ++t) Z += exp(logit[t] - m);
+        *L = m + log(Z);
+        for (int t = lo; t < hi; ++t) {
+            int64_t page = block_table[i * table_stride + t / page_size];
+            int slot = t % page_size;
+            double w = exp(logit[t - lo] - m) / Z;
+            for (int d = 0; d < d_v; ++d)
+                o[d] += w * kv_elem(kv_pool, kv_dtype, kv_scales, page, slot, d, d_qk, page_size);
+        }
+        free(logit);
+    }
+    return 0;
+}
+
+/*
  * Merge of partial attention results over disjoint KV ranges:
  *   L = ln sum_j exp(L_j),  O = sum_j exp(L_j - L) * O_j.
  * Parts with L_j = -inf contribute nothing; if every part is -inf, O = 0 and

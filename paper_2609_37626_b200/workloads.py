@@ -48,6 +48,12 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
     return r.astype(np.uint16)
 
 
+def make_query_rows(seed: int, B: int, H: int, R: int) -> np.ndarray:
+    """R query rows per request and head, [B][H][R][576] bf16 bit patterns (N(0,1), a stream of its own)."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 7])))
+    return f32_to_bf16_bits(rng.standard_normal((B, H, R, D_QK), dtype=np.float32))
+
+
 def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
     """bf16 bit patterns -> float32 (exact)."""
     return (np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)

@@ -134,6 +134,76 @@ def test_dominant_key_selects_its_row():
     assert abs(lse[0, 0] - SCALE * 8.0 * math.fsum(qv.astype(np.float64) ** 2)) < 1e-9
 
 
+# ---------------------------------------------------------------- several causal query rows per request
+def run_rows(w, q4, **kw):
+    args = dict(softmax_scale=w.softmax_scale, kv_scales=w.kv_scales, head_begin=w.head_begin,
+                head_end=w.head_end, kv_begin=w.kv_begin, kv_end=w.kv_end)
+    args.update(kw)
+    return oracle.mla_decode_rows(q4, w.kv_pool, w.block_table, w.seq_lens, **args)
+
+
+@pytest.mark.parametrize("kv_dtype", [0, 1])
+def test_rows_one_row_is_plain_decode(kv_dtype):
+    w = W.make_workload("rows1", 61 + kv_dtype, [1, 64, 130], H=5, kv_dtype=kv_dtype)
+    out, lse = run(w)
+    out4, lse4 = run_rows(w, np.ascontiguousarray(w.q[:, :, None, :]))
+    assert np.array_equal(out4[:, :, 0], out) and np.array_equal(lse4[:, :, 0], lse)
+
+
+@pytest.mark.parametrize("R", [2, 3, 8])
+def test_rows_each_row_is_plain_decode_over_its_causal_prefix(R):
+    # row r of an R-row call = the one-row decode of the same query over the first s - (R-1-r) tokens:
+    # reduces every row to the single-row oracle pinned above (bit for bit, same loops)
+    lens = [R, R + 1, 64, 65, 200]
+    w = W.make_workload("rowsR", 63 + R, lens, H=3)
+    q4 = W.make_query_rows(63 + R, w.B, w.H, R)
+    out4, lse4 = run_rows(w, q4)
+    for r in range(R):
+        shorter = (w.seq_lens - (R - 1 - r)).astype(np.int32)
+        o, l = oracle.mla_decode(np.ascontiguousarray(q4[:, :, r]), w.kv_pool, w.block_table, shorter,
+                                 softmax_scale=w.softmax_scale)
+        assert np.array_equal(out4[:, :, r], o) and np.array_equal(lse4[:, :, r], l)
+
+
+def test_rows_match_dense_causal_library_attention():
+    R = 4
+    w = W.make_workload("rowslib", 67, [4, 70, 131], H=4)
+    q4 = W.make_query_rows(67, w.B, w.H, R)
+    out4, lse4 = run_rows(w, q4)
+    for i in range(w.B):
+        rows = torch.from_numpy(dense_rows(w, i)); s = rows.shape[0]
+        q = torch.from_numpy(f32(q4[i]))                              # [H][R][576]
+        mask = torch.arange(s)[None, :] <= (s - R + torch.arange(R))[:, None]      # row r sees tokens <= its position
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            q[None], rows[None, None].expand(1, w.H, -1, -1),
+            torch.nn.functional.pad(rows[:, :512], (0, 64))[None, None].expand(1, w.H, -1, -1),
+            attn_mask=mask, scale=SCALE)[0, :, :, :512].numpy()
+        assert np.allclose(out4[i], ref, rtol=0, atol=1e-12)
+        logits = SCALE * torch.einsum("hrd,td->hrt", q, rows).masked_fill(~mask[None], -math.inf)
+        assert np.allclose(lse4[i], torch.logsumexp(logits, dim=2).numpy(), rtol=0, atol=1e-12)
+
+
+def test_rows_first_row_of_a_fresh_request_sees_one_token_and_ranges_can_empty_a_row():
+    R = 3
+    w = W.make_workload("rowsedge", 69, [3, 100], H=2)
+    q4 = W.make_query_rows(69, w.B, w.H, R)
+    out4, lse4 = run_rows(w, q4)
+    # request 0 has exactly R tokens: row 0 attends token 0 only -> O = that row's latent part, LSE = scale q.k
+    k0 = f32(w.kv_pool[w.block_table[0, 0], 0])
+    for g in range(w.H):
+        assert np.array_equal(out4[0, g, 0], k0[:512])
+        assert abs(lse4[0, g, 0] - SCALE * float(f32(q4[0, g, 0]) @ k0)) < 1e-12
+    # a range that starts at the last token: only the last row has anything to attend
+    kb = (w.seq_lens - 1).astype(np.int32)
+    out4, lse4 = run_rows(w, q4, kv_begin=kb)
+    assert np.all(np.isneginf(lse4[:, :, : R - 1])) and np.all(out4[:, :, : R - 1] == 0.0)
+    assert np.all(np.isfinite(lse4[:, :, R - 1]))
+    # fewer tokens than rows: the oldest rows have an empty range
+    w1 = W.make_workload("rowsshort", 70, [2], H=2)
+    o, l = run_rows(w1, W.make_query_rows(70, 1, 2, 4))
+    assert np.all(np.isneginf(l[0, :, :2])) and np.all(np.isfinite(l[0, :, 2:]))
+
+
 # ---------------------------------------------------------------- library and brute force
 @pytest.mark.parametrize("kv_dtype", [0, 1])
 def test_matches_dense_library_attention(kv_dtype):
