@@ -91,7 +91,7 @@ typedef struct splash_mla_shape {
     int64_t out_stride_request, out_stride_head; /* multiples of 4 */
     int64_t lse_stride_request;
     uint32_t flags;              /* SPLASH_FLAG_* bits, 0 for the default path */
-    uint32_t reserved;           /* must be 0 */
+    uint32_t q_rows;             /* R: query rows per request, 0 or 1 = one row (decode); see splash_mla_decode */
 } splash_mla_shape;
 
 /*
@@ -104,6 +104,18 @@ typedef struct splash_mla_shape {
  *     lse    = ln sum_{t in R_i} exp(l_t)                          (natural log, scale included)
  *     out[d] = sum_{t in R_i} exp(l_t - lse) * row_t[d],  d < 512
  * An empty R_i gives out = 0, lse = -inf.
+ *
+ * Several query rows per request (shape.q_rows = R > 1; a multi-token decode step or a
+ * short prefill chunk: the batch entry of a request carries q_i > 1 rows, Sec. 4.1): the R
+ * rows are the request's R newest tokens, whose cache rows are already written; row r sits
+ * at position seq_lens[i] - R + r and attends causally, i.e. its range is
+ *     [max(0, kv_begin[i]), min(kv_end[i], seq_lens[i] - (R - 1 - r))),
+ * each row on its own with the formulas above.  The rows of a head are dense:
+ *     q   (i, g, r, d) at q  [i*q_stride_request   + g*q_stride_head   + r*576 + d], q_stride_head   = R*576
+ *     out (i, g, r, d) at out[i*out_stride_request + g*out_stride_head + r*512 + d], out_stride_head = R*512
+ *     lse (i, g, r)    at lse[i*lse_stride_request + g*R + r]
+ * 1 <= R <= 8.  A slice of more than 128 / R heads is served 128 (head, row) pairs at a
+ * time, each pass reading the cache once.
  *
  *   q            bf16, 16-byte aligned
  *   kv_pool      [num_pool_pages][64][576] bf16 (73,728 B / page) or e4m3 bytes

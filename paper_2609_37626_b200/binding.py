@@ -52,7 +52,7 @@ class MlaShape(ctypes.Structure):
         ("out_stride_head", ctypes.c_int64),
         ("lse_stride_request", ctypes.c_int64),
         ("flags", ctypes.c_uint32),
-        ("reserved", ctypes.c_uint32),
+        ("q_rows", ctypes.c_uint32),
     ]
 
 
@@ -114,17 +114,25 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]):
 
 def make_shape(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch.Tensor, out: torch.Tensor,
                lse: torch.Tensor, softmax_scale: float, flags: int = 0) -> MlaShape:
-    B, H, dqk = q.shape
-    assert q.stride(2) == 1 and out.stride(2) == 1 and lse.stride(1) == 1
+    """q [B][H][576] (one row per request) or [B][H][R][576] (R causal rows per request)."""
+    q_rows = 0
+    if q.dim() == 4:
+        q_rows = q.shape[2]
+        assert q.stride(3) == 1 and q.stride(2) == q.shape[3] and out.dim() == 4 and out.stride(3) == 1
+        assert out.stride(2) == out.shape[3] and lse.dim() == 3 and lse.stride(2) == 1 and lse.stride(1) == q_rows
+        B, H, _, dqk = q.shape
+    else:
+        B, H, dqk = q.shape
+        assert q.stride(2) == 1 and out.stride(2) == 1 and lse.stride(1) == 1
     kv_dtype = SPLASH_KV_BF16 if kv_pool.dtype == torch.bfloat16 else SPLASH_KV_E4M3_TOKEN_SCALE
     return MlaShape(
-        struct_size=ctypes.sizeof(MlaShape), num_requests=B, num_heads=H, d_qk=dqk, d_v=out.shape[2],
+        struct_size=ctypes.sizeof(MlaShape), num_requests=B, num_heads=H, d_qk=dqk, d_v=out.shape[-1],
         page_size=kv_pool.shape[1], num_pool_pages=kv_pool.shape[0],
         block_table_stride=block_table.stride(0) if block_table.dim() == 2 and B > 0 else 0,
         kv_dtype=kv_dtype, softmax_scale=float(softmax_scale),
         q_stride_request=q.stride(0), q_stride_head=q.stride(1),
         out_stride_request=out.stride(0), out_stride_head=out.stride(1),
-        lse_stride_request=lse.stride(0), flags=flags, reserved=0)
+        lse_stride_request=lse.stride(0), flags=flags, q_rows=q_rows)
 
 
 def splash_mla_decode_workspace_bytes(shape: MlaShape, head_begin: int, head_end: int) -> int:
@@ -155,16 +163,19 @@ def splash_mla_decode(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch
     kv_scales [P][64] fp32; block_table [B][stride] int32; seq_lens, kv_begin, kv_end
     [B] int32.  out [B][H][512] fp32 and lse [B][H] fp32 are allocated (uninitialised
     outside the head slice) unless given.  Returns (out, lse).
+    A 4-D q [B][H][R][576] asks for R causal query rows per request (the request's R
+    newest tokens); out is then [B][H][R][512] and lse [B][H][R].
     """
     lib = load()
     assert q.is_cuda and q.dtype == torch.bfloat16
-    B, H, _ = q.shape
+    B, H = q.shape[0], q.shape[1]
+    rows = (q.shape[2],) if q.dim() == 4 else ()
     if head_end is None:
         head_end = H
     if out is None:
-        out = torch.empty((B, H, D_V), dtype=torch.float32, device=q.device)
+        out = torch.empty((B, H) + rows + (D_V,), dtype=torch.float32, device=q.device)
     if lse is None:
-        lse = torch.empty((B, H), dtype=torch.float32, device=q.device)
+        lse = torch.empty((B, H) + rows, dtype=torch.float32, device=q.device)
     assert block_table.dtype == torch.int32 and seq_lens.dtype == torch.int32
     shape = make_shape(q, kv_pool, block_table, out, lse, softmax_scale, flags)
     if workspace is None:

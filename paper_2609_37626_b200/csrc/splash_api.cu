@@ -79,14 +79,30 @@ int check_shape(const splash_mla_shape *s, int32_t head_begin, int32_t head_end)
     }
     if (s->lse_stride_request < s->num_heads && s->num_requests > 1) { set_error("lse_stride_request < num_heads"); return SPLASH_INVALID_ARG; }
     if (!(s->softmax_scale == s->softmax_scale)) { set_error("softmax_scale is NaN"); return SPLASH_INVALID_ARG; }
+    if (s->q_rows > (uint32_t)kMaxQRows) { set_error("q_rows must be in [1, %d] (0 = 1)", kMaxQRows); return SPLASH_UNSUPPORTED; }
+    if (s->q_rows > 1) {
+        const int64_t R = s->q_rows;
+        if (s->q_stride_head != R * kDQK || s->out_stride_head != R * kDV) {
+            set_error("with q_rows = R > 1 the rows of a head are dense: q_stride_head = R * 576, out_stride_head = R * 512");
+            return SPLASH_INVALID_ARG;
+        }
+        if (s->lse_stride_request < s->num_heads * R && s->num_requests > 1) { set_error("lse_stride_request < num_heads * q_rows"); return SPLASH_INVALID_ARG; }
+        if (s->flags & SPLASH_FLAG_NO_PAIR) { set_error("q_rows > 1 runs on the CTA-pair kernels only"); return SPLASH_UNSUPPORTED; }
+    }
     return SPLASH_OK;
 }
 
 // How one decode call is cut into CTAs.
 struct Tiling { int heads_per_group, num_groups, num_workers; };
 
+// h = width of the slice in (virtual) heads
 Tiling choose_tiling(const splash_mla_shape *s, int h, int sm_count, bool simt) {
     Tiling t;
+    if (!simt && s->q_rows > 1) {      // several query rows per request: always a CTA pair, whatever the width
+        t.heads_per_group = 64; t.num_groups = 2;
+        t.num_workers = sm_count / 2 > 0 ? sm_count / 2 : 1;
+        return t;
+    }
     if (simt) {
         t.heads_per_group = simt_heads_per_group();
         t.num_groups = (h + t.heads_per_group - 1) / t.heads_per_group;
@@ -122,7 +138,10 @@ size_t splash_mla_decode_workspace_bytes(const splash_mla_shape *shape, int32_t 
     if (check_shape(shape, head_begin, head_end) != SPLASH_OK) return 0;
     DeviceInfo dev;
     if (!current_device_info(dev)) return 0;
-    const int h = head_end - head_begin;
+    // with R query rows per request the call runs over virtual heads, at most kMaxHeads of them at a time
+    const int R = shape->q_rows > 1 ? (int)shape->q_rows : 1;
+    int h = (head_end - head_begin) * R;
+    if (R > 1 && h > kMaxHeads) h = kMaxHeads;
     if (h == 0 || shape->num_requests == 0) return 256;
     // the larger of the two kernels' needs, so one workspace serves both paths
     size_t need = 0;
@@ -141,8 +160,8 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     g_launches = 0;
     int rc = check_shape(shape, head_begin, head_end);
     if (rc != SPLASH_OK) return rc;
-    const int B = shape->num_requests, h = head_end - head_begin;
-    if (B == 0 || h == 0) return SPLASH_OK;   // idle rank: nothing to do
+    const int B = shape->num_requests;
+    if (B == 0 || head_end == head_begin) return SPLASH_OK;   // idle rank: nothing to do
     if (!q || !kv_pool || !block_table || !seq_lens || !out || !lse || !workspace) {
         set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG;
     }
@@ -158,6 +177,16 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     if (dev.cc_major != 10) { set_error("device compute capability %d.x is not 10.x", dev.cc_major); return SPLASH_UNSUPPORTED_DEVICE; }
 
     const bool simt = (shape->flags & SPLASH_FLAG_SIMT) != 0;
+    // R query rows per request: the kernels see R * num_heads virtual heads (head g, row r -> g * R + r: the rows
+    // of a head are dense, so a virtual head is 576 / 512 elements from the next) and mask causally by
+    // (virtual head mod R); a slice wider than 128 virtual heads is served 128 at a time.
+    const int R = shape->q_rows > 1 ? (int)shape->q_rows : 1;
+    const int vbegin = head_begin * R, vend = head_end * R;
+    const int vstep = R > 1 ? kMaxHeads : vend - vbegin;
+    cudaError_t e = cudaSuccess;
+    for (int vb = vbegin; vb < vend && e == cudaSuccess; vb += vstep) {
+    const int ve = vb + vstep < vend ? vb + vstep : vend;
+    const int h = ve - vb;
     Tiling t = choose_tiling(shape, h, dev.sm_count, simt);
     PlanView v = make_plan_view(workspace, B, t.num_workers, h);
     if (workspace_bytes < v.bytes) {
@@ -169,10 +198,10 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     memset(&p, 0, sizeof p);
     p.q = q; p.kv_pool = kv_pool; p.kv_scales = kv_scales; p.block_table = block_table; p.seq_lens = seq_lens;
     p.out = out; p.lse = lse;
-    p.q_stride_request = shape->q_stride_request; p.q_stride_head = shape->q_stride_head;
-    p.out_stride_request = shape->out_stride_request; p.out_stride_head = shape->out_stride_head;
+    p.q_stride_request = shape->q_stride_request; p.q_stride_head = R > 1 ? kDQK : shape->q_stride_head;
+    p.out_stride_request = shape->out_stride_request; p.out_stride_head = R > 1 ? kDV : shape->out_stride_head;
     p.lse_stride_request = shape->lse_stride_request;
-    p.B = B; p.H = shape->num_heads; p.head_begin = head_begin; p.head_end = head_end;
+    p.B = B; p.H = shape->num_heads * R; p.head_begin = vb; p.head_end = ve; p.q_rows = R;
     p.table_stride = shape->block_table_stride; p.num_pool_pages = shape->num_pool_pages;
     p.heads_per_group = t.heads_per_group; p.num_groups = t.num_groups; p.num_workers = t.num_workers;
     p.softmax_scale = shape->softmax_scale;
@@ -186,7 +215,7 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     else if (pair)
         p.request_overhead_tiles = kRequestOverheadTilesPair;
 
-    cudaError_t e = record_timing_event(0, stream);
+    e = record_timing_event(0, stream);
     if (e == cudaSuccess)
         e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
                         v.cost_start, v.worker_begin, v.split_list, v.status, stream);
@@ -199,6 +228,7 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     if (e == cudaSuccess) e = launch_split_combine(p, v.req_wfirst, v.req_wlast, v.split_list, stream);
     if (e == cudaSuccess) e = record_timing_event(3, stream);
     if (e == cudaSuccess && g_timing) g_events_recorded = true;
+    }
     if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
     return SPLASH_OK;
 }

@@ -11,6 +11,7 @@
 namespace splash {
 
 constexpr int kDQK = 576;        // d_c + d_r (absorbed MLA row width)
+constexpr int kMaxQRows = 8;      // query rows per request (multi-token decode steps, short prefill chunks)
 constexpr int kDV = 512;         // d_c (value width)
 constexpr int kDRope = 64;
 constexpr int kPage = 64;        // tokens per page
@@ -91,6 +92,8 @@ struct DecodeParams {
     int32_t head_begin, head_end;
     int32_t table_stride;
     int32_t num_pool_pages;
+    int32_t q_rows;            // R query rows per request; the heads of a call are then virtual heads g * R + r, and
+                               // row r attends causally: tokens below seq_len - (R - 1 - r)
     int32_t heads_per_group;   // heads one CTA computes
     int32_t num_groups;        // head groups per KV worker
     float softmax_scale;

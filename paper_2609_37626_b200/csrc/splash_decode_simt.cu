@@ -63,6 +63,9 @@ decode_simt_kernel(const DecodeParams p) {
         __syncthreads();
 
         const int first_page = seg.lo / kPage;
+        // several query rows per request: (virtual) head g is row g mod R and sees the tokens below its causal end
+        const int s_len = p.q_rows > 1 ? p.seq_lens[seg.request] : 0;
+        auto causal_end = [&](int hd) { return p.q_rows > 1 ? s_len - (p.q_rows - 1 - (head0 + hd) % p.q_rows) : 0x3fffffff; };
         for (int tile = seg.tile_begin; tile < seg.tile_end; ++tile) {
             const int page_idx = first_page + tile;
             const int t0 = page_idx * kPage;
@@ -105,7 +108,7 @@ decode_simt_kernel(const DecodeParams p) {
             for (int idx = tid; idx < kSimtHeads * kPage; idx += kSimtThreads) {
                 int hd = idx / kPage, t = idx % kPage;
                 float sv = -INFINITY;
-                if (t >= a && t < b) {
+                if (t >= a && t < min(b, causal_end(hd) - t0)) {
                     float dot = 0.f;
                     const uint4 *row = reinterpret_cast<const uint4 *>(&sm.rows[t][0]);
                     const float *qh = sm.q[hd];
@@ -126,19 +129,20 @@ decode_simt_kernel(const DecodeParams p) {
             // ---- online softmax: warp `wid` owns head `wid` --------------------------
             {
                 const int hd = wid;
+                const int bh = min(b, causal_end(hd) - t0);      // this head's end within the tile
                 float s0 = sm.s[hd][lane], s1 = sm.s[hd][lane + 32];
                 float mx = fmaxf(s0, s1);
                 for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
                 float m_old = sm.m[hd];
-                float m_new = fmaxf(m_old, mx);           // finite: every tile holds a valid token
-                float p0 = (lane >= a && lane < b) ? __expf(s0 - m_new) : 0.f;
-                float p1 = (lane + 32 >= a && lane + 32 < b) ? __expf(s1 - m_new) : 0.f;
+                float m_new = fmaxf(m_old, mx);           // -inf only while the head has seen no token
+                float p0 = (lane >= a && lane < bh) ? __expf(s0 - m_new) : 0.f;
+                float p1 = (lane + 32 >= a && lane + 32 < bh) ? __expf(s1 - m_new) : 0.f;
                 float sum = p0 + p1;
                 for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
                 float al = (m_old == -INFINITY) ? 0.f : __expf(m_old - m_new);
                 if (KV_DTYPE == 1) { p0 *= sm.tok_scale[lane < b ? lane : 0]; p1 *= sm.tok_scale[lane + 32 < b ? lane + 32 : 0]; }
-                if (!(lane >= a && lane < b)) p0 = 0.f;
-                if (!(lane + 32 >= a && lane + 32 < b)) p1 = 0.f;
+                if (!(lane >= a && lane < bh)) p0 = 0.f;
+                if (!(lane + 32 >= a && lane + 32 < bh)) p1 = 0.f;
                 sm.s[hd][lane] = p0; sm.s[hd][lane + 32] = p1;
                 if (lane == 0) { sm.alpha[hd] = al; sm.m[hd] = m_new; sm.l[hd] = sm.l[hd] * al + sum; }
             }
@@ -167,9 +171,9 @@ decode_simt_kernel(const DecodeParams p) {
             int g = head0 + hd;
             if (g >= p.head_end) continue;
             float l = sm.l[hd];
-            float inv = 1.f / l;
+            float inv = l > 0.f ? 1.f / l : 0.f;          // no token at all: O = 0, LSE = -inf
             float2 o = make_float2(acc[hd][0] * inv, acc[hd][1] * inv);
-            float L = sm.m[hd] + logf(l);
+            float L = l > 0.f ? sm.m[hd] + logf(l) : -INFINITY;
             if (seg.slot < 0) {
                 float *dst = p.out + (int64_t)seg.request * p.out_stride_request + (int64_t)g * p.out_stride_head;
                 *reinterpret_cast<float2 *>(dst + 2 * tid) = o;

@@ -417,6 +417,9 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
             if (lane == 0) mbar_arrive(bar(kBarQsRead));
             float m = -INFINITY, l = 0.f;
             const int nsuper = (seg.tile_end - seg.tile_begin + 1) >> 1;
+            // several query rows per request: this thread's (virtual) head is row (head mod R) and sees the
+            // tokens below causal_end only
+            const int causal_end = p.q_rows > 1 ? p.seq_lens[seg.request] - (p.q_rows - 1 - (head0 + hd) % p.q_rows) : 0x3fffffff;   // (far above any token index, and safe to subtract a negative offset from)
             for (int s = 0; s < nsuper; ++s, ++st_it) {
                 const PairGeom g = pair_geom(s);
                 const TileGeom geo = pg ? g.b : g.a;
@@ -444,9 +447,15 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                 tcgen05_fence_before();
                 __syncwarp();
                 if (lane == 0) arrive_on_leader(kBarSEmpty + b);
-                const uint32_t valid = __ballot_sync(0xffffffffu, 32 * cf + lane >= geo.r_lo && 32 * cf + lane < geo.r_hi);
+                uint32_t valid = __ballot_sync(0xffffffffu, 32 * cf + lane >= geo.r_lo && 32 * cf + lane < geo.r_hi);
+                {
+                    // how many of this thread's 32 tokens lie below its head's causal end: token j of the thread is
+                    // token (page index) * 64 + tok0 + 32 cf + j of the request
+                    const int lim = causal_end - ((seg.lo / kPage + seg.tile_begin + 2 * s + pg) * kPage + geo.tok0 + 32 * cf);
+                    if (lim < 32) valid &= lim <= 0 ? 0u : (1u << lim) - 1u;
+                }
                 float mt = -INFINITY;
-                if (valid == 0xffffffffu) {
+                if (__all_sync(0xffffffffu, valid == 0xffffffffu)) {
 #pragma unroll
                     for (int j2 = 0; j2 < 16; ++j2) {
                         const float4 t = tok_a[j2];
@@ -474,7 +483,7 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                 float al = 1.f;
                 if (mt > m + kTau) { al = (m == -INFINITY) ? 0.f : fast_exp2(m - mt); m = mt; l *= al; grew = true; }
                 if (slot4 == 0) alpha_s[hd] = al;
-                const float off = kLift - m;
+                const float off = kLift - (m == -INFINITY ? 0.f : m);   // a head that has seen no token yet: all weights 0, not NaN
                 uint32_t phi[8], plo[8];
 #pragma unroll
                 for (int j4 = 0; j4 < 8; ++j4) {
@@ -535,10 +544,10 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
             if (slot4 == 0) {
                 const float4 x4 = *reinterpret_cast<const float4 *>(&xch[hd * 4]);
                 const float lt = (x4.x + x4.y) + (x4.z + x4.w);
-                l_s[hd] = 1.f / lt;
+                l_s[hd] = lt > 0.f ? 1.f / lt : 0.f;       // no token at all (an empty causal range): O = 0, LSE = -inf
                 const int gh = head0 + hd;
                 if (gh < p.head_end) {
-                    float lse = (m - kLift + log2f(lt)) * kLn2;
+                    float lse = lt > 0.f ? (m - kLift + log2f(lt)) * kLn2 : -INFINITY;
                     if (seg.slot < 0) p.lse[(int64_t)seg.request * p.lse_stride_request + gh] = lse;
                     else p.partial_lse[(int64_t)seg.slot * h + (gh - p.head_begin)] = lse;
                 }

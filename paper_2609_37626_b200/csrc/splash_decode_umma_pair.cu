@@ -300,6 +300,9 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
         while (it.next(p, seg)) {
             float m = -INFINITY, l = 0.f;               // running maximum in scaled log2 units
             const int first_page = seg.lo / kPage;
+            // several query rows per request: this thread's (virtual) head is row (head mod R) and sees the
+            // tokens below causal_end only
+            const int causal_end = p.q_rows > 1 ? p.seq_lens[seg.request] - (p.q_rows - 1 - (head0 + hd) % p.q_rows) : 0x3fffffff;   // (far above any token index, and safe to subtract a negative offset from)
             for (int tile = seg.tile_begin; tile < seg.tile_end; ++tile, ++kv_it) {
                 const TileGeom geo = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
                 const uint32_t b = kv_it & 1;
@@ -320,11 +323,13 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                 tcgen05_fence_before();
                 __syncwarp();
                 if (lane == 0) arrive_on_leader(kBarSEmpty + b);
-                // rows outside [r_lo, r_hi) are zero fill or tokens outside the request's range
-                if (row0 < geo.r_lo || row0 + 16 > geo.r_hi) {
+                // rows outside [r_lo, r_hi) are zero fill or tokens outside the request's range (or beyond this
+                // head's causal end: row r of the tile holds token (first_page + tile) * 64 + tok0 + r)
+                const int r_hi = min(geo.r_hi, causal_end - ((first_page + tile) * kPage + geo.tok0));
+                if (row0 < geo.r_lo || row0 + 16 > r_hi) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (row0 + j < geo.r_lo || row0 + j >= geo.r_hi) sv[j] = -INFINITY;
+                        if (row0 + j < geo.r_lo || row0 + j >= r_hi) sv[j] = -INFINITY;
                 }
                 float mt = sv[0];
 #pragma unroll
@@ -340,10 +345,11 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                 float al = 1.f;
                 if (mt > m + kTau) { al = (m == -INFINITY) ? 0.f : fast_exp2(m - mt); m = mt; l *= al; grew = true; }
                 if (slot4 == 0) alpha_s[hd] = al;
+                const float mref = m == -INFINITY ? 0.f : m;   // a head that has seen no token yet: all weights 0, not NaN
                 uint32_t pk[8];
 #pragma unroll
                 for (int j = 0; j < 16; j += 2) {
-                    const float u0 = fast_exp2(sv[j] - m), u1 = fast_exp2(sv[j + 1] - m);
+                    const float u0 = fast_exp2(sv[j] - mref), u1 = fast_exp2(sv[j + 1] - mref);
                     l += u0 + u1;
                     pk[j >> 1] = pack_bf16x2(u0, u1);
                 }
@@ -386,10 +392,10 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
             if (slot4 == 0) {
                 const float4 x4 = *reinterpret_cast<const float4 *>(&xch[hd * 4]);
                 const float lt = (x4.x + x4.y) + (x4.z + x4.w);
-                l_s[hd] = 1.f / lt;
+                l_s[hd] = lt > 0.f ? 1.f / lt : 0.f;       // no token at all (an empty causal range): O = 0, LSE = -inf
                 const int gh = head0 + hd;
                 if (gh < p.head_end) {
-                    float lse = (m + log2f(lt)) * kLn2;
+                    float lse = lt > 0.f ? (m + log2f(lt)) * kLn2 : -INFINITY;
                     if (seg.slot < 0) p.lse[(int64_t)seg.request * p.lse_stride_request + gh] = lse;
                     else p.partial_lse[(int64_t)seg.slot * h + (gh - p.head_begin)] = lse;
                 }

@@ -86,6 +86,11 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
     if ((c & 31) == 0) red_s[c >> 5] = m;
     __syncthreads();
     m = fmaxf(fmaxf(red_s[0], red_s[1]), fmaxf(red_s[2], red_s[3]));
+    if (m == -INFINITY) {                  // no piece saw a token (a query row whose causal range is empty)
+        o4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c == 0) *lse = -INFINITY;
+        return;
+    }
     for (int j = c; j < nparts; j += kMergeThreads) w_s[j] = expf(w_s[j] - m);     // 0 for dead workers
     __syncthreads();
     float Z = 0.f;

@@ -47,7 +47,7 @@ def good_shape(**kw):
     s = binding.MlaShape(struct_size=ctypes.sizeof(binding.MlaShape), num_requests=2, num_heads=16, d_qk=576,
                          d_v=512, page_size=64, num_pool_pages=8, block_table_stride=4, kv_dtype=0,
                          softmax_scale=0.07, q_stride_request=16 * 576, q_stride_head=576,
-                         out_stride_request=16 * 512, out_stride_head=512, lse_stride_request=16, flags=0, reserved=0)
+                         out_stride_request=16 * 512, out_stride_head=512, lse_stride_request=16, flags=0, q_rows=0)
     for k, v in kw.items():
         setattr(s, k, v)
     return s
