@@ -226,6 +226,31 @@ class GpuBench:
                "tokens": w.total_tokens(), "requests": w.B, "heads": w.head_end - w.head_begin}
         return res, dw, out, lse
 
+    def rows_workload(self, w, R, steps, warmup, peaks):
+        """R causal query rows per request over the same cache (a multi-token decode step): whole-call time,
+        roofline from the algorithmic bytes (each cache row once) and flops (every row of every head)."""
+        torch, binding = self.torch, self.binding
+        dw = binding.DeviceWorkload(w, self.device)
+        q4 = torch.from_numpy(W.make_query_rows(1234, w.B, w.H, R).view(np.int16)).to(self.device).view(torch.bfloat16)
+        out = torch.empty((w.B, w.H, R, W.D_V), dtype=torch.float32, device=self.device)
+        lse = torch.empty((w.B, w.H, R), dtype=torch.float32, device=self.device)
+        step = lambda: binding.splash_mla_decode(q4, dw.kv_pool, dw.block_table, dw.seq_lens, softmax_scale=w.softmax_scale,
+                                                 kv_scales=dw.kv_scales, head_begin=w.head_begin, head_end=w.head_end,
+                                                 out=out, lse=lse)
+        ms = self.timed(step, steps, warmup)
+        h = w.head_end - w.head_begin
+        rows_bytes = w.B * h * (R - 1) * (W.D_QK * 2 + W.D_V * 4 + 4)        # the extra q rows read, out / lse rows written
+        alg_bytes, alg_flops = w.algorithmic_bytes() + rows_bytes, w.algorithmic_flops() * R
+        t_hbm, t_tensor = alg_bytes / (peaks["hbm_gbs"] * 1e9), alg_flops / (peaks["bf16_tflops"] * 1e12)
+        p50 = float(np.median(ms))
+        return {"q_rows": R, "ms_per_step": float(ms.mean()), "ms_p50": p50, "ms_p95": float(np.percentile(ms, 95)),
+                "query_rows_per_s": w.B * R / (ms.mean() * 1e-3),
+                "roofline": {"bound": "hbm" if t_hbm >= t_tensor else "tensor", "roofline_ms": max(t_hbm, t_tensor) * 1e3,
+                             "frac": max(t_hbm, t_tensor) * 1e3 / p50, "of": "whole call, p50", "peak_source": peaks["source"],
+                             "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
+                             "passes_over_the_cache": -(-h * R // 128)},
+                "launches_per_step": binding.splash_last_launch_count()}
+
     def e2e(self, w, dw, steps, warmup):
         """Same call with the step's inputs coming from pinned host memory and the
         results going back to it inside the timed region."""
@@ -411,6 +436,13 @@ def main():
                     torch.cuda.empty_cache()
                 except Exception as exc:  # report, do not hide
                     extra[name] = {"error": repr(exc)}
+            # several causal query rows per request on the main workload's cache (multi-token decode steps)
+            for R in (2, 4):
+                try:
+                    extra["%s_rows%d" % (args.workload, R)] = gb.rows_workload(w, R, max(5, args.steps // 2), args.warmup, peaks)
+                    torch.cuda.empty_cache()
+                except Exception as exc:
+                    extra["%s_rows%d" % (args.workload, R)] = {"error": repr(exc)}
 
     if rank == 0:
         line = {
