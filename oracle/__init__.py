@@ -211,3 +211,44 @@ def kv_page_migrate(src_pool, dst_pool, src_page_ids, dst_page_ids, block_table,
         ctypes.c_int64(src_page_ids.size),
         ctypes.c_int32(src_id_base), ctypes.c_int32(dst_id_base),
         _ptr(block_table, ctypes.c_int32), ctypes.c_int64(block_table.size))
+
+
+# ---------------------------------------------------------------------------------------------
+# DOP transfer layout changes (App. E): a tensor in global-row, local-head order is regrouped into
+# owner-row, all-head order and back.  Pure permutations of whole rows of bytes, written here with
+# explicit loops over (position, head) so that they can be read against the text.
+def dop_pack_rows(a, b, send_row):
+    """Send buffer of the forward exchange.  a [N][h][da], b [N][h][db] or None (the no-position and
+    rotary parts of the query, fused into one row), send_row [n]: the source row of send position p
+    (rows grouped by destination owner; row identity and head order are kept).  -> [n][h][da+db]."""
+    n, h = len(send_row), a.shape[1]
+    da = a.shape[2]
+    db = 0 if b is None else b.shape[2]
+    out = np.zeros((n, h, da + db), dtype=a.dtype)
+    for p in range(n):
+        for j in range(h):
+            out[p, j, :da] = a[send_row[p], j]
+            if b is not None:
+                out[p, j, da:] = b[send_row[p], j]
+    return out
+
+
+def dop_unpack_rows(recv, send_row, num_rows, out=None):
+    """Reverse exchange, last step: position p of recv [n][h][d] goes back to row send_row[p] of
+    out [num_rows][h][d]; rows that are not listed keep what ``out`` held (zeros when allocated here)."""
+    if out is None:
+        out = np.zeros((num_rows,) + recv.shape[1:], dtype=recv.dtype)
+    for p in range(len(send_row)):
+        out[send_row[p]] = recv[p]
+    return out
+
+
+def dop_swap_outer(x):
+    """[A][B][...] -> [B][A][...]: receive buffer in source-rank-major order [T][n][h][d] to owner-row,
+    all-head order [n][T*h][d] (head s*h + j comes from rank s: global head order), and its inverse."""
+    A, B = x.shape[0], x.shape[1]
+    out = np.zeros((B, A) + x.shape[2:], dtype=x.dtype)
+    for s in range(A):
+        for r in range(B):
+            out[r, s] = x[s, r]
+    return out
