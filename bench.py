@@ -251,6 +251,34 @@ class GpuBench:
                              "passes_over_the_cache": -(-h * R // 128)},
                 "launches_per_step": binding.splash_last_launch_count()}
 
+    def dop_workload(self, steps, warmup, peaks, N=16384, T=8, h=16):
+        """DOP transfer layout changes at a rank's size of a large batch: N query rows, h = H/T local heads;
+        bytes read + written over the measured copy bandwidth."""
+        torch, binding = self.torch, self.binding
+        g = torch.Generator(device=self.device); g.manual_seed(77)
+        nope = torch.randint(-2 ** 15, 2 ** 15, (N, h, 512), dtype=torch.int16, device=self.device, generator=g).view(torch.bfloat16)
+        rope = torch.randint(-2 ** 15, 2 ** 15, (N, h, 64), dtype=torch.int16, device=self.device, generator=g).view(torch.bfloat16)
+        send_row = torch.randperm(N, device=self.device, generator=g).to(torch.int32)
+        send = torch.empty((N, h, 576), dtype=torch.bfloat16, device=self.device)
+        res = {}
+        def report(name, ms, nbytes):
+            p50 = float(np.median(ms))
+            res[name] = {"ms_p50": p50, "gbs": nbytes / (p50 * 1e-3) / 1e9, "frac_of_hbm": nbytes / (p50 * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "bytes": nbytes}
+        ms = self.timed(lambda: binding.splash_dop_pack_rows(nope, rope, send_row, out=send), steps, warmup)
+        report("pack_rows", ms, 2 * send.numel() * 2 + N * 4)
+        recv = send.view(T, N // T, h, 576)
+        swapped = torch.empty((N // T, T, h, 576), dtype=torch.bfloat16, device=self.device)
+        ms = self.timed(lambda: binding.splash_dop_swap_outer(recv, out=swapped), steps, warmup)
+        report("swap_outer", ms, 2 * recv.numel() * 2)
+        del nope, rope, send, swapped
+        o_recv = torch.empty((N, h, 512), dtype=torch.float32, device=self.device).normal_(generator=g)
+        o_out = torch.empty((N, h, 512), dtype=torch.float32, device=self.device)
+        ms = self.timed(lambda: binding.splash_dop_unpack_rows(o_recv, send_row, o_out), steps, warmup)
+        report("unpack_rows", ms, 2 * o_recv.numel() * 4 + N * 4)
+        res["shape"] = {"rows": N, "ranks": T, "local_heads": h}
+        return res
+
     def e2e(self, w, dw, steps, warmup):
         """Same call with the step's inputs coming from pinned host memory and the
         results going back to it inside the timed region."""
@@ -436,6 +464,11 @@ def main():
                     torch.cuda.empty_cache()
                 except Exception as exc:  # report, do not hide
                     extra[name] = {"error": repr(exc)}
+            try:
+                extra["dop_layout_changes"] = gb.dop_workload(max(5, args.steps // 2), args.warmup, peaks)
+                torch.cuda.empty_cache()
+            except Exception as exc:
+                extra["dop_layout_changes"] = {"error": repr(exc)}
             # several causal query rows per request on the main workload's cache (multi-token decode steps)
             for R in (2, 4):
                 try:

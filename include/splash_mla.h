@@ -232,6 +232,40 @@ SPLASH_API int splash_kv_page_migrate_static(const void *src_pool, const float *
                                              int32_t src_id_base, int32_t dst_id_base, int32_t max_page_id,
                                              int32_t *block_table, int64_t num_table_entries, void *stream);
 
+/*
+ * DOP transfer layout changes (App. E): the regrouping steps on either side of the two
+ * all-to-alls that turn a tensor in global-row, local-head order (every rank holds its head
+ * slice of all N rows) into owner-row, all-head order (every rank holds all heads of the rows
+ * it owns) and back.  The collectives themselves are the caller's; these calls move whole
+ * rows of bytes on one GPU, byte-exact, and keep row identity, head order and positions.
+ * Sizes and pitches are in BYTES and must be even; when every pointer, size and pitch is a
+ * multiple of 16 a 16-byte vector path is taken, otherwise a 2-byte scalar one.  n = 0 is a
+ * successful no-op (ranks that own no rows still take part in the exchange).
+ *
+ * splash_dop_pack_rows: builds the send buffer of the forward exchange,
+ *     send[p][j] = a[send_row[p]][j] ++ b[send_row[p]][j],    p < n, j < h,
+ * where send_row lists the source rows grouped by destination owner (the caller derives the
+ * all-to-all split sizes from the per-owner row counts) and a / b are the no-position and the
+ * rotary part of the query (a_part_bytes / b_part_bytes per head; b may be NULL with
+ * b_part_bytes = 0), fused so that one collective moves both.  Element (r, j) of a starts at
+ * a + r*a_row_pitch + j*a_head_pitch.  send is dense: [n][h][a_part_bytes + b_part_bytes].
+ *
+ * splash_dop_swap_outer: out[r][s] = in[s][r] for blocks of inner_bytes, s < A, r < B.  With
+ * A = T ranks, B = n owned rows and inner = h heads it turns the receive buffer of the forward
+ * exchange (source-rank major) into all-head order [n][T*h] (head s*h + j from rank s); with
+ * the roles swapped it builds the send buffer of the reverse exchange.
+ *
+ * splash_dop_unpack_rows: the reverse exchange's last step, out[send_row[p]] = recv[p] for rows
+ * of row_bytes (recv dense, out rows out_row_pitch apart); rows not listed are left untouched.
+ * send_row must not list a row twice.
+ */
+SPLASH_API int splash_dop_pack_rows(const void *a, int64_t a_part_bytes, int64_t a_row_pitch, int64_t a_head_pitch,
+                                    const void *b, int64_t b_part_bytes, int64_t b_row_pitch, int64_t b_head_pitch,
+                                    const int32_t *send_row, int64_t n, int32_t h, void *send, void *stream);
+SPLASH_API int splash_dop_swap_outer(const void *in, int64_t A, int64_t B, int64_t inner_bytes, void *out, void *stream);
+SPLASH_API int splash_dop_unpack_rows(const void *recv, const int32_t *send_row, int64_t n, int64_t row_bytes,
+                                      void *out, int64_t out_row_pitch, void *stream);
+
 /* Host-side helpers. */
 SPLASH_API const char *splash_status_string(int status);
 SPLASH_API const char *splash_last_error(void);

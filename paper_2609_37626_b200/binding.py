@@ -82,6 +82,12 @@ def load() -> ctypes.CDLL:
     lib.splash_kv_page_migrate_static.argtypes = [vp, vp, vp, vp, i64, vp, vp, i64, i32, i32, i32, vp, i64, vp]
     lib.splash_kv_page_migrate_workspace_bytes.restype = sz
     lib.splash_kv_page_migrate_workspace_bytes.argtypes = [i32]
+    lib.splash_dop_pack_rows.restype = ctypes.c_int
+    lib.splash_dop_pack_rows.argtypes = [vp, i64, i64, i64, vp, i64, i64, i64, vp, i64, i32, vp, vp]
+    lib.splash_dop_swap_outer.restype = ctypes.c_int
+    lib.splash_dop_swap_outer.argtypes = [vp, i64, i64, i64, vp, vp]
+    lib.splash_dop_unpack_rows.restype = ctypes.c_int
+    lib.splash_dop_unpack_rows.argtypes = [vp, vp, i64, i64, vp, i64, vp]
     lib.splash_status_string.restype = ctypes.c_char_p
     lib.splash_status_string.argtypes = [ctypes.c_int]
     lib.splash_last_error.restype = ctypes.c_char_p
@@ -223,6 +229,61 @@ def splash_kv_page_migrate(src_pool: torch.Tensor, dst_pool: torch.Tensor, src_p
                                       _ptr(src_page_ids), _ptr(dst_page_ids), n, src_id_base, dst_id_base,
                                       max_page_id, _ptr(block_table), block_table.numel(), _ptr(workspace),
                                       workspace.numel(), _stream_ptr(stream)))
+
+
+def splash_dop_pack_rows(a: torch.Tensor, b: Optional[torch.Tensor], send_row: torch.Tensor,
+                         out: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """Send buffer of the DOP forward exchange: out[p][j] = a[send_row[p]][j] ++ b[send_row[p]][j].
+
+    a [N][h][da], b [N][h][db] or None (last dimension contiguous, any row / head strides), send_row [n] int32.
+    Returns out [n][h][da+db] (dense)."""
+    lib = load()
+    assert a.dim() == 3 and (a.numel() == 0 or a.stride(2) == 1) and send_row.dtype == torch.int32
+    assert send_row.numel() == 0 or send_row.is_contiguous()
+    es = a.element_size()
+    n, h, da = send_row.numel(), a.shape[1], a.shape[2]
+    db = 0
+    if b is not None:
+        assert b.dim() == 3 and (b.numel() == 0 or b.stride(2) == 1) and b.dtype == a.dtype and b.shape[:2] == a.shape[:2]
+        db = b.shape[2]
+    if out is None:
+        out = torch.empty((n, h, da + db), dtype=a.dtype, device=a.device)
+    assert out.is_contiguous() and tuple(out.shape) == (n, h, da + db)
+    _check(lib.splash_dop_pack_rows(_ptr(a), da * es, a.stride(0) * es, a.stride(1) * es,
+                                    _ptr(b), db * es, (b.stride(0) * es) if b is not None else 0,
+                                    (b.stride(1) * es) if b is not None else 0,
+                                    _ptr(send_row), n, h, _ptr(out), _stream_ptr(stream)))
+    return out
+
+
+def splash_dop_swap_outer(x: torch.Tensor, out: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None):
+    """[A][B][...] -> [B][A][...] (contiguous in, contiguous out)."""
+    lib = load()
+    assert x.is_contiguous() and x.dim() >= 2
+    A, B = x.shape[0], x.shape[1]
+    inner = x.element_size()
+    for d in x.shape[2:]:
+        inner *= d
+    if out is None:
+        out = torch.empty((B, A) + tuple(x.shape[2:]), dtype=x.dtype, device=x.device)
+    assert out.is_contiguous()
+    _check(lib.splash_dop_swap_outer(_ptr(x), A, B, inner, _ptr(out), _stream_ptr(stream)))
+    return out
+
+
+def splash_dop_unpack_rows(recv: torch.Tensor, send_row: torch.Tensor, out: torch.Tensor,
+                           stream: Optional[torch.cuda.Stream] = None):
+    """out[send_row[p]] = recv[p]; recv [n][...] contiguous, out [N][...] with contiguous rows."""
+    lib = load()
+    assert recv.is_contiguous() and send_row.dtype == torch.int32 and send_row.is_contiguous()
+    assert recv.shape[1:] == out.shape[1:] and out[0].is_contiguous() if out.shape[0] else True
+    n = send_row.numel()
+    row_bytes = recv.element_size()
+    for d in recv.shape[1:]:
+        row_bytes *= d
+    _check(lib.splash_dop_unpack_rows(_ptr(recv), _ptr(send_row), n, row_bytes, _ptr(out),
+                                      out.stride(0) * out.element_size(), _stream_ptr(stream)))
+    return out
 
 
 def splash_kv_page_migrate_static(src_pool: torch.Tensor, dst_pool: torch.Tensor, src_page_ids: torch.Tensor,

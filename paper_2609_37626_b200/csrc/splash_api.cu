@@ -348,6 +348,62 @@ int splash_set_kernel_timing(int enable) {
     return SPLASH_OK;
 }
 
+int splash_dop_pack_rows(const void *a, int64_t a_part_bytes, int64_t a_row_pitch, int64_t a_head_pitch,
+                         const void *b, int64_t b_part_bytes, int64_t b_row_pitch, int64_t b_head_pitch,
+                         const int32_t *send_row, int64_t n, int32_t h, void *send, void *stream_) {
+    g_launches = 0;
+    if (n < 0 || h < 0 || a_part_bytes <= 0 || b_part_bytes < 0) { set_error("negative size"); return SPLASH_INVALID_ARG; }
+    if (n == 0 || h == 0) return SPLASH_OK;
+    if (!a || !send || !send_row || (b_part_bytes > 0 && !b)) { set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG; }
+    if (b_part_bytes == 0) { b = nullptr; b_row_pitch = b_head_pitch = 0; }
+    if (((a_part_bytes | b_part_bytes | a_row_pitch | a_head_pitch | b_row_pitch | b_head_pitch) & 1) || !aligned(a, 2) ||
+        !aligned(send, 2) || (b && !aligned(b, 2)) || !aligned(send_row, 4)) {
+        set_error("sizes, pitches and pointers must be even"); return SPLASH_INVALID_ARG;
+    }
+    if (a_head_pitch < a_part_bytes || (b && b_head_pitch < b_part_bytes)) { set_error("head pitch smaller than the part"); return SPLASH_INVALID_ARG; }
+    if (n > 0x7fffffffLL) { set_error("too many rows"); return SPLASH_INVALID_ARG; }
+    DeviceInfo dev;
+    if (!current_device_info(dev)) return SPLASH_CUDA_ERROR;
+    cudaError_t e = launch_dop_pack_rows(a, b, send, send_row, n, h, a_part_bytes, b_part_bytes, a_row_pitch, a_head_pitch,
+                                         b_row_pitch, b_head_pitch, dev.sm_count, static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    return SPLASH_OK;
+}
+
+int splash_dop_swap_outer(const void *in, int64_t A, int64_t B, int64_t inner_bytes, void *out, void *stream_) {
+    g_launches = 0;
+    if (A < 0 || B < 0 || inner_bytes < 0 || (inner_bytes & 1)) { set_error("negative or odd size"); return SPLASH_INVALID_ARG; }
+    if (A == 0 || B == 0 || inner_bytes == 0) return SPLASH_OK;
+    if (!in || !out || !aligned(in, 2) || !aligned(out, 2)) { set_error("a required pointer is NULL or odd"); return SPLASH_INVALID_ARG; }
+    {
+        const char *pi = static_cast<const char *>(in), *po = static_cast<const char *>(out);
+        const int64_t bytes = A * B * inner_bytes;
+        if (po < pi + bytes && pi < po + bytes) { set_error("out overlaps in"); return SPLASH_INVALID_ARG; }
+    }
+    DeviceInfo dev;
+    if (!current_device_info(dev)) return SPLASH_CUDA_ERROR;
+    cudaError_t e = launch_dop_swap_outer(in, out, A, B, inner_bytes, dev.sm_count, static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    return SPLASH_OK;
+}
+
+int splash_dop_unpack_rows(const void *recv, const int32_t *send_row, int64_t n, int64_t row_bytes, void *out,
+                           int64_t out_row_pitch, void *stream_) {
+    g_launches = 0;
+    if (n < 0 || row_bytes < 0 || ((row_bytes | out_row_pitch) & 1)) { set_error("negative or odd size"); return SPLASH_INVALID_ARG; }
+    if (n == 0 || row_bytes == 0) return SPLASH_OK;
+    if (!recv || !out || !send_row || !aligned(recv, 2) || !aligned(out, 2) || !aligned(send_row, 4)) {
+        set_error("a required pointer is NULL or misaligned"); return SPLASH_INVALID_ARG;
+    }
+    if (out_row_pitch < row_bytes) { set_error("out_row_pitch smaller than a row"); return SPLASH_INVALID_ARG; }
+    DeviceInfo dev;
+    if (!current_device_info(dev)) return SPLASH_CUDA_ERROR;
+    cudaError_t e = launch_dop_unpack_rows(recv, out, send_row, n, row_bytes, out_row_pitch, dev.sm_count,
+                                           static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    return SPLASH_OK;
+}
+
 int splash_get_kernel_timing(float *plan_ms, float *decode_ms, float *combine_ms) {
     if (!g_events_recorded) { set_error("no timed decode call on this thread"); return SPLASH_INVALID_ARG; }
     cudaError_t e = cudaEventSynchronize(g_events[3]);

@@ -202,6 +202,13 @@ cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const in
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
                         int32_t *status, cudaStream_t stream);
+cudaError_t launch_dop_pack_rows(const void *a, const void *b, void *out, const int32_t *send_row, int64_t n, int h,
+                                 int64_t a_bytes, int64_t b_bytes, int64_t a_row_pitch, int64_t a_head_pitch,
+                                 int64_t b_row_pitch, int64_t b_head_pitch, int sm_count, cudaStream_t stream);
+cudaError_t launch_dop_unpack_rows(const void *recv, void *out, const int32_t *send_row, int64_t n, int64_t row_bytes,
+                                   int64_t out_row_pitch, int sm_count, cudaStream_t stream);
+cudaError_t launch_dop_swap_outer(const void *in, void *out, int64_t A, int64_t Bn, int64_t inner_bytes, int sm_count,
+                                  cudaStream_t stream);
 cudaError_t launch_decode_simt(const DecodeParams &p, int kv_dtype, cudaStream_t stream);
 int simt_heads_per_group();
 // tcgen05 kernel: how it cuts a head slice of width h into CTAs, and its launcher

@@ -89,3 +89,19 @@ def test_merge_and_migrate_reject_bad_arguments(lib):
     assert lib.splash_kv_page_migrate(p, p, p, None, 73728, p, p, 1, 0, 0, 16, p, 8, p, 4096, None) == binding.SPLASH_INVALID_ARG
     assert lib.splash_kv_page_migrate(p, None, p, None, 73728, p, p, 1, 0, 0, 1 << 20, p, 8, p, 64, None) == binding.SPLASH_INVALID_ARG
     assert lib.splash_kv_page_migrate_workspace_bytes(1000) >= 4000
+
+
+def test_dop_layout_changes_reject_bad_arguments(lib):
+    p, q = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x100000)
+    # empty work is legal (a rank that owns no rows still takes part in the exchange)
+    assert lib.splash_dop_pack_rows(p, 1024, 4096, 1024, p, 128, 512, 128, p, 0, 4, q, None) == binding.SPLASH_OK
+    assert lib.splash_dop_swap_outer(p, 4, 0, 64, q, None) == binding.SPLASH_OK
+    assert lib.splash_dop_unpack_rows(p, p, 0, 64, q, 64, None) == binding.SPLASH_OK
+    # odd sizes, missing pointers, a head pitch shorter than the part, overlapping buffers
+    assert lib.splash_dop_pack_rows(p, 1023, 4096, 1024, None, 0, 0, 0, p, 3, 4, q, None) == binding.SPLASH_INVALID_ARG
+    assert lib.splash_dop_pack_rows(p, 1024, 4096, 1024, None, 128, 512, 128, p, 3, 4, q, None) == binding.SPLASH_INVALID_ARG
+    assert lib.splash_dop_pack_rows(p, 1024, 4096, 512, None, 0, 0, 0, p, 3, 4, q, None) == binding.SPLASH_INVALID_ARG
+    assert lib.splash_dop_pack_rows(p, 1024, 4096, 1024, None, 0, 0, 0, None, 3, 4, q, None) == binding.SPLASH_INVALID_ARG
+    assert lib.splash_dop_swap_outer(p, 4, 4, 64, ctypes.c_void_p(0x1100), None) == binding.SPLASH_INVALID_ARG
+    assert lib.splash_dop_swap_outer(p, 4, 4, 63, q, None) == binding.SPLASH_INVALID_ARG
+    assert lib.splash_dop_unpack_rows(p, p, 3, 64, q, 32, None) == binding.SPLASH_INVALID_ARG
