@@ -354,6 +354,61 @@ class GpuBench:
                 "note": "includes the block-table restore copy issued before each call"}
 
 
+    def overlap_workload(self, w, dw, steps, warmup, layers=4):
+        """Layer-pipelined migration under decode (Sec. 4.1 "Handoff"): layer l's pages move on a second stream while
+        layer l - 1 decodes; decode of layer l waits for its pages.  All layers use this workload's arrays (the
+        migration writes the second pool and a copy of the table, so the decodes' inputs never change).  Reports the
+        time the migration adds to the decode-only sequence, in units of one layer's migration."""
+        torch, binding = self.torch, self.binding
+        total = w.num_pool_pages
+        extra_pages = int(np.ceil(len(w.used_pages) * 0.3))
+        n_src = total - extra_pages
+        src, dst = W.migration_plan(W.BASE_SEED + 55, w.used_pages, extra_pages, 0.3)
+        dsrc, ddst = torch.from_numpy(src).to(self.device), torch.from_numpy(dst).to(self.device)
+        table_next = dw.block_table.clone()
+        out = torch.empty((w.B, w.H, W.D_V), dtype=torch.float32, device=self.device)
+        lse = torch.empty((w.B, w.H), dtype=torch.float32, device=self.device)
+        side = torch.cuda.Stream(device=self.device)
+        mig_ws = torch.empty(int(binding.load().splash_kv_page_migrate_workspace_bytes(total)) + 256, dtype=torch.uint8, device=self.device)
+
+        def migrate(stream):
+            binding.splash_kv_page_migrate(dw.kv_pool[:n_src], dw.kv_pool[n_src:], dsrc, ddst, table_next,
+                                           src_scales=dw.kv_scales[:n_src], dst_scales=dw.kv_scales[n_src:],
+                                           src_id_base=0, dst_id_base=n_src, max_page_id=total, workspace=mig_ws, stream=stream)
+
+        def decode_only():
+            for _ in range(layers):
+                dw.decode(out=out, lse=lse)
+
+        def migrate_only():
+            for _ in range(layers):
+                migrate(None)
+
+        def pipelined():
+            main = torch.cuda.current_stream()
+            side.wait_stream(main)
+            started = None
+            for l in range(layers):
+                # layer l's pages move while layer l - 1 decodes
+                if started is not None:
+                    side.wait_event(started)
+                with torch.cuda.stream(side):
+                    migrate(side)
+                    moved = torch.cuda.Event(); moved.record(side)
+                main.wait_event(moved)
+                started = torch.cuda.Event(); started.record(main)
+                dw.decode(out=out, lse=lse)
+            main.wait_stream(side)
+
+        t_dec = float(np.median(self.timed(decode_only, steps, warmup)))
+        t_mig = float(np.median(self.timed(migrate_only, steps, warmup)))
+        t_pipe = float(np.median(self.timed(pipelined, steps, warmup)))
+        return {"layers": layers, "decode_only_ms": t_dec, "migrate_only_ms": t_mig, "pipelined_ms": t_pipe,
+                "serial_ms": t_dec + t_mig, "exposed_ms": t_pipe - t_dec,
+                "exposed_in_layer_migrations": (t_pipe - t_dec) / (t_mig / layers),
+                "pages_per_layer": int(len(src))}
+
+
 def run_reference(args, rank):
     """The oracle as the reference arm: each step is a bounded sample of the workload."""
     if rank != 0:
@@ -458,6 +513,7 @@ def main():
                         r["cp"] = gb.cp_workload(wx, max(5, args.steps // 2), args.warmup)
                     if name == "c5":
                         r["page_migrate"] = gb.migrate_workload(wx, dwx, max(5, args.steps // 2), args.warmup, peaks)
+                        r["migrate_under_decode"] = gb.overlap_workload(wx, dwx, max(5, args.steps // 2), args.warmup)
                     extra[name] = r
                     del wx, ox, lx
                     dwx = None
