@@ -60,7 +60,7 @@ def load_traffic():
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled every 200 ms while running."""
+    """nvidia-smi clocks and throttle reasons sampled every 100 ms while running."""
 
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -75,7 +75,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except Exception:
             self.proc = None
@@ -279,6 +279,22 @@ class GpuBench:
         res["shape"] = {"rows": N, "ranks": T, "local_heads": h}
         return res
 
+    def in_kernel_clock(self, dw, out, lse):
+        """SM clock seen by the decode kernel itself: cycles / nanoseconds of its main loop, per CTA, from the
+        library's diagnostic trace (written by the CTA-pair kernels; None for the others)."""
+        torch, binding = self.torch, self.binding
+        buf = torch.zeros(64 * 8 + 512, dtype=torch.int64, device=self.device)
+        binding.splash_debug_set_trace(buf)
+        try:
+            dw.decode(out=out, lse=lse)
+            torch.cuda.synchronize()
+        finally:
+            binding.splash_debug_set_trace(None)
+        t = buf.cpu().numpy()
+        cyc, ns = t[512:512 + 148].astype(np.float64), t[768:768 + 148].astype(np.float64)
+        ok = (cyc > 0) & (ns > 0)
+        return float(np.median(cyc[ok] / ns[ok]) * 1e3) if ok.any() else None
+
     def e2e(self, w, dw, steps, warmup):
         """Same call with the step's inputs coming from pinned host memory and the
         results going back to it inside the timed region."""
@@ -480,9 +496,18 @@ def main():
     sampler.start()
     main_res, dw, out, lse = gb.decode_workload(w, args.steps, args.warmup, peaks, traffic, args.workload)
     torch.cuda.synchronize()
+    # the timed region lasts a few milliseconds, less than one nvidia-smi sampling period: keep the same step
+    # running for about a second so that the sampler sees the clocks under this load
+    t_end = time.time() + 1.0
+    while time.time() < t_end:
+        for _ in range(20):
+            gb.flush_l2(); dw.decode(out=out, lse=lse)
+        torch.cuda.synchronize()
+    in_kernel_mhz = gb.in_kernel_clock(dw, out, lse)
     if world > 1:
         dist.barrier()
     clocks = sampler.stop()
+    clocks["sm_mhz_in_kernel"] = in_kernel_mhz
     e2e = gb.e2e(w, dw, args.steps, args.warmup)
 
     ms = main_res["ms_per_step"]
