@@ -58,7 +58,6 @@ enum BarrierId {
     kBarSFull,                         // [2]
     kBarSEmpty = kBarSFull + 2,        // [2]
     kBarPFull = kBarSEmpty + 2,
-    kBarPEmpty,
     kBarOFull,
     kBarOEmpty,
     kNumBarriers
@@ -156,7 +155,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
         for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kMmaWarps); }
         mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), L::kAcc);
         for (int b = 0; b < L::kSBufs; ++b) { mbar_init(bar(kBarSFull + b), L::kAcc); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxWarps); }
-        mbar_init(bar(kBarPFull), kNumSoftmaxWarps); mbar_init(bar(kBarPEmpty), 1);   // (PEmpty unused)
+        mbar_init(bar(kBarPFull), kNumSoftmaxWarps);
         mbar_init(bar(kBarOFull), kMmaWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxWarps);
         misc[1] = 0; misc[2] = 0; misc[3] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

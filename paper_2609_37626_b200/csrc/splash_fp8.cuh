@@ -56,14 +56,5 @@ __device__ __forceinline__ float fast_rcp(float x) {
     return y;
 }
 
-// Split x into hi + lo with hi carrying 4 significant bits (an e4m3 value when it is in
-// e4m3's normal range): Veltkamp's splitting with 2^20 + 1, all in the fp32 pipe.  The
-// intrinsics keep the compiler from contracting the steps into FMAs, which would undo it.
-__device__ __forceinline__ void split4(float x, float &hi, float &lo) {
-    const float c = __fmul_rn(x, 1048577.0f);
-    hi = __fsub_rn(c, __fsub_rn(c, x));
-    lo = __fsub_rn(x, hi);
-}
-
 }  // namespace umma
 }  // namespace splash

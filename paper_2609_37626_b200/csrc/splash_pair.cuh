@@ -21,9 +21,6 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
 // Arrival on a barrier of the other CTA that carries no data with it: a release at cluster scope
 // stalls the arriving thread for ~300 cycles and takes ~500 to land, the relaxed form ~20 and
 // ~200.  It is used where what the arrival announces is already in place on this SM when it is

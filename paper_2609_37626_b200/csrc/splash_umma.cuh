@@ -80,12 +80,6 @@ __device__ __forceinline__ bool mbar_wait(const Ctx &ctx, uint32_t bar, uint32_t
     return mbar_wait_slow(ctx, bar, parity, bar_id);
 }
 
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-
 // TMA store of a shared-memory tile (bulk async-group completion); coordinates outside the
 // tensor are clipped
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2) {
