@@ -180,14 +180,14 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                             tma_load_4d_pair(k0, &tmap_half, leader_bar(kBarKFull + stage), 0, g.tok0 + kHalf * (int)rank, 0, page);
                             // A stage is held from its load until P.V has read it, about three tiles, so the
                             // load of tile t + 3 starts only when the issuers are about to need it: have its
-                            // page in L2 by then (one CTA of the pair asks for even pages, the other for odd).
+                            // half of the page in L2 by then.
                             const int tf = tile + kPrefetchAhead;
-                            if (tf < seg.tile_end && ((tf & 1) == (int)rank)) {
+                            if (tf < seg.tile_end) {
                                 const int page_f = table[first_page + tf];
-                                if (page_f >= 0 && page_f < p.num_pool_pages) {
-                                    tma_prefetch_4d(&tmap_half, 0, 0, 0, page_f);
-                                    tma_prefetch_4d(&tmap_half, 0, kHalf, 0, page_f);
-                                }
+                                // this CTA's half of the page is 32 consecutive rows: one contiguous range
+                                if (page_f >= 0 && page_f < p.num_pool_pages)
+                                    bulk_prefetch_l2(static_cast<const uint8_t *>(p.kv_pool) + ((size_t)page_f * kPage + kHalf * rank) * (kDQK * 2),
+                                                     kStageBytes);
                             }
                         }
                     } else {
