@@ -99,6 +99,22 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
     const float inv_z = 1.f / Z;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     int j = 0;
+    // sixteen, then four part loads in flight per thread: one long context cut into a piece per worker is merged by
+    // one block per head, and the part loop is a chain of round trips to L2 / HBM
+    for (; j + 16 <= nparts; j += 16) {
+        float4 v[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u)
+            v[u] = reinterpret_cast<const float4 *>(p.partial_out + ((int64_t)slot_s[j + u] * h + k) * kDV)[c];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+            const float wgt = w_s[j + u] * inv_z;
+            if (wgt != 0.f) {          // a dead worker's slot holds stale bytes
+                acc.x = fmaf(wgt, v[u].x, acc.x); acc.y = fmaf(wgt, v[u].y, acc.y);
+                acc.z = fmaf(wgt, v[u].z, acc.z); acc.w = fmaf(wgt, v[u].w, acc.w);
+            }
+        }
+    }
     for (; j + 4 <= nparts; j += 4) {
         float4 v[4];
 #pragma unroll
