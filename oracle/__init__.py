@@ -175,6 +175,47 @@ def mla_decode_rows(q, kv_pool, block_table, seq_lens, *, softmax_scale, kv_scal
     return out, lse
 
 
+SPARSE_ROW_BYTES = 656
+
+
+def mla_decode_sparse(q, kv_pool, block_table, seq_lens, sel, sel_count, *, softmax_scale,
+                      head_begin=0, head_end=None, page_size=64):
+    """Decode attention over the listed tokens of a cache of 656-byte rows (see splash_oracle.c).
+
+    q [B][H][576] uint16 (bf16 bits); kv_pool [P][page_size][656] uint8; sel [B][K] int32 token
+    positions, request i uses the first sel_count[i].  Returns (out [B][H][512], lse [B][H]) float64,
+    NaN outside [head_begin, head_end).
+    """
+    lib = _load()
+    assert q.dtype == np.uint16 and q.ndim == 3 and q.strides[2] == 2 and q.shape[2] == 576
+    B, H, _ = q.shape
+    kv_pool = np.ascontiguousarray(kv_pool)
+    assert kv_pool.dtype == np.uint8 and kv_pool.shape[-1] == SPARSE_ROW_BYTES and kv_pool.shape[-2] == page_size
+    block_table = np.ascontiguousarray(block_table, dtype=np.int32)
+    if block_table.ndim == 1:
+        block_table = block_table.reshape(B, -1) if B else block_table.reshape(0, 1)
+    seq_lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    sel = np.ascontiguousarray(sel, dtype=np.int32)
+    if sel.ndim == 1:
+        sel = sel.reshape(B, -1) if B else sel.reshape(0, 1)
+    sel_count = np.ascontiguousarray(sel_count, dtype=np.int32)
+    assert sel_count.shape == (B,) and (B == 0 or sel_count.max() <= sel.shape[1])
+    if head_end is None:
+        head_end = H
+    out = np.full((B, H, 512), np.nan, dtype=np.float64)
+    lse = np.full((B, H), np.nan, dtype=np.float64)
+    rc = lib.oracle_mla_decode_sparse(
+        ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(page_size),
+        _ptr(q, ctypes.c_uint16), ctypes.c_int64(q.strides[0] // 2), ctypes.c_int64(q.strides[1] // 2),
+        _ptr(kv_pool, ctypes.c_uint8), _ptr(block_table, ctypes.c_int32), ctypes.c_int64(block_table.shape[1]),
+        _ptr(seq_lens, ctypes.c_int32), _ptr(sel, ctypes.c_int32), ctypes.c_int64(sel.shape[1]),
+        _ptr(sel_count, ctypes.c_int32), ctypes.c_int(head_begin), ctypes.c_int(head_end),
+        ctypes.c_double(float(softmax_scale)), _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"oracle_mla_decode_sparse rejected its arguments (rc={rc})")
+    return out, lse
+
+
 def lse_merge(part_out, part_lse):
     """Merge [parts][rows][d_v] partial outputs by their [parts][rows] LSE."""
     lib = _load()

@@ -18,8 +18,8 @@
  *     partial results are combined through their log-sum-exp.
  *
  * The attention formula itself is the textbook softmax attention; the paper
- * does not print it.  Readings of everything the paper leaves open (row
- * layout, LSE base, empty ranges, fp8 format) are listed in the design doc.
+ * does not print it; what the paper leaves open (row layout, LSE base, empty
+ * ranges, fp8 format) is stated at each function.
  *
  * Pins (tests/test_oracle_pins.py): closed forms (n = 1, n = 2, identical
  * V rows, q = 0), invariants (key shift, permutation of tokens and of page
@@ -135,6 +135,97 @@ int oracle_mla_decode(int B, int H, int d_qk, int d_v, int page_size,
             double w = exp(logit[t - lo] - m) / Z;
             for (int d = 0; d < d_v; ++d)
                 o[d] += w * kv_elem(kv_pool, kv_dtype, kv_scales, page, slot, d, d_qk, page_size);
+        }
+        free(logit);
+    }
+    return 0;
+}
+
+/*
+ * Sparse decode in the cache format of the paper's runs.
+ *
+ * The serving stack of the evaluation runs a SPARSE absorbed-MLA backend (Sec. 5,
+ * "Setup"): for every decode query an indexer has picked the tokens of the request's
+ * history that the query attends over, and attention is the same softmax attention as
+ * oracle_mla_decode restricted to that token list.  The cache row of that stack holds an
+ * FP8 latent with its scales and a BF16 rope part (App. B, the per-token KV payload;
+ * Sec. 5 "FP8 E4M3 KV").  The paper gives the contents, not the offsets; the byte layout
+ * read here is, per token, 656 bytes:
+ *     [0, 512)    e4m3 codes c_d of the latent, d = 0..511
+ *     [512, 528)  four float scales s_b, one per block of 128 latent dims
+ *     [528, 656)  64 bf16 rope values r_j
+ * so that the row's 576 key columns are  k_d = c_d * s_{d / 128}  (d < 512),  k_{512+j} = r_j,
+ * and the value read back is the latent, v_d = k_d (d < 512).
+ *
+ *   q           [B][H][576] bf16 bits, strides in elements
+ *   kv_pool     [P][page_size][656] bytes
+ *   sel         [B][sel_stride] int32: token positions within the request, in any order;
+ *               request i uses its first sel_count[i] entries.  An entry outside
+ *               [0, seq_lens[i]) is an argument error (returns -2, nothing defined).
+ *   out         [B][H][512] double, lse [B][H] double, written for heads [head_begin, head_end)
+ *
+ * A request with sel_count = 0 gives out = 0, lse = -inf.  A token listed twice counts twice.
+ */
+enum { SPARSE_ROW_BYTES = 656, SPARSE_D_LATENT = 512, SPARSE_D_ROPE = 64, SPARSE_BLOCK = 128 };
+
+static double sparse_row_elem(const uint8_t *row, int d) {
+    if (d < SPARSE_D_LATENT) {
+        float s;
+        memcpy(&s, row + SPARSE_D_LATENT + 4 * (d / SPARSE_BLOCK), sizeof s);
+        return oracle_e4m3_to_double(row[d]) * (double)s;
+    }
+    uint16_t bits;
+    memcpy(&bits, row + SPARSE_D_LATENT + 16 + 2 * (d - SPARSE_D_LATENT), sizeof bits);
+    return bf16_to_double(bits);
+}
+
+int oracle_mla_decode_sparse(int B, int H, int page_size,
+                             const uint16_t *q, int64_t q_stride_b, int64_t q_stride_h,
+                             const uint8_t *kv_pool,
+                             const int32_t *block_table, int64_t table_stride,
+                             const int32_t *seq_lens,
+                             const int32_t *sel, int64_t sel_stride, const int32_t *sel_count,
+                             int head_begin, int head_end, double softmax_scale,
+                             double *out, double *lse) {
+    const int d_qk = SPARSE_D_LATENT + SPARSE_D_ROPE, d_v = SPARSE_D_LATENT;
+    int h = head_end - head_begin;
+    if (h < 0 || head_begin < 0 || head_end > H) return -1;
+    for (int i = 0; i < B; ++i)
+        for (int j = 0; j < sel_count[i]; ++j) {
+            int t = sel[i * sel_stride + j];
+            if (t < 0 || t >= seq_lens[i]) return -2;
+        }
+    int64_t total = (int64_t)B * h;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t job = 0; job < total; ++job) {
+        int i = (int)(job / h), g = head_begin + (int)(job % h);
+        int n = sel_count[i];
+        double *o = out + ((int64_t)i * H + g) * d_v;
+        double *L = lse + (int64_t)i * H + g;
+        for (int d = 0; d < d_v; ++d) o[d] = 0.0;
+        if (n <= 0) { *L = -INFINITY; continue; }
+        const uint16_t *qrow = q + i * q_stride_b + g * q_stride_h;
+        double *logit = (double *)malloc(sizeof(double) * (size_t)n);
+        double m = -INFINITY;
+        for (int j = 0; j < n; ++j) {
+            int t = sel[i * sel_stride + j];
+            int64_t page = block_table[i * table_stride + t / page_size];
+            const uint8_t *row = kv_pool + (page * page_size + t % page_size) * SPARSE_ROW_BYTES;
+            double acc = 0.0;
+            for (int d = 0; d < d_qk; ++d) acc += bf16_to_double(qrow[d]) * sparse_row_elem(row, d);
+            logit[j] = softmax_scale * acc;
+            if (logit[j] > m) m = logit[j];
+        }
+        double Z = 0.0;
+        for (int j = 0; j < n; ++j) Z += exp(logit[j] - m);
+        *L = m + log(Z);
+        for (int j = 0; j < n; ++j) {
+            int t = sel[i * sel_stride + j];
+            int64_t page = block_table[i * table_stride + t / page_size];
+            const uint8_t *row = kv_pool + (page * page_size + t % page_size) * SPARSE_ROW_BYTES;
+            double w = exp(logit[j] - m) / Z;
+            for (int d = 0; d < d_v; ++d) o[d] += w * sparse_row_elem(row, d);
         }
         free(logit);
     }

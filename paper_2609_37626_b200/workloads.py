@@ -76,11 +76,57 @@ def quantize_e4m3_per_token(x: np.ndarray):
     return codes, scale
 
 
+SPARSE_ROW_BYTES = 656        # 512 e4m3 latent codes, 4 float block scales, 64 bf16 rope values
+SPARSE_BLOCK = 128            # latent dims per scale
+
+
+def pack_sparse_rows(x: np.ndarray) -> np.ndarray:
+    """Rows of 576 float32 -> rows of 656 bytes: the latent quantised to e4m3 in blocks of 128 dims
+    (scale = max|x| / 448 over the block, 1 for an all-zero block; code = RNE(clamp(x / scale, +-448))),
+    the four scales, the rope part rounded to bf16."""
+    import torch
+
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    n = x.shape[0]
+    lat = x[:, :D_LATENT].reshape(n, D_LATENT // SPARSE_BLOCK, SPARSE_BLOCK)
+    amax = np.abs(lat).max(axis=-1)
+    scale = np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
+    y = np.clip(lat / scale[..., None], -448.0, 448.0).astype(np.float32)
+    codes = torch.from_numpy(y).to(torch.float8_e4m3fn).view(torch.uint8).numpy().reshape(n, D_LATENT)
+    out = np.empty((n, SPARSE_ROW_BYTES), dtype=np.uint8)
+    out[:, :D_LATENT] = codes
+    out[:, D_LATENT:D_LATENT + 16] = scale.view(np.uint8).reshape(n, 16)
+    out[:, D_LATENT + 16:] = f32_to_bf16_bits(x[:, D_LATENT:]).view(np.uint8).reshape(n, 2 * D_ROPE)
+    return out
+
+
+def select_tokens(seed: int, seq_lens, topk: int):
+    """The token list an indexer would hand to sparse decode: for every request min(topk, s) distinct
+    positions drawn uniformly from its history, in random order (the worst case for locality).
+    Returns (sel [B][topk] int32, -1 beyond the count; sel_count [B] int32)."""
+    seq_lens = np.asarray(seq_lens, dtype=np.int32)
+    B = int(seq_lens.shape[0])
+    sel = np.full((B, max(topk, 1)), -1, dtype=np.int32)
+    cnt = np.minimum(seq_lens, topk).astype(np.int32)
+    for i in range(B):
+        rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 11, i])))
+        s, k = int(seq_lens[i]), int(cnt[i])
+        if k:
+            sel[i, :k] = rng.permutation(s)[:k] if s <= 4 * k else rng.choice(s, size=k, replace=False)
+    return sel, cnt
+
+
+def sparse_algorithmic_bytes(sel_count, h: int) -> int:
+    """Sparse decode: every listed row once (656 B) and its list entry, the q slice read, out + lse written."""
+    n, B = int(np.asarray(sel_count).sum()), len(sel_count)
+    return n * (SPARSE_ROW_BYTES + 4) + B * h * D_QK * 2 + B * h * (D_V + 1) * 4 + 8 * B
+
+
 @dataclasses.dataclass
 class Workload:
     name: str
     q: np.ndarray                       # [B][H][576] uint16 (bf16 bits)
-    kv_pool: np.ndarray                 # [P][64][576] uint16 (bf16) or uint8 (e4m3)
+    kv_pool: np.ndarray                 # [P][64][576] uint16 (bf16) or uint8 (e4m3), or [P][64][656] uint8 (kv_dtype 2)
     kv_scales: Optional[np.ndarray]     # [P][64] float32 for e4m3, else None
     block_table: np.ndarray             # [B][stride] int32, -1 beyond the last page
     seq_lens: np.ndarray                # [B] int32
@@ -102,7 +148,9 @@ class Workload:
 
     @property
     def kv_dtype(self) -> int:
-        return 0 if self.kv_pool.dtype == np.uint16 else 1
+        if self.kv_pool.dtype == np.uint16:
+            return 0
+        return 1 if self.kv_pool.shape[-1] == D_QK else 2
 
     @property
     def num_pool_pages(self) -> int:
@@ -134,8 +182,9 @@ def make_workload(name: str, seed: int, seq_lens, H: int, *, head_begin: int = 0
                   extra_pool_pages: int = 0) -> Workload:
     """Draw q and a paged latent cache for the given context lengths.
 
-    Values are i.i.d. N(0,1) (rotary columns times ``rope_scale``) rounded to bf16,
-    or quantised to e4m3 with one scale per token.  Pages are dealt to requests in
+    Values are i.i.d. N(0,1) (rotary columns times ``rope_scale``) rounded to bf16 (``kv_dtype`` 0),
+    quantised to e4m3 with one scale per token (1), or packed into 656-byte rows (2: e4m3 latent with a
+    scale per 128 dims, bf16 rope; ``pack_sparse_rows``).  Pages are dealt to requests in
     order from a seeded permutation of the pool (``placement``: "permute",
     "identity" or "reversed").  Every byte the attention must not read (unused
     pages, slots past the end of a request's last page, table padding) is poisoned
@@ -186,6 +235,10 @@ def make_workload(name: str, seed: int, seq_lens, H: int, *, head_begin: int = 0
             kv_pool[:, 1::2, :] = BF16_INF
         else:
             kv_pool[...] = 0
+    elif kv_dtype == 2:
+        kv_pool = np.empty((total_pages, PAGE_SIZE, SPARSE_ROW_BYTES), dtype=np.uint8)
+        kv_scales = None
+        kv_pool[...] = 0xFF if poison else 0          # NaN as an e4m3 code, as a float scale and as a bf16
     else:
         kv_pool = np.empty((total_pages, PAGE_SIZE, D_QK), dtype=np.uint8)
         kv_scales = np.empty((total_pages, PAGE_SIZE), dtype=np.float32)
@@ -230,6 +283,12 @@ def make_workload(name: str, seed: int, seq_lens, H: int, *, head_begin: int = 0
                 kv_pool[ids[:full]] = bits[:full * PAGE_SIZE].reshape(full, PAGE_SIZE, D_QK)
             if rem:
                 kv_pool[ids[full], :rem] = bits[full * PAGE_SIZE:]
+        elif kv_dtype == 2:
+            packed = pack_sparse_rows(rows)
+            if full:
+                kv_pool[ids[:full]] = packed[:full * PAGE_SIZE].reshape(full, PAGE_SIZE, SPARSE_ROW_BYTES)
+            if rem:
+                kv_pool[ids[full], :rem] = packed[full * PAGE_SIZE:]
         else:
             codes, sc = quantize_e4m3_per_token(rows)
             if full:
