@@ -54,7 +54,14 @@ typedef enum splash_status {
     SPLASH_DEVICE_TIMEOUT = -5      /* (status word only) a bounded device wait gave up */
 } splash_status;
 
-enum { SPLASH_KV_BF16 = 0, SPLASH_KV_E4M3_TOKEN_SCALE = 1 };
+enum {
+    SPLASH_KV_BF16 = 0,
+    SPLASH_KV_E4M3_TOKEN_SCALE = 1,
+    /* 656-byte rows: 512 e4m3 latent codes, 4 fp32 scales (one per 128 latent dims), 64 bf16 rope values.
+     * Only splash_mla_decode_sparse reads this format. */
+    SPLASH_KV_E4M3_BLOCK_SCALE_BF16_ROPE = 2
+};
+#define SPLASH_SPARSE_ROW_BYTES 656
 
 /* shape.flags bits */
 enum {
@@ -152,6 +159,46 @@ SPLASH_API int splash_mla_decode(const splash_mla_shape *shape,
  * count.  Returns 0 on invalid arguments. */
 SPLASH_API size_t splash_mla_decode_workspace_bytes(const splash_mla_shape *shape,
                                          int32_t head_begin, int32_t head_end);
+
+/*
+ * Sparse decode: attention over a LIST of tokens per request instead of a range (the sparse
+ * absorbed-MLA backend of the paper's runs, Sec. 5 "Setup": an indexer has selected the tokens
+ * each decode query attends over), reading the cache row format of those runs (FP8 latent with
+ * its scales, BF16 rope; Sec. 5, App. B payload).  Per token the row is 656 bytes:
+ *     [0, 512)    e4m3 codes c_d of the latent
+ *     [512, 528)  four fp32 scales s_b, b = d / 128
+ *     [528, 656)  64 bf16 rope values r_j
+ * with key columns k_d = c_d * s_{d/128} (d < 512), k_{512+j} = r_j and value v_d = k_d (d < 512).
+ * For request i and head g in [head_begin, head_end), with T_i the first sel_count[i] entries
+ * of sel_tokens[i * sel_stride ...] (token positions of request i, any order):
+ *     l_t = softmax_scale * q[i][g] . k(t),  lse = ln sum_{t in T_i} exp(l_t),
+ *     out = sum_{t in T_i} exp(l_t - lse) v(t)
+ * sel_count[i] = 0 gives out = 0, lse = -inf; a position listed twice counts twice.
+ *
+ *   shape        kv_dtype = SPLASH_KV_E4M3_BLOCK_SCALE_BF16_ROPE, q_rows 0 or 1; the other fields
+ *                as for splash_mla_decode
+ *   kv_pool      [num_pool_pages][64][656] bytes (41,984 B / page), 128-byte aligned
+ *   sel_tokens   int32; entry j of request i at sel_tokens[i * sel_stride + j]; entries at or
+ *                beyond sel_count[i] are never read
+ *   sel_count    [num_requests] int32, each in [0, max_selected]
+ *   max_selected bound on sel_count (the indexer's k, e.g. 2048); sizes the workspace
+ *   workspace    at least splash_mla_decode_sparse_workspace_bytes() bytes, 256-byte aligned
+ *
+ * All pointers are device pointers.  A list entry outside [0, seq_lens[i]), a page id outside
+ * the pool or a count outside [0, max_selected] is never dereferenced; the outputs of that
+ * request are then NaN.  Two stages on the device: the listed rows are gathered and dequantised
+ * (code times block scale, rounded to bf16) into a dense bf16 cache inside the workspace, then
+ * the dense decode kernels run over it.
+ */
+SPLASH_API int splash_mla_decode_sparse(const splash_mla_shape *shape, const void *q, const void *kv_pool,
+                             const int32_t *block_table, const int32_t *seq_lens,
+                             const int32_t *sel_tokens, int64_t sel_stride, const int32_t *sel_count,
+                             int32_t max_selected, int32_t head_begin, int32_t head_end,
+                             float *out, float *lse, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Workspace size for splash_mla_decode_sparse (host computation).  Returns 0 on invalid arguments. */
+SPLASH_API size_t splash_mla_decode_sparse_workspace_bytes(const splash_mla_shape *shape, int32_t max_selected,
+                                                int32_t head_begin, int32_t head_end);
 
 /*
  * Merge partial attention results over disjoint KV ranges (the CP combination step;

@@ -22,6 +22,8 @@ SPLASH_CUDA_ERROR = -4
 SPLASH_DEVICE_TIMEOUT = -5
 SPLASH_KV_BF16 = 0
 SPLASH_KV_E4M3_TOKEN_SCALE = 1
+SPLASH_KV_E4M3_BLOCK_SCALE_BF16_ROPE = 2
+SPLASH_SPARSE_ROW_BYTES = 656
 SPLASH_FLAG_SIMT = 1
 SPLASH_FLAG_NO_PAIR = 2
 
@@ -74,6 +76,10 @@ def load() -> ctypes.CDLL:
     lib.splash_mla_decode.argtypes = [ctypes.POINTER(MlaShape), vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.splash_mla_decode_workspace_bytes.restype = sz
     lib.splash_mla_decode_workspace_bytes.argtypes = [ctypes.POINTER(MlaShape), i32, i32]
+    lib.splash_mla_decode_sparse.restype = ctypes.c_int
+    lib.splash_mla_decode_sparse.argtypes = [ctypes.POINTER(MlaShape), vp, vp, vp, vp, vp, i64, vp, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.splash_mla_decode_sparse_workspace_bytes.restype = sz
+    lib.splash_mla_decode_sparse_workspace_bytes.argtypes = [ctypes.POINTER(MlaShape), i32, i32, i32]
     lib.splash_lse_merge.restype = ctypes.c_int
     lib.splash_lse_merge.argtypes = [i32, i64, i32, vp, vp, vp, vp, vp]
     lib.splash_kv_page_migrate.restype = ctypes.c_int
@@ -130,7 +136,10 @@ def make_shape(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch.Tensor
     else:
         B, H, dqk = q.shape
         assert q.stride(2) == 1 and out.stride(2) == 1 and lse.stride(1) == 1
-    kv_dtype = SPLASH_KV_BF16 if kv_pool.dtype == torch.bfloat16 else SPLASH_KV_E4M3_TOKEN_SCALE
+    if kv_pool.dtype == torch.bfloat16:
+        kv_dtype = SPLASH_KV_BF16
+    else:
+        kv_dtype = SPLASH_KV_E4M3_BLOCK_SCALE_BF16_ROPE if kv_pool.shape[-1] == SPLASH_SPARSE_ROW_BYTES else SPLASH_KV_E4M3_TOKEN_SCALE
     return MlaShape(
         struct_size=ctypes.sizeof(MlaShape), num_requests=B, num_heads=H, d_qk=dqk, d_v=out.shape[-1],
         page_size=kv_pool.shape[1], num_pool_pages=kv_pool.shape[0],
@@ -191,6 +200,51 @@ def splash_mla_decode(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch
                                _ptr(seq_lens), head_begin, head_end, _ptr(kv_begin), _ptr(kv_end),
                                _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel() * workspace.element_size(),
                                _stream_ptr(stream))
+    _check(rc)
+    return out, lse
+
+
+def splash_mla_decode_sparse_workspace_bytes(shape: MlaShape, max_selected: int, head_begin: int, head_end: int) -> int:
+    return int(load().splash_mla_decode_sparse_workspace_bytes(ctypes.byref(shape), max_selected, head_begin, head_end))
+
+
+def splash_mla_decode_sparse(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch.Tensor, seq_lens: torch.Tensor,
+                             sel_tokens: torch.Tensor, sel_count: torch.Tensor, *, softmax_scale: float,
+                             max_selected: Optional[int] = None, head_begin: int = 0, head_end: Optional[int] = None,
+                             out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                             workspace: Optional[torch.Tensor] = None, stream: Optional[torch.cuda.Stream] = None,
+                             flags: int = 0):
+    """Decode attention over a token list per request; see ``splash_mla_decode_sparse`` in include/splash_mla.h.
+
+    q [B][H][576] bf16; kv_pool [P][64][656] uint8 (e4m3 latent, four block scales, bf16 rope per row);
+    sel_tokens [B][K] int32 token positions, request i uses the first sel_count[i] (<= max_selected, default K).
+    Returns (out [B][H][512] fp32, lse [B][H] fp32).
+    """
+    lib = load()
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.dim() == 3
+    assert kv_pool.dtype == torch.uint8 and kv_pool.shape[-1] == SPLASH_SPARSE_ROW_BYTES and kv_pool.is_contiguous()
+    assert sel_tokens.dtype == torch.int32 and sel_count.dtype == torch.int32 and sel_tokens.dim() == 2
+    assert sel_tokens.numel() == 0 or sel_tokens.stride(1) == 1
+    assert block_table.dtype == torch.int32 and seq_lens.dtype == torch.int32
+    B, H = q.shape[0], q.shape[1]
+    if head_end is None:
+        head_end = H
+    if max_selected is None:
+        max_selected = sel_tokens.shape[1]
+    if out is None:
+        out = torch.empty((B, H, D_V), dtype=torch.float32, device=q.device)
+    if lse is None:
+        lse = torch.empty((B, H), dtype=torch.float32, device=q.device)
+    shape = make_shape(q, kv_pool, block_table, out, lse, softmax_scale, flags)
+    if workspace is None:
+        need = splash_mla_decode_sparse_workspace_bytes(shape, max_selected, head_begin, head_end)
+        if need == 0:
+            _check(SPLASH_INVALID_ARG)
+        workspace = _workspace(q.device, need, "decode")
+    rc = lib.splash_mla_decode_sparse(ctypes.byref(shape), _ptr(q), _ptr(kv_pool), _ptr(block_table), _ptr(seq_lens),
+                                      _ptr(sel_tokens), sel_tokens.stride(0) if B > 0 else 0, _ptr(sel_count), max_selected,
+                                      head_begin, head_end, _ptr(out), _ptr(lse), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream_ptr(stream))
     _check(rc)
     return out, lse
 
@@ -357,7 +411,7 @@ class DeviceWorkload:
             self.kv_scales = None
         else:
             self.kv_pool = torch.from_numpy(w.kv_pool).to(dev)
-            self.kv_scales = torch.from_numpy(w.kv_scales).to(dev)
+            self.kv_scales = None if w.kv_scales is None else torch.from_numpy(w.kv_scales).to(dev)
         self.block_table = torch.from_numpy(w.block_table).to(dev)
         self.seq_lens = torch.from_numpy(w.seq_lens).to(dev)
         self.kv_begin = None if w.kv_begin is None else torch.from_numpy(w.kv_begin).to(dev)

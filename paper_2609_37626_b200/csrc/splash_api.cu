@@ -233,6 +233,81 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     return SPLASH_OK;
 }
 
+namespace {
+
+// Workspace of a sparse call: [dense decode workspace][dense lens B][dense table B * ppr][dense cache].
+struct SparseView {
+    splash_mla_shape dense;        // the shape of the dense call over the gathered cache
+    int pages_per_request;
+    size_t inner_bytes, off_lens, off_table, off_pool, bytes;
+};
+
+bool make_sparse_view(const splash_mla_shape *shape, int32_t max_selected, int32_t head_begin, int32_t head_end, SparseView &v) {
+    if (shape == nullptr || shape->struct_size != sizeof(splash_mla_shape)) { set_error("shape is NULL or of another version"); return false; }
+    if (shape->kv_dtype != SPLASH_KV_E4M3_BLOCK_SCALE_BF16_ROPE) { set_error("sparse decode reads kv_dtype 2 (656-byte rows) only"); return false; }
+    if (shape->q_rows > 1) { set_error("sparse decode takes one query row per request"); return false; }
+    if (max_selected < 0 || max_selected > (1 << 20)) { set_error("max_selected must be in [0, 2^20]"); return false; }
+    v.dense = *shape;
+    v.dense.kv_dtype = SPLASH_KV_BF16;
+    v.pages_per_request = max_selected > 0 ? (max_selected + kPage - 1) / kPage : 1;
+    const int64_t pages = (int64_t)shape->num_requests * v.pages_per_request;
+    if (pages > 0x7fffffffLL / kPage) { set_error("num_requests * max_selected is too large"); return false; }
+    v.dense.num_pool_pages = (int32_t)pages;
+    v.dense.block_table_stride = v.pages_per_request;
+    if (check_shape(&v.dense, head_begin, head_end) != SPLASH_OK) return false;
+    v.inner_bytes = splash_mla_decode_workspace_bytes(&v.dense, head_begin, head_end);
+    if (v.inner_bytes == 0) return false;
+    size_t off = align_up(v.inner_bytes, 256);
+    v.off_lens = off; off = align_up(off + sizeof(int32_t) * (size_t)shape->num_requests, 256);
+    v.off_table = off; off = align_up(off + sizeof(int32_t) * (size_t)pages, 256);
+    v.off_pool = off; off += (size_t)pages * kPage * kDQK * 2;
+    v.bytes = align_up(off, 256);
+    return true;
+}
+
+}  // namespace
+
+size_t splash_mla_decode_sparse_workspace_bytes(const splash_mla_shape *shape, int32_t max_selected, int32_t head_begin,
+                                                int32_t head_end) {
+    SparseView v;
+    return make_sparse_view(shape, max_selected, head_begin, head_end, v) ? v.bytes : 0;
+}
+
+int splash_mla_decode_sparse(const splash_mla_shape *shape, const void *q, const void *kv_pool, const int32_t *block_table,
+                             const int32_t *seq_lens, const int32_t *sel_tokens, int64_t sel_stride, const int32_t *sel_count,
+                             int32_t max_selected, int32_t head_begin, int32_t head_end, float *out, float *lse,
+                             void *workspace, size_t workspace_bytes, void *stream_) {
+    g_launches = 0;
+    SparseView v;
+    if (!make_sparse_view(shape, max_selected, head_begin, head_end, v)) return SPLASH_INVALID_ARG;
+    const int B = shape->num_requests;
+    if (B == 0 || head_end == head_begin) return SPLASH_OK;
+    if (!q || !kv_pool || !block_table || !seq_lens || !sel_count || !out || !lse || !workspace || (max_selected > 0 && !sel_tokens)) {
+        set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG;
+    }
+    if (!aligned(kv_pool, 128) || !aligned(workspace, 256) || !aligned(sel_tokens, 4) || !aligned(sel_count, 4) ||
+        !aligned(block_table, 4) || !aligned(seq_lens, 4)) {
+        set_error("misaligned pointer (kv_pool 128 B, workspace 256 B)"); return SPLASH_INVALID_ARG;
+    }
+    if (sel_stride < max_selected && B > 1) { set_error("sel_stride < max_selected"); return SPLASH_INVALID_ARG; }
+    if (workspace_bytes < v.bytes) { set_error("workspace has %zu bytes, %zu needed", workspace_bytes, v.bytes); return SPLASH_INVALID_ARG; }
+    DeviceInfo dev;
+    if (!current_device_info(dev)) return SPLASH_CUDA_ERROR;
+    if (dev.cc_major != 10) { set_error("device compute capability %d.x is not 10.x", dev.cc_major); return SPLASH_UNSUPPORTED_DEVICE; }
+    char *ws = static_cast<char *>(workspace);
+    int32_t *dense_lens = reinterpret_cast<int32_t *>(ws + v.off_lens);
+    int32_t *dense_table = reinterpret_cast<int32_t *>(ws + v.off_table);
+    void *dense_pool = ws + v.off_pool;
+    cudaError_t e = launch_sparse_gather(B, max_selected, v.pages_per_request, kv_pool, shape->num_pool_pages, block_table,
+                                         shape->block_table_stride, seq_lens, sel_tokens, sel_stride, sel_count, dense_pool,
+                                         dense_table, dense_lens, dev.sm_count, static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+    const int rc = splash_mla_decode(&v.dense, q, dense_pool, nullptr, dense_table, dense_lens, head_begin, head_end, nullptr,
+                                     nullptr, out, lse, workspace, v.inner_bytes, stream_);
+    count_launch();      // the gather kernel, on top of the dense call's launches
+    return rc;
+}
+
 int splash_lse_merge(int32_t num_parts, int64_t rows, int32_t d_v, const float *part_out, const float *part_lse,
                      float *out, float *lse, void *stream_) {
     g_launches = 0;

@@ -14,6 +14,7 @@ constexpr int kDQK = 576;        // d_c + d_r (absorbed MLA row width)
 constexpr int kMaxQRows = 8;      // query rows per request (multi-token decode steps, short prefill chunks)
 constexpr int kDV = 512;         // d_c (value width)
 constexpr int kDRope = 64;
+constexpr int kDLatent = 512;
 constexpr int kPage = 64;        // tokens per page
 constexpr int kMaxHeads = 128;
 // largest page id (exclusive) the allocation-free migrate entry point can remap: 1 MiB of table
@@ -202,6 +203,10 @@ cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const in
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
                         int32_t *status, cudaStream_t stream);
+cudaError_t launch_sparse_gather(int B, int max_sel, int pages_per_request, const void *kv_pool, int num_pool_pages,
+                                 const int32_t *block_table, int64_t table_stride, const int32_t *seq_lens,
+                                 const int32_t *sel, int64_t sel_stride, const int32_t *sel_count, void *dense_pool,
+                                 int32_t *dense_table, int32_t *dense_lens, int sm_count, cudaStream_t stream);
 cudaError_t launch_dop_pack_rows(const void *a, const void *b, void *out, const int32_t *send_row, int64_t n, int h,
                                  int64_t a_bytes, int64_t b_bytes, int64_t a_row_pitch, int64_t a_head_pitch,
                                  int64_t b_row_pitch, int64_t b_head_pitch, int sm_count, cudaStream_t stream);
