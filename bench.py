@@ -251,6 +251,47 @@ class GpuBench:
                              "passes_over_the_cache": -(-h * R // 128)},
                 "launches_per_step": binding.splash_last_launch_count()}
 
+    def sparse_workload(self, seq_lens, H, steps, warmup, peaks, topk=2048):
+        """Sparse decode: every request attends over the (at most) topk tokens of a seeded list, cache rows in the
+        656-byte format.  Whole-call time; the roofline is each LISTED row once over the measured copy bandwidth."""
+        torch, binding = self.torch, self.binding
+        w = W.make_workload("sparse_top%d" % topk, W.BASE_SEED + 60, seq_lens, H=H, kv_dtype=2)
+        sel_h, cnt_h = W.select_tokens(W.BASE_SEED + 60, w.seq_lens, topk)
+        dw = binding.DeviceWorkload(w, self.device)
+        sel, cnt = torch.from_numpy(sel_h).to(self.device), torch.from_numpy(cnt_h).to(self.device)
+        out = torch.empty((w.B, w.H, W.D_V), dtype=torch.float32, device=self.device)
+        lse = torch.empty((w.B, w.H), dtype=torch.float32, device=self.device)
+        step = lambda: binding.splash_mla_decode_sparse(dw.q, dw.kv_pool, dw.block_table, dw.seq_lens, sel, cnt,
+                                                        softmax_scale=w.softmax_scale, out=out, lse=lse)
+        ms = self.timed(step, steps, warmup)
+        launches = binding.splash_last_launch_count()
+        binding.splash_set_kernel_timing(True)
+        kt = []
+        for _ in range(steps):
+            self.flush_l2(); step()
+            kt.append(binding.splash_get_kernel_timing())
+        binding.splash_set_kernel_timing(False)
+        kt = np.array(kt)
+        rc, detail = binding.splash_workspace_status(binding.decode_workspace(torch.device(self.device)))
+        if rc != 0:
+            raise RuntimeError(f"device status {rc} {detail}")
+        n_sel = int(cnt_h.sum())
+        alg_bytes = W.sparse_algorithmic_bytes(cnt_h, H)
+        alg_flops = 2 * H * (W.D_QK + W.D_V) * n_sel
+        t_hbm, t_tensor = alg_bytes / (peaks["hbm_gbs"] * 1e9), alg_flops / (peaks["bf16_tflops"] * 1e12)
+        p50 = float(np.median(ms))
+        return {"requests": w.B, "heads": H, "topk": topk, "listed_tokens": n_sel, "context_tokens": w.total_tokens(),
+                "row_bytes": W.SPARSE_ROW_BYTES, "ms_per_step": float(ms.mean()), "ms_p50": p50,
+                "ms_p95": float(np.percentile(ms, 95)), "tokens_per_s": w.B / (ms.mean() * 1e-3),
+                "stages_ms": {"gather_dequant": p50 - float(kt.sum(axis=1).mean()), "plan": float(kt[:, 0].mean()),
+                              "dense_decode": float(kt[:, 1].mean()), "combine": float(kt[:, 2].mean()),
+                              "note": "gather = whole call p50 minus the three timed kernels"},
+                "roofline": {"bound": "hbm" if t_hbm >= t_tensor else "tensor", "roofline_ms": max(t_hbm, t_tensor) * 1e3,
+                             "frac": max(t_hbm, t_tensor) * 1e3 / p50, "of": "whole call, p50", "peak_source": peaks["source"],
+                             "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
+                             "bytes_moved_by_the_two_stages": n_sel * (W.SPARSE_ROW_BYTES + 2 * W.D_QK * 2)},
+                "launches_per_step": launches}
+
     def dop_workload(self, steps, warmup, peaks, N=16384, T=8, h=16):
         """DOP transfer layout changes at a rank's size of a large batch: N query rows, h = H/T local heads;
         bytes read + written over the measured copy bandwidth."""
@@ -505,6 +546,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--only-main", action="store_true", help="skip the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sparse-only", action="store_true", help="print only the sparse-decode workload's numbers")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -535,6 +577,10 @@ def main():
         w = W.make_workload(w.name, W.BASE_SEED + idx + 100 * rank, w.seq_lens, H=w.H, head_begin=w.head_begin,
                             head_end=w.head_end, kv_dtype=w.kv_dtype)
     gen_s = time.time() - t_gen
+
+    if args.sparse_only:
+        print(json.dumps({"sparse_top2048": gb.sparse_workload(w.seq_lens, w.H, args.steps, args.warmup, peaks)}))
+        return
 
     sampler = ClockSampler(local_rank)
     if world > 1:
@@ -597,6 +643,12 @@ def main():
                 torch.cuda.empty_cache()
             except Exception as exc:
                 extra["dop_layout_changes"] = {"error": repr(exc)}
+            # sparse decode over the main workload's context lengths, 2048 listed tokens per request
+            try:
+                extra["sparse_top2048"] = gb.sparse_workload(w.seq_lens, w.H, max(5, args.steps // 2), args.warmup, peaks)
+                torch.cuda.empty_cache()
+            except Exception as exc:
+                extra["sparse_top2048"] = {"error": repr(exc)}
             # several causal query rows per request on the main workload's cache (multi-token decode steps)
             for R in (2, 4):
                 try:
