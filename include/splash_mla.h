@@ -188,7 +188,8 @@ SPLASH_API size_t splash_mla_decode_workspace_bytes(const splash_mla_shape *shap
  * the pool or a count outside [0, max_selected] is never dereferenced; the outputs of that
  * request are then NaN.  Two stages on the device: the listed rows are gathered and dequantised
  * (code times block scale, rounded to bf16) into a dense bf16 cache inside the workspace, then
- * the dense decode kernels run over it.
+ * the dense decode kernels run over it (launch order: plan over the list counts, gather,
+ * decode kernel, combine).
  */
 SPLASH_API int splash_mla_decode_sparse(const splash_mla_shape *shape, const void *q, const void *kv_pool,
                              const int32_t *block_table, const int32_t *seq_lens,
@@ -327,7 +328,8 @@ SPLASH_API int splash_last_launch_count(void);
  * kernels (plan, decode, split combine); the events are created on first use.
  * splash_get_kernel_timing() synchronises on the last call's final event and returns
  * the three durations in milliseconds (host pointers, each may be NULL).  Off by
- * default; enabling it adds four event records per call and nothing else.
+ * default; enabling it adds four event records per call and nothing else.  For
+ * splash_mla_decode_sparse the decode figure covers the gather kernel and the decode kernel.
  */
 SPLASH_API int splash_set_kernel_timing(int enable);
 SPLASH_API int splash_get_kernel_timing(float *plan_ms, float *decode_ms, float *combine_ms);

@@ -153,10 +153,28 @@ size_t splash_mla_decode_workspace_bytes(const splash_mla_shape *shape, int32_t 
     return align_up(need, 256);
 }
 
-int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *kv_pool, const float *kv_scales,
-                      const int32_t *block_table, const int32_t *seq_lens, int32_t head_begin, int32_t head_end,
-                      const int32_t *kv_begin, const int32_t *kv_end, float *out, float *lse,
-                      void *workspace, size_t workspace_bytes, void *stream_) {
+}  // extern "C"
+
+namespace {
+
+// The first stage of a sparse call: gathers the listed rows into the dense cache that the decode then reads.
+struct SparseStage {
+    const void *pool656;
+    int num_pool_pages;
+    const int32_t *block_table;
+    int64_t table_stride;
+    const int32_t *ctx_lens, *sel, *sel_count;
+    int64_t sel_stride;
+    int max_selected, pages_per_request;
+    int32_t *dense_table;
+};
+
+// One dense decode call: plan, decode kernel, combine.  With a sparse stage, seq_lens are the list counts, kv_pool
+// and block_table the dense cache and its table, and the gather kernel runs between the plan and the decode kernel.
+int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_pool, const float *kv_scales,
+                 const int32_t *block_table, const int32_t *seq_lens, int32_t head_begin, int32_t head_end,
+                 const int32_t *kv_begin, const int32_t *kv_end, float *out, float *lse,
+                 void *workspace, size_t workspace_bytes, void *stream_, const SparseStage *sparse) {
     g_launches = 0;
     int rc = check_shape(shape, head_begin, head_end);
     if (rc != SPLASH_OK) return rc;
@@ -208,6 +226,7 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     p.tile_start = v.tile_start; p.req_lo = v.req_lo; p.req_hi = v.req_hi; p.worker_begin = v.worker_begin;
     p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
     p.trace = g_trace;
+    p.len_cap = sparse ? sparse->max_selected : -1;
     p.request_overhead_tiles = kRequestOverheadTilesDefault;
     const bool pair = !simt && t.num_groups == 2 && t.heads_per_group == 64 && !(shape->flags & SPLASH_FLAG_NO_PAIR);
     if (!simt && shape->kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE)
@@ -220,6 +239,10 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
         e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
                         v.cost_start, v.worker_begin, v.split_list, v.status, stream);
     if (e == cudaSuccess) e = record_timing_event(1, stream);
+    if (e == cudaSuccess && sparse)
+        e = launch_sparse_gather(B, sparse->max_selected, sparse->pages_per_request, sparse->pool656, sparse->num_pool_pages,
+                                 sparse->block_table, sparse->table_stride, sparse->ctx_lens, sparse->sel, sparse->sel_stride,
+                                 sparse->sel_count, const_cast<void *>(kv_pool), sparse->dense_table, dev.sm_count, stream);
     if (e == cudaSuccess) {
         if (simt) e = launch_decode_simt(p, shape->kv_dtype, stream);
         else e = launch_decode_umma(p, *shape, stream);
@@ -233,13 +256,25 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
     return SPLASH_OK;
 }
 
+}  // namespace
+
+extern "C" {
+
+int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *kv_pool, const float *kv_scales,
+                      const int32_t *block_table, const int32_t *seq_lens, int32_t head_begin, int32_t head_end,
+                      const int32_t *kv_begin, const int32_t *kv_end, float *out, float *lse,
+                      void *workspace, size_t workspace_bytes, void *stream_) {
+    return decode_dense(shape, q, kv_pool, kv_scales, block_table, seq_lens, head_begin, head_end, kv_begin, kv_end, out, lse,
+                        workspace, workspace_bytes, stream_, nullptr);
+}
+
 namespace {
 
-// Workspace of a sparse call: [dense decode workspace][dense lens B][dense table B * ppr][dense cache].
+// Workspace of a sparse call: [dense decode workspace][dense table B * ppr][dense cache].
 struct SparseView {
     splash_mla_shape dense;        // the shape of the dense call over the gathered cache
     int pages_per_request;
-    size_t inner_bytes, off_lens, off_table, off_pool, bytes;
+    size_t inner_bytes, off_table, off_pool, bytes;
 };
 
 bool make_sparse_view(const splash_mla_shape *shape, int32_t max_selected, int32_t head_begin, int32_t head_end, SparseView &v) {
@@ -258,7 +293,6 @@ bool make_sparse_view(const splash_mla_shape *shape, int32_t max_selected, int32
     v.inner_bytes = splash_mla_decode_workspace_bytes(&v.dense, head_begin, head_end);
     if (v.inner_bytes == 0) return false;
     size_t off = align_up(v.inner_bytes, 256);
-    v.off_lens = off; off = align_up(off + sizeof(int32_t) * (size_t)shape->num_requests, 256);
     v.off_table = off; off = align_up(off + sizeof(int32_t) * (size_t)pages, 256);
     v.off_pool = off; off += (size_t)pages * kPage * kDQK * 2;
     v.bytes = align_up(off, 256);
@@ -295,17 +329,14 @@ int splash_mla_decode_sparse(const splash_mla_shape *shape, const void *q, const
     if (!current_device_info(dev)) return SPLASH_CUDA_ERROR;
     if (dev.cc_major != 10) { set_error("device compute capability %d.x is not 10.x", dev.cc_major); return SPLASH_UNSUPPORTED_DEVICE; }
     char *ws = static_cast<char *>(workspace);
-    int32_t *dense_lens = reinterpret_cast<int32_t *>(ws + v.off_lens);
-    int32_t *dense_table = reinterpret_cast<int32_t *>(ws + v.off_table);
-    void *dense_pool = ws + v.off_pool;
-    cudaError_t e = launch_sparse_gather(B, max_selected, v.pages_per_request, kv_pool, shape->num_pool_pages, block_table,
-                                         shape->block_table_stride, seq_lens, sel_tokens, sel_stride, sel_count, dense_pool,
-                                         dense_table, dense_lens, dev.sm_count, static_cast<cudaStream_t>(stream_));
-    if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
-    const int rc = splash_mla_decode(&v.dense, q, dense_pool, nullptr, dense_table, dense_lens, head_begin, head_end, nullptr,
-                                     nullptr, out, lse, workspace, v.inner_bytes, stream_);
-    count_launch();      // the gather kernel, on top of the dense call's launches
-    return rc;
+    SparseStage st;
+    st.pool656 = kv_pool; st.num_pool_pages = shape->num_pool_pages; st.block_table = block_table;
+    st.table_stride = shape->block_table_stride; st.ctx_lens = seq_lens; st.sel = sel_tokens; st.sel_count = sel_count;
+    st.sel_stride = sel_stride; st.max_selected = max_selected; st.pages_per_request = v.pages_per_request;
+    st.dense_table = reinterpret_cast<int32_t *>(ws + v.off_table);
+    // plan (over the list counts) -> gather into the dense cache -> decode kernel over the dense cache -> combine
+    return decode_dense(&v.dense, q, ws + v.off_pool, nullptr, st.dense_table, sel_count, head_begin, head_end, nullptr, nullptr,
+                        out, lse, workspace, v.inner_bytes, stream_, &st);
 }
 
 int splash_lse_merge(int32_t num_parts, int64_t rows, int32_t d_v, const float *part_out, const float *part_lse,

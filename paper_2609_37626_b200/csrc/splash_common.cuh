@@ -102,6 +102,7 @@ struct DecodeParams {
     const int32_t *tile_start, *req_lo, *req_hi, *worker_begin;
     int32_t *status;
     float *partial_lse, *partial_out;
+    int32_t len_cap;           // >= 0: seq_lens holds list counts; one outside [0, len_cap] counts as 1 (sparse decode)
     int32_t num_workers;
     int32_t request_overhead_tiles;   // per-request cost the plan adds to the tile count
     long long *trace;          // optional device buffer for pipeline timestamps (diagnostics), or NULL
@@ -206,7 +207,7 @@ cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const in
 cudaError_t launch_sparse_gather(int B, int max_sel, int pages_per_request, const void *kv_pool, int num_pool_pages,
                                  const int32_t *block_table, int64_t table_stride, const int32_t *seq_lens,
                                  const int32_t *sel, int64_t sel_stride, const int32_t *sel_count, void *dense_pool,
-                                 int32_t *dense_table, int32_t *dense_lens, int sm_count, cudaStream_t stream);
+                                 int32_t *dense_table, int sm_count, cudaStream_t stream);
 cudaError_t launch_dop_pack_rows(const void *a, const void *b, void *out, const int32_t *send_row, int64_t n, int h,
                                  int64_t a_bytes, int64_t b_bytes, int64_t a_row_pitch, int64_t a_head_pitch,
                                  int64_t b_row_pitch, int64_t b_head_pitch, int sm_count, cudaStream_t stream);

@@ -21,7 +21,7 @@ constexpr int kPlanSmemRequests = 4096;
 constexpr int kPlanSmemWorkers = 512;
 
 __global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ kv_begin,
+plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ kv_begin,
             const int32_t *__restrict__ kv_end, int32_t *tile_start,
             int32_t *__restrict__ req_lo, int32_t *__restrict__ req_hi,
             int32_t *__restrict__ req_wfirst, int32_t *__restrict__ req_wlast,
@@ -47,6 +47,7 @@ plan_kernel(int B, int W, int overhead, const int32_t *__restrict__ seq_lens, co
         long long n = 0;
         if (i < B) {
             int s = seq_lens[i];
+            if (len_cap >= 0 && (s < 0 || s > len_cap)) s = 1;     // a list count out of bounds: one (poisoned) row
             int lo = kv_begin ? kv_begin[i] : 0;
             int hi = kv_end ? kv_end[i] : s;
             if (lo < 0) lo = 0;
@@ -132,7 +133,7 @@ cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const in
     if (first_use_on_device(configured)) {
         cudaFuncSetAttribute(plan_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     }
-    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.seq_lens, kv_begin, kv_end, tile_start,
+    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.len_cap, p.seq_lens, kv_begin, kv_end, tile_start,
                                                 req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, split_list, status);
     count_launch();
     return cudaGetLastError();
