@@ -12,7 +12,7 @@
  *                       giving partial (O, LSE) that splash_lse_merge combines.
  * The cache is the head-shared latent cache of absorbed MLA: one row of
  * d_qk = d_c + d_r = 512 + 64 elements per token, the value being its first
- * d_v = d_c = 512 elements (Sec. 3 "Cost": d_q = d_c + d_r, d_z = d_c; App. B
+ * d_v = d_c = 512 elements (Sec. 3 "Cost": d_q = d_c + d_r, d_z = d_c; App. A
  * dimensions).  splash_kv_page_migrate is the local part of a layout switch: the
  * "discard" primitive's repack of kept blocks into the destination view (Sec. 3,
  * Sec. 4.1 "Reuse"), after which every query must still read its complete history

@@ -10,7 +10,7 @@
  *     (the paper's premise: "one head-shared latent history per token", Sec. 1);
  *   - absorbed MLA: a query row and a cache row are d_q = d_c + d_r wide and the
  *     value read back per head is d_z = d_c wide (Sec. 3, "Cost" paragraph of
- *     DOP, Eq. "dop-traffic"); with the DeepSeek-V3 dimensions of App. B,
+ *     DOP, Eq. "dop-traffic"); with the DeepSeek-V3 dimensions of App. A,
  *     d_c = 512 and d_r = 64;
  *   - decode presents one query row per request and every head attends over the
  *     request's complete history (Sec. 3 "Computation"; Sec. 4.1 "Handoff");

@@ -2,7 +2,7 @@
 //
 // The attention time of a decode step is set by the KV bytes read and the
 // contraction work, both linear in the context length (the paper's per-step cost
-// model, App. C: t_att = max{F_att / Phi_att, K_read / beta_KV}), so the plan
+// model, App. B: t_att = max{F_att / Phi_att, K_read / beta_KV}), so the plan
 // spreads page tiles -- not requests -- evenly over the CTAs: the global sequence of
 // (request, page tile) pairs is cut into `num_workers` contiguous runs of equal cost,
 // where a non-empty request costs its tile count plus a fixed overhead.  A run that

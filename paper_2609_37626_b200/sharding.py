@@ -2,7 +2,7 @@
 
 The attention shard of a rank is fixed by the layout (Sec. 3 of the paper): a head
 slice of H/T heads under TP / DOP, the requests it owns under DP-attention (assigned
-round-robin so that counts are balanced, App. C), or a contiguous 1/T of every
+round-robin so that counts are balanced, App. B), or a contiguous 1/T of every
 request's tokens under position-sharded CP (App. E).  Head and request slices are
 independent units -- no exchange happens inside attention -- so several ranks simply
 run their own calls; only CP ends with one exchange (an all-gather of the per-rank

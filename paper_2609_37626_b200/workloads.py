@@ -9,7 +9,7 @@ Workload shapes follow the paper's serving regimes ("many short vs a few very
 long requests", Sec. 1; fixed-length batches, Sec. 5): a DP-attention request
 slice, a TP/DOP head slice at 32K context, a position-sharded CP request at
 256K, and an RL-rollout batch with a long-tailed length mix and fp8 KV.  The
-dimensions are the DeepSeek-V3 ones of App. B: 128 heads, a 512-wide latent and
+dimensions are the DeepSeek-V3 ones of App. A: 128 heads, a 512-wide latent and
 a 64-wide rotary part, softmax scale 1/sqrt(128 + 64).
 
 Arrays are numpy: bf16 as uint16 bit patterns, e4m3 as uint8 codes.
@@ -29,7 +29,7 @@ D_ROPE = 64
 D_QK = D_LATENT + D_ROPE
 D_V = D_LATENT
 PAGE_SIZE = 64
-BASE_SEED = 20260922  # the PCG64 seed the paper uses for its own Monte-Carlo (App. C)
+BASE_SEED = 20260922  # the PCG64 seed the paper uses for its own Monte-Carlo (App. B)
 SOFTMAX_SCALE = 1.0 / math.sqrt(192.0)
 
 BF16_NAN = 0x7FC0
