@@ -5,7 +5,11 @@
 // dense decode kernels then run over that cache with the list lengths as context lengths.
 //
 // One warp per listed row: 41 16-byte loads in, 72 16-byte stores out, both coalesced.  HBM-bound:
-// 656 B read + 1152 B written per listed token (and 1152 B read again by the decode kernel).
+// 656 B read + 1152 B written per listed token (and 1152 B read again by the decode kernel).  With
+// rows picked uniformly at random the kernel sits at about half of the DRAM rate (4.2 TB/s of reads
+// plus writes); a variant that moved the rows as 656-byte bulk copies through shared memory, with
+// 2.5 times the bytes in flight per SM, ran at the same rate, so the limit is on the DRAM side
+// (isolated 656-byte reads between write bursts), not the SMs' latency hiding.
 #include <cuda_bf16.h>
 
 #include "splash_common.cuh"
@@ -17,7 +21,7 @@ namespace {
 
 constexpr int kSparseRowBytes = 656;
 constexpr int kGatherThreads = 256;
-constexpr int kRowsInFlight = 8;              // rows a warp loads before it converts any (a multiple of 4)
+constexpr int kRowsInFlight = 4;              // rows a warp loads before it converts any (a multiple of 4)
 constexpr uint32_t kBf16NanPair = 0x7FC07FC0u;
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -32,7 +36,7 @@ __device__ __forceinline__ uint2 dequant4(uint32_t w, float s) {
 }
 
 // Grid-stride over the B * pages_per_request * 64 row slots of the dense cache, in groups of 32 slots per warp.
-__global__ void __launch_bounds__(kGatherThreads)
+__global__ void __launch_bounds__(kGatherThreads, 4)
 sparse_gather_kernel(int B, int max_sel, int pages_per_request, const uint8_t *__restrict__ kv_pool, int num_pool_pages,
                      const int32_t *__restrict__ block_table, int64_t table_stride, const int32_t *__restrict__ seq_lens,
                      const int32_t *__restrict__ sel, int64_t sel_stride, const int32_t *__restrict__ sel_count,
@@ -58,7 +62,7 @@ sparse_gather_kernel(int B, int max_sel, int pages_per_request, const uint8_t *_
     // address hangs on a chain of three loads (count, list entry, page id): the chain of the NEXT group advances one
     // link per batch of rows of the current group, so its latency hides behind the row loads.
     constexpr int kGroup = 32, kBatches = kGroup / kRowsInFlight;
-    static_assert(kBatches == 4, "one link of the next group's address chain per batch");
+    static_assert(kBatches >= 4, "one link of the next group's address chain per batch");
     const int64_t num_groups = (total + kGroup - 1) / kGroup;
     int n_req = 0, n_idx = 0, n_cnt = 0, n_len = 0, n_tok = 0, n_page = 0, n_state = 0;
     auto link = [&](int step, int64_t group) {
@@ -93,7 +97,7 @@ sparse_gather_kernel(int B, int max_sel, int pages_per_request, const uint8_t *_
         const int k = lane >> 3;
 #pragma unroll
         for (int b = 0; b < kBatches; ++b) {
-            link(b, group + num_warps);
+            if (b < 4) link(b, group + num_warps);
             int state[kRowsInFlight];
             uint4 lat[kRowsInFlight], rope[kRowsInFlight / 4];
             float scale[kRowsInFlight];
