@@ -113,3 +113,15 @@ def test_sparse_argument_checks():
     out, lse = binding.splash_mla_decode_sparse(dw.q, dw.kv_pool, dw.block_table, dw.seq_lens, sel, cnt, softmax_scale=0.1)
     torch.cuda.synchronize()
     assert torch.isfinite(out).all()
+
+
+def test_sparse_at_the_size_the_benchmark_times():
+    # c2's 64 context lengths, 2,048 listed tokens per request, all 128 heads: every output against the oracle
+    c2 = W.config(2)
+    w = W.make_workload("sparse_top2048", W.BASE_SEED + 60, c2.seq_lens, H=128, kv_dtype=2)
+    del c2
+    sel, cnt = W.select_tokens(W.BASE_SEED + 60, w.seq_lens, 2048)
+    assert cnt.max() == 2048 and cnt.sum() > 100000
+    ref = oracle.mla_decode_sparse(w.q, w.kv_pool, w.block_table, w.seq_lens, sel, cnt, softmax_scale=w.softmax_scale)
+    out, lse = gpu_sparse(w, sel, cnt)
+    compare_sparse(out, lse, *ref, 0, 128, "bench size")
