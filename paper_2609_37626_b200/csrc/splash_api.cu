@@ -167,6 +167,7 @@ struct SparseStage {
     int64_t sel_stride;
     int max_selected, pages_per_request;
     int32_t *dense_table;
+    bool fused;        // one kernel gathers, dequantises and multiplies (CTA pairs); else gather kernel + dense kernels
 };
 
 // One dense decode call: plan, decode kernel, combine.  With a sparse stage, seq_lens are the list counts, kv_pool
@@ -206,6 +207,8 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     const int ve = vb + vstep < vend ? vb + vstep : vend;
     const int h = ve - vb;
     Tiling t = choose_tiling(shape, h, dev.sm_count, simt);
+    const bool fused_sparse = sparse && sparse->fused && !simt;
+    if (fused_sparse) { t.heads_per_group = 64; t.num_groups = 2; t.num_workers = dev.sm_count / 2 > 0 ? dev.sm_count / 2 : 1; }
     PlanView v = make_plan_view(workspace, B, t.num_workers, h);
     if (workspace_bytes < v.bytes) {
         set_error("workspace has %zu bytes, %zu needed", workspace_bytes, v.bytes); return SPLASH_INVALID_ARG;
@@ -227,6 +230,11 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
     p.trace = g_trace;
     p.len_cap = sparse ? sparse->max_selected : -1;
+    if (fused_sparse) {
+        p.kv_pool = sparse->pool656; p.block_table = sparse->block_table; p.table_stride = sparse->table_stride;
+        p.num_pool_pages = sparse->num_pool_pages; p.sel = sparse->sel; p.sel_stride = sparse->sel_stride;
+        p.ctx_lens = sparse->ctx_lens;
+    }
     p.request_overhead_tiles = kRequestOverheadTilesDefault;
     const bool pair = !simt && t.num_groups == 2 && t.heads_per_group == 64 && !(shape->flags & SPLASH_FLAG_NO_PAIR);
     if (!simt && shape->kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE)
@@ -239,12 +247,13 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
         e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
                         v.cost_start, v.worker_begin, v.split_list, v.status, stream);
     if (e == cudaSuccess) e = record_timing_event(1, stream);
-    if (e == cudaSuccess && sparse)
+    if (e == cudaSuccess && sparse && !fused_sparse)
         e = launch_sparse_gather(B, sparse->max_selected, sparse->pages_per_request, sparse->pool656, sparse->num_pool_pages,
                                  sparse->block_table, sparse->table_stride, sparse->ctx_lens, sparse->sel, sparse->sel_stride,
                                  sparse->sel_count, const_cast<void *>(kv_pool), sparse->dense_table, dev.sm_count, stream);
     if (e == cudaSuccess) {
         if (simt) e = launch_decode_simt(p, shape->kv_dtype, stream);
+        else if (fused_sparse) e = launch_decode_sparse_pair(p, stream);
         else e = launch_decode_umma(p, *shape, stream);
     }
     if (e == cudaSuccess) e = record_timing_event(2, stream);
@@ -334,6 +343,7 @@ int splash_mla_decode_sparse(const splash_mla_shape *shape, const void *q, const
     st.table_stride = shape->block_table_stride; st.ctx_lens = seq_lens; st.sel = sel_tokens; st.sel_count = sel_count;
     st.sel_stride = sel_stride; st.max_selected = max_selected; st.pages_per_request = v.pages_per_request;
     st.dense_table = reinterpret_cast<int32_t *>(ws + v.off_table);
+    st.fused = (shape->flags & (SPLASH_FLAG_NO_PAIR | SPLASH_FLAG_SIMT)) == 0;
     // plan (over the list counts) -> gather into the dense cache -> decode kernel over the dense cache -> combine
     return decode_dense(&v.dense, q, ws + v.off_pool, nullptr, st.dense_table, sel_count, head_begin, head_end, nullptr, nullptr,
                         out, lse, workspace, v.inner_bytes, stream_, &st);

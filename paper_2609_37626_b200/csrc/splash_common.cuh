@@ -103,6 +103,10 @@ struct DecodeParams {
     int32_t *status;
     float *partial_lse, *partial_out;
     int32_t len_cap;           // >= 0: seq_lens holds list counts; one outside [0, len_cap] counts as 1 (sparse decode)
+    // fused sparse decode: kv_pool holds 656-byte rows, block_table / num_pool_pages describe it, and request i
+    // attends over the tokens sel[i * sel_stride + j], j < seq_lens[i], each below ctx_lens[i]
+    const int32_t *sel, *ctx_lens;
+    int64_t sel_stride;
     int32_t num_workers;
     int32_t request_overhead_tiles;   // per-request cost the plan adds to the tile count
     long long *trace;          // optional device buffer for pipeline timestamps (diagnostics), or NULL
@@ -204,6 +208,7 @@ cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const in
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
                         int32_t *status, cudaStream_t stream);
+cudaError_t launch_decode_sparse_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_sparse_gather(int B, int max_sel, int pages_per_request, const void *kv_pool, int num_pool_pages,
                                  const int32_t *block_table, int64_t table_stride, const int32_t *seq_lens,
                                  const int32_t *sel, int64_t sel_stride, const int32_t *sel_count, void *dense_pool,

@@ -1,0 +1,656 @@
+// Sparse decode kernel: attention over a LIST of tokens per request, cache rows in the 656-byte
+// format (512 e4m3 latent codes, four float scales -- one per 128 latent dims --, 64 bf16 rope
+// values; Sec. 5 setup, App. B payload), on a CLUSTER OF TWO CTAs per KV worker issuing
+// tcgen05 cta_group::2 MMAs.
+//
+// The contractions, the softmax, the accumulators and the epilogue are those of the bf16
+// CTA-pair kernel: per tile of 64 listed tokens
+//   S [128 heads x 64 tokens] = Q K^T      M = 128 (64 heads per CTA), N = 64: each CTA supplies 32 tokens
+//   O [128 heads x 256 dv]   += P V        M = 128, N = 256 (x 2 halves of dv): each CTA supplies 128 dv columns
+// over a bf16 tile in shared memory (9 chunk slabs of 32 tokens x 128 B, 128-byte swizzle; after
+// QK^T the four latent slots this CTA does not multiply are overwritten with the peer's tokens'
+// columns that it does).  What differs is where the tile comes from: no TMA can fetch scattered
+// 656-byte rows into that layout, so
+//   * an address warp walks the token list a few tiles ahead: list entry -> page id -> row
+//     address, four tiles abreast so that the chain of dependent loads is paid once per four
+//     tiles; it leaves the addresses in a ring in shared memory and pulls the rows into L2;
+//   * three converter warps copy the raw rows into a staging buffer with 16-byte asynchronous
+//     copies (no registers held while the rows travel), then dequantise from there (code x block
+//     scale, rounded to bf16) into the swizzled tile: this CTA's 32 tokens in full for QK^T, and
+//     the peer's 32 tokens' 256 columns for P.V once QK^T has retired.  Each warp copies and
+//     converts its own rows only, so the staging buffer needs no barrier of its own.
+// Every listed row crosses HBM once (twice through L2: the peer reads it too).
+//
+// Roles per CTA (576 threads): address warp, 4 QK^T issuers and 2 P.V issuers (leader CTA only;
+// the first issuer warp of either CTA also loads that CTA's query rows), 8 softmax warps,
+// 3 converter warps.  Barriers that the issuers wait on live in the leader; the peer's warps
+// arrive on them across the cluster (relaxed arrivals: what they announce is already in place on
+// the peer's SM).
+#include <cuda_bf16.h>
+
+#include "splash_fp8.cuh"
+#include "splash_pair.cuh"
+
+namespace splash {
+
+namespace {
+
+using namespace umma;
+
+constexpr int kQkWarps = 4, kPvWarps = 2, kSoftmaxWarps = 8;
+constexpr int kWarpAddr = 0;
+constexpr int kWarpQk = 1;
+constexpr int kWarpPv = kWarpQk + kQkWarps;
+constexpr int kWarpSoftmax = kWarpPv + kPvWarps;       // 7: TMEM quadrant = warp & 3
+constexpr int kConvWarps = 3;
+constexpr int kWarpConv = kWarpSoftmax + kSoftmaxWarps;
+constexpr int kThreads = (kWarpConv + kConvWarps) * 32;   // 18 warps = 576 threads
+constexpr int kN = 64;                              // heads per CTA
+constexpr int kHalf = 32;                           // tokens per CTA and tile
+constexpr uint32_t kSlab = kHalf * 128;             // one chunk of a half-page: 32 tokens x 128 B
+constexpr uint32_t kStageBytes = 9 * kSlab;         // 36,864
+constexpr uint32_t kQSlab = kN * 128;               // one chunk of the query rows: 64 heads x 128 B
+constexpr uint32_t kQBytes = 9 * kQSlab;            // 73,728
+constexpr uint32_t kPHalfBytes = kN * 64;           // P of one half-page: 64 heads x 32 tokens bf16
+constexpr int kStages = 3;
+constexpr int kRing = 8;                            // tiles of row addresses the address warp may be ahead
+constexpr int kAddrBatch = 4;                       // tiles whose addresses are resolved abreast
+constexpr uint32_t kRowBytes = 656;                 // a cache row: 512 codes, 4 scales, 64 bf16 rope values
+constexpr uint32_t kVRowBytes = 272;                // what P.V needs of a peer row: 2 x 128 codes, 4 scales
+constexpr float kTau = 8.0f;                        // O is rescaled only when a row maximum grows by more than 2^8
+
+enum BarrierId {
+    kBarKFull = 0,                        // [3] leader: both CTAs' 32 tokens converted (all converter warps of both)
+    kBarQkDone = kBarKFull + kStages,     // [3] QK^T of the stage retired (multicast commit): peer columns may be written
+    kBarVFull = kBarQkDone + kStages,     // [3] leader: both CTAs' peer columns converted
+    kBarStageEmpty = kBarVFull + kStages, // [3] P.V of the stage retired (multicast commit): stage and P buffers
+                                          //     are free, O is up to date
+    kBarQFull = kBarStageEmpty + kStages, // leader: query rows of both CTAs landed
+    kBarQEmpty,                           // last QK^T of the request retired (multicast commit)
+    kBarSFull,                            // [2] S buffer written (multicast commit)
+    kBarSEmpty = kBarSFull + 2,           // [2] S buffer read (leader: by both CTAs)
+    kBarPFull = kBarSEmpty + 2,           // [2] P buffer written (leader: by both CTAs)
+    kBarOFull = kBarPFull + 2,            // last P.V of the request retired (multicast commit)
+    kBarOEmpty,                           // O drained (leader: by both CTAs)
+    kBarAddrFull,                         // [8] local: row addresses of a tile written to the ring
+    kBarAddrEmpty = kBarAddrFull + kRing, // [8] local: the converter warps are done with the ring slot
+    kNumBarriers = kBarAddrEmpty + kRing
+};
+
+constexpr uint32_t kOffK = 0;                                   // [3 stages] 9 chunk slots of 32 tokens
+constexpr uint32_t kOffQ = kOffK + kStages * kStageBytes;       // 9 chunks x 64 heads x 128 B
+constexpr uint32_t kOffP1 = kOffQ + kQBytes;                    // [2 buffers] P of half-page 1: 64 heads x 64 B
+constexpr uint32_t kOffRawK = kOffP1 + 2 * kPHalfBytes;         // raw rows of this CTA's 32 tokens: 32 x 656 B
+constexpr uint32_t kOffRawV = kOffRawK + kHalf * kRowBytes;     // the peer's 32 tokens, the 272 bytes P.V needs of each
+constexpr uint32_t kOffRing = kOffRawV + kHalf * kVRowBytes;    // uint64 [8][64] row addresses (0: zero row, 1: poisoned row)
+constexpr uint32_t kOffAlpha = kOffRing + kRing * 64 * 8;       // float [64]
+constexpr uint32_t kOffL = kOffAlpha + kN * 4;                  // float [64]
+constexpr uint32_t kOffXch = kOffL + kN * 4;                    // float [64][4]
+constexpr uint32_t kOffBar = kOffXch + kN * 16;
+constexpr uint32_t kOffMisc = (kOffBar + kNumBarriers * 8 + 15) / 16 * 16;
+constexpr uint32_t kSmemBytes = kOffMisc + 32;
+static_assert(kSmemBytes <= 232448, "shared memory overflow");
+static_assert(kOffQ % 1024 == 0 && kOffP1 % 1024 == 0 && kSlab % 1024 == 0, "swizzle atoms need 1024-byte alignment");
+static_assert(kOffRawK % 16 == 0 && kOffRawV % 16 == 0 && kOffRing % 8 == 0 && kOffBar % 8 == 0, "alignment");
+// tensor memory: O two halves of dv x 128 columns, then 2 S buffers x 4 partials x 32 columns
+constexpr uint32_t kColO = 0, kColS = 256;
+
+// 4 e4m3 codes (one 32-bit word) times a scale -> 4 bf16 (two words)
+__device__ __forceinline__ uint2 dequant4(uint32_t w, float s) {
+    const float2 a = from_e4m3x2((uint16_t)(w & 0xffffu)), b = from_e4m3x2((uint16_t)(w >> 16));
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a.x * s, a.y * s), hi = __floats2bfloat162_rn(b.x * s, b.y * s);
+    return make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+}
+
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmap_q) {
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const uint32_t sbase = smem_u32(smem);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t rank = cluster_ctarank();             // 0 = leader: issues the MMAs
+    const int worker = blockIdx.x >> 1;
+    const int head0 = p.head_begin + (int)rank * kN;
+    const int h = p.head_end - p.head_begin;
+
+    volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + kOffMisc);
+    Ctx ctx{misc + 1, p.status};
+    auto bar = [&](int id) -> uint32_t { return sbase + kOffBar + 8u * (uint32_t)id; };
+    auto leader_bar = [&](int id) -> uint32_t { return map_to_cta(sbase + kOffBar + 8u * (uint32_t)id, 0); };
+    // one arrival of a warp of either CTA on a barrier that lives in the leader
+    auto arrive_on_leader = [&](int id) {
+        if (rank == 0) mbar_arrive(bar(id));
+        else mbar_arrive_cluster_relaxed(leader_bar(id));
+    };
+
+    if (tid == 0) {
+        // barriers the leader's issuers wait on count the warps of both CTAs (the peer's copies are unused)
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar(kBarKFull + s), 2 * kConvWarps); mbar_init(bar(kBarQkDone + s), kQkWarps);
+            mbar_init(bar(kBarVFull + s), 2 * kConvWarps); mbar_init(bar(kBarStageEmpty + s), kPvWarps);
+        }
+        for (int s = 0; s < kRing; ++s) { mbar_init(bar(kBarAddrFull + s), 1); mbar_init(bar(kBarAddrEmpty + s), kConvWarps); }
+        mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), kQkWarps);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), 2 * kSoftmaxWarps);
+            mbar_init(bar(kBarPFull + b), 2 * kSoftmaxWarps);
+        }
+        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), 2 * kSoftmaxWarps);
+        misc[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(sbase + kOffMisc), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                   // barriers of both CTAs exist before anyone signals them
+    tcgen05_fence_after();
+    const uint32_t tmem_base = misc[0];
+    grid_dependency_wait();                               // the plan kernel's output is read from here on
+    const long long t_start = clock64();
+    const unsigned long long ns_start = global_timer_ns();
+
+    SegmentIter it;
+    it.init(p, worker);
+    Segment seg;
+    seg.lo = seg.hi = seg.tile_begin = seg.tile_end = 0;
+
+    if (warp == kWarpAddr) {
+        // ===================================================== address warp
+        // Box row R of a tile holds list entry tile * 64 + tok0 + R (tile_geom with lo = 0: a short last tile is
+        // aligned to the end of the box, the rows before it are zero).  Lane l resolves rows l and 32 + l of each
+        // of four consecutive tiles at once, so the two dependent loads (list entry, page id) cost one round trip
+        // each per four tiles.  Address 0 stands for a zero row, 1 for a poisoned one (a list entry outside the
+        // request, a page id outside the pool, a count outside [0, len_cap]).
+        unsigned long long *ring = reinterpret_cast<unsigned long long *>(smem + kOffRing);
+        const uint8_t *pool = static_cast<const uint8_t *>(p.kv_pool);
+        uint32_t kv_it = 0;
+        bool ok = true, more = it.next(p, seg);
+        int tile = more ? seg.tile_begin : 0;
+        while (ok && more) {
+            int n_tiles = 0;
+            int tok[kAddrBatch][2], len[kAddrBatch];
+            const int32_t *table[kAddrBatch];
+            unsigned long long addr[kAddrBatch][2];
+#pragma unroll
+            for (int u = 0; u < kAddrBatch; ++u) {
+                tok[u][0] = tok[u][1] = -1; len[u] = 0; table[u] = p.block_table; addr[u][0] = addr[u][1] = 0ull;
+                if (!more) continue;
+                n_tiles = u + 1;
+                const int cnt = p.seq_lens[seg.request];
+                const bool bad_count = cnt < 0 || cnt > p.len_cap;
+                const TileGeom g = tile_geom(seg.lo, seg.hi, tile * kPage);
+                const int32_t *list = p.sel + (int64_t)seg.request * p.sel_stride;
+                len[u] = p.ctx_lens[seg.request];
+                table[u] = p.block_table + (int64_t)seg.request * p.table_stride;
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int R = 32 * e + lane;
+                    if (R >= g.r_lo && R < g.r_hi) {
+                        addr[u][e] = 1ull;                                           // poisoned unless resolved below
+                        if (!bad_count) tok[u][e] = __ldg(list + tile * kPage + g.tok0 + R);
+                    }
+                }
+                if (++tile == seg.tile_end) { more = it.next(p, seg); tile = more ? seg.tile_begin : 0; }
+            }
+            int page[kAddrBatch][2];
+#pragma unroll
+            for (int u = 0; u < kAddrBatch; ++u)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool live = addr[u][e] == 1ull && tok[u][e] >= 0 && tok[u][e] < len[u];
+                    page[u][e] = live ? __ldg(table[u] + tok[u][e] / kPage) : -1;
+                }
+#pragma unroll
+            for (int u = 0; u < kAddrBatch; ++u) {
+                if (u >= n_tiles) continue;
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    if (page[u][e] >= 0 && page[u][e] < p.num_pool_pages)
+                        addr[u][e] = reinterpret_cast<unsigned long long>(pool + ((int64_t)page[u][e] * kPage + tok[u][e] % kPage) * kRowBytes);
+                const uint32_t slot = kv_it % kRing, ph = (kv_it / kRing) & 1;
+                if (lane == 0) ok = mbar_wait(ctx, bar(kBarAddrEmpty + slot), ph ^ 1, kBarAddrEmpty + slot);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                ring[slot * 64 + lane] = addr[u][0];
+                ring[slot * 64 + 32 + lane] = addr[u][1];
+                // this CTA's own 32 tokens of the tile: into L2 ahead of the converter warps' copies
+                const unsigned long long own = rank == 0 ? addr[u][0] : addr[u][1];
+                if (own > 1ull) bulk_prefetch_l2(reinterpret_cast<const void *>(own), kRowBytes);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(kBarAddrFull + slot));
+                ++kv_it;
+            }
+        }
+    } else if (warp >= kWarpConv) {
+        // ===================================================== converter warps
+        // Warp c takes rows c, c + 3, ... of this CTA's 32 tokens (all 576 columns, for QK^T and as this CTA's
+        // own half of P.V) and of the peer's 32 tokens (the 256 latent columns this CTA multiplies in P.V).
+        const int c = warp - kWarpConv;
+        const unsigned long long *ring = reinterpret_cast<const unsigned long long *>(smem + kOffRing);
+        uint8_t *raw_k = smem + kOffRawK, *raw_v = smem + kOffRawV;
+        const uint32_t raw_k_s = sbase + kOffRawK, raw_v_s = sbase + kOffRawV;
+        // total number of tiles of this worker (the role does not care about request boundaries)
+        uint32_t total = 0;
+        while (it.next(p, seg)) total += (uint32_t)(seg.tile_end - seg.tile_begin);
+        bool ok = true;
+        auto cp16 = [](uint32_t dst, const void *src) {
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+        };
+        auto commit = []() { asm volatile("cp.async.commit_group;" ::: "memory"); };
+        // raw rows of tile kv: this CTA's tokens in full, then the peer's tokens' P.V columns, one copy group each
+        auto issue_k = [&](uint32_t kv) {
+            if (kv < total && ok) {
+                const uint32_t slot = kv % kRing;
+                if (lane == 0) ok = mbar_wait(ctx, bar(kBarAddrFull + slot), (kv / kRing) & 1, kBarAddrFull + slot);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (ok) {
+                    for (int t = c; t < kHalf; t += kConvWarps) {
+                        const unsigned long long a = ring[slot * 64 + 32 * rank + t];
+                        if (a > 1ull) {
+                            const uint8_t *row = reinterpret_cast<const uint8_t *>(a);
+                            cp16(raw_k_s + t * kRowBytes + 16 * lane, row + 16 * lane);
+                            if (lane < 9) cp16(raw_k_s + t * kRowBytes + 512 + 16 * lane, row + 512 + 16 * lane);
+                        }
+                    }
+                }
+            }
+            commit();
+        };
+        auto issue_v = [&](uint32_t kv) {
+            if (kv < total && ok) {
+                const uint32_t slot = kv % kRing;
+                for (int t = c; t < kHalf; t += kConvWarps) {
+                    const unsigned long long a = ring[slot * 64 + 32 * (1 - rank) + t];
+                    if (a > 1ull && lane < 17) {
+                        // units 0-7: codes [128 r, + 128); 8-15: codes [256 + 128 r, + 128); 16: the four scales
+                        const uint8_t *row = reinterpret_cast<const uint8_t *>(a);
+                        const uint32_t off = lane < 8 ? 128 * rank + 16 * lane : lane < 16 ? 256 + 128 * rank + 16 * (lane - 8) : 512;
+                        cp16(raw_v_s + t * kVRowBytes + 16 * lane, row + off);
+                    }
+                }
+            }
+            commit();
+        };
+        issue_k(0);
+        issue_v(0);
+        for (uint32_t kv = 0; kv < total && ok; ++kv) {
+            const uint32_t stage = kv % kStages, sph = (kv / kStages) & 1, slot = kv % kRing;
+            uint8_t *k0 = smem + kOffK + stage * kStageBytes;
+            // ---- this CTA's tokens: all but the latest copy group (the peer columns of this tile) have landed
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) ok = mbar_wait(ctx, bar(kBarStageEmpty + stage), sph ^ 1, kBarStageEmpty + stage);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            for (int t = c; t < kHalf; t += kConvWarps) {
+                const unsigned long long a = ring[slot * 64 + 32 * rank + t];
+                uint4 lo, hi, rope;
+                if (a > 1ull) {
+                    // lane l: codes [16 l, 16 l + 16) = units 2 (l & 3), + 1 of chunk l >> 2; lanes 0-7: rope unit l
+                    const uint8_t *src = raw_k + t * kRowBytes;
+                    const uint4 lat = *reinterpret_cast<const uint4 *>(src + 16 * lane);
+                    const float s = *reinterpret_cast<const float *>(src + 512 + 4 * (lane >> 3));
+                    if (lane < 8) rope = *reinterpret_cast<const uint4 *>(src + 528 + 16 * lane);
+                    const uint2 x0 = dequant4(lat.x, s), x1 = dequant4(lat.y, s), x2 = dequant4(lat.z, s), x3 = dequant4(lat.w, s);
+                    lo = make_uint4(x0.x, x0.y, x1.x, x1.y); hi = make_uint4(x2.x, x2.y, x3.x, x3.y);
+                } else {
+                    const uint32_t fill = a == 0ull ? 0u : 0x7FC07FC0u;
+                    lo = hi = rope = make_uint4(fill, fill, fill, fill);
+                }
+                uint8_t *dst = k0 + (lane >> 2) * kSlab + t * 128;
+                const uint32_t u0 = 2 * (lane & 3);
+                *reinterpret_cast<uint4 *>(dst + ((u0 ^ (t & 7)) << 4)) = lo;
+                *reinterpret_cast<uint4 *>(dst + (((u0 + 1) ^ (t & 7)) << 4)) = hi;
+                if (lane < 8) *reinterpret_cast<uint4 *>(k0 + 8 * kSlab + t * 128 + ((lane ^ (t & 7)) << 4)) = rope;
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) arrive_on_leader(kBarKFull + stage);
+            issue_k(kv + 1);
+            // ---- the peer's tokens: their copy group has landed (only the group just issued may be pending);
+            // the slots they go to are dead once QK^T of the stage has retired
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) ok = mbar_wait(ctx, bar(kBarQkDone + stage), sph, kBarQkDone + stage);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            {
+                // lane l = 16 n + 8 e + w: codes [8 w, + 8) of chunk 4 n + 2 rank + e -> unit w of slot 4 n + 2 (1 - rank) + e
+                const int n = lane >> 4, e = (lane >> 3) & 1, w = lane & 7;
+                uint8_t *dst_slot = k0 + (4 * n + 2 * (1 - (int)rank) + e) * kSlab;
+                for (int t = c; t < kHalf; t += kConvWarps) {
+                    const unsigned long long a = ring[slot * 64 + 32 * (1 - rank) + t];
+                    uint4 v;
+                    if (a > 1ull) {
+                        const uint8_t *src = raw_v + t * kVRowBytes;
+                        const uint2 codes = *reinterpret_cast<const uint2 *>(src + 8 * lane);
+                        const float s = *reinterpret_cast<const float *>(src + 256 + 4 * (2 * n + (int)rank));
+                        const uint2 x0 = dequant4(codes.x, s), x1 = dequant4(codes.y, s);
+                        v = make_uint4(x0.x, x0.y, x1.x, x1.y);
+                    } else {
+                        const uint32_t fill = a == 0ull ? 0u : 0x7FC07FC0u;
+                        v = make_uint4(fill, fill, fill, fill);
+                    }
+                    *reinterpret_cast<uint4 *>(dst_slot + t * 128 + ((w ^ (t & 7)) << 4)) = v;
+                }
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) { arrive_on_leader(kBarVFull + stage); mbar_arrive(bar(kBarAddrEmpty + slot)); }
+            issue_v(kv + 1);
+        }
+    } else if (warp >= kWarpQk && warp < kWarpQk + kQkWarps && rank == 0) {
+        // ===================================================== QK^T issuers (leader CTA)
+        // One thread sustains one tcgen05.mma per ~65 cycles and a chain of MMAs into one accumulator
+        // runs at the MMA latency, so the 36 K = 16 steps of a tile go to four issuers with a partial
+        // accumulator each.
+        if (lane == 0) {
+            const int a = warp - kWarpQk;
+            constexpr uint32_t kIdescQK = make_idesc(128, 64, 0, 0);
+            uint32_t kv_it = 0, seg_it = 0;
+            bool ok = true;
+            while (ok && it.next(p, seg)) {
+                if (a == 0) {
+                    // the query rows of the request, once the last QK^T of the previous one has retired
+                    ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(kBarQFull), 2 * kQBytes);      // the rows of both CTAs
+                    tma_load_4d_pair(sbase + kOffQ, &tmap_q, leader_bar(kBarQFull), 0, head0, 0, seg.request);
+                }
+                ok = mbar_wait_cluster(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
+                for (int tile = seg.tile_begin; ok && tile < seg.tile_end; ++tile, ++kv_it) {
+                    const uint32_t stage = kv_it % kStages, b = kv_it & 1;
+                    ok = mbar_wait_cluster(ctx, bar(kBarKFull + stage), (kv_it / kStages) & 1, kBarKFull + stage) &&
+                         mbar_wait_cluster(ctx, bar(kBarSEmpty + b), ((kv_it >> 1) & 1) ^ 1, kBarSEmpty + b);
+                    if (!ok) break;
+                    tcgen05_fence_after();
+                    const uint32_t k0 = sbase + kOffK + stage * kStageBytes;
+                    const uint32_t d = tmem_base + kColS + (b * kQkWarps + a) * kHalf;
+#pragma unroll
+                    for (int t = 0; t < 36 / kQkWarps; ++t) {
+                        const int idx = t * kQkWarps + a, c = idx >> 2, k = idx & 3;
+                        uint64_t dq = make_desc(sbase + kOffQ + c * kQSlab + k * 32, 16, 1024);   // A: 2 x 64 heads x 16
+                        uint64_t dk = make_desc(k0 + c * kSlab + k * 32, 16, 1024);             // B: 2 x 32 tokens x 16
+                        umma_bf16_pair(d, dq, dk, kIdescQK, t != 0);
+                    }
+                    umma_commit_pair(bar(kBarSFull + b));
+                    umma_commit_pair(bar(kBarQkDone + stage));
+                }
+                if (ok) umma_commit_pair(bar(kBarQEmpty));
+                ++seg_it;
+            }
+        }
+    } else if (warp >= kWarpPv && warp < kWarpPv + kPvWarps && rank == 0) {
+        // ===================================================== P.V issuers (leader CTA)
+        if (lane == 0) {
+            const int n = warp - kWarpPv;                 // dv half: columns [256 n, 256 n + 256)
+            constexpr uint32_t kIdescPV = make_idesc(128, 256, 0, 1);
+            uint32_t kv_it = 0, seg_it = 0;
+            bool ok = true;
+            while (ok && it.next(p, seg)) {
+                for (int tile = seg.tile_begin; ok && tile < seg.tile_end; ++tile, ++kv_it) {
+                    const uint32_t stage = kv_it % kStages, pb = kv_it & 1;
+                    ok = mbar_wait_cluster(ctx, bar(kBarVFull + stage), (kv_it / kStages) & 1, kBarVFull + stage) &&
+                         mbar_wait_cluster(ctx, bar(kBarPFull + pb), (kv_it >> 1) & 1, kBarPFull + pb);
+                    if (ok && tile == seg.tile_begin) ok = mbar_wait_cluster(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty);
+                    if (!ok) break;
+                    tcgen05_fence_after();
+                    const uint32_t k0 = sbase + kOffK + stage * kStageBytes;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // 16 tokens of half-page g.  A: P rows (heads), 32 bytes of the 64-byte row (g = 0: in the
+                        // stage's rope slot, g = 1: in its own buffer);
+                        // B: slots 4n + 2g, + 1 (two 64-wide dv chunks, LBO apart), 16 token rows, MN-major
+                        const int g = j >> 1;
+                        const uint32_t p0 = g == 0 ? k0 + 8 * kSlab : sbase + kOffP1 + pb * kPHalfBytes;
+                        uint64_t da = make_desc_sw64(p0 + (j & 1) * 32, 16, 512);
+                        uint64_t db = make_desc(k0 + (4 * n + 2 * g) * kSlab + (j & 1) * 2048, kSlab, 1024);
+                        umma_bf16_pair(tmem_base + kColO + n * 128, da, db, kIdescPV, (tile != seg.tile_begin) || j != 0);
+                    }
+                    umma_commit_pair(bar(kBarStageEmpty + stage));
+                    if (tile + 1 == seg.tile_end) umma_commit_pair(bar(kBarOFull));
+                }
+                ++seg_it;
+            }
+        }
+    } else if (warp == kWarpQk) {
+        // peer CTA: its first issuer warp only loads the query rows of this CTA's heads
+        if (lane == 0) {
+            uint32_t seg_it = 0;
+            bool ok = true;
+            while (ok && it.next(p, seg)) {
+                ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
+                if (ok) tma_load_4d_pair(sbase + kOffQ, &tmap_q, leader_bar(kBarQFull), 0, head0, 0, seg.request);
+                ++seg_it;
+            }
+        }
+    } else if (warp >= kWarpQk && warp < kWarpSoftmax) {
+        // the other issuer warps of the peer CTA have nothing to do
+    } else {
+        // ===================================================== softmax + epilogue warps
+        // S partial layout per CTA: TMEM lane L < 64 = head L, tokens of half-page 0 in 32 columns;
+        // lane 64 + L = head L, tokens of half-page 1.  Two warps per quadrant take 16 columns each,
+        // so a thread owns ONE head and 16 tokens of one half-page.
+        const int sw = warp - kWarpSoftmax;             // 0..7
+        const int q4 = warp & 3;                        // TMEM lane quadrant
+        const int cf = sw >> 2;                         // column half: tokens [16 cf, 16 cf + 16) of the half-page
+        const int g = q4 >> 1;                          // half-page
+        const int hd = 32 * (q4 & 1) + lane;            // this thread's head (0..63 within the CTA)
+        const int half_id = q4 & 1;                     // heads 0-31 or 32-63: the four warps that share them sync on bar 2 + half_id
+        const int row0 = kHalf * g + 16 * cf;           // first of this thread's 16 rows of the 64-row tile
+        const uint32_t lane_addr = (uint32_t)(32 * q4) << 16;
+        float *alpha_s = reinterpret_cast<float *>(smem + kOffAlpha);
+        float *l_s = reinterpret_cast<float *>(smem + kOffL);
+        float *xch = reinterpret_cast<float *>(smem + kOffXch);
+        const float scale_log2 = p.softmax_scale * kLog2e;
+        const int slot4 = g * 2 + cf;                   // this thread's slot among the 4 threads of its head
+        uint32_t kv_it = 0, seg_it = 0;
+        // A failed (timed-out) wait only clears `ok`; the role keeps walking its tiles so that every
+        // thread still meets the named barriers -- once the CTA aborts, waits return at once.
+        bool ok = true;
+        while (it.next(p, seg)) {
+            float m = -INFINITY, l = 0.f;               // running maximum in scaled log2 units
+            const int first_page = seg.lo / kPage;
+            // several query rows per request: this thread's (virtual) head is row (head mod R) and sees the
+            // tokens below causal_end only
+            const int causal_end = p.q_rows > 1 ? p.seq_lens[seg.request] - (p.q_rows - 1 - (head0 + hd) % p.q_rows) : 0x3fffffff;   // (far above any token index, and safe to subtract a negative offset from)
+            for (int tile = seg.tile_begin; tile < seg.tile_end; ++tile, ++kv_it) {
+                const TileGeom geo = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);   // (lo = 0: list positions)
+                const uint32_t b = kv_it & 1;
+                ok &= mbar_wait(ctx, bar(kBarSFull + b), (kv_it >> 1) & 1, kBarSFull + b);
+                tcgen05_fence_after();
+                float sv[16];
+                {
+                    float pa[16], pb[16], pc[16];
+                    const uint32_t sb = tmem_base + lane_addr + kColS + (b * kQkWarps) * kHalf + 16 * cf;
+                    tmem_ld16(sb, sv);
+                    tmem_ld16(sb + kHalf, pa);
+                    tmem_ld16(sb + 2 * kHalf, pb);
+                    tmem_ld16(sb + 3 * kHalf, pc);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) sv[j] = ((sv[j] + pa[j]) + (pb[j] + pc[j])) * scale_log2;
+                }
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) arrive_on_leader(kBarSEmpty + b);
+                // rows outside [r_lo, r_hi) are zero fill or tokens outside the request's range (or beyond this
+                // head's causal end: row r of the tile holds token (first_page + tile) * 64 + tok0 + r)
+                const int r_hi = min(geo.r_hi, causal_end - ((first_page + tile) * kPage + geo.tok0));
+                if (row0 < geo.r_lo || row0 + 16 > r_hi) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (row0 + j < geo.r_lo || row0 + j >= r_hi) sv[j] = -INFINITY;
+                }
+                float mt = sv[0];
+#pragma unroll
+                for (int j = 1; j < 16; ++j) mt = fmaxf(mt, sv[j]);
+                // row maximum over the 4 threads of this head (2 half-pages x 2 column halves, 4 different warps)
+                xch[hd * 4 + slot4] = mt;
+                named_bar_sync_dyn<128>(2 + half_id);
+                {
+                    const float4 x4 = *reinterpret_cast<const float4 *>(&xch[hd * 4]);
+                    mt = fmaxf(fmaxf(x4.x, x4.y), fmaxf(x4.z, x4.w));
+                }
+                bool grew = false;
+                float al = 1.f;
+                if (mt > m + kTau) { al = (m == -INFINITY) ? 0.f : fast_exp2(m - mt); m = mt; l *= al; grew = true; }
+                if (slot4 == 0) alpha_s[hd] = al;
+                const float mref = m == -INFINITY ? 0.f : m;   // a head that has seen no token yet: all weights 0, not NaN
+                uint32_t pk[8];
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    const float u0 = fast_exp2(sv[j] - mref), u1 = fast_exp2(sv[j + 1] - mref);
+                    l += u0 + u1;
+                    pk[j >> 1] = pack_bf16x2(u0, u1);
+                }
+                const bool rescale = named_bar_or<1, kSoftmaxWarps * 32>(grew);
+                // P.V of the tile that last used the P buffer of half-page 1 (two back) must be done; a rescale
+                // of O also needs the previous tile's P.V
+                if (kv_it > 1) ok &= mbar_wait(ctx, bar(kBarStageEmpty + (kv_it - 2) % kStages), ((kv_it - 2) / kStages) & 1, kBarStageEmpty);
+                if (rescale && tile != seg.tile_begin) {
+                    ok &= mbar_wait(ctx, bar(kBarStageEmpty + (kv_it - 1) % kStages), ((kv_it - 1) / kStages) & 1, kBarStageEmpty);
+                    tcgen05_fence_after();
+                    // O rows are TMEM lanes: this thread scales its lane's columns [128 cf, 128 cf + 128)
+                    const float a_row = alpha_s[hd];
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        float o[32];
+                        const uint32_t addr = tmem_base + lane_addr + kColO + 128 * cf + c * 32;
+                        tmem_ld32(addr, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) o[k] *= a_row;
+                        tmem_st16(addr, *reinterpret_cast<float(*)[16]>(&o[0]));
+                        tmem_st16(addr + 16, *reinterpret_cast<float(*)[16]>(&o[16]));
+                    }
+                    tmem_wait_st();
+                }
+                {
+                    // P of this half-page: K-major, 64-byte swizzle; row = head, bytes [32 cf, 32 cf + 32)
+                    uint8_t *ph = g == 0 ? smem + kOffK + (kv_it % kStages) * kStageBytes + 8 * kSlab : smem + kOffP1 + b * kPHalfBytes;
+                    *reinterpret_cast<uint4 *>(ph + sw64((uint32_t)hd, (uint32_t)(32 * cf))) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4 *>(ph + sw64((uint32_t)hd, (uint32_t)(32 * cf + 16))) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                }
+                fence_proxy_async();
+                tcgen05_fence_before();
+                __syncwarp();
+                if (lane == 0) arrive_on_leader(kBarPFull + b);
+            }
+            // ---- row sums of the 4 threads of a head
+            xch[hd * 4 + slot4] = l;
+            named_bar_sync<1, kSoftmaxWarps * 32>();
+            if (slot4 == 0) {
+                const float4 x4 = *reinterpret_cast<const float4 *>(&xch[hd * 4]);
+                const float lt = (x4.x + x4.y) + (x4.z + x4.w);
+                l_s[hd] = lt > 0.f ? 1.f / lt : 0.f;       // no token at all (an empty causal range): O = 0, LSE = -inf
+                const int gh = head0 + hd;
+                if (gh < p.head_end) {
+                    // (a poisoned row makes the sum NaN: it is passed on, so that the request's LSE is NaN like its output)
+                    float lse = lt > 0.f ? (m + log2f(lt)) * kLn2 : (lt == 0.f ? -INFINITY : lt);
+                    if (seg.slot < 0) p.lse[(int64_t)seg.request * p.lse_stride_request + gh] = lse;
+                    else p.partial_lse[(int64_t)seg.slot * h + (gh - p.head_begin)] = lse;
+                }
+            }
+            named_bar_sync<1, kSoftmaxWarps * 32>();
+            // ---- epilogue: lane L < 64 holds head L, dv [256 n, 256 n + 128) in columns n * 128 + j;
+            // lane 64 + L holds head L, dv [256 n + 128, 256 n + 256).  The two warps of a quadrant
+            // take one n each.  Read in the accumulator fragment layout (16 lanes at a time: thread T
+            // gets rows T/4 and T/4 + 8, two columns of every eight), so that a store instruction
+            // writes whole 32-byte sectors: 8 rows x 4 lanes x 8 bytes.
+            ok &= mbar_wait(ctx, bar(kBarOFull), seg_it & 1, kBarOFull);
+            tcgen05_fence_after();
+            {
+                float *obase;
+                int64_t ostride;
+                if (seg.slot < 0) {
+                    obase = p.out + (int64_t)seg.request * p.out_stride_request + (int64_t)head0 * p.out_stride_head;
+                    ostride = p.out_stride_head;
+                } else {
+                    obase = p.partial_out + ((int64_t)seg.slot * h + (head0 - p.head_begin)) * kDV;
+                    ostride = kDV;
+                }
+                const int n = cf;
+                const int dv0 = 256 * n + 128 * g + 2 * (lane & 3);
+                const int nvalid = min(kN, p.head_end - head0);
+#pragma unroll 1
+                for (int hc = 0; hc < 4; ++hc) {
+                    const int half = hc >> 1, c = hc & 1;
+                    const int hA = 32 * (q4 & 1) + 16 * half + (lane >> 2), hB = hA + 8;
+                    float o[32];
+                    tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * q4 + 16 * half) << 16) + kColO + n * 128 + c * 64, o);
+                    const float iA = l_s[hA], iB = l_s[hB];
+                    float *rowA = obase + (int64_t)hA * ostride + dv0 + c * 64, *rowB = obase + (int64_t)hB * ostride + dv0 + c * 64;
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (hA < nvalid) *reinterpret_cast<float2 *>(rowA + 8 * k) = make_float2(o[4 * k] * iA, o[4 * k + 1] * iA);
+                        if (hB < nvalid) *reinterpret_cast<float2 *>(rowB + 8 * k) = make_float2(o[4 * k + 2] * iB, o[4 * k + 3] * iB);
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) arrive_on_leader(kBarOEmpty);
+            ++seg_it;
+        }
+    }
+
+    asm volatile("cp.async.wait_all;" ::: "memory");
+    fill_empty_requests(p, worker, head0, kN, tid, kThreads);
+    if (p.trace != nullptr && tid == 0) {   // per-CTA cycles and nanoseconds
+        p.trace[512 + blockIdx.x] = clock64() - t_start;
+        if (blockIdx.x < 256) p.trace[768 + blockIdx.x] = (long long)(global_timer_ns() - ns_start);
+    }
+
+    // ---- teardown: nobody leaves while its partner may still touch its shared memory or barriers
+    if (*ctx.abort_flag) {
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) { __nanosleep(1000); }
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 0) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_decode_sparse_pair(const DecodeParams &p, cudaStream_t stream) {
+    alignas(64) CUtensorMap mq;
+    if (!make_map_4d(&mq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, p.q, (uint64_t)p.H,
+                     (uint64_t)p.B, (uint64_t)p.q_stride_head * 2, 128,
+                     (uint64_t)(p.B > 1 ? p.q_stride_request : p.q_stride_head * p.H) * 2, (uint32_t)kN, 9))
+        return cudaErrorInvalidValue;
+    static bool configured[64] = {};
+    cudaError_t e = cudaSuccess;
+    if (first_use_on_device(configured)) {
+        e = cudaFuncSetAttribute(decode_sparse_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        if (e != cudaSuccess) return e;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(p.num_workers * 2)); cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];      // (the cluster shape is part of the kernel's declaration)
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, decode_sparse_pair_kernel, p, mq);
+    count_launch();
+    return e;
+}
+
+}  // namespace splash

@@ -15,6 +15,16 @@ TOL_O = TOL[1]["abs_o"]
 TOL_LSE = TOL[1]["lse"]
 
 
+# 0: the fused kernel (gather + dequantise + attention on CTA pairs); 2 (the no-pair flag): the gather kernel followed by
+# the dense kernels
+PATHS = {"fused": 0, "two_stage": 2}
+
+
+@pytest.fixture(params=list(PATHS))
+def flags(request):
+    return PATHS[request.param]
+
+
 def gpu_sparse(w, sel, cnt, sentinel=None, **kw):
     import torch
     from paper_2609_37626_b200 import binding
@@ -53,49 +63,49 @@ def compare_sparse(out, lse, ref_out, ref_lse, hb, he, what):
     (64, [700, 0, 129, 4000, 1], 300),              # an empty request, a list that ends inside a page
     (8, [100000], 1000),                            # one long context, a sparse pick
 ])
-def test_sparse_matches_the_oracle(H, lens, topk):
+def test_sparse_matches_the_oracle(flags, H, lens, topk):
     w = W.make_workload("sparse", 900 + H, lens, H=H, kv_dtype=2)
     sel, cnt = W.select_tokens(900 + H, w.seq_lens, topk)
     ref = oracle.mla_decode_sparse(w.q, w.kv_pool, w.block_table, w.seq_lens, sel, cnt, softmax_scale=w.softmax_scale)
-    out, lse = gpu_sparse(w, sel, cnt)
+    out, lse = gpu_sparse(w, sel, cnt, flags=flags)
     compare_sparse(out, lse, *ref, 0, H, f"H={H} topk={topk}")
 
 
-def test_sparse_head_slice_leaves_the_rest_untouched_and_is_reproducible():
+def test_sparse_head_slice_leaves_the_rest_untouched_and_is_reproducible(flags):
     H, hb, he = 32, 8, 24
     w = W.make_workload("sparseslice", 910, [900, 70, 3000, 129, 6], H=H, kv_dtype=2, head_begin=hb, head_end=he)
     sel, cnt = W.select_tokens(910, w.seq_lens, 256)
     cnt[1] = 0                                                # an empty list for a non-empty request
     ref = oracle.mla_decode_sparse(w.q, w.kv_pool, w.block_table, w.seq_lens, sel, cnt, softmax_scale=w.softmax_scale,
                                    head_begin=hb, head_end=he)
-    a = gpu_sparse(w, sel, cnt, sentinel=7.0)
+    a = gpu_sparse(w, sel, cnt, sentinel=7.0, flags=flags)
     compare_sparse(*a, *ref, hb, he, "slice")
     assert np.all(a[0][:, :hb] == 7.0) and np.all(a[0][:, he:] == 7.0) and np.all(a[1][:, :hb] == 7.0) and np.all(a[1][:, he:] == 7.0)
-    b = gpu_sparse(w, sel, cnt, sentinel=7.0)
+    b = gpu_sparse(w, sel, cnt, sentinel=7.0, flags=flags)
     assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
 
 
-def test_sparse_duplicates_and_wide_list_stride():
+def test_sparse_duplicates_and_wide_list_stride(flags):
     w = W.make_workload("sparsedup", 920, [500, 64], H=16, kv_dtype=2)
     rng = np.random.Generator(np.random.PCG64(920))
     sel = np.full((2, 200), -1, dtype=np.int32)               # a stride wider than max_selected
     sel[0, :90] = rng.integers(0, 500, size=90); sel[1, :70] = rng.integers(0, 64, size=70)     # with repeats
     cnt = np.array([90, 70], dtype=np.int32)
     ref = oracle.mla_decode_sparse(w.q, w.kv_pool, w.block_table, w.seq_lens, sel, cnt, softmax_scale=w.softmax_scale)
-    out, lse = gpu_sparse(w, sel, cnt, max_selected=96)
+    out, lse = gpu_sparse(w, sel, cnt, max_selected=96, flags=flags)
     compare_sparse(out, lse, *ref, 0, 16, "duplicates")
 
 
-def test_sparse_bad_entries_give_nan_for_that_request_only():
+def test_sparse_bad_entries_give_nan_for_that_request_only(flags):
     w = W.make_workload("sparsebad", 930, [300, 300, 300], H=16, kv_dtype=2)
     sel, cnt = W.select_tokens(930, w.seq_lens, 64)
     good = oracle.mla_decode_sparse(w.q, w.kv_pool, w.block_table, w.seq_lens, sel, cnt, softmax_scale=w.softmax_scale)
     bad = sel.copy(); bad[1, 17] = 300                        # one position past the end of request 1
-    out, lse = gpu_sparse(w, bad, cnt)
+    out, lse = gpu_sparse(w, bad, cnt, flags=flags)
     assert np.isnan(out[1]).all() and np.isnan(lse[1]).all()
     assert np.abs(out[[0, 2]] - good[0][[0, 2]]).max() <= TOL_O
     cnt2 = cnt.copy(); cnt2[2] = 65                           # a count above max_selected
-    out, lse = gpu_sparse(w, sel, cnt2, max_selected=64)
+    out, lse = gpu_sparse(w, sel, cnt2, max_selected=64, flags=flags)
     assert np.isnan(out[2]).all() and np.isfinite(out[:2]).all()
 
 
@@ -115,7 +125,7 @@ def test_sparse_argument_checks():
     assert torch.isfinite(out).all()
 
 
-def test_sparse_at_the_size_the_benchmark_times():
+def test_sparse_at_the_size_the_benchmark_times(flags):
     # c2's 64 context lengths, 2,048 listed tokens per request, all 128 heads: every output against the oracle
     c2 = W.config(2)
     w = W.make_workload("sparse_top2048", W.BASE_SEED + 60, c2.seq_lens, H=128, kv_dtype=2)
@@ -123,5 +133,5 @@ def test_sparse_at_the_size_the_benchmark_times():
     sel, cnt = W.select_tokens(W.BASE_SEED + 60, w.seq_lens, 2048)
     assert cnt.max() == 2048 and cnt.sum() > 100000
     ref = oracle.mla_decode_sparse(w.q, w.kv_pool, w.block_table, w.seq_lens, sel, cnt, softmax_scale=w.softmax_scale)
-    out, lse = gpu_sparse(w, sel, cnt)
+    out, lse = gpu_sparse(w, sel, cnt, flags=flags)
     compare_sparse(out, lse, *ref, 0, 128, "bench size")
