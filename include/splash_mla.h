@@ -70,7 +70,10 @@ enum {
     SPLASH_FLAG_SIMT = 1u,
     /* slices of 65..128 heads: use two independent 64-head CTAs per KV worker instead of a CTA
      * pair issuing cta_group::2 MMAs.  A diagnostic path. */
-    SPLASH_FLAG_NO_PAIR = 2u
+    SPLASH_FLAG_NO_PAIR = 2u,
+    /* splash_mla_decode_sparse only: one kernel that gathers, dequantises and multiplies (CTA pairs) instead of
+     * the gather kernel followed by the dense kernels.  Correct, not yet the faster of the two. */
+    SPLASH_FLAG_SPARSE_FUSED = 4u
 };
 
 /*

@@ -26,6 +26,7 @@ SPLASH_KV_E4M3_BLOCK_SCALE_BF16_ROPE = 2
 SPLASH_SPARSE_ROW_BYTES = 656
 SPLASH_FLAG_SIMT = 1
 SPLASH_FLAG_NO_PAIR = 2
+SPLASH_FLAG_SPARSE_FUSED = 4
 
 D_QK, D_V, PAGE_SIZE = 576, 512, 64
 

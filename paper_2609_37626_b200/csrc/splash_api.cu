@@ -343,7 +343,7 @@ int splash_mla_decode_sparse(const splash_mla_shape *shape, const void *q, const
     st.table_stride = shape->block_table_stride; st.ctx_lens = seq_lens; st.sel = sel_tokens; st.sel_count = sel_count;
     st.sel_stride = sel_stride; st.max_selected = max_selected; st.pages_per_request = v.pages_per_request;
     st.dense_table = reinterpret_cast<int32_t *>(ws + v.off_table);
-    st.fused = (shape->flags & (SPLASH_FLAG_NO_PAIR | SPLASH_FLAG_SIMT)) == 0;
+    st.fused = (shape->flags & SPLASH_FLAG_SPARSE_FUSED) != 0 && (shape->flags & (SPLASH_FLAG_NO_PAIR | SPLASH_FLAG_SIMT)) == 0;
     // plan (over the list counts) -> gather into the dense cache -> decode kernel over the dense cache -> combine
     return decode_dense(&v.dense, q, ws + v.off_pool, nullptr, st.dense_table, sel_count, head_begin, head_end, nullptr, nullptr,
                         out, lse, workspace, v.inner_bytes, stream_, &st);

@@ -14,16 +14,16 @@
 //   * an address warp walks the token list a few tiles ahead: list entry -> page id -> row
 //     address, four tiles abreast so that the chain of dependent loads is paid once per four
 //     tiles; it leaves the addresses in a ring in shared memory and pulls the rows into L2;
-//   * three converter warps copy the raw rows into a staging buffer with 16-byte asynchronous
-//     copies (no registers held while the rows travel), then dequantise from there (code x block
-//     scale, rounded to bf16) into the swizzled tile: this CTA's 32 tokens in full for QK^T, and
-//     the peer's 32 tokens' 256 columns for P.V once QK^T has retired.  Each warp copies and
-//     converts its own rows only, so the staging buffer needs no barrier of its own.
+//   * converter warps copy the raw rows into staging buffers with 16-byte asynchronous copies
+//     (no registers held while the rows travel), then dequantise from there (code x block
+//     scale, rounded to bf16) into the swizzled tile: three warps this CTA's 32 tokens in full
+//     for QK^T, three others the peer's 32 tokens' 256 columns for P.V once QK^T has retired.
+//     Each warp copies and converts its own rows only, so the staging buffers need no barrier.
 // Every listed row crosses HBM once (twice through L2: the peer reads it too).
 //
-// Roles per CTA (576 threads): address warp, 4 QK^T issuers and 2 P.V issuers (leader CTA only;
+// Roles per CTA (672 threads): address warp, 4 QK^T issuers and 2 P.V issuers (leader CTA only;
 // the first issuer warp of either CTA also loads that CTA's query rows), 8 softmax warps,
-// 3 converter warps.  Barriers that the issuers wait on live in the leader; the peer's warps
+// 3 + 3 converter warps.  Barriers that the issuers wait on live in the leader; the peer's warps
 // arrive on them across the cluster (relaxed arrivals: what they announce is already in place on
 // the peer's SM).
 #include <cuda_bf16.h>
@@ -42,9 +42,10 @@ constexpr int kWarpAddr = 0;
 constexpr int kWarpQk = 1;
 constexpr int kWarpPv = kWarpQk + kQkWarps;
 constexpr int kWarpSoftmax = kWarpPv + kPvWarps;       // 7: TMEM quadrant = warp & 3
-constexpr int kConvWarps = 3;
-constexpr int kWarpConv = kWarpSoftmax + kSoftmaxWarps;
-constexpr int kThreads = (kWarpConv + kConvWarps) * 32;   // 18 warps = 576 threads
+constexpr int kConvWarps = 3;                           // converter warps per duty (this CTA's tokens / the peer's columns)
+constexpr int kWarpConvK = kWarpSoftmax + kSoftmaxWarps;
+constexpr int kWarpConvV = kWarpConvK + kConvWarps;
+constexpr int kThreads = (kWarpConvV + kConvWarps) * 32;  // 21 warps = 672 threads
 constexpr int kN = 64;                              // heads per CTA
 constexpr int kHalf = 32;                           // tokens per CTA and tile
 constexpr uint32_t kSlab = kHalf * 128;             // one chunk of a half-page: 32 tokens x 128 B
@@ -52,7 +53,7 @@ constexpr uint32_t kStageBytes = 9 * kSlab;         // 36,864
 constexpr uint32_t kQSlab = kN * 128;               // one chunk of the query rows: 64 heads x 128 B
 constexpr uint32_t kQBytes = 9 * kQSlab;            // 73,728
 constexpr uint32_t kPHalfBytes = kN * 64;           // P of one half-page: 64 heads x 32 tokens bf16
-constexpr int kStages = 3;
+constexpr int kStages = 2;
 constexpr int kRing = 8;                            // tiles of row addresses the address warp may be ahead
 constexpr int kAddrBatch = 4;                       // tiles whose addresses are resolved abreast
 constexpr uint32_t kRowBytes = 656;                 // a cache row: 512 codes, 4 scales, 64 bf16 rope values
@@ -60,10 +61,10 @@ constexpr uint32_t kVRowBytes = 272;                // what P.V needs of a peer 
 constexpr float kTau = 8.0f;                        // O is rescaled only when a row maximum grows by more than 2^8
 
 enum BarrierId {
-    kBarKFull = 0,                        // [3] leader: both CTAs' 32 tokens converted (all converter warps of both)
-    kBarQkDone = kBarKFull + kStages,     // [3] QK^T of the stage retired (multicast commit): peer columns may be written
-    kBarVFull = kBarQkDone + kStages,     // [3] leader: both CTAs' peer columns converted
-    kBarStageEmpty = kBarVFull + kStages, // [3] P.V of the stage retired (multicast commit): stage and P buffers
+    kBarKFull = 0,                        // [2] leader: both CTAs' 32 tokens converted (all converter warps of both)
+    kBarQkDone = kBarKFull + kStages,     // [2] QK^T of the stage retired (multicast commit): peer columns may be written
+    kBarVFull = kBarQkDone + kStages,     // [2] leader: both CTAs' peer columns converted
+    kBarStageEmpty = kBarVFull + kStages, // [2] P.V of the stage retired (multicast commit): stage and P buffers
                                           //     are free, O is up to date
     kBarQFull = kBarStageEmpty + kStages, // leader: query rows of both CTAs landed
     kBarQEmpty,                           // last QK^T of the request retired (multicast commit)
@@ -77,12 +78,13 @@ enum BarrierId {
     kNumBarriers = kBarAddrEmpty + kRing
 };
 
-constexpr uint32_t kOffK = 0;                                   // [3 stages] 9 chunk slots of 32 tokens
+constexpr uint32_t kOffK = 0;                                   // [2 stages] 9 chunk slots of 32 tokens
 constexpr uint32_t kOffQ = kOffK + kStages * kStageBytes;       // 9 chunks x 64 heads x 128 B
 constexpr uint32_t kOffP1 = kOffQ + kQBytes;                    // [2 buffers] P of half-page 1: 64 heads x 64 B
-constexpr uint32_t kOffRawK = kOffP1 + 2 * kPHalfBytes;         // raw rows of this CTA's 32 tokens: 32 x 656 B
-constexpr uint32_t kOffRawV = kOffRawK + kHalf * kRowBytes;     // the peer's 32 tokens, the 272 bytes P.V needs of each
-constexpr uint32_t kOffRing = kOffRawV + kHalf * kVRowBytes;    // uint64 [8][64] row addresses (0: zero row, 1: poisoned row)
+constexpr uint32_t kRawKBytes = kHalf * kRowBytes, kRawVBytes = kHalf * kVRowBytes;
+constexpr uint32_t kOffRawK = kOffP1 + 2 * kPHalfBytes;         // [2 buffers] raw rows of this CTA's 32 tokens: 32 x 656 B
+constexpr uint32_t kOffRawV = kOffRawK + 2 * kRawKBytes;        // [2 buffers] the peer's 32 tokens, the 272 bytes P.V needs of each
+constexpr uint32_t kOffRing = kOffRawV + 2 * kRawVBytes;        // uint64 [8][64] row addresses (0: zero row, 1: poisoned row)
 constexpr uint32_t kOffAlpha = kOffRing + kRing * 64 * 8;       // float [64]
 constexpr uint32_t kOffL = kOffAlpha + kN * 4;                  // float [64]
 constexpr uint32_t kOffXch = kOffL + kN * 4;                    // float [64][4]
@@ -136,7 +138,7 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
             mbar_init(bar(kBarKFull + s), 2 * kConvWarps); mbar_init(bar(kBarQkDone + s), kQkWarps);
             mbar_init(bar(kBarVFull + s), 2 * kConvWarps); mbar_init(bar(kBarStageEmpty + s), kPvWarps);
         }
-        for (int s = 0; s < kRing; ++s) { mbar_init(bar(kBarAddrFull + s), 1); mbar_init(bar(kBarAddrEmpty + s), kConvWarps); }
+        for (int s = 0; s < kRing; ++s) { mbar_init(bar(kBarAddrFull + s), 1); mbar_init(bar(kBarAddrEmpty + s), 2 * kConvWarps); }
         mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), kQkWarps);
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), 2 * kSoftmaxWarps);
@@ -231,123 +233,146 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
                 ++kv_it;
             }
         }
-    } else if (warp >= kWarpConv) {
+    } else if (warp >= kWarpConvK) {
         // ===================================================== converter warps
-        // Warp c takes rows c, c + 3, ... of this CTA's 32 tokens (all 576 columns, for QK^T and as this CTA's
-        // own half of P.V) and of the peer's 32 tokens (the 256 latent columns this CTA multiplies in P.V).
-        const int c = warp - kWarpConv;
+        // Three warps build this CTA's 32 tokens of every tile (all 576 columns: its half of the B operand of
+        // QK^T, and its own tokens' share of P.V), three others the peer's 32 tokens' 256 latent columns that this
+        // CTA multiplies in P.V, which go to slots that are dead once QK^T of the stage has retired.  Warp c of
+        // either trio takes rows c, c + 3, ...; it copies exactly the raw rows it later converts (two buffers: the
+        // copies of tile kv + 2 start when tile kv is converted), so the staging area needs no barrier.
+        const bool is_v = warp >= kWarpConvV;
+        const int c = (warp - kWarpConvK) % kConvWarps;
         const unsigned long long *ring = reinterpret_cast<const unsigned long long *>(smem + kOffRing);
-        uint8_t *raw_k = smem + kOffRawK, *raw_v = smem + kOffRawV;
-        const uint32_t raw_k_s = sbase + kOffRawK, raw_v_s = sbase + kOffRawV;
-        // total number of tiles of this worker (the role does not care about request boundaries)
-        uint32_t total = 0;
+        uint32_t total = 0;         // tiles of this worker (the role does not care about request boundaries)
         while (it.next(p, seg)) total += (uint32_t)(seg.tile_end - seg.tile_begin);
         bool ok = true;
         auto cp16 = [](uint32_t dst, const void *src) {
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
         };
-        auto commit = []() { asm volatile("cp.async.commit_group;" ::: "memory"); };
-        // raw rows of tile kv: this CTA's tokens in full, then the peer's tokens' P.V columns, one copy group each
-        auto issue_k = [&](uint32_t kv) {
+        const int half_of_rows = is_v ? 1 - (int)rank : (int)rank;       // which 32 rows of the 64-row box
+        // the raw rows of tile kv into staging buffer kv & 1: one copy group (possibly empty)
+        auto issue = [&](uint32_t kv) {
             if (kv < total && ok) {
                 const uint32_t slot = kv % kRing;
                 if (lane == 0) ok = mbar_wait(ctx, bar(kBarAddrFull + slot), (kv / kRing) & 1, kBarAddrFull + slot);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (ok) {
+                    const uint32_t raw = sbase + (is_v ? kOffRawV + (kv & 1) * kRawVBytes : kOffRawK + (kv & 1) * kRawKBytes);
                     for (int t = c; t < kHalf; t += kConvWarps) {
-                        const unsigned long long a = ring[slot * 64 + 32 * rank + t];
-                        if (a > 1ull) {
-                            const uint8_t *row = reinterpret_cast<const uint8_t *>(a);
-                            cp16(raw_k_s + t * kRowBytes + 16 * lane, row + 16 * lane);
-                            if (lane < 9) cp16(raw_k_s + t * kRowBytes + 512 + 16 * lane, row + 512 + 16 * lane);
+                        const unsigned long long a = ring[slot * 64 + 32 * half_of_rows + t];
+                        if (a <= 1ull) continue;
+                        const uint8_t *row = reinterpret_cast<const uint8_t *>(a);
+                        if (!is_v) {
+                            cp16(raw + t * kRowBytes + 16 * lane, row + 16 * lane);
+                            if (lane < 9) cp16(raw + t * kRowBytes + 512 + 16 * lane, row + 512 + 16 * lane);
+                        } else if (lane < 17) {
+                            // units 0-7: codes [128 r, + 128); 8-15: codes [256 + 128 r, + 128); 16: the four scales
+                            const uint32_t off = lane < 8 ? 128 * rank + 16 * lane : lane < 16 ? 256 + 128 * rank + 16 * (lane - 8) : 512;
+                            cp16(raw + t * kVRowBytes + 16 * lane, row + off);
                         }
                     }
                 }
             }
-            commit();
+            asm volatile("cp.async.commit_group;" ::: "memory");
         };
-        auto issue_v = [&](uint32_t kv) {
-            if (kv < total && ok) {
-                const uint32_t slot = kv % kRing;
-                for (int t = c; t < kHalf; t += kConvWarps) {
-                    const unsigned long long a = ring[slot * 64 + 32 * (1 - rank) + t];
-                    if (a > 1ull && lane < 17) {
-                        // units 0-7: codes [128 r, + 128); 8-15: codes [256 + 128 r, + 128); 16: the four scales
-                        const uint8_t *row = reinterpret_cast<const uint8_t *>(a);
-                        const uint32_t off = lane < 8 ? 128 * rank + 16 * lane : lane < 16 ? 256 + 128 * rank + 16 * (lane - 8) : 512;
-                        cp16(raw_v_s + t * kVRowBytes + 16 * lane, row + off);
-                    }
-                }
-            }
-            commit();
-        };
-        issue_k(0);
-        issue_v(0);
+        long long *const trace = (blockIdx.x == 0 && c == 0 && lane == 0) ? p.trace : nullptr;
+        auto mark = [&](uint32_t tile, int ev) { if (trace != nullptr && tile < 64) trace[tile * 8 + ev + (is_v ? 4 : 0)] = clock64(); };
+        issue(0);
+        issue(1);
         for (uint32_t kv = 0; kv < total && ok; ++kv) {
             const uint32_t stage = kv % kStages, sph = (kv / kStages) & 1, slot = kv % kRing;
             uint8_t *k0 = smem + kOffK + stage * kStageBytes;
-            // ---- this CTA's tokens: all but the latest copy group (the peer columns of this tile) have landed
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
+            mark(kv, 0);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");      // all but the latest group: tile kv has landed
             __syncwarp();
-            if (lane == 0) ok = mbar_wait(ctx, bar(kBarStageEmpty + stage), sph ^ 1, kBarStageEmpty + stage);
+            // this CTA's tokens go to a stage that P.V has left; the peer's columns to slots QK^T has left
+            if (lane == 0)
+                ok = is_v ? mbar_wait(ctx, bar(kBarQkDone + stage), sph, kBarQkDone + stage)
+                          : mbar_wait(ctx, bar(kBarStageEmpty + stage), sph ^ 1, kBarStageEmpty + stage);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
-            for (int t = c; t < kHalf; t += kConvWarps) {
-                const unsigned long long a = ring[slot * 64 + 32 * rank + t];
-                uint4 lo, hi, rope;
-                if (a > 1ull) {
-                    // lane l: codes [16 l, 16 l + 16) = units 2 (l & 3), + 1 of chunk l >> 2; lanes 0-7: rope unit l
-                    const uint8_t *src = raw_k + t * kRowBytes;
-                    const uint4 lat = *reinterpret_cast<const uint4 *>(src + 16 * lane);
-                    const float s = *reinterpret_cast<const float *>(src + 512 + 4 * (lane >> 3));
-                    if (lane < 8) rope = *reinterpret_cast<const uint4 *>(src + 528 + 16 * lane);
-                    const uint2 x0 = dequant4(lat.x, s), x1 = dequant4(lat.y, s), x2 = dequant4(lat.z, s), x3 = dequant4(lat.w, s);
-                    lo = make_uint4(x0.x, x0.y, x1.x, x1.y); hi = make_uint4(x2.x, x2.y, x3.x, x3.y);
-                } else {
-                    const uint32_t fill = a == 0ull ? 0u : 0x7FC07FC0u;
-                    lo = hi = rope = make_uint4(fill, fill, fill, fill);
+            mark(kv, 1);
+            const unsigned long long *addr_row = ring + slot * 64 + 32 * half_of_rows;
+            if (!is_v) {
+                const uint8_t *raw = smem + kOffRawK + (kv & 1) * kRawKBytes;
+                // lane l: codes [16 l, 16 l + 16) = units 2 (l & 3), + 1 of chunk l >> 2; lanes 0-7: rope unit l.
+                // Four rows at a time: all their loads first, then the arithmetic.
+                for (int t0 = c; t0 < kHalf; t0 += 4 * kConvWarps) {
+                    uint4 lat[4], rope[4];
+                    float sc[4];
+                    unsigned long long a[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int t = t0 + u * kConvWarps;
+                        a[u] = t < kHalf ? addr_row[t] : 0ull;
+                        if (t < kHalf && a[u] > 1ull) {
+                            const uint8_t *src = raw + t * kRowBytes;
+                            lat[u] = *reinterpret_cast<const uint4 *>(src + 16 * lane);
+                            sc[u] = *reinterpret_cast<const float *>(src + 512 + 4 * (lane >> 3));
+                            if (lane < 8) rope[u] = *reinterpret_cast<const uint4 *>(src + 528 + 16 * lane);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int t = t0 + u * kConvWarps;
+                        if (t >= kHalf) continue;
+                        uint4 lo, hi, rp = rope[u];
+                        if (a[u] > 1ull) {
+                            const uint2 x0 = dequant4(lat[u].x, sc[u]), x1 = dequant4(lat[u].y, sc[u]), x2 = dequant4(lat[u].z, sc[u]),
+                                        x3 = dequant4(lat[u].w, sc[u]);
+                            lo = make_uint4(x0.x, x0.y, x1.x, x1.y); hi = make_uint4(x2.x, x2.y, x3.x, x3.y);
+                        } else {
+                            const uint32_t fill = a[u] == 0ull ? 0u : 0x7FC07FC0u;
+                            lo = hi = rp = make_uint4(fill, fill, fill, fill);
+                        }
+                        uint8_t *dst = k0 + (lane >> 2) * kSlab + t * 128;
+                        const uint32_t u0 = 2 * (lane & 3);
+                        *reinterpret_cast<uint4 *>(dst + ((u0 ^ (t & 7)) << 4)) = lo;
+                        *reinterpret_cast<uint4 *>(dst + (((u0 + 1) ^ (t & 7)) << 4)) = hi;
+                        if (lane < 8) *reinterpret_cast<uint4 *>(k0 + 8 * kSlab + t * 128 + ((lane ^ (t & 7)) << 4)) = rp;
+                    }
                 }
-                uint8_t *dst = k0 + (lane >> 2) * kSlab + t * 128;
-                const uint32_t u0 = 2 * (lane & 3);
-                *reinterpret_cast<uint4 *>(dst + ((u0 ^ (t & 7)) << 4)) = lo;
-                *reinterpret_cast<uint4 *>(dst + (((u0 + 1) ^ (t & 7)) << 4)) = hi;
-                if (lane < 8) *reinterpret_cast<uint4 *>(k0 + 8 * kSlab + t * 128 + ((lane ^ (t & 7)) << 4)) = rope;
-            }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) arrive_on_leader(kBarKFull + stage);
-            issue_k(kv + 1);
-            // ---- the peer's tokens: their copy group has landed (only the group just issued may be pending);
-            // the slots they go to are dead once QK^T of the stage has retired
-            asm volatile("cp.async.wait_group 1;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) ok = mbar_wait(ctx, bar(kBarQkDone + stage), sph, kBarQkDone + stage);
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-            if (!ok) break;
-            {
+            } else {
+                const uint8_t *raw = smem + kOffRawV + (kv & 1) * kRawVBytes;
                 // lane l = 16 n + 8 e + w: codes [8 w, + 8) of chunk 4 n + 2 rank + e -> unit w of slot 4 n + 2 (1 - rank) + e
                 const int n = lane >> 4, e = (lane >> 3) & 1, w = lane & 7;
                 uint8_t *dst_slot = k0 + (4 * n + 2 * (1 - (int)rank) + e) * kSlab;
-                for (int t = c; t < kHalf; t += kConvWarps) {
-                    const unsigned long long a = ring[slot * 64 + 32 * (1 - rank) + t];
-                    uint4 v;
-                    if (a > 1ull) {
-                        const uint8_t *src = raw_v + t * kVRowBytes;
-                        const uint2 codes = *reinterpret_cast<const uint2 *>(src + 8 * lane);
-                        const float s = *reinterpret_cast<const float *>(src + 256 + 4 * (2 * n + (int)rank));
-                        const uint2 x0 = dequant4(codes.x, s), x1 = dequant4(codes.y, s);
-                        v = make_uint4(x0.x, x0.y, x1.x, x1.y);
-                    } else {
-                        const uint32_t fill = a == 0ull ? 0u : 0x7FC07FC0u;
-                        v = make_uint4(fill, fill, fill, fill);
+                for (int t0 = c; t0 < kHalf; t0 += 4 * kConvWarps) {
+                    uint2 codes[4];
+                    float sc[4];
+                    unsigned long long a[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int t = t0 + u * kConvWarps;
+                        a[u] = t < kHalf ? addr_row[t] : 0ull;
+                        if (t < kHalf && a[u] > 1ull) {
+                            const uint8_t *src = raw + t * kVRowBytes;
+                            codes[u] = *reinterpret_cast<const uint2 *>(src + 8 * lane);
+                            sc[u] = *reinterpret_cast<const float *>(src + 256 + 4 * (2 * n + (int)rank));
+                        }
                     }
-                    *reinterpret_cast<uint4 *>(dst_slot + t * 128 + ((w ^ (t & 7)) << 4)) = v;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int t = t0 + u * kConvWarps;
+                        if (t >= kHalf) continue;
+                        uint4 v;
+                        if (a[u] > 1ull) {
+                            const uint2 x0 = dequant4(codes[u].x, sc[u]), x1 = dequant4(codes[u].y, sc[u]);
+                            v = make_uint4(x0.x, x0.y, x1.x, x1.y);
+                        } else {
+                            const uint32_t fill = a[u] == 0ull ? 0u : 0x7FC07FC0u;
+                            v = make_uint4(fill, fill, fill, fill);
+                        }
+                        *reinterpret_cast<uint4 *>(dst_slot + t * 128 + ((w ^ (t & 7)) << 4)) = v;
+                    }
                 }
             }
             fence_proxy_async();
             __syncwarp();
-            if (lane == 0) { arrive_on_leader(kBarVFull + stage); mbar_arrive(bar(kBarAddrEmpty + slot)); }
-            issue_v(kv + 1);
+            if (lane == 0) { arrive_on_leader((is_v ? kBarVFull : kBarKFull) + stage); mbar_arrive(bar(kBarAddrEmpty + slot)); }
+            mark(kv, 2);
+            issue(kv + 2);
+            mark(kv, 3);
         }
     } else if (warp >= kWarpQk && warp < kWarpQk + kQkWarps && rank == 0) {
         // ===================================================== QK^T issuers (leader CTA)

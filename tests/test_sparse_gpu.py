@@ -15,9 +15,8 @@ TOL_O = TOL[1]["abs_o"]
 TOL_LSE = TOL[1]["lse"]
 
 
-# 0: the fused kernel (gather + dequantise + attention on CTA pairs); 2 (the no-pair flag): the gather kernel followed by
-# the dense kernels
-PATHS = {"fused": 0, "two_stage": 2}
+# 0: the gather kernel followed by the dense kernels; 4: the fused kernel (gather + dequantise + attention on CTA pairs)
+PATHS = {"two_stage": 0, "fused": 4}
 
 
 @pytest.fixture(params=list(PATHS))
