@@ -16,14 +16,15 @@
 //     tiles; it leaves the addresses in a ring in shared memory and pulls the rows into L2;
 //   * converter warps copy the raw rows into staging buffers with 16-byte asynchronous copies
 //     (no registers held while the rows travel), then dequantise from there (code x block
-//     scale, rounded to bf16) into the swizzled tile: three warps this CTA's 32 tokens in full
-//     for QK^T, three others the peer's 32 tokens' 256 columns for P.V once QK^T has retired.
+//     scale, as f16 -- tile, query rows and P are f16 in this kernel) into the swizzled tile: six
+//     warps this CTA's 32 tokens in full for QK^T, three others the peer's 32 tokens' 256 columns
+//     for P.V once QK^T has retired.
 //     Each warp copies and converts its own rows only, so the staging buffers need no barrier.
 // Every listed row crosses HBM once (twice through L2: the peer reads it too).
 //
-// Roles per CTA (672 threads): address warp, 4 QK^T issuers and 2 P.V issuers (leader CTA only;
+// Roles per CTA (768 threads): address warp, 4 QK^T issuers and 2 P.V issuers (leader CTA only;
 // the first issuer warp of either CTA also loads that CTA's query rows), 8 softmax warps,
-// 3 + 3 converter warps.  Barriers that the issuers wait on live in the leader; the peer's warps
+// 6 + 3 converter warps.  Barriers that the issuers wait on live in the leader; the peer's warps
 // arrive on them across the cluster (relaxed arrivals: what they announce is already in place on
 // the peer's SM).
 #include <cuda_bf16.h>
@@ -42,10 +43,10 @@ constexpr int kWarpAddr = 0;
 constexpr int kWarpQk = 1;
 constexpr int kWarpPv = kWarpQk + kQkWarps;
 constexpr int kWarpSoftmax = kWarpPv + kPvWarps;       // 7: TMEM quadrant = warp & 3
-constexpr int kConvWarps = 3;                           // converter warps per duty (this CTA's tokens / the peer's columns)
+constexpr int kConvKWarps = 6, kConvVWarps = 3;         // converter warps: this CTA's tokens / the peer's columns
 constexpr int kWarpConvK = kWarpSoftmax + kSoftmaxWarps;
-constexpr int kWarpConvV = kWarpConvK + kConvWarps;
-constexpr int kThreads = (kWarpConvV + kConvWarps) * 32;  // 21 warps = 672 threads
+constexpr int kWarpConvV = kWarpConvK + kConvKWarps;
+constexpr int kThreads = (kWarpConvV + kConvVWarps) * 32; // 24 warps = 768 threads
 constexpr int kN = 64;                              // heads per CTA
 constexpr int kHalf = 32;                           // tokens per CTA and tile
 constexpr uint32_t kSlab = kHalf * 128;             // one chunk of a half-page: 32 tokens x 128 B
@@ -66,7 +67,8 @@ enum BarrierId {
     kBarVFull = kBarQkDone + kStages,     // [2] leader: both CTAs' peer columns converted
     kBarStageEmpty = kBarVFull + kStages, // [2] P.V of the stage retired (multicast commit): stage and P buffers
                                           //     are free, O is up to date
-    kBarQFull = kBarStageEmpty + kStages, // leader: query rows of both CTAs landed
+    kBarQFull = kBarStageEmpty + kStages, // leader: query rows of both CTAs converted to f16 (all softmax warps of both)
+    kBarQLanded,                          // local: this CTA's query rows (bf16) landed
     kBarQEmpty,                           // last QK^T of the request retired (multicast commit)
     kBarSFull,                            // [2] S buffer written (multicast commit)
     kBarSEmpty = kBarSFull + 2,           // [2] S buffer read (leader: by both CTAs)
@@ -75,7 +77,8 @@ enum BarrierId {
     kBarOEmpty,                           // O drained (leader: by both CTAs)
     kBarAddrFull,                         // [8] local: row addresses of a tile written to the ring
     kBarAddrEmpty = kBarAddrFull + kRing, // [8] local: the converter warps are done with the ring slot
-    kNumBarriers = kBarAddrEmpty + kRing
+    kBarRaw = kBarAddrEmpty + kRing,      // [9 warps][2 buffers] local: a converter warp's raw rows landed (tx bytes)
+    kNumBarriers = kBarRaw + 2 * (kConvKWarps + kConvVWarps)
 };
 
 constexpr uint32_t kOffK = 0;                                   // [2 stages] 9 chunk slots of 32 tokens
@@ -97,11 +100,35 @@ static_assert(kOffRawK % 16 == 0 && kOffRawV % 16 == 0 && kOffRing % 8 == 0 && k
 // tensor memory: O two halves of dv x 128 columns, then 2 S buffers x 4 partials x 32 columns
 constexpr uint32_t kColO = 0, kColS = 256;
 
-// 4 e4m3 codes (one 32-bit word) times a scale -> 4 bf16 (two words)
-__device__ __forceinline__ uint2 dequant4(uint32_t w, float s) {
-    const float2 a = from_e4m3x2((uint16_t)(w & 0xffffu)), b = from_e4m3x2((uint16_t)(w >> 16));
-    __nv_bfloat162 lo = __floats2bfloat162_rn(a.x * s, a.y * s), hi = __floats2bfloat162_rn(b.x * s, b.y * s);
-    return make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+// The tile, the query rows and P are F16 here, not BF16: an e4m3 code becomes f16 exactly in one instruction and
+// the block scale is one packed multiply, where the way to bf16 leads through fp32 and costs three times the
+// instructions -- and the converter warps are what bounds this kernel.  (f16 also keeps three more significant
+// bits of code x scale.  Its range, 6e-5 .. 65504 for normal numbers, holds latent values and queries with room
+// to spare; a block scale above 146 would overflow.)
+constexpr uint32_t kF16Formats = ~((1u << 7) | (1u << 10));     // instruction descriptor: A and B formats F16 (0), not BF16 (1)
+constexpr uint32_t kF16NanPair = 0x7E007E00u;
+
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
+    return pack_f16x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint16_t v) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(v));
+    return r;
+}
+__device__ __forceinline__ uint32_t hmul2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+// 4 e4m3 codes (one 32-bit word) times a scale (the same in both halves of s2) -> 4 f16 (two words)
+__device__ __forceinline__ uint2 dequant4(uint32_t w, uint32_t s2) {
+    return make_uint2(hmul2(e4m3x2_to_f16x2((uint16_t)(w & 0xffffu)), s2), hmul2(e4m3x2_to_f16x2((uint16_t)(w >> 16)), s2));
 }
 
 __device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -135,11 +162,12 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     if (tid == 0) {
         // barriers the leader's issuers wait on count the warps of both CTAs (the peer's copies are unused)
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar(kBarKFull + s), 2 * kConvWarps); mbar_init(bar(kBarQkDone + s), kQkWarps);
-            mbar_init(bar(kBarVFull + s), 2 * kConvWarps); mbar_init(bar(kBarStageEmpty + s), kPvWarps);
+            mbar_init(bar(kBarKFull + s), 2 * kConvKWarps); mbar_init(bar(kBarQkDone + s), kQkWarps);
+            mbar_init(bar(kBarVFull + s), 2 * kConvVWarps); mbar_init(bar(kBarStageEmpty + s), kPvWarps);
         }
-        for (int s = 0; s < kRing; ++s) { mbar_init(bar(kBarAddrFull + s), 1); mbar_init(bar(kBarAddrEmpty + s), 2 * kConvWarps); }
-        mbar_init(bar(kBarQFull), 1); mbar_init(bar(kBarQEmpty), kQkWarps);
+        for (int s = 0; s < 2 * (kConvKWarps + kConvVWarps); ++s) mbar_init(bar(kBarRaw + s), 1);
+        for (int s = 0; s < kRing; ++s) { mbar_init(bar(kBarAddrFull + s), 1); mbar_init(bar(kBarAddrEmpty + s), kConvKWarps + kConvVWarps); }
+        mbar_init(bar(kBarQFull), 2 * kSoftmaxWarps); mbar_init(bar(kBarQLanded), 1); mbar_init(bar(kBarQEmpty), kQkWarps);
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), 2 * kSoftmaxWarps);
             mbar_init(bar(kBarPFull + b), 2 * kSoftmaxWarps);
@@ -235,45 +263,51 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         }
     } else if (warp >= kWarpConvK) {
         // ===================================================== converter warps
-        // Three warps build this CTA's 32 tokens of every tile (all 576 columns: its half of the B operand of
+        // Six warps build this CTA's 32 tokens of every tile (all 576 columns: its half of the B operand of
         // QK^T, and its own tokens' share of P.V), three others the peer's 32 tokens' 256 latent columns that this
         // CTA multiplies in P.V, which go to slots that are dead once QK^T of the stage has retired.  Warp c of
-        // either trio takes rows c, c + 3, ...; it copies exactly the raw rows it later converts (two buffers: the
+        // either group takes every sixth / third row; it copies exactly the raw rows it later converts (two buffers: the
         // copies of tile kv + 2 start when tile kv is converted), so the staging area needs no barrier.
         const bool is_v = warp >= kWarpConvV;
-        const int c = (warp - kWarpConvK) % kConvWarps;
+        const int c = is_v ? warp - kWarpConvV : warp - kWarpConvK;
+        const int nw = is_v ? kConvVWarps : kConvKWarps;
         const unsigned long long *ring = reinterpret_cast<const unsigned long long *>(smem + kOffRing);
         uint32_t total = 0;         // tiles of this worker (the role does not care about request boundaries)
         while (it.next(p, seg)) total += (uint32_t)(seg.tile_end - seg.tile_begin);
         bool ok = true;
-        auto cp16 = [](uint32_t dst, const void *src) {
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-        };
         const int half_of_rows = is_v ? 1 - (int)rank : (int)rank;       // which 32 rows of the 64-row box
-        // the raw rows of tile kv into staging buffer kv & 1: one copy group (possibly empty)
+        const int raw_bar = kBarRaw + 2 * (warp - kWarpConvK);
+        // The raw rows of tile kv into staging buffer kv & 1, as bulk copies that complete on this warp's barrier of
+        // that buffer: lane j takes the warp's j-th row.  (Per-lane 16-byte asynchronous copies do the same job
+        // through the load/store unit, and at 1,900 of them per tile they held up every shared-memory access of the SM.)
         auto issue = [&](uint32_t kv) {
             if (kv < total && ok) {
-                const uint32_t slot = kv % kRing;
+                const uint32_t slot = kv % kRing, buf = kv & 1;
                 if (lane == 0) ok = mbar_wait(ctx, bar(kBarAddrFull + slot), (kv / kRing) & 1, kBarAddrFull + slot);
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (ok) {
-                    const uint32_t raw = sbase + (is_v ? kOffRawV + (kv & 1) * kRawVBytes : kOffRawK + (kv & 1) * kRawKBytes);
-                    for (int t = c; t < kHalf; t += kConvWarps) {
-                        const unsigned long long a = ring[slot * 64 + 32 * half_of_rows + t];
-                        if (a <= 1ull) continue;
+                    const int t = c + lane * nw;
+                    const unsigned long long a = t < kHalf ? ring[slot * 64 + 32 * half_of_rows + t] : 0ull;
+                    const bool valid = a > 1ull;
+                    const unsigned m = __ballot_sync(0xffffffffu, valid);
+                    fence_proxy_async();          // the buffer was last read through the generic proxy
+                    __syncwarp();
+                    if (lane == 0) mbar_expect_tx(bar(raw_bar + buf), (uint32_t)__popc(m) * (is_v ? kVRowBytes : kRowBytes));
+                    __syncwarp();
+                    if (valid) {
                         const uint8_t *row = reinterpret_cast<const uint8_t *>(a);
                         if (!is_v) {
-                            cp16(raw + t * kRowBytes + 16 * lane, row + 16 * lane);
-                            if (lane < 9) cp16(raw + t * kRowBytes + 512 + 16 * lane, row + 512 + 16 * lane);
-                        } else if (lane < 17) {
-                            // units 0-7: codes [128 r, + 128); 8-15: codes [256 + 128 r, + 128); 16: the four scales
-                            const uint32_t off = lane < 8 ? 128 * rank + 16 * lane : lane < 16 ? 256 + 128 * rank + 16 * (lane - 8) : 512;
-                            cp16(raw + t * kVRowBytes + 16 * lane, row + off);
+                            bulk_load(sbase + kOffRawK + buf * kRawKBytes + t * kRowBytes, row, kRowBytes, bar(raw_bar + buf));
+                        } else {
+                            // codes [128 r, + 128), codes [256 + 128 r, + 128), the four scales
+                            const uint32_t dst = sbase + kOffRawV + buf * kRawVBytes + t * kVRowBytes;
+                            bulk_load(dst, row + 128 * rank, 128, bar(raw_bar + buf));
+                            bulk_load(dst + 128, row + 256 + 128 * rank, 128, bar(raw_bar + buf));
+                            bulk_load(dst + 256, row + 512, 16, bar(raw_bar + buf));
                         }
                     }
                 }
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
         };
         long long *const trace = (blockIdx.x == 0 && c == 0 && lane == 0) ? p.trace : nullptr;
         auto mark = [&](uint32_t tile, int ev) { if (trace != nullptr && tile < 64) trace[tile * 8 + ev + (is_v ? 4 : 0)] = clock64(); };
@@ -283,8 +317,9 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
             const uint32_t stage = kv % kStages, sph = (kv / kStages) & 1, slot = kv % kRing;
             uint8_t *k0 = smem + kOffK + stage * kStageBytes;
             mark(kv, 0);
-            asm volatile("cp.async.wait_group 1;" ::: "memory");      // all but the latest group: tile kv has landed
-            __syncwarp();
+            ok = mbar_wait(ctx, bar(raw_bar + (kv & 1)), (kv >> 1) & 1, raw_bar);      // the raw rows of tile kv have landed
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
             // this CTA's tokens go to a stage that P.V has left; the peer's columns to slots QK^T has left
             if (lane == 0)
                 ok = is_v ? mbar_wait(ctx, bar(kBarQkDone + stage), sph, kBarQkDone + stage)
@@ -293,78 +328,58 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
             if (!ok) break;
             mark(kv, 1);
             const unsigned long long *addr_row = ring + slot * 64 + 32 * half_of_rows;
+            // One row per iteration and no unrolling: the loop bodies are a few dozen instructions that stay in the
+            // instruction cache.  (Unrolled four rows deep for instruction-level parallelism, the straight-line code
+            // ran at a twelfth of an instruction per cycle: each warp walks it once per tile, alone.)
             if (!is_v) {
                 const uint8_t *raw = smem + kOffRawK + (kv & 1) * kRawKBytes;
-                // lane l: codes [16 l, 16 l + 16) = units 2 (l & 3), + 1 of chunk l >> 2; lanes 0-7: rope unit l.
-                // Four rows at a time: all their loads first, then the arithmetic.
-                for (int t0 = c; t0 < kHalf; t0 += 4 * kConvWarps) {
-                    uint4 lat[4], rope[4];
-                    float sc[4];
-                    unsigned long long a[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int t = t0 + u * kConvWarps;
-                        a[u] = t < kHalf ? addr_row[t] : 0ull;
-                        if (t < kHalf && a[u] > 1ull) {
-                            const uint8_t *src = raw + t * kRowBytes;
-                            lat[u] = *reinterpret_cast<const uint4 *>(src + 16 * lane);
-                            sc[u] = *reinterpret_cast<const float *>(src + 512 + 4 * (lane >> 3));
-                            if (lane < 8) rope[u] = *reinterpret_cast<const uint4 *>(src + 528 + 16 * lane);
-                        }
+                // lane l: codes [16 l, 16 l + 16) = units 2 (l & 3), + 1 of chunk l >> 2; rope word l of the ninth chunk
+                uint8_t *dst_lane = k0 + (lane >> 2) * kSlab;
+                const uint32_t u0 = 2 * (lane & 3);
+#pragma unroll 1
+                for (int t = c; t < kHalf; t += nw) {
+                    const unsigned long long a = addr_row[t];
+                    uint4 lo, hi;
+                    uint32_t rp;
+                    if (a > 1ull) {
+                        const uint8_t *src = raw + t * kRowBytes;
+                        const uint4 lat = *reinterpret_cast<const uint4 *>(src + 16 * lane);
+                        const uint32_t sc = pack_f16x2(*reinterpret_cast<const float *>(src + 512 + 4 * (lane >> 3)), 0.f);
+                        rp = bf16x2_to_f16x2(*reinterpret_cast<const uint32_t *>(src + 528 + 4 * lane));
+                        const uint32_t s2 = __byte_perm(sc, sc, 0x1010);          // the scale in both halves
+                        const uint2 x0 = dequant4(lat.x, s2), x1 = dequant4(lat.y, s2), x2 = dequant4(lat.z, s2), x3 = dequant4(lat.w, s2);
+                        lo = make_uint4(x0.x, x0.y, x1.x, x1.y); hi = make_uint4(x2.x, x2.y, x3.x, x3.y);
+                    } else {
+                        const uint32_t fill = a == 0ull ? 0u : kF16NanPair;
+                        lo = hi = make_uint4(fill, fill, fill, fill);
+                        rp = fill;
                     }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int t = t0 + u * kConvWarps;
-                        if (t >= kHalf) continue;
-                        uint4 lo, hi, rp = rope[u];
-                        if (a[u] > 1ull) {
-                            const uint2 x0 = dequant4(lat[u].x, sc[u]), x1 = dequant4(lat[u].y, sc[u]), x2 = dequant4(lat[u].z, sc[u]),
-                                        x3 = dequant4(lat[u].w, sc[u]);
-                            lo = make_uint4(x0.x, x0.y, x1.x, x1.y); hi = make_uint4(x2.x, x2.y, x3.x, x3.y);
-                        } else {
-                            const uint32_t fill = a[u] == 0ull ? 0u : 0x7FC07FC0u;
-                            lo = hi = rp = make_uint4(fill, fill, fill, fill);
-                        }
-                        uint8_t *dst = k0 + (lane >> 2) * kSlab + t * 128;
-                        const uint32_t u0 = 2 * (lane & 3);
-                        *reinterpret_cast<uint4 *>(dst + ((u0 ^ (t & 7)) << 4)) = lo;
-                        *reinterpret_cast<uint4 *>(dst + (((u0 + 1) ^ (t & 7)) << 4)) = hi;
-                        if (lane < 8) *reinterpret_cast<uint4 *>(k0 + 8 * kSlab + t * 128 + ((lane ^ (t & 7)) << 4)) = rp;
-                    }
+                    uint8_t *dst = dst_lane + t * 128;
+                    *reinterpret_cast<uint4 *>(dst + ((u0 ^ (t & 7)) << 4)) = lo;
+                    *reinterpret_cast<uint4 *>(dst + (((u0 + 1) ^ (t & 7)) << 4)) = hi;
+                    *reinterpret_cast<uint32_t *>(k0 + 8 * kSlab + t * 128 + ((((lane >> 2) ^ (t & 7))) << 4) + 4 * (lane & 3)) = rp;
                 }
             } else {
                 const uint8_t *raw = smem + kOffRawV + (kv & 1) * kRawVBytes;
                 // lane l = 16 n + 8 e + w: codes [8 w, + 8) of chunk 4 n + 2 rank + e -> unit w of slot 4 n + 2 (1 - rank) + e
                 const int n = lane >> 4, e = (lane >> 3) & 1, w = lane & 7;
                 uint8_t *dst_slot = k0 + (4 * n + 2 * (1 - (int)rank) + e) * kSlab;
-                for (int t0 = c; t0 < kHalf; t0 += 4 * kConvWarps) {
-                    uint2 codes[4];
-                    float sc[4];
-                    unsigned long long a[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int t = t0 + u * kConvWarps;
-                        a[u] = t < kHalf ? addr_row[t] : 0ull;
-                        if (t < kHalf && a[u] > 1ull) {
-                            const uint8_t *src = raw + t * kVRowBytes;
-                            codes[u] = *reinterpret_cast<const uint2 *>(src + 8 * lane);
-                            sc[u] = *reinterpret_cast<const float *>(src + 256 + 4 * (2 * n + (int)rank));
-                        }
+#pragma unroll 1
+                for (int t = c; t < kHalf; t += nw) {
+                    const unsigned long long a = addr_row[t];
+                    uint4 v;
+                    if (a > 1ull) {
+                        const uint8_t *src = raw + t * kVRowBytes;
+                        const uint2 codes = *reinterpret_cast<const uint2 *>(src + 8 * lane);
+                        const uint32_t sc = pack_f16x2(*reinterpret_cast<const float *>(src + 256 + 4 * (2 * n + (int)rank)), 0.f);
+                        const uint32_t s2 = __byte_perm(sc, sc, 0x1010);
+                        const uint2 x0 = dequant4(codes.x, s2), x1 = dequant4(codes.y, s2);
+                        v = make_uint4(x0.x, x0.y, x1.x, x1.y);
+                    } else {
+                        const uint32_t fill = a == 0ull ? 0u : kF16NanPair;
+                        v = make_uint4(fill, fill, fill, fill);
                     }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int t = t0 + u * kConvWarps;
-                        if (t >= kHalf) continue;
-                        uint4 v;
-                        if (a[u] > 1ull) {
-                            const uint2 x0 = dequant4(codes[u].x, sc[u]), x1 = dequant4(codes[u].y, sc[u]);
-                            v = make_uint4(x0.x, x0.y, x1.x, x1.y);
-                        } else {
-                            const uint32_t fill = a[u] == 0ull ? 0u : 0x7FC07FC0u;
-                            v = make_uint4(fill, fill, fill, fill);
-                        }
-                        *reinterpret_cast<uint4 *>(dst_slot + t * 128 + ((w ^ (t & 7)) << 4)) = v;
-                    }
+                    *reinterpret_cast<uint4 *>(dst_slot + t * 128 + ((w ^ (t & 7)) << 4)) = v;
                 }
             }
             fence_proxy_async();
@@ -381,7 +396,7 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         // accumulator each.
         if (lane == 0) {
             const int a = warp - kWarpQk;
-            constexpr uint32_t kIdescQK = make_idesc(128, 64, 0, 0);
+            constexpr uint32_t kIdescQK = make_idesc(128, 64, 0, 0) & kF16Formats;
             uint32_t kv_it = 0, seg_it = 0;
             bool ok = true;
             while (ok && it.next(p, seg)) {
@@ -389,8 +404,8 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
                     // the query rows of the request, once the last QK^T of the previous one has retired
                     ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
                     if (!ok) break;
-                    mbar_expect_tx(bar(kBarQFull), 2 * kQBytes);      // the rows of both CTAs
-                    tma_load_4d_pair(sbase + kOffQ, &tmap_q, leader_bar(kBarQFull), 0, head0, 0, seg.request);
+                    mbar_expect_tx(bar(kBarQLanded), kQBytes);
+                    tma_load_4d(sbase + kOffQ, &tmap_q, bar(kBarQLanded), 0, head0, 0, seg.request);
                 }
                 ok = mbar_wait_cluster(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
                 for (int tile = seg.tile_begin; ok && tile < seg.tile_end; ++tile, ++kv_it) {
@@ -419,7 +434,7 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         // ===================================================== P.V issuers (leader CTA)
         if (lane == 0) {
             const int n = warp - kWarpPv;                 // dv half: columns [256 n, 256 n + 256)
-            constexpr uint32_t kIdescPV = make_idesc(128, 256, 0, 1);
+            constexpr uint32_t kIdescPV = make_idesc(128, 256, 0, 1) & kF16Formats;
             uint32_t kv_it = 0, seg_it = 0;
             bool ok = true;
             while (ok && it.next(p, seg)) {
@@ -455,7 +470,10 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
             bool ok = true;
             while (ok && it.next(p, seg)) {
                 ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
-                if (ok) tma_load_4d_pair(sbase + kOffQ, &tmap_q, leader_bar(kBarQFull), 0, head0, 0, seg.request);
+                if (ok) {
+                    mbar_expect_tx(bar(kBarQLanded), kQBytes);
+                    tma_load_4d(sbase + kOffQ, &tmap_q, bar(kBarQLanded), 0, head0, 0, seg.request);
+                }
                 ++seg_it;
             }
         }
@@ -486,6 +504,20 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         while (it.next(p, seg)) {
             float m = -INFINITY, l = 0.f;               // running maximum in scaled log2 units
             const int first_page = seg.lo / kPage;
+            {
+                // the query rows arrive as bf16; the tile is f16 (see the converter warps), so they are rewritten in
+                // place, element for element (exact: eight significant bits fit f16's eleven), before QK^T may read them
+                ok &= mbar_wait(ctx, bar(kBarQLanded), seg_it & 1, kBarQLanded);
+                uint4 *qv = reinterpret_cast<uint4 *>(smem + kOffQ);
+                for (int i = sw * 32 + lane; i < (int)(kQBytes / 16); i += kSoftmaxWarps * 32) {
+                    uint4 x = qv[i];
+                    x.x = bf16x2_to_f16x2(x.x); x.y = bf16x2_to_f16x2(x.y); x.z = bf16x2_to_f16x2(x.z); x.w = bf16x2_to_f16x2(x.w);
+                    qv[i] = x;
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) arrive_on_leader(kBarQFull);
+            }
             // several query rows per request: this thread's (virtual) head is row (head mod R) and sees the
             // tokens below causal_end only
             const int causal_end = p.q_rows > 1 ? p.seq_lens[seg.request] - (p.q_rows - 1 - (head0 + hd) % p.q_rows) : 0x3fffffff;   // (far above any token index, and safe to subtract a negative offset from)
@@ -537,7 +569,7 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
                 for (int j = 0; j < 16; j += 2) {
                     const float u0 = fast_exp2(sv[j] - mref), u1 = fast_exp2(sv[j + 1] - mref);
                     l += u0 + u1;
-                    pk[j >> 1] = pack_bf16x2(u0, u1);
+                    pk[j >> 1] = pack_f16x2(u0, u1);
                 }
                 const bool rescale = named_bar_or<1, kSoftmaxWarps * 32>(grew);
                 // P.V of the tile that last used the P buffer of half-page 1 (two back) must be done; a rescale
@@ -631,7 +663,6 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         }
     }
 
-    asm volatile("cp.async.wait_all;" ::: "memory");
     fill_empty_requests(p, worker, head0, kN, tid, kThreads);
     if (p.trace != nullptr && tid == 0) {   // per-CTA cycles and nanoseconds
         p.trace[512 + blockIdx.x] = clock64() - t_start;
