@@ -78,6 +78,22 @@ def test_request_counts_and_skewed_lengths(flags, B):
     compare(out, lse, *ref, kv_dtype=0, what=f"B={B}")
 
 
+def test_more_requests_than_the_plan_stages_in_shared_memory():
+    # 4,500 short requests (the plan kernel keeps its prefix arrays in shared memory up to 4,096): sampled outputs
+    # against the oracle, every output finite, empty requests zero
+    B = 4500
+    rng = np.random.default_rng(77)
+    lens = rng.integers(0, 200, size=B)
+    w = W.make_workload("manyreq", 377, lens, H=16)
+    out, lse = gpu_run(w)
+    pairs = np.array(sorted({(int(rng.integers(0, B)), int(rng.integers(0, 16))) for _ in range(300)}), np.int32)
+    ref_o, ref_l = oracle_run(w, pairs=pairs)
+    compare(out, lse, ref_o, ref_l, kv_dtype=0, rows=[tuple(p) for p in pairs], what="B=4500")
+    assert np.isfinite(out).all()
+    empty = lens == 0
+    assert np.all(out[empty] == 0) and np.all(np.isneginf(lse[empty])) and np.isfinite(lse[~empty]).all()
+
+
 def test_empty_batch_and_empty_slice_are_no_ops(flags):
     import torch
     from paper_2609_37626_b200 import binding
