@@ -72,7 +72,8 @@ enum {
      * pair issuing cta_group::2 MMAs.  A diagnostic path. */
     SPLASH_FLAG_NO_PAIR = 2u,
     /* splash_mla_decode_sparse only: one kernel that gathers, dequantises and multiplies (CTA pairs) instead of
-     * the gather kernel followed by the dense kernels.  Correct, not yet the faster of the two. */
+     * the gather kernel followed by the dense kernels.  Every listed row crosses HBM once; tile, query rows and
+     * P are f16 in that kernel (values must lie within f16's range).  Correct, not yet the faster of the two. */
     SPLASH_FLAG_SPARSE_FUSED = 4u
 };
 

@@ -14,17 +14,17 @@
 //   * an address warp walks the token list a few tiles ahead: list entry -> page id -> row
 //     address, four tiles abreast so that the chain of dependent loads is paid once per four
 //     tiles; it leaves the addresses in a ring in shared memory and pulls the rows into L2;
-//   * converter warps copy the raw rows into staging buffers with 16-byte asynchronous copies
-//     (no registers held while the rows travel), then dequantise from there (code x block
-//     scale, as f16 -- tile, query rows and P are f16 in this kernel) into the swizzled tile: six
-//     warps this CTA's 32 tokens in full for QK^T, three others the peer's 32 tokens' 256 columns
-//     for P.V once QK^T has retired.
-//     Each warp copies and converts its own rows only, so the staging buffers need no barrier.
+//   * the eight softmax warps copy the raw rows into a staging area (one bulk copy per row, no
+//     registers held while the rows travel) and, between the softmax of one tile and the next,
+//     dequantise from there (code x block scale, as f16 -- tile, query rows and P are f16 in
+//     this kernel) into the swizzled tile: this CTA's 32 tokens in full for QK^T, and the peer's
+//     32 tokens' 256 columns for P.V once QK^T has retired.  Each warp copies and converts its
+//     own four rows only, so the staging area needs no barrier.
 // Every listed row crosses HBM once (twice through L2: the peer reads it too).
 //
-// Roles per CTA (768 threads): address warp, 4 QK^T issuers and 2 P.V issuers (leader CTA only;
-// the first issuer warp of either CTA also loads that CTA's query rows), 8 softmax warps,
-// 6 + 3 converter warps.  Barriers that the issuers wait on live in the leader; the peer's warps
+// Roles per CTA (480 threads): address warp, 4 QK^T issuers and 2 P.V issuers (leader CTA only;
+// the first issuer warp of either CTA also loads that CTA's query rows), 8 softmax warps that
+// also copy and convert the rows.  Barriers that the issuers wait on live in the leader; the peer's warps
 // arrive on them across the cluster (relaxed arrivals: what they announce is already in place on
 // the peer's SM).
 #include <cuda_bf16.h>
@@ -43,10 +43,8 @@ constexpr int kWarpAddr = 0;
 constexpr int kWarpQk = 1;
 constexpr int kWarpPv = kWarpQk + kQkWarps;
 constexpr int kWarpSoftmax = kWarpPv + kPvWarps;       // 7: TMEM quadrant = warp & 3
-constexpr int kConvKWarps = 6, kConvVWarps = 3;         // converter warps: this CTA's tokens / the peer's columns
-constexpr int kWarpConvK = kWarpSoftmax + kSoftmaxWarps;
-constexpr int kWarpConvV = kWarpConvK + kConvKWarps;
-constexpr int kThreads = (kWarpConvV + kConvVWarps) * 32; // 24 warps = 768 threads
+constexpr int kThreads = (kWarpSoftmax + kSoftmaxWarps) * 32;   // 15 warps = 480 threads
+constexpr int kRowsPerWarp = 4;                         // raw rows a softmax warp copies and converts per tile and duty
 constexpr int kN = 64;                              // heads per CTA
 constexpr int kHalf = 32;                           // tokens per CTA and tile
 constexpr uint32_t kSlab = kHalf * 128;             // one chunk of a half-page: 32 tokens x 128 B
@@ -58,7 +56,7 @@ constexpr int kStages = 2;
 constexpr int kRing = 8;                            // tiles of row addresses the address warp may be ahead
 constexpr int kAddrBatch = 4;                       // tiles whose addresses are resolved abreast
 constexpr uint32_t kRowBytes = 656;                 // a cache row: 512 codes, 4 scales, 64 bf16 rope values
-constexpr uint32_t kVRowBytes = 272;                // what P.V needs of a peer row: 2 x 128 codes, 4 scales
+constexpr uint32_t kVRowBytes = 528;                // a peer row without its rope part: 512 codes, 4 scales (P.V reads half the codes)
 constexpr float kTau = 8.0f;                        // O is rescaled only when a row maximum grows by more than 2^8
 
 enum BarrierId {
@@ -77,17 +75,17 @@ enum BarrierId {
     kBarOEmpty,                           // O drained (leader: by both CTAs)
     kBarAddrFull,                         // [8] local: row addresses of a tile written to the ring
     kBarAddrEmpty = kBarAddrFull + kRing, // [8] local: the converter warps are done with the ring slot
-    kBarRaw = kBarAddrEmpty + kRing,      // [9 warps][2 buffers] local: a converter warp's raw rows landed (tx bytes)
-    kNumBarriers = kBarRaw + 2 * (kConvKWarps + kConvVWarps)
+    kBarRaw = kBarAddrEmpty + kRing,      // [8 warps][own tokens, peer columns] local: a softmax warp's raw rows landed (tx bytes)
+    kNumBarriers = kBarRaw + 2 * kSoftmaxWarps
 };
 
 constexpr uint32_t kOffK = 0;                                   // [2 stages] 9 chunk slots of 32 tokens
 constexpr uint32_t kOffQ = kOffK + kStages * kStageBytes;       // 9 chunks x 64 heads x 128 B
 constexpr uint32_t kOffP1 = kOffQ + kQBytes;                    // [2 buffers] P of half-page 1: 64 heads x 64 B
 constexpr uint32_t kRawKBytes = kHalf * kRowBytes, kRawVBytes = kHalf * kVRowBytes;
-constexpr uint32_t kOffRawK = kOffP1 + 2 * kPHalfBytes;         // [2 buffers] raw rows of this CTA's 32 tokens: 32 x 656 B
-constexpr uint32_t kOffRawV = kOffRawK + 2 * kRawKBytes;        // [2 buffers] the peer's 32 tokens, the 272 bytes P.V needs of each
-constexpr uint32_t kOffRing = kOffRawV + 2 * kRawVBytes;        // uint64 [8][64] row addresses (0: zero row, 1: poisoned row)
+constexpr uint32_t kOffRawK = kOffP1 + 2 * kPHalfBytes;         // raw rows of this CTA's 32 tokens: 32 x 656 B
+constexpr uint32_t kOffRawV = kOffRawK + kRawKBytes;            // the peer's 32 tokens, codes and scales: 32 x 528 B
+constexpr uint32_t kOffRing = kOffRawV + kRawVBytes;            // uint64 [8][64] row addresses (0: zero row, 1: poisoned row)
 constexpr uint32_t kOffAlpha = kOffRing + kRing * 64 * 8;       // float [64]
 constexpr uint32_t kOffL = kOffAlpha + kN * 4;                  // float [64]
 constexpr uint32_t kOffXch = kOffL + kN * 4;                    // float [64][4]
@@ -162,11 +160,11 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
     if (tid == 0) {
         // barriers the leader's issuers wait on count the warps of both CTAs (the peer's copies are unused)
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar(kBarKFull + s), 2 * kConvKWarps); mbar_init(bar(kBarQkDone + s), kQkWarps);
-            mbar_init(bar(kBarVFull + s), 2 * kConvVWarps); mbar_init(bar(kBarStageEmpty + s), kPvWarps);
+            mbar_init(bar(kBarKFull + s), 2 * kSoftmaxWarps); mbar_init(bar(kBarQkDone + s), kQkWarps);
+            mbar_init(bar(kBarVFull + s), 2 * kSoftmaxWarps); mbar_init(bar(kBarStageEmpty + s), kPvWarps);
         }
-        for (int s = 0; s < 2 * (kConvKWarps + kConvVWarps); ++s) mbar_init(bar(kBarRaw + s), 1);
-        for (int s = 0; s < kRing; ++s) { mbar_init(bar(kBarAddrFull + s), 1); mbar_init(bar(kBarAddrEmpty + s), kConvKWarps + kConvVWarps); }
+        for (int s = 0; s < 2 * kSoftmaxWarps; ++s) mbar_init(bar(kBarRaw + s), 1);
+        for (int s = 0; s < kRing; ++s) { mbar_init(bar(kBarAddrFull + s), 1); mbar_init(bar(kBarAddrEmpty + s), kSoftmaxWarps); }
         mbar_init(bar(kBarQFull), 2 * kSoftmaxWarps); mbar_init(bar(kBarQLanded), 1); mbar_init(bar(kBarQEmpty), kQkWarps);
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), 2 * kSoftmaxWarps);
@@ -260,134 +258,6 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
                 if (lane == 0) mbar_arrive(bar(kBarAddrFull + slot));
                 ++kv_it;
             }
-        }
-    } else if (warp >= kWarpConvK) {
-        // ===================================================== converter warps
-        // Six warps build this CTA's 32 tokens of every tile (all 576 columns: its half of the B operand of
-        // QK^T, and its own tokens' share of P.V), three others the peer's 32 tokens' 256 latent columns that this
-        // CTA multiplies in P.V, which go to slots that are dead once QK^T of the stage has retired.  Warp c of
-        // either group takes every sixth / third row; it copies exactly the raw rows it later converts (two buffers: the
-        // copies of tile kv + 2 start when tile kv is converted), so the staging area needs no barrier.
-        const bool is_v = warp >= kWarpConvV;
-        const int c = is_v ? warp - kWarpConvV : warp - kWarpConvK;
-        const int nw = is_v ? kConvVWarps : kConvKWarps;
-        const unsigned long long *ring = reinterpret_cast<const unsigned long long *>(smem + kOffRing);
-        uint32_t total = 0;         // tiles of this worker (the role does not care about request boundaries)
-        while (it.next(p, seg)) total += (uint32_t)(seg.tile_end - seg.tile_begin);
-        bool ok = true;
-        const int half_of_rows = is_v ? 1 - (int)rank : (int)rank;       // which 32 rows of the 64-row box
-        const int raw_bar = kBarRaw + 2 * (warp - kWarpConvK);
-        // The raw rows of tile kv into staging buffer kv & 1, as bulk copies that complete on this warp's barrier of
-        // that buffer: lane j takes the warp's j-th row.  (Per-lane 16-byte asynchronous copies do the same job
-        // through the load/store unit, and at 1,900 of them per tile they held up every shared-memory access of the SM.)
-        auto issue = [&](uint32_t kv) {
-            if (kv < total && ok) {
-                const uint32_t slot = kv % kRing, buf = kv & 1;
-                if (lane == 0) ok = mbar_wait(ctx, bar(kBarAddrFull + slot), (kv / kRing) & 1, kBarAddrFull + slot);
-                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                if (ok) {
-                    const int t = c + lane * nw;
-                    const unsigned long long a = t < kHalf ? ring[slot * 64 + 32 * half_of_rows + t] : 0ull;
-                    const bool valid = a > 1ull;
-                    const unsigned m = __ballot_sync(0xffffffffu, valid);
-                    fence_proxy_async();          // the buffer was last read through the generic proxy
-                    __syncwarp();
-                    if (lane == 0) mbar_expect_tx(bar(raw_bar + buf), (uint32_t)__popc(m) * (is_v ? kVRowBytes : kRowBytes));
-                    __syncwarp();
-                    if (valid) {
-                        const uint8_t *row = reinterpret_cast<const uint8_t *>(a);
-                        if (!is_v) {
-                            bulk_load(sbase + kOffRawK + buf * kRawKBytes + t * kRowBytes, row, kRowBytes, bar(raw_bar + buf));
-                        } else {
-                            // codes [128 r, + 128), codes [256 + 128 r, + 128), the four scales
-                            const uint32_t dst = sbase + kOffRawV + buf * kRawVBytes + t * kVRowBytes;
-                            bulk_load(dst, row + 128 * rank, 128, bar(raw_bar + buf));
-                            bulk_load(dst + 128, row + 256 + 128 * rank, 128, bar(raw_bar + buf));
-                            bulk_load(dst + 256, row + 512, 16, bar(raw_bar + buf));
-                        }
-                    }
-                }
-            }
-        };
-        long long *const trace = (blockIdx.x == 0 && c == 0 && lane == 0) ? p.trace : nullptr;
-        auto mark = [&](uint32_t tile, int ev) { if (trace != nullptr && tile < 64) trace[tile * 8 + ev + (is_v ? 4 : 0)] = clock64(); };
-        issue(0);
-        issue(1);
-        for (uint32_t kv = 0; kv < total && ok; ++kv) {
-            const uint32_t stage = kv % kStages, sph = (kv / kStages) & 1, slot = kv % kRing;
-            uint8_t *k0 = smem + kOffK + stage * kStageBytes;
-            mark(kv, 0);
-            ok = mbar_wait(ctx, bar(raw_bar + (kv & 1)), (kv >> 1) & 1, raw_bar);      // the raw rows of tile kv have landed
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-            if (!ok) break;
-            // this CTA's tokens go to a stage that P.V has left; the peer's columns to slots QK^T has left
-            if (lane == 0)
-                ok = is_v ? mbar_wait(ctx, bar(kBarQkDone + stage), sph, kBarQkDone + stage)
-                          : mbar_wait(ctx, bar(kBarStageEmpty + stage), sph ^ 1, kBarStageEmpty + stage);
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-            if (!ok) break;
-            mark(kv, 1);
-            const unsigned long long *addr_row = ring + slot * 64 + 32 * half_of_rows;
-            // One row per iteration and no unrolling: the loop bodies are a few dozen instructions that stay in the
-            // instruction cache.  (Unrolled four rows deep for instruction-level parallelism, the straight-line code
-            // ran at a twelfth of an instruction per cycle: each warp walks it once per tile, alone.)
-            if (!is_v) {
-                const uint8_t *raw = smem + kOffRawK + (kv & 1) * kRawKBytes;
-                // lane l: codes [16 l, 16 l + 16) = units 2 (l & 3), + 1 of chunk l >> 2; rope word l of the ninth chunk
-                uint8_t *dst_lane = k0 + (lane >> 2) * kSlab;
-                const uint32_t u0 = 2 * (lane & 3);
-#pragma unroll 1
-                for (int t = c; t < kHalf; t += nw) {
-                    const unsigned long long a = addr_row[t];
-                    uint4 lo, hi;
-                    uint32_t rp;
-                    if (a > 1ull) {
-                        const uint8_t *src = raw + t * kRowBytes;
-                        const uint4 lat = *reinterpret_cast<const uint4 *>(src + 16 * lane);
-                        const uint32_t sc = pack_f16x2(*reinterpret_cast<const float *>(src + 512 + 4 * (lane >> 3)), 0.f);
-                        rp = bf16x2_to_f16x2(*reinterpret_cast<const uint32_t *>(src + 528 + 4 * lane));
-                        const uint32_t s2 = __byte_perm(sc, sc, 0x1010);          // the scale in both halves
-                        const uint2 x0 = dequant4(lat.x, s2), x1 = dequant4(lat.y, s2), x2 = dequant4(lat.z, s2), x3 = dequant4(lat.w, s2);
-                        lo = make_uint4(x0.x, x0.y, x1.x, x1.y); hi = make_uint4(x2.x, x2.y, x3.x, x3.y);
-                    } else {
-                        const uint32_t fill = a == 0ull ? 0u : kF16NanPair;
-                        lo = hi = make_uint4(fill, fill, fill, fill);
-                        rp = fill;
-                    }
-                    uint8_t *dst = dst_lane + t * 128;
-                    *reinterpret_cast<uint4 *>(dst + ((u0 ^ (t & 7)) << 4)) = lo;
-                    *reinterpret_cast<uint4 *>(dst + (((u0 + 1) ^ (t & 7)) << 4)) = hi;
-                    *reinterpret_cast<uint32_t *>(k0 + 8 * kSlab + t * 128 + ((((lane >> 2) ^ (t & 7))) << 4) + 4 * (lane & 3)) = rp;
-                }
-            } else {
-                const uint8_t *raw = smem + kOffRawV + (kv & 1) * kRawVBytes;
-                // lane l = 16 n + 8 e + w: codes [8 w, + 8) of chunk 4 n + 2 rank + e -> unit w of slot 4 n + 2 (1 - rank) + e
-                const int n = lane >> 4, e = (lane >> 3) & 1, w = lane & 7;
-                uint8_t *dst_slot = k0 + (4 * n + 2 * (1 - (int)rank) + e) * kSlab;
-#pragma unroll 1
-                for (int t = c; t < kHalf; t += nw) {
-                    const unsigned long long a = addr_row[t];
-                    uint4 v;
-                    if (a > 1ull) {
-                        const uint8_t *src = raw + t * kVRowBytes;
-                        const uint2 codes = *reinterpret_cast<const uint2 *>(src + 8 * lane);
-                        const uint32_t sc = pack_f16x2(*reinterpret_cast<const float *>(src + 256 + 4 * (2 * n + (int)rank)), 0.f);
-                        const uint32_t s2 = __byte_perm(sc, sc, 0x1010);
-                        const uint2 x0 = dequant4(codes.x, s2), x1 = dequant4(codes.y, s2);
-                        v = make_uint4(x0.x, x0.y, x1.x, x1.y);
-                    } else {
-                        const uint32_t fill = a == 0ull ? 0u : kF16NanPair;
-                        v = make_uint4(fill, fill, fill, fill);
-                    }
-                    *reinterpret_cast<uint4 *>(dst_slot + t * 128 + ((w ^ (t & 7)) << 4)) = v;
-                }
-            }
-            fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) { arrive_on_leader((is_v ? kBarVFull : kBarKFull) + stage); mbar_arrive(bar(kBarAddrEmpty + slot)); }
-            mark(kv, 2);
-            issue(kv + 2);
-            mark(kv, 3);
         }
     } else if (warp >= kWarpQk && warp < kWarpQk + kQkWarps && rank == 0) {
         // ===================================================== QK^T issuers (leader CTA)
@@ -501,6 +371,150 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
         // A failed (timed-out) wait only clears `ok`; the role keeps walking its tiles so that every
         // thread still meets the named barriers -- once the CTA aborts, waits return at once.
         bool ok = true;
+
+        // ---- the same eight warps also build the tiles (separate converter warps ran an order of magnitude below
+        // their instruction count: a dozen roles per SM wait on instruction fetch; eight warps that walk the same
+        // loops do not).  Warp sw owns rows 4 sw .. 4 sw + 3 of this CTA's 32 tokens (all 576 columns) and of the
+        // peer's 32 tokens (the 256 latent columns this CTA multiplies in P.V): it copies the raw rows (one bulk
+        // copy per row, lane u < 4 issues row u; they complete on the warp's own barrier) and later converts the
+        // rows it copied, so the staging area needs no barrier of its own.  Tile kv + 1 is built while P.V of tile
+        // kv - 1 has long retired (after the softmax of tile kv); the peer columns of tile kv follow at once, QK^T
+        // of tile kv having retired before its softmax could start.
+        const unsigned long long *ring = reinterpret_cast<const unsigned long long *>(smem + kOffRing);
+        uint32_t total = 0;         // tiles of this worker: the building duties do not care about request boundaries
+        {
+            SegmentIter it2 = it;
+            Segment seg2;
+            while (it2.next(p, seg2)) total += (uint32_t)(seg2.tile_end - seg2.tile_begin);
+        }
+        const int raw_bar_k = kBarRaw + 2 * sw, raw_bar_v = raw_bar_k + 1;
+        // Ask for the raw rows of two tiles at once: this CTA's tokens of tile kv_own (lanes 0-3, one row each) and the
+        // peer's tokens of tile kv_peer (lanes 4-7).  What becomes of each row -- copied, zero, poisoned -- is kept in
+        // two 4-bit masks per duty, so that the builders need not read the ring again.
+        uint32_t own_valid = 0, own_poison = 0, peer_valid = 0, peer_poison = 0;
+        auto issue_rows = [&](uint32_t kv_own, uint32_t kv_peer) {
+            const bool do_own = kv_own < total, do_peer = kv_peer < total;
+            if (!do_own && !do_peer) return;
+            if (do_own) ok &= mbar_wait(ctx, bar(kBarAddrFull + kv_own % kRing), (kv_own / kRing) & 1, kBarAddrFull);
+            if (do_peer) ok &= mbar_wait(ctx, bar(kBarAddrFull + kv_peer % kRing), (kv_peer / kRing) & 1, kBarAddrFull);
+            const int duty = lane >> 2, u = lane & 3;          // lanes 0-3: own rows, 4-7: peer rows
+            const bool mine = ok && lane < 8 && (duty == 0 ? do_own : do_peer);
+            const int t = kRowsPerWarp * sw + u;
+            const uint32_t slot = (duty == 0 ? kv_own : kv_peer) % kRing;
+            const int half_of_rows = duty == 0 ? (int)rank : 1 - (int)rank;
+            const unsigned long long a = mine ? ring[slot * 64 + 32 * half_of_rows + t] : 0ull;
+            const unsigned valid = __ballot_sync(0xffffffffu, a > 1ull), poison = __ballot_sync(0xffffffffu, a == 1ull);
+            if (do_own) { own_valid = valid & 15u; own_poison = poison & 15u; }
+            if (do_peer) { peer_valid = (valid >> 4) & 15u; peer_poison = (poison >> 4) & 15u; }
+            fence_proxy_async();          // the rows' staging space was last read through the generic proxy
+            __syncwarp();
+            if (lane == 0) {
+                if (do_own) mbar_expect_tx(bar(raw_bar_k), (uint32_t)__popc(valid & 15u) * kRowBytes);
+                if (do_peer) mbar_expect_tx(bar(raw_bar_v), (uint32_t)__popc(valid & 0xf0u) * kVRowBytes);
+            }
+            __syncwarp();
+            if (a > 1ull) {
+                if (duty == 0) bulk_load(sbase + kOffRawK + t * kRowBytes, reinterpret_cast<const void *>(a), kRowBytes, bar(raw_bar_k));
+                else bulk_load(sbase + kOffRawV + t * kVRowBytes, reinterpret_cast<const void *>(a), kVRowBytes, bar(raw_bar_v));
+            }
+        };
+        // this CTA's tokens of tile kv: raw rows -> f16 rows of the stage (needs P.V of tile kv - kStages retired).
+        // All loads of the four rows first, then the arithmetic and the stores.
+        auto build_own = [&](uint32_t kv) {
+            if (kv >= total) return;
+            const uint32_t stage = kv % kStages, sph = (kv / kStages) & 1;
+            ok &= mbar_wait(ctx, bar(raw_bar_k), kv & 1, raw_bar_k);
+            ok &= mbar_wait(ctx, bar(kBarStageEmpty + stage), sph ^ 1, kBarStageEmpty + stage);
+            uint8_t *k0 = smem + kOffK + stage * kStageBytes;
+            // lane l: codes [16 l, 16 l + 16) = units 2 (l & 3), + 1 of chunk l >> 2; rope word l of the ninth chunk
+            uint8_t *dst_lane = k0 + (lane >> 2) * kSlab;
+            const uint32_t u0 = 2 * (lane & 3);
+            const uint32_t valid = ok ? own_valid : 0u;
+            uint4 lat[kRowsPerWarp];
+            float scf[kRowsPerWarp];
+            uint32_t rope[kRowsPerWarp];
+#pragma unroll
+            for (int u = 0; u < kRowsPerWarp; ++u) {
+                const uint8_t *src = smem + kOffRawK + (kRowsPerWarp * sw + u) * kRowBytes;
+                if ((valid >> u) & 1u) {
+                    lat[u] = *reinterpret_cast<const uint4 *>(src + 16 * lane);
+                    scf[u] = *reinterpret_cast<const float *>(src + 512 + 4 * (lane >> 3));
+                    rope[u] = *reinterpret_cast<const uint32_t *>(src + 528 + 4 * lane);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kRowsPerWarp; ++u) {
+                const int t = kRowsPerWarp * sw + u;
+                uint4 lo, hi;
+                uint32_t rp;
+                if ((valid >> u) & 1u) {
+                    const uint32_t sc = pack_f16x2(scf[u], 0.f);
+                    const uint32_t s2 = __byte_perm(sc, sc, 0x1010);          // the scale in both halves
+                    const uint2 x0 = dequant4(lat[u].x, s2), x1 = dequant4(lat[u].y, s2), x2 = dequant4(lat[u].z, s2), x3 = dequant4(lat[u].w, s2);
+                    lo = make_uint4(x0.x, x0.y, x1.x, x1.y); hi = make_uint4(x2.x, x2.y, x3.x, x3.y);
+                    rp = bf16x2_to_f16x2(rope[u]);
+                } else {
+                    const uint32_t fill = ((own_poison >> u) & 1u) ? kF16NanPair : 0u;
+                    lo = hi = make_uint4(fill, fill, fill, fill);
+                    rp = fill;
+                }
+                uint8_t *dst = dst_lane + t * 128;
+                *reinterpret_cast<uint4 *>(dst + ((u0 ^ (t & 7)) << 4)) = lo;
+                *reinterpret_cast<uint4 *>(dst + (((u0 + 1) ^ (t & 7)) << 4)) = hi;
+                *reinterpret_cast<uint32_t *>(k0 + 8 * kSlab + t * 128 + ((((lane >> 2) ^ (t & 7))) << 4) + 4 * (lane & 3)) = rp;
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) arrive_on_leader(kBarKFull + stage);
+        };
+        // the peer's tokens of tile kv, the columns this CTA multiplies in P.V: into the slots QK^T of the tile has left
+        auto build_peer = [&](uint32_t kv) {
+            const uint32_t stage = kv % kStages, sph = (kv / kStages) & 1, slot = kv % kRing;
+            ok &= mbar_wait(ctx, bar(raw_bar_v), kv & 1, raw_bar_v);
+            ok &= mbar_wait(ctx, bar(kBarQkDone + stage), sph, kBarQkDone + stage);
+            uint8_t *k0 = smem + kOffK + stage * kStageBytes;
+            // lane l = 16 n + 8 e + w: codes [8 w, + 8) of chunk 4 n + 2 rank + e -> unit w of slot 4 n + 2 (1 - rank) + e
+            const int n = lane >> 4, e = (lane >> 3) & 1, w = lane & 7;
+            uint8_t *dst_slot = k0 + (4 * n + 2 * (1 - (int)rank) + e) * kSlab;
+            const uint32_t code_off = (4 * n + 2 * (int)rank + e) * 64 + 8 * w, scale_off = 512 + 4 * (2 * n + (int)rank);
+            const uint32_t valid = ok ? peer_valid : 0u;
+            uint2 codes[kRowsPerWarp];
+            float scf[kRowsPerWarp];
+#pragma unroll
+            for (int u = 0; u < kRowsPerWarp; ++u) {
+                const uint8_t *src = smem + kOffRawV + (kRowsPerWarp * sw + u) * kVRowBytes;
+                if ((valid >> u) & 1u) {
+                    codes[u] = *reinterpret_cast<const uint2 *>(src + code_off);
+                    scf[u] = *reinterpret_cast<const float *>(src + scale_off);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kRowsPerWarp; ++u) {
+                const int t = kRowsPerWarp * sw + u;
+                uint4 v;
+                if ((valid >> u) & 1u) {
+                    const uint32_t sc = pack_f16x2(scf[u], 0.f);
+                    const uint32_t s2 = __byte_perm(sc, sc, 0x1010);
+                    const uint2 x0 = dequant4(codes[u].x, s2), x1 = dequant4(codes[u].y, s2);
+                    v = make_uint4(x0.x, x0.y, x1.x, x1.y);
+                } else {
+                    const uint32_t fill = ((peer_poison >> u) & 1u) ? kF16NanPair : 0u;
+                    v = make_uint4(fill, fill, fill, fill);
+                }
+                *reinterpret_cast<uint4 *>(dst_slot + t * 128 + ((w ^ (t & 7)) << 4)) = v;
+            }
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) { arrive_on_leader(kBarVFull + stage); mbar_arrive(bar(kBarAddrEmpty + slot)); }
+        };
+        // diagnostic timeline of the first softmax warp of CTA 0: S landed, P written, own tokens of the next tile
+        // built, peer columns built, next rows asked for
+        long long *const trace = (blockIdx.x == 0 && sw == 0 && lane == 0) ? p.trace : nullptr;
+        auto mark = [&](uint32_t tile, int ev) { if (trace != nullptr && tile < 64) trace[tile * 8 + ev] = clock64(); };
+        issue_rows(0, 0);
+        build_own(0);
+        issue_rows(1, 0xffffffffu);       // (the masks now describe tile 1 / tile 0: the builders of the loop run before the next request)
+
         while (it.next(p, seg)) {
             float m = -INFINITY, l = 0.f;               // running maximum in scaled log2 units
             const int first_page = seg.lo / kPage;
@@ -524,7 +538,9 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
             for (int tile = seg.tile_begin; tile < seg.tile_end; ++tile, ++kv_it) {
                 const TileGeom geo = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);   // (lo = 0: list positions)
                 const uint32_t b = kv_it & 1;
+                mark(kv_it, 0);
                 ok &= mbar_wait(ctx, bar(kBarSFull + b), (kv_it >> 1) & 1, kBarSFull + b);
+                mark(kv_it, 1);
                 tcgen05_fence_after();
                 float sv[16];
                 {
@@ -603,6 +619,14 @@ decode_sparse_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensor
                 tcgen05_fence_before();
                 __syncwarp();
                 if (lane == 0) arrive_on_leader(kBarPFull + b);
+                // ---- the tiles ahead: this CTA's tokens of the next tile, then the peer's columns of this one
+                mark(kv_it, 2);
+                build_own(kv_it + 1);
+                mark(kv_it, 3);
+                build_peer(kv_it);
+                mark(kv_it, 4);
+                issue_rows(kv_it + 2, kv_it + 1);
+                mark(kv_it, 5);
             }
             // ---- row sums of the 4 threads of a head
             xch[hd * 4 + slot4] = l;
