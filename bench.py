@@ -275,6 +275,14 @@ class GpuBench:
         rc, detail = binding.splash_workspace_status(binding.decode_workspace(torch.device(self.device)))
         if rc != 0:
             raise RuntimeError(f"device status {rc} {detail}")
+        # the fused kernel (one kernel gathers, dequantises and multiplies), for comparison: not the default path
+        fused = lambda: binding.splash_mla_decode_sparse(dw.q, dw.kv_pool, dw.block_table, dw.seq_lens, sel, cnt,
+                                                         softmax_scale=w.softmax_scale, out=out, lse=lse,
+                                                         flags=binding.SPLASH_FLAG_SPARSE_FUSED)
+        ms_fused = self.timed(fused, steps, warmup)
+        rc, detail = binding.splash_workspace_status(binding.decode_workspace(torch.device(self.device)))
+        if rc != 0:
+            raise RuntimeError(f"device status {rc} {detail} (fused sparse kernel)")
         n_sel = int(cnt_h.sum())
         alg_bytes = W.sparse_algorithmic_bytes(cnt_h, H)
         alg_flops = 2 * H * (W.D_QK + W.D_V) * n_sel
@@ -290,6 +298,8 @@ class GpuBench:
                              "frac": max(t_hbm, t_tensor) * 1e3 / p50, "of": "whole call, p50", "peak_source": peaks["source"],
                              "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
                              "bytes_moved_by_the_two_stages": n_sel * (W.SPARSE_ROW_BYTES + 2 * W.D_QK * 2)},
+                "fused_kernel_variant": {"ms_p50": float(np.median(ms_fused)), "launches_per_step": binding.splash_last_launch_count(),
+                                         "note": "SPLASH_FLAG_SPARSE_FUSED: every listed row crosses HBM once; not the default while slower"},
                 "launches_per_step": launches}
 
     def dop_workload(self, steps, warmup, peaks, N=16384, T=8, h=16):
