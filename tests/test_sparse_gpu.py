@@ -134,3 +134,16 @@ def test_sparse_at_the_size_the_benchmark_times(flags):
     ref = oracle.mla_decode_sparse(w.q, w.kv_pool, w.block_table, w.seq_lens, sel, cnt, softmax_scale=w.softmax_scale)
     out, lse = gpu_sparse(w, sel, cnt, flags=flags)
     compare_sparse(out, lse, *ref, 0, 128, "bench size")
+
+
+def test_sparse_all_lists_empty_and_zero_capacity(flags):
+    import torch
+    from paper_2609_37626_b200 import binding
+    w = W.make_workload("sparseempty", 950, [100, 7], H=16, kv_dtype=2)
+    dw = binding.DeviceWorkload(w)
+    cnt = torch.zeros(2, dtype=torch.int32, device="cuda")
+    for sel in (torch.zeros((2, 0), dtype=torch.int32, device="cuda"), torch.full((2, 5), -1, dtype=torch.int32, device="cuda")):
+        out, lse = binding.splash_mla_decode_sparse(dw.q, dw.kv_pool, dw.block_table, dw.seq_lens, sel, cnt,
+                                                    softmax_scale=w.softmax_scale, flags=flags)
+        torch.cuda.synchronize()
+        assert torch.all(out == 0) and torch.all(torch.isneginf(lse))
