@@ -227,6 +227,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     p.heads_per_group = t.heads_per_group; p.num_groups = t.num_groups; p.num_workers = t.num_workers;
     p.softmax_scale = shape->softmax_scale;
     p.tile_start = v.tile_start; p.req_lo = v.req_lo; p.req_hi = v.req_hi; p.worker_begin = v.worker_begin;
+    p.worker_req = v.worker_req;
     p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
     p.trace = g_trace;
     p.len_cap = sparse ? sparse->max_selected : -1;
@@ -245,7 +246,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     e = record_timing_event(0, stream);
     if (e == cudaSuccess)
         e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
-                        v.cost_start, v.worker_begin, v.split_list, v.status, stream);
+                        v.cost_start, v.worker_begin, v.split_list, v.worker_req, v.status, stream);
     if (e == cudaSuccess) e = record_timing_event(1, stream);
     if (e == cudaSuccess && sparse && !fused_sparse)
         e = launch_sparse_gather(B, sparse->max_selected, sparse->pages_per_request, sparse->pool656, sparse->num_pool_pages,

@@ -45,6 +45,7 @@ struct PlanView {
     int32_t *cost_start;    // [B+1] exclusive prefix of per-request cost (tiles + overhead)
     int32_t *worker_begin;  // [W+1] global tile index where each worker starts
     int32_t *split_list;    // [W+1] requests computed in more than one piece (count in status[8])
+    int32_t *worker_req;    // [W+1] the request that holds a worker's first tile (what the kernels would bisect for)
     float *partial_lse;     // [2W][h]
     float *partial_out;     // [2W][h][512]
     int32_t num_workers;    // W
@@ -67,6 +68,7 @@ inline __host__ PlanView make_plan_view(void *workspace, int B, int W, int h) {
     v.cost_start = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(B + 1);
     v.worker_begin = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
     v.split_list = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
+    v.worker_req = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
     off = align_up(off, 256);
     v.partial_lse = reinterpret_cast<float *>(p + off); off += sizeof(float) * (size_t)2 * W * h;
     off = align_up(off, 256);
@@ -100,6 +102,7 @@ struct DecodeParams {
     float softmax_scale;
     // plan (device pointers into the workspace)
     const int32_t *tile_start, *req_lo, *req_hi, *worker_begin;
+    const int32_t *worker_req;   // request holding each worker's first tile, from the plan
     int32_t *status;
     float *partial_lse, *partial_out;
     int32_t len_cap;           // >= 0: seq_lens holds list counts; one outside [0, len_cap] counts as 1 (sparse decode)
@@ -129,12 +132,9 @@ struct SegmentIter {
     __device__ void init(const DecodeParams &p, int worker) {
         ts = p.tile_start; B = p.B; w = worker;
         wb = p.worker_begin[worker]; x = wb; end = p.worker_begin[worker + 1];
-        i = 0;
-        if (x < end) {   // request containing tile x: last i with ts[i] <= x and ts[i+1] > x
-            int lo = 0, hi = B;           // invariant: ts[lo] <= x < ts[hi]
-            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (ts[mid] <= x) lo = mid; else hi = mid; }
-            i = lo;
-        }
+        // the request containing tile x (last i with ts[i] <= x and ts[i+1] > x): the plan has it, which saves every
+        // role of every CTA a bisection of a dozen dependent global loads before its first tile
+        i = x < end ? p.worker_req[worker] : 0;
     }
     __device__ bool next(const DecodeParams &p, Segment &s) {
         if (x >= end) return false;
@@ -206,7 +206,7 @@ void count_launch(int n = 1);
 // kernels' host launchers
 cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
-                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
+                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list, int32_t *worker_req,
                         int32_t *status, cudaStream_t stream);
 cudaError_t launch_decode_sparse_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_sparse_gather(int B, int max_sel, int pages_per_request, const void *kv_pool, int num_pool_pages,

@@ -25,7 +25,8 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
             const int32_t *__restrict__ kv_end, int32_t *tile_start,
             int32_t *__restrict__ req_lo, int32_t *__restrict__ req_hi,
             int32_t *__restrict__ req_wfirst, int32_t *__restrict__ req_wlast,
-            int32_t *cost_start, int32_t *worker_begin, int32_t *__restrict__ split_list, int32_t *__restrict__ status) {
+            int32_t *cost_start, int32_t *worker_begin, int32_t *__restrict__ split_list, int32_t *__restrict__ worker_req,
+            int32_t *__restrict__ status) {
     __shared__ long long warp_tot_tiles[32], warp_tot_cost[32];
     __shared__ long long carry_tiles, carry_cost;
     __shared__ int n_split;
@@ -80,7 +81,7 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
     // bisection, and a start that falls into the request's fixed overhead snaps to
     // its first tile.
     for (int w = tid; w <= W; w += kPlanThreads) {
-        int g = total_tiles;
+        int g = total_tiles, first_req = 0;
         if (w < W && total_cost > 0) {
             long long target = (total_cost * w) / W;
             int lo = 0, hi = B;   // invariant cost_start[lo] <= target < cost_start[hi]
@@ -89,8 +90,10 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
             long long off = target - cost_start[lo] - overhead;
             if (off < 0) off = 0;
             g = tile_start[lo] + (int)off;
+            first_req = lo;
         }
         worker_begin[w] = g;
+        worker_req[w] = first_req;
     }
     __threadfence_block();
     __syncthreads();
@@ -127,14 +130,14 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
 cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
-                        int32_t *status, cudaStream_t stream) {
+                        int32_t *worker_req, int32_t *status, cudaStream_t stream) {
     // same shared-memory carve-out as the decode kernel that follows: no reconfiguration between them
     static bool configured[64] = {};
     if (first_use_on_device(configured)) {
         cudaFuncSetAttribute(plan_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     }
     plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.len_cap, p.seq_lens, kv_begin, kv_end, tile_start,
-                                                req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, split_list, status);
+                                                req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, split_list, worker_req, status);
     count_launch();
     return cudaGetLastError();
 }
