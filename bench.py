@@ -332,9 +332,12 @@ class GpuBench:
 
     def in_kernel_clock(self, dw, out, lse):
         """SM clock seen by the decode kernel itself: cycles / nanoseconds of its main loop, per CTA, from the
-        library's diagnostic trace (written by the CTA-pair kernels; None for the others)."""
+        library's diagnostic trace (written by the CTA-pair kernels; None for the others), and the longest CTA's
+        main loop in microseconds (after an L2 flush, like the timed steps): what the kernel executes, without the
+        launch and completion latency that the CUDA-event duration of a single launch includes."""
         torch, binding = self.torch, self.binding
         buf = torch.zeros(64 * 8 + 512, dtype=torch.int64, device=self.device)
+        self.flush_l2()
         binding.splash_debug_set_trace(buf)
         try:
             dw.decode(out=out, lse=lse)
@@ -344,7 +347,9 @@ class GpuBench:
         t = buf.cpu().numpy()
         cyc, ns = t[512:512 + 148].astype(np.float64), t[768:768 + 148].astype(np.float64)
         ok = (cyc > 0) & (ns > 0)
-        return float(np.median(cyc[ok] / ns[ok]) * 1e3) if ok.any() else None
+        if not ok.any():
+            return None, None
+        return float(np.median(cyc[ok] / ns[ok]) * 1e3), float(ns[ok].max() * 1e-3)
 
     def e2e(self, w, dw, steps, warmup):
         """Same call with the step's inputs coming from pinned host memory and the
@@ -606,11 +611,12 @@ def main():
         for _ in range(20):
             gb.flush_l2(); dw.decode(out=out, lse=lse)
         torch.cuda.synchronize()
-    in_kernel_mhz = gb.in_kernel_clock(dw, out, lse)
+    in_kernel_mhz, longest_cta_us = gb.in_kernel_clock(dw, out, lse)
     if world > 1:
         dist.barrier()
     clocks = sampler.stop()
     clocks["sm_mhz_in_kernel"] = in_kernel_mhz
+    main_res["roofline"]["longest_cta_main_loop_us"] = longest_cta_us      # context for kernel_ms, not used in frac
     e2e = gb.e2e(w, dw, args.steps, args.warmup)
 
     ms = main_res["ms_per_step"]
