@@ -147,3 +147,21 @@ def test_sparse_all_lists_empty_and_zero_capacity(flags):
                                                     softmax_scale=w.softmax_scale, flags=flags)
         torch.cuda.synchronize()
         assert torch.all(out == 0) and torch.all(torch.isneginf(lse))
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_sparse_random_shapes_and_slices(flags, seed):
+    rng = np.random.default_rng(1000 + seed)
+    B = int(rng.integers(1, 24))
+    H = int(rng.choice([1, 3, 8, 16, 24, 40, 64, 72, 128]))
+    lens = rng.integers(0, 2500, size=B)
+    topk = int(rng.choice([1, 7, 64, 65, 200, 513]))
+    hb = int(rng.integers(0, H)); he = int(rng.integers(hb + 1, H + 1))
+    w = W.make_workload("sparserand", 1000 + seed, lens, H=H, kv_dtype=2, head_begin=hb, head_end=he)
+    sel, cnt = W.select_tokens(1000 + seed, w.seq_lens, topk)
+    cnt[rng.integers(0, B)] = 0                                   # one request with an empty list
+    ref = oracle.mla_decode_sparse(w.q, w.kv_pool, w.block_table, w.seq_lens, sel, cnt, softmax_scale=w.softmax_scale,
+                                   head_begin=hb, head_end=he)
+    out, lse = gpu_sparse(w, sel, cnt, sentinel=3.0, flags=flags)
+    compare_sparse(out, lse, *ref, hb, he, f"seed {seed}: B={B} H={H} slice [{hb},{he}) topk={topk}")
+    assert np.all(out[:, :hb] == 3.0) and np.all(out[:, he:] == 3.0)
