@@ -246,7 +246,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     e = record_timing_event(0, stream);
     if (e == cudaSuccess)
         e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
-                        v.cost_start, v.worker_begin, v.split_list, v.worker_req, v.status, stream);
+                        v.cost_start, v.worker_begin, v.split_list, v.worker_req, v.split_rec, v.status, stream);
     if (e == cudaSuccess) e = record_timing_event(1, stream);
     if (e == cudaSuccess && sparse && !fused_sparse)
         e = launch_sparse_gather(B, sparse->max_selected, sparse->pages_per_request, sparse->pool656, sparse->num_pool_pages,
@@ -258,7 +258,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
         else e = launch_decode_umma(p, *shape, stream);
     }
     if (e == cudaSuccess) e = record_timing_event(2, stream);
-    if (e == cudaSuccess) e = launch_split_combine(p, v.req_wfirst, v.req_wlast, v.split_list, stream);
+    if (e == cudaSuccess) e = launch_split_combine(p, v.req_wfirst, v.req_wlast, v.split_rec, stream);
     if (e == cudaSuccess) e = record_timing_event(3, stream);
     if (e == cudaSuccess && g_timing) g_events_recorded = true;
     }

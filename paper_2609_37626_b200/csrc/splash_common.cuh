@@ -46,6 +46,7 @@ struct PlanView {
     int32_t *worker_begin;  // [W+1] global tile index where each worker starts
     int32_t *split_list;    // [W+1] requests computed in more than one piece (count in status[8])
     int32_t *worker_req;    // [W+1] the request that holds a worker's first tile (what the kernels would bisect for)
+    int4 *split_rec;        // [W+1] per entry of split_list: (request, first worker, last worker, first tile of the request)
     float *partial_lse;     // [2W][h]
     float *partial_out;     // [2W][h][512]
     int32_t num_workers;    // W
@@ -69,6 +70,8 @@ inline __host__ PlanView make_plan_view(void *workspace, int B, int W, int h) {
     v.worker_begin = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
     v.split_list = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
     v.worker_req = reinterpret_cast<int32_t *>(p + off); off += sizeof(int32_t) * (size_t)(W + 1);
+    off = align_up(off, 16);
+    v.split_rec = reinterpret_cast<int4 *>(p + off); off += sizeof(int4) * (size_t)(W + 1);
     off = align_up(off, 256);
     v.partial_lse = reinterpret_cast<float *>(p + off); off += sizeof(float) * (size_t)2 * W * h;
     off = align_up(off, 256);
@@ -206,7 +209,7 @@ void count_launch(int n = 1);
 // kernels' host launchers
 cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
-                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list, int32_t *worker_req,
+                        int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list, int32_t *worker_req, int4 *split_rec,
                         int32_t *status, cudaStream_t stream);
 cudaError_t launch_decode_sparse_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_sparse_gather(int B, int max_sel, int pages_per_request, const void *kv_pool, int num_pool_pages,
@@ -229,7 +232,7 @@ cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_decode_umma_fp8_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_decode_umma_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
-                                 const int32_t *split_list, cudaStream_t stream);
+                                 const int4 *split_rec, cudaStream_t stream);
 cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *part_out,
                              const float *part_lse, float *out, float *lse, cudaStream_t stream);
 cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, void *dst_pool,

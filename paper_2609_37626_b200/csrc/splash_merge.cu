@@ -54,7 +54,7 @@ constexpr int kMaxParts = 512;     // >= number of workers of any launch (one pe
 
 __global__ void __launch_bounds__(kMergeThreads)
 split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirst,
-                     const int32_t *__restrict__ req_wlast, const int32_t *__restrict__ split_list) {
+                     const int32_t *__restrict__ req_wlast, const int4 *__restrict__ split_rec) {
     __shared__ float w_s[kMaxParts];
     __shared__ int slot_s[kMaxParts];
     __shared__ float red_s[kMergeThreads / 32];
@@ -62,22 +62,31 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
     const int k = blockIdx.x % h, entry = blockIdx.x / h;
     const int g = p.head_begin + k;
     grid_dependency_wait();       // the decode kernel's partial slots (and the plan) are read from here on
-    if (entry >= p.status[8]) return;
-    const int i = split_list[entry];
-    const int wf = req_wfirst[i], wl = req_wlast[i];
+    // Three rounds of loads, each independent within itself (the plan's arrays have long left L2 by now, so every
+    // dependent load is a trip to DRAM): the list length and this entry's record; then the worker boundaries and the
+    // LSE of every candidate slot; then the partial outputs.
+    const int n_entries = p.status[8];
+    const int4 rec = split_rec[entry];             // (request, first worker, last worker, first tile); unused past the list's end
+    if (entry >= n_entries) return;
+    const int i = rec.x, wf = rec.y, wl = rec.z;
     float4 *o4 = reinterpret_cast<float4 *>(p.out + (int64_t)i * p.out_stride_request + (int64_t)g * p.out_stride_head);
     float *lse = p.lse + (int64_t)i * p.lse_stride_request + g;
     const int c = threadIdx.x;             // 128 threads x float4 = 512 columns
     // workers between the first and the last may own no tiles at all (their start snapped to
     // the same tile as their successor's): they wrote no slot and get weight 0
-    const int rs = p.tile_start[i];
+    const int rs = rec.w;
     const int nparts = wl - wf + 1;
     float m = -INFINITY;
     for (int j = c; j < nparts; j += kMergeThreads) {
         const int w = wf + j;
-        const bool live = p.worker_begin[w + 1] > p.worker_begin[w];
-        const int slot = 2 * w + (rs <= p.worker_begin[w] ? 0 : 1);
-        const float L = live ? p.partial_lse[(int64_t)slot * h + k] : -INFINITY;
+        // slot 2 w + 1 can only be the first worker's (the request starts inside its run); both candidates' LSEs are
+        // fetched beside the boundaries that decide between them (a slot nobody wrote holds stale bytes: not used)
+        const int wb0 = p.worker_begin[w], wb1 = p.worker_begin[w + 1];
+        const float L0 = p.partial_lse[(int64_t)(2 * w) * h + k];
+        const float L1 = j == 0 ? p.partial_lse[(int64_t)(2 * w + 1) * h + k] : 0.f;
+        const bool live = wb1 > wb0;
+        const int slot = 2 * w + (rs <= wb0 ? 0 : 1);
+        const float L = live ? ((slot & 1) ? L1 : L0) : -INFINITY;
         slot_s[j] = slot;
         w_s[j] = L;
         m = fmaxf(m, L);
@@ -151,7 +160,7 @@ cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *
 }
 
 cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
-                                 const int32_t *split_list, cudaStream_t stream) {
+                                 const int4 *split_rec, cudaStream_t stream) {
     // at most one request straddles each boundary between consecutive workers
     const int max_split = p.num_workers < p.B ? p.num_workers : p.B;
     dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * max_split));
@@ -159,7 +168,7 @@ cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirs
     if (first_use_on_device(configured)) {   // keep the decode kernel's shared-memory carve-out
         cudaFuncSetAttribute(split_combine_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     }
-    cudaError_t e = launch_dependent(split_combine_kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_list);
+    cudaError_t e = launch_dependent(split_combine_kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_rec);
     count_launch();
     return e;
 }

@@ -26,7 +26,7 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
             int32_t *__restrict__ req_lo, int32_t *__restrict__ req_hi,
             int32_t *__restrict__ req_wfirst, int32_t *__restrict__ req_wlast,
             int32_t *cost_start, int32_t *worker_begin, int32_t *__restrict__ split_list, int32_t *__restrict__ worker_req,
-            int32_t *__restrict__ status) {
+            int4 *__restrict__ split_rec, int32_t *__restrict__ status) {
     __shared__ long long warp_tot_tiles[32], warp_tot_cost[32];
     __shared__ long long carry_tiles, carry_cost;
     __shared__ int n_split;
@@ -115,7 +115,11 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
         req_wfirst[i] = wf; req_wlast[i] = wl;
         // requests cut into several pieces are listed for the combine kernel (at most W - 1 of them;
         // the list order varies from run to run, the results do not depend on it)
-        if (wf != wl) split_list[atomicAdd(&n_split, 1)] = i;
+        if (wf != wl) {
+            const int e = atomicAdd(&n_split, 1);
+            split_list[e] = i;
+            split_rec[e] = make_int4(i, wf, wl, rs);      // all the combine kernel needs to know about the request, in one load
+        }
     }
     __syncthreads();
     if (tid == 0) status[8] = n_split;
@@ -130,14 +134,14 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
 cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
-                        int32_t *worker_req, int32_t *status, cudaStream_t stream) {
+                        int32_t *worker_req, int4 *split_rec, int32_t *status, cudaStream_t stream) {
     // same shared-memory carve-out as the decode kernel that follows: no reconfiguration between them
     static bool configured[64] = {};
     if (first_use_on_device(configured)) {
         cudaFuncSetAttribute(plan_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     }
     plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.len_cap, p.seq_lens, kv_begin, kv_end, tile_start,
-                                                req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, split_list, worker_req, status);
+                                                req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, split_list, worker_req, split_rec, status);
     count_launch();
     return cudaGetLastError();
 }
