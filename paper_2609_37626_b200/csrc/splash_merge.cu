@@ -108,7 +108,7 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
     const float inv_z = 1.f / Z;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     int j = 0;
-    // sixteen, then four part loads in flight per thread: one long context cut into a piece per worker is merged by
+    // sixteen, then (up to) four part loads in flight per thread: one long context cut into a piece per worker is merged by
     // one block per head, and the part loop is a chain of round trips to L2 / HBM
     for (; j + 16 <= nparts; j += 16) {
         float4 v[16];
@@ -124,26 +124,20 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
             }
         }
     }
-    for (; j + 4 <= nparts; j += 4) {
+    // the rest four at a time as well, loads first: taken one by one, each part's load would wait for the previous
+    // part's arithmetic, and a request cut into two or three pieces (the usual case) would pay a round trip per piece
+    for (; j < nparts; j += 4) {
         float4 v[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u)
-            v[u] = reinterpret_cast<const float4 *>(p.partial_out + ((int64_t)slot_s[j + u] * h + k) * kDV)[c];
+            if (j + u < nparts) v[u] = reinterpret_cast<const float4 *>(p.partial_out + ((int64_t)slot_s[j + u] * h + k) * kDV)[c];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const float wgt = w_s[j + u] * inv_z;
+            const float wgt = j + u < nparts ? w_s[j + u] * inv_z : 0.f;
             if (wgt != 0.f) {          // a dead worker's slot holds stale bytes
                 acc.x = fmaf(wgt, v[u].x, acc.x); acc.y = fmaf(wgt, v[u].y, acc.y);
                 acc.z = fmaf(wgt, v[u].z, acc.z); acc.w = fmaf(wgt, v[u].w, acc.w);
             }
-        }
-    }
-    for (; j < nparts; ++j) {
-        const float wgt = w_s[j] * inv_z;
-        if (wgt != 0.f) {
-            float4 v = reinterpret_cast<const float4 *>(p.partial_out + ((int64_t)slot_s[j] * h + k) * kDV)[c];
-            acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
-            acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
         }
     }
     o4[c] = acc;
