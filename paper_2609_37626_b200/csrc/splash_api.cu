@@ -242,6 +242,8 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
         p.request_overhead_tiles = pair ? kRequestOverheadTilesFp8Pair : kRequestOverheadTilesFp8;
     else if (pair)
         p.request_overhead_tiles = kRequestOverheadTilesPair;
+    // the bf16 CTA-pair kernel writes its partial outputs as f16
+    p.partial_f16 = (pair && shape->kv_dtype == SPLASH_KV_BF16 && !fused_sparse) ? 1 : 0;
 
     e = record_timing_event(0, stream);
     if (e == cudaSuccess)

@@ -108,6 +108,8 @@ struct DecodeParams {
     const int32_t *worker_req;   // request holding each worker's first tile, from the plan
     int32_t *status;
     float *partial_lse, *partial_out;
+    int32_t partial_f16;       // 1: the partial outputs are f16 (same slot order, rows of 512 halves): half the bytes for the
+                               // decode kernel to write and the combine kernel to read; 11 significant bits of a normalised O
     int32_t len_cap;           // >= 0: seq_lens holds list counts; one outside [0, len_cap] counts as 1 (sparse decode)
     // fused sparse decode: kv_pool holds 656-byte rows, block_table / num_pool_pages describe it, and request i
     // attends over the tokens sel[i * sel_stride + j], j < seq_lens[i], each below ctx_lens[i]

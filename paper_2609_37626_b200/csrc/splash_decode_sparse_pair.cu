@@ -106,11 +106,6 @@ constexpr uint32_t kColO = 0, kColS = 256;
 constexpr uint32_t kF16Formats = ~((1u << 7) | (1u << 10));     // instruction descriptor: A and B formats F16 (0), not BF16 (1)
 constexpr uint32_t kF16NanPair = 0x7E007E00u;
 
-__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
-    uint32_t r;
-    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-    return r;
-}
 __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
     return pack_f16x2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
 }

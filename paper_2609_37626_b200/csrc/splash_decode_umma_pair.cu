@@ -28,6 +28,8 @@
 // issuers wait on live in the leader; the peer's warps arrive on them across the cluster
 // (relaxed arrivals: what they announce is already in place on the peer's SM), and TMA loads
 // of the peer complete on them too.
+#include <cuda_fp16.h>
+
 #include "splash_pair.cuh"
 
 namespace splash {
@@ -430,10 +432,35 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                     const float iA = l_s[hA], iB = l_s[hB];
                     float *rowA = obase + (int64_t)hA * ostride + dv0 + c * 64, *rowB = obase + (int64_t)hB * ostride + dv0 + c * 64;
                     tmem_wait_ld();
+                    if (seg.slot >= 0) {
+                        // a partial piece: f16 rows of the slot (the combine kernel weighs and sums them in fp32)
+                        __half *base16 = reinterpret_cast<__half *>(p.partial_out) + ((int64_t)seg.slot * h + (head0 - p.head_begin)) * kDV;
+                        // A thread holds columns 8 k + 2 i, + 1 (i = lane & 3) of its two rows.  Neighbouring lanes swap one
+                        // packed pair per two k, so that every lane owns four consecutive columns (8 bytes) and a store
+                        // instruction writes whole 32-byte sectors: even lanes columns 16 k' + 2 i .. + 3, odd lanes
+                        // 16 k' + 8 + 2 (i - 1) .. + 3.
+                        const int i4 = lane & 3;
+                        const int col = (i4 & 1) ? 8 + 2 * (i4 - 1) : 2 * i4;
+                        uint2 *hrowA = reinterpret_cast<uint2 *>(base16 + (int64_t)hA * kDV + 256 * n + 128 * g + c * 64 + col);
+                        uint2 *hrowB = reinterpret_cast<uint2 *>(base16 + (int64_t)hB * kDV + 256 * n + 128 * g + c * 64 + col);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        if (hA < nvalid) *reinterpret_cast<float2 *>(rowA + 8 * k) = make_float2(o[4 * k] * iA, o[4 * k + 1] * iA);
-                        if (hB < nvalid) *reinterpret_cast<float2 *>(rowB + 8 * k) = make_float2(o[4 * k + 2] * iB, o[4 * k + 3] * iB);
+                        for (int kk = 0; kk < 4; ++kk) {
+                            const uint32_t a0 = pack_f16x2(o[8 * kk] * iA, o[8 * kk + 1] * iA), a1 = pack_f16x2(o[8 * kk + 4] * iA, o[8 * kk + 5] * iA);
+                            const uint32_t b0 = pack_f16x2(o[8 * kk + 2] * iB, o[8 * kk + 3] * iB), b1 = pack_f16x2(o[8 * kk + 6] * iB, o[8 * kk + 7] * iB);
+                            // even lanes keep the first of their two pairs and get the partner's first; odd lanes the second
+                            const uint32_t ra = __shfl_xor_sync(0xffffffffu, (i4 & 1) ? a0 : a1, 1);
+                            const uint32_t rb = __shfl_xor_sync(0xffffffffu, (i4 & 1) ? b0 : b1, 1);
+                            const uint2 va = (i4 & 1) ? make_uint2(ra, a1) : make_uint2(a0, ra);
+                            const uint2 vb = (i4 & 1) ? make_uint2(rb, b1) : make_uint2(b0, rb);
+                            if (hA < nvalid) hrowA[4 * kk] = va;          // 16 halves on
+                            if (hB < nvalid) hrowB[4 * kk] = vb;
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            if (hA < nvalid) *reinterpret_cast<float2 *>(rowA + 8 * k) = make_float2(o[4 * k] * iA, o[4 * k + 1] * iA);
+                            if (hB < nvalid) *reinterpret_cast<float2 *>(rowB + 8 * k) = make_float2(o[4 * k + 2] * iB, o[4 * k + 3] * iB);
+                        }
                     }
                 }
             }

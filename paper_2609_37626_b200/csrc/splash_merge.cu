@@ -2,6 +2,10 @@
 // the decode kernels' split-KV partial slots.  Both compute, per row,
 //     L = ln sum_j exp(L_j),   O = sum_j exp(L_j - L) O_j,
 // parts with L_j = -inf contributing nothing.  Pure fp32, HBM-bound.
+#include <cuda_fp16.h>
+
+#include <type_traits>
+
 #include "splash_common.cuh"
 
 namespace splash {
@@ -52,6 +56,7 @@ lse_merge_kernel(int num_parts, int64_t rows, int d_v, const float *__restrict__
 // float4 column over the parts with several loads in flight.
 constexpr int kMaxParts = 512;     // >= number of workers of any launch (one per SM at most)
 
+template <bool kF16>      // the partial outputs are f16 (rows of 512 halves) or fp32
 __global__ void __launch_bounds__(kMergeThreads)
 split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirst,
                      const int32_t *__restrict__ req_wlast, const int4 *__restrict__ split_rec) {
@@ -106,37 +111,55 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
     for (int j = 0; j < nparts; ++j) Z += w_s[j];          // same order in every thread: one value of Z
     const float L = m + logf(Z);
     const float inv_z = 1.f / Z;
+    // this thread's four columns of a slot's row as they lie in memory (loads first, conversions with the arithmetic:
+    // a conversion next to its load would make every load wait for the one before it)
+    using Raw = typename std::conditional<kF16, uint2, float4>::type;
+    auto load_part = [&](int slot) -> Raw {
+        const int64_t row = (int64_t)slot * h + k;
+        if constexpr (kF16) return reinterpret_cast<const uint2 *>(reinterpret_cast<const __half *>(p.partial_out) + row * kDV)[c];
+        else return reinterpret_cast<const float4 *>(p.partial_out + row * kDV)[c];
+    };
+    auto widen = [](const Raw &r) -> float4 {
+        if constexpr (kF16) {
+            const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&r.x)), b = __half22float2(*reinterpret_cast<const __half2 *>(&r.y));
+            return make_float4(a.x, a.y, b.x, b.y);
+        } else {
+            return r;
+        }
+    };
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     int j = 0;
     // sixteen, then (up to) four part loads in flight per thread: one long context cut into a piece per worker is merged by
     // one block per head, and the part loop is a chain of round trips to L2 / HBM
     for (; j + 16 <= nparts; j += 16) {
-        float4 v[16];
+        Raw raw[16];
 #pragma unroll
         for (int u = 0; u < 16; ++u)
-            v[u] = reinterpret_cast<const float4 *>(p.partial_out + ((int64_t)slot_s[j + u] * h + k) * kDV)[c];
+            raw[u] = load_part(slot_s[j + u]);
 #pragma unroll
         for (int u = 0; u < 16; ++u) {
             const float wgt = w_s[j + u] * inv_z;
             if (wgt != 0.f) {          // a dead worker's slot holds stale bytes
-                acc.x = fmaf(wgt, v[u].x, acc.x); acc.y = fmaf(wgt, v[u].y, acc.y);
-                acc.z = fmaf(wgt, v[u].z, acc.z); acc.w = fmaf(wgt, v[u].w, acc.w);
+                const float4 v = widen(raw[u]);
+                acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
+                acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
             }
         }
     }
     // the rest four at a time as well, loads first: taken one by one, each part's load would wait for the previous
     // part's arithmetic, and a request cut into two or three pieces (the usual case) would pay a round trip per piece
     for (; j < nparts; j += 4) {
-        float4 v[4];
+        Raw raw[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u)
-            if (j + u < nparts) v[u] = reinterpret_cast<const float4 *>(p.partial_out + ((int64_t)slot_s[j + u] * h + k) * kDV)[c];
+            if (j + u < nparts) raw[u] = load_part(slot_s[j + u]);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const float wgt = j + u < nparts ? w_s[j + u] * inv_z : 0.f;
             if (wgt != 0.f) {          // a dead worker's slot holds stale bytes
-                acc.x = fmaf(wgt, v[u].x, acc.x); acc.y = fmaf(wgt, v[u].y, acc.y);
-                acc.z = fmaf(wgt, v[u].z, acc.z); acc.w = fmaf(wgt, v[u].w, acc.w);
+                const float4 v = widen(raw[u]);
+                acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
+                acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
             }
         }
     }
@@ -160,9 +183,12 @@ cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirs
     dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * max_split));
     static bool configured[64] = {};
     if (first_use_on_device(configured)) {   // keep the decode kernel's shared-memory carve-out
-        cudaFuncSetAttribute(split_combine_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(split_combine_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(split_combine_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     }
-    cudaError_t e = launch_dependent(split_combine_kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_rec);
+    cudaError_t e = p.partial_f16
+        ? launch_dependent(split_combine_kernel<true>, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_rec)
+        : launch_dependent(split_combine_kernel<false>, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_rec);
     count_launch();
     return e;
 }
