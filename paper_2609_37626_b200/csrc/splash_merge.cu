@@ -56,8 +56,12 @@ lse_merge_kernel(int num_parts, int64_t rows, int d_v, const float *__restrict__
 // float4 column over the parts with several loads in flight.
 constexpr int kMaxParts = 512;     // >= number of workers of any launch (one per SM at most)
 
-template <bool kF16>      // the partial outputs are f16 (rows of 512 halves) or fp32
-__global__ void __launch_bounds__(kMergeThreads)
+// kF16: the partial outputs are f16 (rows of 512 halves) or fp32.  kLean: a variant for launches whose requests are cut
+// into few pieces each (many requests per worker): at most four part loads in flight, few enough registers for twelve
+// resident blocks per SM instead of eight -- its blocks are short chains of round trips to DRAM, and what bounds
+// the kernel is how many of them an SM holds at a time.
+template <bool kF16, bool kLean>
+__global__ void __launch_bounds__(kMergeThreads, kLean ? 12 : 8)
 split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirst,
                      const int32_t *__restrict__ req_wlast, const int4 *__restrict__ split_rec) {
     __shared__ float w_s[kMaxParts];
@@ -131,7 +135,7 @@ split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirs
     int j = 0;
     // sixteen, then (up to) four part loads in flight per thread: one long context cut into a piece per worker is merged by
     // one block per head, and the part loop is a chain of round trips to L2 / HBM
-    for (; j + 16 <= nparts; j += 16) {
+    for (; !kLean && j + 16 <= nparts; j += 16) {
         Raw raw[16];
 #pragma unroll
         for (int u = 0; u < 16; ++u)
@@ -183,12 +187,16 @@ cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirs
     dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * max_split));
     static bool configured[64] = {};
     if (first_use_on_device(configured)) {   // keep the decode kernel's shared-memory carve-out
-        cudaFuncSetAttribute(split_combine_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-        cudaFuncSetAttribute(split_combine_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(split_combine_kernel<false, false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(split_combine_kernel<true, false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(split_combine_kernel<false, true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        cudaFuncSetAttribute(split_combine_kernel<true, true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     }
-    cudaError_t e = p.partial_f16
-        ? launch_dependent(split_combine_kernel<true>, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_rec)
-        : launch_dependent(split_combine_kernel<false>, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_rec);
+    // many requests per worker: every request is cut into a few pieces at most
+    const bool lean = (int64_t)p.B * 4 >= p.num_workers;
+    auto kernel = p.partial_f16 ? (lean ? split_combine_kernel<true, true> : split_combine_kernel<true, false>)
+                                : (lean ? split_combine_kernel<false, true> : split_combine_kernel<false, false>);
+    cudaError_t e = launch_dependent(kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_rec);
     count_launch();
     return e;
 }
