@@ -57,11 +57,11 @@ lse_merge_kernel(int num_parts, int64_t rows, int d_v, const float *__restrict__
 constexpr int kMaxParts = 512;     // >= number of workers of any launch (one per SM at most)
 
 // kF16: the partial outputs are f16 (rows of 512 halves) or fp32.  kLean: a variant for launches whose requests are cut
-// into few pieces each (many requests per worker): at most four part loads in flight, few enough registers for twelve
+// into few pieces each (many requests per worker): at most four part loads in flight, few enough registers for sixteen
 // resident blocks per SM instead of eight -- its blocks are short chains of round trips to DRAM, and what bounds
 // the kernel is how many of them an SM holds at a time.
 template <bool kF16, bool kLean>
-__global__ void __launch_bounds__(kMergeThreads, kLean ? 12 : 8)
+__global__ void __launch_bounds__(kMergeThreads, kLean ? 16 : 8)
 split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirst,
                      const int32_t *__restrict__ req_wlast, const int4 *__restrict__ split_rec) {
     __shared__ float w_s[kMaxParts];
