@@ -332,9 +332,8 @@ class GpuBench:
 
     def in_kernel_clock(self, dw, out, lse):
         """SM clock seen by the decode kernel itself: cycles / nanoseconds of its main loop, per CTA, from the
-        library's diagnostic trace (written by the CTA-pair kernels; None for the others), and the longest CTA's
-        main loop in microseconds (after an L2 flush, like the timed steps): what the kernel executes, without the
-        launch and completion latency that the CUDA-event duration of a single launch includes."""
+        library's diagnostic trace (written by the CTA-pair kernels; None for the others), and the longest span in
+        microseconds of the thread that writes the trace (the producer warp's: it ends a few tiles before its CTA)."""
         torch, binding = self.torch, self.binding
         buf = torch.zeros(64 * 8 + 512, dtype=torch.int64, device=self.device)
         self.flush_l2()
@@ -616,7 +615,6 @@ def main():
         dist.barrier()
     clocks = sampler.stop()
     clocks["sm_mhz_in_kernel"] = in_kernel_mhz
-    main_res["roofline"]["longest_cta_main_loop_us"] = longest_cta_us      # context for kernel_ms, not used in frac
     e2e = gb.e2e(w, dw, args.steps, args.warmup)
 
     ms = main_res["ms_per_step"]
