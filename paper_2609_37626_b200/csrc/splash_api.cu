@@ -260,7 +260,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
         else e = launch_decode_umma(p, *shape, stream);
     }
     if (e == cudaSuccess) e = record_timing_event(2, stream);
-    if (e == cudaSuccess) e = launch_split_combine(p, v.req_wfirst, v.req_wlast, v.split_rec, stream);
+    if (e == cudaSuccess) e = launch_split_combine(p, v.split_rec, stream);
     if (e == cudaSuccess) e = record_timing_event(3, stream);
     if (e == cudaSuccess && g_timing) g_events_recorded = true;
     }

@@ -233,8 +233,7 @@ cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &sh
 cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_decode_umma_fp8_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_decode_umma_pair(const DecodeParams &p, cudaStream_t stream);
-cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
-                                 const int4 *split_rec, cudaStream_t stream);
+cudaError_t launch_split_combine(const DecodeParams &p, const int4 *split_rec, cudaStream_t stream);
 cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *part_out,
                              const float *part_lse, float *out, float *lse, cudaStream_t stream);
 cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, void *dst_pool,

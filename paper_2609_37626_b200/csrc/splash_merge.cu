@@ -62,8 +62,7 @@ constexpr int kMaxParts = 512;     // >= number of workers of any launch (one pe
 // the kernel is how many of them an SM holds at a time.
 template <bool kF16, bool kLean>
 __global__ void __launch_bounds__(kMergeThreads, kLean ? 16 : 8)
-split_combine_kernel(const DecodeParams p, const int32_t *__restrict__ req_wfirst,
-                     const int32_t *__restrict__ req_wlast, const int4 *__restrict__ split_rec) {
+split_combine_kernel(const DecodeParams p, const int4 *__restrict__ split_rec) {
     __shared__ float w_s[kMaxParts];
     __shared__ int slot_s[kMaxParts];
     __shared__ float red_s[kMergeThreads / 32];
@@ -180,8 +179,7 @@ cudaError_t launch_lse_merge(int num_parts, int64_t rows, int d_v, const float *
     return cudaGetLastError();
 }
 
-cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirst, const int32_t *req_wlast,
-                                 const int4 *split_rec, cudaStream_t stream) {
+cudaError_t launch_split_combine(const DecodeParams &p, const int4 *split_rec, cudaStream_t stream) {
     // at most one request straddles each boundary between consecutive workers
     const int max_split = p.num_workers < p.B ? p.num_workers : p.B;
     dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * max_split));
@@ -196,7 +194,7 @@ cudaError_t launch_split_combine(const DecodeParams &p, const int32_t *req_wfirs
     const bool lean = (int64_t)p.B * 4 >= p.num_workers;
     auto kernel = p.partial_f16 ? (lean ? split_combine_kernel<true, true> : split_combine_kernel<true, false>)
                                 : (lean ? split_combine_kernel<false, true> : split_combine_kernel<false, false>);
-    cudaError_t e = launch_dependent(kernel, grid, dim3(kMergeThreads), 0, stream, p, req_wfirst, req_wlast, split_rec);
+    cudaError_t e = launch_dependent(kernel, grid, dim3(kMergeThreads), 0, stream, p, split_rec);
     count_launch();
     return e;
 }
