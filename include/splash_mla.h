@@ -28,6 +28,12 @@
  *     error of the calling thread.
  *   - Empty work (no requests, an empty head slice, n = 0 pages) is a successful
  *     no-op: idle ranks are legal (App. E: ranks that own no rows still take part).
+ *   - Stream capture: every call may be recorded into a CUDA graph (Sec. 4.1: the
+ *     steps after a switch replay graphs captured at startup; App. G "Graph capture").  Nothing in a call depends on values the host cannot see at
+ *     capture time -- lengths, ranges, token lists and page tables are read on the
+ *     device, the split-KV plan is computed there -- so a replay follows buffers that
+ *     changed in place.  Make the first call of each kind on a device outside the
+ *     capture (it sets kernel attributes), and leave kernel timing off while capturing.
  */
 #ifndef SPLASH_MLA_H_
 #define SPLASH_MLA_H_
