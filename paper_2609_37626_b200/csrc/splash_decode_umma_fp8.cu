@@ -400,11 +400,8 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     lA = fmaf(a0, t2.y, lA); lA = fmaf(a1, t2.w, lA);
                     lB = fmaf(b0, t2.y, lB); lB = fmaf(b1, t2.w, lB);
                     // hi = the e4m3 value nearest to the weight, lo = what is left, kept as e5m2
-                    phiA[k] = to_e4m3x2(a0, a1);
-                    phiB[k] = to_e4m3x2(b0, b1);
-                    const float2 ba = from_e4m3x2(phiA[k]), bb = from_e4m3x2(phiB[k]);
-                    ploA[k] = to_e5m2x2(a0 - ba.x, a1 - ba.y);
-                    ploB[k] = to_e5m2x2(b0 - bb.x, b1 - bb.y);
+                    split_e4m3_e5m2_x2(a0, a1, phiA[k], ploA[k]);
+                    split_e4m3_e5m2_x2(b0, b1, phiB[k], ploB[k]);
                 }
                 const bool rescale = named_bar_or<1, kNumSoftmaxThreads>(grew);
                 // the P.V that read this P buffer (two tiles back) must be done; a rescale of O^T also

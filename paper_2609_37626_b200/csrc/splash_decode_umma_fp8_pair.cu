@@ -495,10 +495,11 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                         u[e] = fast_exp2(sv[4 * j4 + e] + off);
                         l = fmaf(u[e], rts[e], l);
                     }
-                    const uint16_t h01 = to_e4m3x2(u[0], u[1]), h23 = to_e4m3x2(u[2], u[3]);
-                    const float2 b01 = from_e4m3x2(h01), b23 = from_e4m3x2(h23);
+                    uint16_t h01, h23, r01, r23;
+                    split_e4m3_e5m2_x2(u[0], u[1], h01, r01);
+                    split_e4m3_e5m2_x2(u[2], u[3], h23, r23);
                     phi[j4] = (uint32_t)h01 | ((uint32_t)h23 << 16);
-                    plo[j4] = (uint32_t)to_e5m2x2(u[0] - b01.x, u[1] - b01.y) | ((uint32_t)to_e5m2x2(u[2] - b23.x, u[3] - b23.y) << 16);
+                    plo[j4] = (uint32_t)r01 | ((uint32_t)r23 << 16);
                 }
                 const bool rescale = named_bar_or<1, kSoftmaxWarps * 32>(grew);
                 // P.V of the supertile that last used this P buffer (two back) must be done; a rescale
