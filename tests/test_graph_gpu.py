@@ -105,3 +105,37 @@ def test_lse_merge_replays_from_a_cuda_graph():
     graph.replay()
     torch.cuda.synchronize()
     assert torch.equal(out, ref_out) and torch.equal(lse, ref_lse)
+
+
+def test_page_migrate_replays_from_a_cuda_graph():
+    """A captured migration, replayed on a fresh copy of the pool and table, moves the same pages and rewrites the
+    same table entries as the oracle."""
+    import torch
+    import oracle
+    from paper_2609_37626_b200 import binding
+    lens = [10, 64, 3000, 129, 700]
+    n_used = sum((s + 63) // 64 for s in lens)
+    w = W.make_workload("miggraph", 4300, lens, H=16, kv_dtype=1, extra_pool_pages=n_used)
+    n_src = w.num_pool_pages - n_used
+    src_ids, dst_ids = W.migration_plan(78, np.unique(w.block_table[w.block_table >= 0]), n_used, 0.3)
+    ref_pool, ref_table, ref_sc = w.kv_pool.copy(), w.block_table.copy(), w.kv_scales.copy()
+    oracle.kv_page_migrate(ref_pool[:n_src], ref_pool[n_src:], src_ids, dst_ids, ref_table, src_scales=ref_sc[:n_src],
+                           dst_scales=ref_sc[n_src:], dst_id_base=n_src)
+    dw = binding.DeviceWorkload(w)
+    pool0, table0, sc0 = dw.kv_pool.clone(), dw.block_table.clone(), dw.kv_scales.clone()
+    src_d, dst_d = torch.from_numpy(src_ids).cuda(), torch.from_numpy(dst_ids).cuda()
+    call = lambda: binding.splash_kv_page_migrate(
+        dw.kv_pool[:n_src], dw.kv_pool[n_src:], src_d, dst_d, dw.block_table, src_scales=dw.kv_scales[:n_src],
+        dst_scales=dw.kv_scales[n_src:], src_id_base=0, dst_id_base=n_src, max_page_id=w.num_pool_pages)
+    call()                                           # eager once: workspace allocation and first-use set-up
+    torch.cuda.synchronize()
+    dw.kv_pool.copy_(pool0); dw.block_table.copy_(table0); dw.kv_scales.copy_(sc0)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        call()
+    dw.kv_pool.copy_(pool0); dw.block_table.copy_(table0); dw.kv_scales.copy_(sc0)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(dw.kv_pool.view(torch.uint8).cpu().numpy().reshape(-1), ref_pool.view(np.uint8).reshape(-1))
+    assert np.array_equal(dw.block_table.cpu().numpy(), ref_table)
+    assert np.array_equal(dw.kv_scales.cpu().numpy().view(np.uint32), ref_sc.view(np.uint32))
