@@ -2,14 +2,21 @@
 """Benchmark of the MLA decode hot path (one attention layer-call over a paged latent
 KV cache) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--impl reference]
 
 A step is one ``splash_mla_decode`` call (work plan, page gather, QK^T, online softmax,
 P.V, epilogue, split-KV combine) over one synthetic batch.  The default workload is the
-DP-attention request slice (64 requests, contexts U[1024, 8192], 128 heads, bf16 KV);
-``--workload`` picks another configuration, and the default run also reports the other
-configurations (head slice at 32K, CP ranges + LSE merge, fp8 rollout + page migration)
-under ``"workloads"``.  Rank 0 prints ONE JSON line.
+RL-rollout batch (512 requests, lognormal contexts, 128 heads, e4m3 KV with one scale per
+token): the largest configuration that one GPU holds and the one in the precision of the
+paper's runs.  ``--workload`` picks another configuration, and the default run also reports
+the other configurations (DP-attention slice, head slice at 32K, CP ranges + LSE merge, page
+migration) under ``"workloads"``, with the roofline fractions of the two target
+configurations repeated under ``"targets"``.  Rank 0 prints ONE JSON line.
+
+``--gpus N`` with N > 1 starts N ranks itself (one process per GPU under
+``torch.distributed.run`` on 127.0.0.1) unless it already runs inside such a launch
+(``WORLD_SIZE`` set); every rank decodes its own request slice, no collective on the data
+path, and rank 0 prints the line with ``n_gpus: N``.
 
 Timing: CUDA events on the launching stream around every step, L2 flushed between
 steps by writing a 256 MiB buffer outside the timed intervals, and every workload's KV
@@ -17,6 +24,13 @@ is larger than the 126 MB L2 anyway.  ``value`` is requests decoded per second f
 layer-call with inputs resident in HBM; ``e2e`` repeats it with the step's inputs
 (q, block table, lengths) copied from pinned host memory and out / lse copied back
 inside the timed region (the KV pool itself is serving state that lives in HBM).
+
+``roofline`` follows the decode kernel's own duration against the MEASURED peaks of this
+pool (copy bandwidth, bf16 GEMM burst rate; for e4m3 KV the tensor peak is taken at the bf16
+rate because every operand choice that meets the tolerance costs the pipe what bf16 costs).
+``roofline.nominal`` repeats the arithmetic for the WHOLE CALL (plan + decode + combine)
+against the nominal peaks of the part -- 8 TB/s, 2.25 PFLOP/s bf16, 4.5 PFLOP/s fp8 for the
+kernels that issue 8-bit MMAs -- which is the stricter reading of the target.
 """
 from __future__ import annotations
 
@@ -39,6 +53,8 @@ METRIC = "mla_decode_tokens_per_s_per_gpu"
 UNIT = "tokens/s"
 WORKLOAD_IDS = {"c1": 1, "c2": 2, "c3": 3, "c4": 4, "c5": 5}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0, "fp8_tflops": 4500.0}
+DTYPES = {0: "bf16", 1: "e4m3 KV with an fp32 scale per token, bf16 q, 8-bit MMAs in two terms, fp32 accumulate"}
 
 
 def load_peaks():
@@ -212,13 +228,23 @@ class GpuBench:
             kernel = "decode_umma_fp8_pair_kernel" if fp8 else "decode_umma_pair_kernel"
         else:
             kernel = "decode_umma_fp8_kernel" if fp8 else "decode_umma_kernel<%d>" % (16 if hs <= 16 else 32 if hs <= 32 else 64)
+        # the stricter reading: the whole call against the nominal peaks of the part (fp8 MMA rate for e4m3 KV)
+        nom_tensor = NOMINAL_PEAKS["fp8_tflops"] if fp8 else NOMINAL_PEAKS["bf16_tflops"]
+        tn_hbm, tn_tensor = alg_bytes / (NOMINAL_PEAKS["hbm_gbs"] * 1e9), alg_flops / (nom_tensor * 1e12)
+        tn = max(tn_hbm, tn_tensor)
+        p50 = float(np.median(ms))
+        roof["frac_whole_call"] = max(t_hbm, t_tensor) * 1e3 / p50
+        roof["nominal"] = {"hbm_gbs": NOMINAL_PEAKS["hbm_gbs"], "tensor_tflops": nom_tensor,
+                           "bound": "hbm" if tn_hbm >= tn_tensor else "tensor", "roofline_ms": tn * 1e3,
+                           "frac_kernel": tn * 1e3 / dec_ms, "frac_whole_call": tn * 1e3 / p50}
         roof.update({"kernel": kernel, "kernel_ms": dec_ms, "peak_source": peaks["source"],
                      "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
                      "roofline_ms": max(t_hbm, t_tensor) * 1e3,
                      "achieved_gbs": alg_bytes / (dec_ms * 1e-3) / 1e9,
                      "achieved_tflops": alg_flops / (dec_ms * 1e-3) / 1e12,
                      "plan_ms": float(kt[:, 0].mean()), "combine_ms": float(kt[:, 2].mean()),
-                     "note": "fp8 KV: tensor peak taken at the bf16 rate" if fp8 else None})
+                     "note": ("e4m3 KV: 'frac' takes the tensor peak at the bf16 rate (two 8-bit terms per operand); "
+                              "'nominal' takes the fp8 rate, under which this workload is HBM-bound") if fp8 else None})
         res = {"ms_per_step": float(ms.mean()), "ms_p50": float(np.median(ms)), "ms_p95": float(np.percentile(ms, 95)),
                "tokens_per_s": w.B / (ms.mean() * 1e-3), "tokens_per_s_78_layers": w.B / (ms.mean() * 1e-3) / 78,
                "launches_per_step": launches, "roofline": roof,
@@ -551,18 +577,54 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+def free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def launch_ranks(n: int, argv) -> int:
+    """Start n ranks of this script on this node (one process per GPU) and wait for them."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+class StubBench:
+    """Stands in for the GPU side when the launcher and the rank plumbing are tested on CPU (``--stub-step``): a step
+    is a short host computation, nothing here is a measurement."""
+
+    def decode_workload(self, w, steps, warmup, *_):
+        times = []
+        for k in range(warmup + steps):
+            t0 = time.perf_counter()
+            float(np.square(w.seq_lens.astype(np.float64)).sum())
+            if k >= warmup:
+                times.append((time.perf_counter() - t0) * 1e3 + 1e-3)
+        ms = np.array(times)
+        return ({"ms_per_step": float(ms.mean()), "ms_p50": float(np.median(ms)), "ms_p95": float(np.percentile(ms, 95)),
+                 "launches_per_step": 0, "roofline": None}, None, None, None)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", choices=sorted(WORKLOAD_IDS), default="c2")
+    ap.add_argument("--workload", choices=sorted(WORKLOAD_IDS), default="c5")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--only-main", action="store_true", help="skip the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sparse-only", action="store_true", help="print only the sparse-decode workload's numbers")
+    ap.add_argument("--stub-step", action="store_true",
+                    help="CPU test of the launcher and the rank plumbing: gloo, a host stand-in for the step, no measurement")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    # N > 1 outside a torch.distributed launch: start the ranks here
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -573,49 +635,68 @@ def main():
 
     import torch
     import torch.distributed as dist
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    device = f"cuda:{local_rank}"
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(device))
+    stub = args.stub_step
+    if stub:
+        device = "cpu"
+        if world > 1:
+            dist.init_process_group("gloo")
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the decode path has no CPU fallback")
+        torch.cuda.set_device(local_rank)
+        device = f"cuda:{local_rank}"
+        if world > 1:
+            dist.init_process_group("nccl", device_id=torch.device(device))
     peaks = load_peaks()
     traffic = load_traffic()
-    gb = GpuBench(device)
+    gb = StubBench() if stub else GpuBench(device)
 
     # every rank owns its own batch (request slices are independent: weak scaling, no collective)
     idx = WORKLOAD_IDS[args.workload]
     t_gen = time.time()
-    w = W.config(idx) if world == 1 else W.config(idx)
-    if world > 1:
+    if stub:
+        w = W.config(1)
+    elif idx == 5:
+        w = W.config(5, extra_pool_factor=0.3 if world == 1 else 0.0)      # with the second pool of the page migration
+    else:
+        w = W.config(idx)
+    if world > 1 and not stub:
         w = W.make_workload(w.name, W.BASE_SEED + idx + 100 * rank, w.seq_lens, H=w.H, head_begin=w.head_begin,
                             head_end=w.head_end, kv_dtype=w.kv_dtype)
     gen_s = time.time() - t_gen
 
     if args.sparse_only:
-        print(json.dumps({"sparse_top2048": gb.sparse_workload(w.seq_lens, w.H, args.steps, args.warmup, peaks)}))
+        w2 = W.config(2)
+        print(json.dumps({"sparse_top2048": gb.sparse_workload(w2.seq_lens, w2.H, args.steps, args.warmup, peaks)}))
         return
 
     sampler = ClockSampler(local_rank)
     if world > 1:
         dist.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    main_res, dw, out, lse = gb.decode_workload(w, args.steps, args.warmup, peaks, traffic, args.workload)
-    torch.cuda.synchronize()
-    # the timed region lasts a few milliseconds, less than one nvidia-smi sampling period: keep the same step
-    # running for about a second so that the sampler sees the clocks under this load
-    t_end = time.time() + 1.0
-    while time.time() < t_end:
-        for _ in range(20):
-            gb.flush_l2(); dw.decode(out=out, lse=lse)
+    if not stub:
         torch.cuda.synchronize()
-    in_kernel_mhz, longest_cta_us = gb.in_kernel_clock(dw, out, lse)
-    if world > 1:
-        dist.barrier()
-    clocks = sampler.stop()
-    clocks["sm_mhz_in_kernel"] = in_kernel_mhz
-    e2e = gb.e2e(w, dw, args.steps, args.warmup)
+        sampler.start()
+    main_res, dw, out, lse = gb.decode_workload(w, args.steps, args.warmup, peaks, traffic, args.workload)
+    if stub:
+        if world > 1:
+            dist.barrier()
+        clocks = {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["stub step: no GPU"]}
+        e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "ms_per_step": main_res["ms_per_step"]}
+    else:
+        torch.cuda.synchronize()
+        # the timed region lasts a few milliseconds, less than one nvidia-smi sampling period: keep the same step
+        # running for about a second so that the sampler sees the clocks under this load
+        t_end = time.time() + 1.0
+        while time.time() < t_end:
+            for _ in range(20):
+                gb.flush_l2(); dw.decode(out=out, lse=lse)
+            torch.cuda.synchronize()
+        in_kernel_mhz, longest_cta_us = gb.in_kernel_clock(dw, out, lse)
+        if world > 1:
+            dist.barrier()
+        clocks = sampler.stop()
+        clocks["sm_mhz_in_kernel"] = in_kernel_mhz
+        e2e = gb.e2e(w, dw, args.steps, args.warmup)
 
     ms = main_res["ms_per_step"]
     e2e_ms = e2e["ms_per_step"]
@@ -624,72 +705,91 @@ def main():
     e2e_value = sharding.weak_scaling_value(w.B, world, e2e_ms)
 
     extra = {}
+    targets = {}
     cpu = None
-    if rank == 0 and world == 1:
+    if main_res["roofline"] is not None and args.workload in ("c3", "c5"):
+        targets[args.workload] = main_res["roofline"]["frac"]
+    if rank == 0 and world == 1 and not stub:
         if not args.no_cpu_baseline:
             cpu, _ = time_oracle(w)
         if not args.only_main:
+            steps2 = max(5, args.steps // 2)
+            if idx == 5:
+                try:
+                    extra["c5"] = {"page_migrate": gb.migrate_workload(w, dw, steps2, args.warmup, peaks),
+                                   "migrate_under_decode": gb.overlap_workload(w, dw, steps2, args.warmup)}
+                except Exception as exc:  # report, do not hide
+                    extra["c5"] = {"error": repr(exc)}
             del dw, out, lse
             torch.cuda.empty_cache()
-            for name in ("c3", "c4", "c5"):
+            w2 = w if idx == 2 else None
+            for name in ("c3", "c2", "c4", "c5"):
                 if name == args.workload:
                     continue
                 try:
-                    if name == "c5":
-                        wx = W.config(5, extra_pool_factor=0.3)
-                    else:
-                        wx = W.config(WORKLOAD_IDS[name])
+                    wx = W.config(5, extra_pool_factor=0.3) if name == "c5" else W.config(WORKLOAD_IDS[name])
+                    if name == "c2":
+                        w2 = wx
                     r, dwx, ox, lx = gb.decode_workload(wx, args.steps, args.warmup, peaks, traffic, name)
+                    if name in ("c3", "c5"):
+                        targets[name] = r["roofline"]["frac"]
                     if name == "c4":
                         del dwx
-                        r["cp"] = gb.cp_workload(wx, max(5, args.steps // 2), args.warmup)
+                        r["cp"] = gb.cp_workload(wx, steps2, args.warmup)
                     if name == "c5":
-                        r["page_migrate"] = gb.migrate_workload(wx, dwx, max(5, args.steps // 2), args.warmup, peaks)
-                        r["migrate_under_decode"] = gb.overlap_workload(wx, dwx, max(5, args.steps // 2), args.warmup)
+                        r["page_migrate"] = gb.migrate_workload(wx, dwx, steps2, args.warmup, peaks)
+                        r["migrate_under_decode"] = gb.overlap_workload(wx, dwx, steps2, args.warmup)
                     extra[name] = r
-                    del wx, ox, lx
+                    del ox, lx
                     dwx = None
+                    if name != "c2":
+                        del wx
                     torch.cuda.empty_cache()
                 except Exception as exc:  # report, do not hide
                     extra[name] = {"error": repr(exc)}
             try:
-                extra["dop_layout_changes"] = gb.dop_workload(max(5, args.steps // 2), args.warmup, peaks)
+                extra["dop_layout_changes"] = gb.dop_workload(steps2, args.warmup, peaks)
                 torch.cuda.empty_cache()
             except Exception as exc:
                 extra["dop_layout_changes"] = {"error": repr(exc)}
-            # sparse decode over the main workload's context lengths, 2048 listed tokens per request
-            try:
-                extra["sparse_top2048"] = gb.sparse_workload(w.seq_lens, w.H, max(5, args.steps // 2), args.warmup, peaks)
-                torch.cuda.empty_cache()
-            except Exception as exc:
-                extra["sparse_top2048"] = {"error": repr(exc)}
-            # several causal query rows per request on the main workload's cache (multi-token decode steps)
-            for R in (2, 4):
+            if w2 is not None:
+                # sparse decode over the DP-attention workload's context lengths, 2048 listed tokens per request
                 try:
-                    extra["%s_rows%d" % (args.workload, R)] = gb.rows_workload(w, R, max(5, args.steps // 2), args.warmup, peaks)
+                    extra["sparse_top2048"] = gb.sparse_workload(w2.seq_lens, w2.H, steps2, args.warmup, peaks)
                     torch.cuda.empty_cache()
                 except Exception as exc:
-                    extra["%s_rows%d" % (args.workload, R)] = {"error": repr(exc)}
+                    extra["sparse_top2048"] = {"error": repr(exc)}
+                # several causal query rows per request on that workload's cache (multi-token decode steps)
+                for R in (2, 4):
+                    try:
+                        extra["c2_rows%d" % R] = gb.rows_workload(w2, R, steps2, args.warmup, peaks)
+                        torch.cuda.empty_cache()
+                    except Exception as exc:
+                        extra["c2_rows%d" % R] = {"error": repr(exc)}
 
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-            "data": "synthetic",
-            "config": {"workload": W.CONFIG_NAMES[idx - 1], "requests_per_gpu": w.B, "heads": w.head_end - w.head_begin,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": DTYPES[w.kv_dtype], "data": "synthetic",
+            "config": {"workload": W.CONFIG_NAMES[idx - 1] if not stub else "stub", "requests_per_gpu": w.B,
+                       "heads": w.head_end - w.head_begin,
                        "tokens_per_gpu": w.total_tokens(), "kv_dtype": "bf16" if w.kv_dtype == 0 else "e4m3+token scale",
                        "page_size": 64, "l2": "256 MiB flush write between steps; KV larger than L2",
                        "parallelism": f"dp{world} (request slices, no collective)"},
             "ms_p50": main_res["ms_p50"], "ms_p95": main_res["ms_p95"],
             "tokens_per_s_78_layers": value / 78,
             "roofline": main_res["roofline"],
+            "targets": targets,
             "cpu_baseline": cpu,
             "e2e": {k: (e2e_value if k == "value" else v) for k, v in e2e.items()},
             "gpu_launches": int(main_res["launches_per_step"]) * args.steps,
             "clocks": clocks,
-            "workloads": extra,
             "input_generation_s": gen_s,
+            "workloads": extra,
         }
+        if stub:
+            line["stub"] = True
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -150,11 +150,12 @@ typedef struct splash_mla_shape {
  *                256-byte aligned; its contents on entry do not matter and two
  *                calls that may overlap on the device need different workspaces
  *
- * Slots of a referenced page at or beyond seq_lens[i] and pages the table does not
- * reference are never used: they may hold NaN / Inf patterns.  Slots below
- * seq_lens[i] of a page that intersects R_i must hold finite values even if they lie
- * outside R_i.  Results are bit-reproducible for a fixed call (same shape,
- * lengths and ranges).
+ * Only the rows of tokens in R_i enter the result.  Every other byte of the cache --
+ * slots of a referenced page outside R_i (below or beyond seq_lens[i]), pages the table
+ * does not reference, the scales of such slots -- may hold anything, NaN / Inf patterns
+ * included: a rank of position-sharded CP owns only its own tokens of a boundary page
+ * (App. E).  Results are bit-reproducible for a fixed call (same shape, lengths and
+ * ranges).
  */
 SPLASH_API int splash_mla_decode(const splash_mla_shape *shape,
                       const void *q, const void *kv_pool, const float *kv_scales,

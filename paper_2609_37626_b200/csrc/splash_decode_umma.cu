@@ -202,12 +202,12 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                     entry = idx < seg.tile_end ? table[first_page + idx] : 0;
                 }
                 const int page = __shfl_sync(0xffffffffu, entry, rel & 31);
+                const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
+                const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
                 if (lane == 0) {
-                    const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
                     ok = mbar_wait(ctx, bar(kBarKvEmpty + stage), ph ^ 1, kBarKvEmpty + stage);
                     mark(kv_it, 0);
-                    if (ok) {
-                        const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
+                    if (ok && !g.both) {
                         mbar_expect_tx(bar(kBarKvFull + stage), kStageBytes);
                         const uint32_t dst = sbase + L::kOffKv + stage * kStageBytes;
                         // one box = the whole page: (64 elements, 64 tokens, 9 chunks) -> [chunk][token][128 B]
@@ -216,6 +216,15 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (ok && g.both) {
+                    // a range cut at both ends inside this page: the warp writes the box itself, zeros outside the range
+                    const uint8_t *src = page >= 0 && page < p.num_pool_pages
+                        ? static_cast<const uint8_t *>(p.kv_pool) + (size_t)page * (kPage * kDQK * 2) : nullptr;
+                    fill_rows_by_hand<128>(smem + L::kOffKv + stage * kStageBytes, kSlabBytes, kPage, src, g.tok0, g.a, g.b, 0, 0, kChunks, lane);
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar(kBarKvFull + stage));
+                }
                 ++kv_it;
             }
             ++seg_it;

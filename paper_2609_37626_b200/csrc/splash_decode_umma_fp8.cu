@@ -135,15 +135,15 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     entry = idx < seg.tile_end ? table[first_page + idx] : 0;
                 }
                 const int page = __shfl_sync(0xffffffffu, entry, rel & 31);
+                const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
+                const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
+                // a page id outside the pool reads as zeros through the tensor map; its
+                // scale page is not fetched (plain addresses are not bounds-checked)
+                const bool in_pool = page >= 0 && page < p.num_pool_pages;
                 if (lane == 0) {
-                    const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
                     ok = mbar_wait(ctx, bar(kBarKvEmpty + stage), ph ^ 1, kBarKvEmpty + stage);
                     mark(kv_it, 0);
-                    if (ok) {
-                        const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
-                        // a page id outside the pool reads as zeros through the tensor map; its
-                        // scale page is not fetched (plain addresses are not bounds-checked)
-                        const bool in_pool = page >= 0 && page < p.num_pool_pages;
+                    if (ok && !g.both) {
                         mbar_expect_tx(bar(kBarKvFull + stage), kStageBytes + (in_pool ? kScaleBytes : 0u));
                         tma_load_4d(sbase + kOffKv + stage * kStageBytes, &tmap_kv, bar(kBarKvFull + stage), 0, g.tok0, 0, page);
                         if (in_pool)
@@ -153,6 +153,23 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (ok && g.both) {
+                    // a range cut at both ends inside this page: the warp writes the box itself, zeros outside the
+                    // range (the scale page still comes by bulk copy; the softmax warps mask the scales themselves)
+                    const uint8_t *src = in_pool ? static_cast<const uint8_t *>(p.kv_pool) + (size_t)page * (kPage * kDQK) : nullptr;
+                    fill_rows_by_hand<64>(smem + kOffKv + stage * kStageBytes, kSlab, kPage, src, g.tok0, g.a, g.b, 0, 0, 9, lane);
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (in_pool) {
+                            mbar_expect_tx(bar(kBarKvFull + stage), kScaleBytes);
+                            bulk_load(sbase + kOffScale + stage * kScaleBytes, p.kv_scales + (int64_t)page * kPage,
+                                      kScaleBytes, bar(kBarKvFull + stage));
+                        } else {
+                            mbar_arrive(bar(kBarKvFull + stage));
+                        }
+                    }
+                }
                 ++kv_it;
             }
         }

@@ -163,7 +163,7 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
         g.a = tile_geom(seg.lo, seg.hi, (first_page + ta) * kPage);
         g.has_b = tb < seg.tile_end;
         if (g.has_b) g.b = tile_geom(seg.lo, seg.hi, (first_page + tb) * kPage);
-        else { g.b.tok0 = 0; g.b.r_lo = 0; g.b.r_hi = 0; }
+        else { g.b.tok0 = 0; g.b.r_lo = 0; g.b.r_hi = 0; g.b.a = 0; g.b.b = 0; g.b.both = false; }
         return g;
     };
 
@@ -181,19 +181,23 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
             for (int s = 0; ok && s < nsuper; ++s, ++st_it) {
                 const PairGeom g = pair_geom(s);
                 const int ta = seg.tile_begin + 2 * s;
+                const uint32_t stage = st_it % kStages, ph = (st_it / kStages) & 1;
+                const uint32_t k0 = sbase + kOffK + stage * kPageBytes;
+                // the page this warp fetches: its CTA's own for QK^T, the other CTA's for the P.V chunks.  A tile cut at
+                // both ends inside its page is written by hand instead (zeros outside the range); only a request whose
+                // whole range lies inside one page has such a tile, and it is page A.
+                const TileGeom &tg = (rank == 0) != is_v ? g.a : g.b;
                 int page_a = 0, page_b = 0;
                 if (lane == 0) {
                     page_a = table[first_page + ta];
                     page_b = g.has_b ? table[first_page + ta + 1] : p.num_pool_pages;   // a page past the pool reads as zeros
-                    const uint32_t stage = st_it % kStages, ph = (st_it / kStages) & 1;
-                    const uint32_t k0 = sbase + kOffK + stage * kPageBytes;
                     if (!is_v) {
                         ok = mbar_wait(ctx, bar(kBarStageEmpty + stage), ph ^ 1, kBarStageEmpty + stage);
                         if (ok) {
                             // the leader's barrier expects the pages of both CTAs
                             if (rank == 0) mbar_expect_tx(bar(kBarKFull + stage), 2 * kPageBytes);
-                            tma_load_4d_pair(k0, &tmap_page, leader_bar(kBarKFull + stage), 0, rank == 0 ? g.a.tok0 : g.b.tok0, 0,
-                                             rank == 0 ? page_a : page_b);
+                            if (!tg.both)
+                                tma_load_4d_pair(k0, &tmap_page, leader_bar(kBarKFull + stage), 0, tg.tok0, 0, rank == 0 ? page_a : page_b);
                             // scale pages of both pages, for this CTA's softmax warps
                             const bool in_a = page_a >= 0 && page_a < p.num_pool_pages;
                             const bool in_b = g.has_b && page_b >= 0 && page_b < p.num_pool_pages;
@@ -215,14 +219,32 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                         if (ok) {
                             if (rank == 0) mbar_expect_tx(bar(kBarVFull + stage), 2 * kPeerBytes);
                             // peer page chunks 4n + 2 rank, + 1 -> slots 4n + 2 (1 - rank), + 1
+                            if (!tg.both) {
 #pragma unroll
-                            for (int n = 0; n < 2; ++n)
-                                tma_load_4d_pair(k0 + (4 * n + 2 * (1 - (int)rank)) * kSlab, &tmap_pair, leader_bar(kBarVFull + stage), 0,
-                                                 rank == 0 ? g.b.tok0 : g.a.tok0, 4 * n + 2 * (int)rank, rank == 0 ? page_b : page_a);
+                                for (int n = 0; n < 2; ++n)
+                                    tma_load_4d_pair(k0 + (4 * n + 2 * (1 - (int)rank)) * kSlab, &tmap_pair, leader_bar(kBarVFull + stage), 0,
+                                                     tg.tok0, 4 * n + 2 * (int)rank, rank == 0 ? page_b : page_a);
+                            }
                         }
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (ok && tg.both) {
+                    const int page = __shfl_sync(0xffffffffu, (rank == 0) != is_v ? page_a : page_b, 0);
+                    const uint8_t *src = page >= 0 && page < p.num_pool_pages
+                        ? static_cast<const uint8_t *>(p.kv_pool) + (size_t)page * (kPage * kDQK) : nullptr;
+                    uint8_t *slabs = smem + kOffK + stage * kPageBytes;
+                    if (!is_v) {
+                        fill_rows_by_hand<64>(slabs, kSlab, kPage, src, tg.tok0, tg.a, tg.b, 0, 0, 9, lane);
+                    } else {
+                        for (int n = 0; n < 2; ++n)
+                            fill_rows_by_hand<64>(slabs, kSlab, kPage, src, tg.tok0, tg.a, tg.b, 4 * n + 2 * (int)rank,
+                                                  4 * n + 2 * (1 - (int)rank), 2, lane);
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_complete_tx_cluster(leader_bar(is_v ? kBarVFull + stage : kBarKFull + stage), is_v ? kPeerBytes : kPageBytes);
+                }
             }
         }
     } else if (warp >= kWarpQk && warp < kWarpQk + kQkWarps && rank == 0) {

@@ -169,17 +169,18 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
             const int first_page = seg.lo / kPage;
             const int32_t *table = p.block_table + (int64_t)seg.request * p.table_stride;
             for (int tile = seg.tile_begin; ok && tile < seg.tile_end; ++tile, ++kv_it) {
+                const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
+                const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
+                const uint32_t k0 = sbase + kOffK + stage * kStageBytes;
+                int page = 0;
                 if (lane == 0) {
-                    const int page = table[first_page + tile];
-                    const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
-                    const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
-                    const uint32_t k0 = sbase + kOffK + stage * kStageBytes;
+                    page = table[first_page + tile];
                     if (!is_v) {
                         ok = mbar_wait(ctx, bar(kBarStageEmpty + stage), ph ^ 1, kBarStageEmpty + stage);
                         if (ok) {
                             // the leader's barrier expects the halves of both CTAs
                             if (rank == 0) mbar_expect_tx(bar(kBarKFull + stage), 2 * kStageBytes);
-                            tma_load_4d_pair(k0, &tmap_half, leader_bar(kBarKFull + stage), 0, g.tok0 + kHalf * (int)rank, 0, page);
+                            if (!g.both) tma_load_4d_pair(k0, &tmap_half, leader_bar(kBarKFull + stage), 0, g.tok0 + kHalf * (int)rank, 0, page);
                             // A stage is held from its load until P.V has read it, about three tiles, so the
                             // load of tile t + 3 starts only when the issuers are about to need it: have its
                             // half of the page in L2 by then.
@@ -197,14 +198,34 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                         if (ok) {
                             if (rank == 0) mbar_expect_tx(bar(kBarVFull + stage), 2 * kPeerBytes);
                             // peer half-page chunks 4n + 2 rank, + 1 -> slots 4n + 2 (1 - rank), + 1
+                            if (!g.both) {
 #pragma unroll
-                            for (int n = 0; n < 2; ++n)
-                                tma_load_4d_pair(k0 + (4 * n + 2 * (1 - (int)rank)) * kSlab, &tmap_peer, leader_bar(kBarVFull + stage), 0,
-                                                 g.tok0 + kHalf * (1 - (int)rank), 4 * n + 2 * (int)rank, page);
+                                for (int n = 0; n < 2; ++n)
+                                    tma_load_4d_pair(k0 + (4 * n + 2 * (1 - (int)rank)) * kSlab, &tmap_peer, leader_bar(kBarVFull + stage), 0,
+                                                     g.tok0 + kHalf * (1 - (int)rank), 4 * n + 2 * (int)rank, page);
+                            }
                         }
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (ok && g.both) {
+                    // a range cut at both ends inside this page: the warp writes what the box(es) would have
+                    // delivered, zeros outside the range, and reports the bytes on the leader's barrier
+                    page = __shfl_sync(0xffffffffu, page, 0);
+                    const uint8_t *src = page >= 0 && page < p.num_pool_pages
+                        ? static_cast<const uint8_t *>(p.kv_pool) + (size_t)page * (kPage * kDQK * 2) : nullptr;
+                    uint8_t *slabs = smem + kOffK + stage * kStageBytes;
+                    if (!is_v) {
+                        fill_rows_by_hand<128>(slabs, kSlab, kHalf, src, g.tok0 + kHalf * (int)rank, g.a, g.b, 0, 0, 9, lane);
+                    } else {
+                        for (int n = 0; n < 2; ++n)
+                            fill_rows_by_hand<128>(slabs, kSlab, kHalf, src, g.tok0 + kHalf * (1 - (int)rank), g.a, g.b,
+                                                   4 * n + 2 * (int)rank, 4 * n + 2 * (1 - (int)rank), 2, lane);
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_complete_tx_cluster(leader_bar(is_v ? kBarVFull + stage : kBarKFull + stage), is_v ? kPeerBytes : kStageBytes);
+                }
             }
             ++seg_it;
         }

@@ -57,6 +57,13 @@ static __device__ __noinline__ bool mbar_wait_cluster(const Ctx &ctx, uint32_t b
         }
     }
 }
+// Reports `bytes` as delivered on a barrier given by its cluster address (this CTA's or the leader's): what a TMA load
+// does on completion, for a tile that a warp wrote by hand.  The cluster-scope fence orders the warp's writes (made
+// visible to the tensor core by fence.proxy.async, gathered by __syncwarp) before the report.
+__device__ __forceinline__ void mbar_complete_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("fence.acq_rel.cluster;" ::: "memory");
+    asm volatile("mbarrier.complete_tx.relaxed.cluster.shared::cluster.b64 [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
 // TMA load whose completion bytes go to a barrier of the pair's leader CTA
 __device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int c0, int c1,
                                                  int c2, int c3) {

@@ -244,15 +244,42 @@ __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_mn_major, 
 }
 
 // Valid rows of a tile after the token shift: page-relative tokens [a, b) land in rows
-// [r_lo, r_hi) of the 64-row box when the box starts at token tok0.
-struct TileGeom { int tok0, r_lo, r_hi; };
+// [r_lo, r_hi) of the 64-row box when the box starts at token tok0.  The shift moves ONE cut
+// end out of the page, where the TMA unit fills zeros; a range cut at both ends inside one
+// page (`both`) cannot be loaded that way -- the rows of tokens [0, a) would arrive with
+// whatever the cache holds there, and 0 x NaN is NaN inside P.V -- so the producers copy such a
+// tile by hand (fill_rows_by_hand) and write zeros for every row outside the range.
+struct TileGeom { int tok0, r_lo, r_hi, a, b; bool both; };
 __device__ __forceinline__ TileGeom tile_geom(int lo, int hi, int t0) {
     int a = max(lo, t0) - t0;
     int b = min(hi, t0 + kPage) - t0;
     TileGeom g;
+    g.a = a; g.b = b; g.both = a > 0 && b < kPage;
     if (b < kPage) { g.tok0 = b - kPage; g.r_lo = kPage - b + a; g.r_hi = kPage; }   // end cut: align the end to the box end
     else { g.tok0 = a; g.r_lo = 0; g.r_hi = kPage - a; }                              // front cut (or none)
     return g;
+}
+
+// What one TMA box would have delivered, written by the 32 lanes of a warp with plain loads and stores: rows
+// [0, nrows) of `nchunks` chunk slabs, row r holding token tok_first + r of the page when that token lies in [a, b) and
+// zeros otherwise.  kChunkBytes = 128: 16-bit elements in the 128-byte swizzle; 64: 8-bit elements in the 64-byte
+// swizzle (a cache row is nine chunks either way).  `slabs` is the stage's first slab (1024-byte aligned), chunk
+// src_chunk0 + c of the row goes to slab dst_slot0 + c; page == nullptr (an id outside the pool) gives zeros.  The caller
+// follows up with fence.proxy.async and its barrier arrival.  Only the rare tile cut at both ends takes this path.
+template <int kChunkBytes>
+__device__ __forceinline__ void fill_rows_by_hand(uint8_t *slabs, uint32_t slab_bytes, int nrows, const uint8_t *page,
+                                                  int tok_first, int a, int b, int src_chunk0, int dst_slot0, int nchunks, int lane) {
+    constexpr int kPieces = kChunkBytes / 16;
+    const int total = nrows * nchunks * kPieces;
+    for (int idx = lane; idx < total; idx += 32) {
+        const int j = idx % kPieces, r = (idx / kPieces) % nrows, c = idx / (kPieces * nrows);
+        const int t = tok_first + r;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (page != nullptr && t >= a && t < b)
+            v = __ldg(reinterpret_cast<const uint4 *>(page + (size_t)t * (9 * kChunkBytes) + (size_t)(src_chunk0 + c) * kChunkBytes + j * 16));
+        const int sw = kChunkBytes == 128 ? (r & 7) : ((r >> 1) & 3);
+        *reinterpret_cast<uint4 *>(slabs + (size_t)(dst_slot0 + c) * slab_bytes + (size_t)r * kChunkBytes + ((j ^ sw) << 4)) = v;
+    }
 }
 
 // ---------------------------------------------------------------- host side

@@ -311,6 +311,27 @@ def make_workload(name: str, seed: int, seq_lens, H: int, *, head_begin: int = 0
                     head_end=H if head_end is None else head_end, used_pages=used)
 
 
+def poison_outside_ranges(w: Workload, kv_begin, kv_end) -> None:
+    """Overwrite, in place, every cache row of every request that lies outside its KV range
+    [kv_begin[i], kv_end[i]) with NaN / Inf patterns (for e4m3 also its scale): the cache of a
+    position-sharded rank holds only the tokens it owns (App. E), the other slots of a boundary
+    page hold whatever was there.  Requests must not share pages."""
+    for i in range(w.B):
+        s = int(w.seq_lens[i])
+        lo, hi = max(0, int(kv_begin[i])), min(s, int(kv_end[i]))
+        hi = max(hi, lo)
+        for t in list(range(0, lo)) + list(range(hi, s)):
+            page, slot = int(w.block_table[i, t // PAGE_SIZE]), t % PAGE_SIZE
+            if w.kv_dtype == 0:
+                w.kv_pool[page, slot, :] = BF16_NAN if (t & 1) else BF16_INF
+                w.kv_pool[page, slot, 5::7] = 0xFF80                     # -Inf
+            elif w.kv_dtype == 1:
+                w.kv_pool[page, slot, :] = E4M3_NAN if (t & 1) else 0xFF  # both NaN codes of e4m3fn
+                w.kv_scales[page, slot] = np.nan if (t % 3) else np.inf
+            else:
+                w.kv_pool[page, slot, :] = 0xFF
+
+
 def rollout_lengths(seed: int, n: int = 512) -> np.ndarray:
     """Lognormal context lengths: median 2048, sigma 1.2, clipped to [16, 131072]."""
     rng = np.random.Generator(np.random.PCG64(seed))
