@@ -57,7 +57,9 @@ typedef enum splash_status {
     SPLASH_UNSUPPORTED = -2,        /* dims / page size / dtype / head count not built */
     SPLASH_UNSUPPORTED_DEVICE = -3, /* the current device is not compute capability 10.x */
     SPLASH_CUDA_ERROR = -4,         /* a CUDA runtime / driver call failed */
-    SPLASH_DEVICE_TIMEOUT = -5      /* (status word only) a bounded device wait gave up */
+    SPLASH_DEVICE_TIMEOUT = -5,     /* (status word only) a bounded device wait gave up */
+    SPLASH_BAD_PAGE_ID = -6         /* (status word only, SPLASH_FLAG_VALIDATE) a block-table entry the call needs
+                                       names no page of the pool */
 } splash_status;
 
 enum {
@@ -80,7 +82,13 @@ enum {
     /* splash_mla_decode_sparse only: one kernel that gathers, dequantises and multiplies (CTA pairs) instead of
      * the gather kernel followed by the dense kernels.  Every listed row crosses HBM once; tile, query rows and
      * P are f16 in that kernel (values must lie within f16's range).  Correct, not yet the faster of the two. */
-    SPLASH_FLAG_SPARSE_FUSED = 4u
+    SPLASH_FLAG_SPARSE_FUSED = 4u,
+    /* splash_mla_decode only: validation mode.  One more (small) kernel between the plan and the decode kernel checks
+     * every block-table entry of a page that intersects a request's range against [0, num_pool_pages) and records
+     * the first bad one in the workspace status word: splash_workspace_status() then returns SPLASH_BAD_PAGE_ID with
+     * detail = (request, page index within the request, the id found).  With or without the flag an id outside the
+     * pool is never dereferenced (the page reads as zeros); the flag makes the mistake visible. */
+    SPLASH_FLAG_VALIDATE = 8u
 };
 
 /*
@@ -355,9 +363,11 @@ SPLASH_API int splash_debug_set_trace(void *device_buffer);
 
 /*
  * Read the device status word at the head of a decode workspace after the caller
- * has synchronised the stream: SPLASH_OK, or SPLASH_DEVICE_TIMEOUT if a bounded wait
- * inside a kernel gave up (the results of that call are then invalid).  Performs a
- * blocking 16-byte device-to-host copy; not for the hot path.
+ * has synchronised the stream: SPLASH_OK, SPLASH_DEVICE_TIMEOUT if a bounded wait
+ * inside a kernel gave up (the results of that call are then invalid), or, for a call
+ * made with SPLASH_FLAG_VALIDATE, SPLASH_BAD_PAGE_ID.  The first event of a call wins
+ * and stays until the next call on that workspace.  Performs a blocking 16-byte
+ * device-to-host copy; not for the hot path.
  */
 SPLASH_API int splash_workspace_status(const void *workspace, int32_t *detail /* host, [3], may be NULL */);
 

@@ -6,8 +6,8 @@
  * check and from the benchmark's CPU-baseline leg.  Nothing here is blocked,
  * fused or reordered beyond the definition:
  *
- *   - the KV cache holds ONE latent row per token, shared by every query head
- *     (the paper's premise: "one head-shared latent history per token", Sec. 1);
+ *   - the KV cache holds ONE latent row per token, with no head axis: all query
+ *     heads read the same history (the premise of the paper's layouts, Sec. 1);
  *   - absorbed MLA: a query row and a cache row are d_q = d_c + d_r wide and the
  *     value read back per head is d_z = d_c wide (Sec. 3, "Cost" paragraph of
  *     DOP, Eq. "dop-traffic"); with the DeepSeek-V3 dimensions of App. A,

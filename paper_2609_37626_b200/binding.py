@@ -20,6 +20,7 @@ SPLASH_UNSUPPORTED = -2
 SPLASH_UNSUPPORTED_DEVICE = -3
 SPLASH_CUDA_ERROR = -4
 SPLASH_DEVICE_TIMEOUT = -5
+SPLASH_BAD_PAGE_ID = -6
 SPLASH_KV_BF16 = 0
 SPLASH_KV_E4M3_TOKEN_SCALE = 1
 SPLASH_KV_E4M3_BLOCK_SCALE_BF16_ROPE = 2
@@ -27,6 +28,7 @@ SPLASH_SPARSE_ROW_BYTES = 656
 SPLASH_FLAG_SIMT = 1
 SPLASH_FLAG_NO_PAIR = 2
 SPLASH_FLAG_SPARSE_FUSED = 4
+SPLASH_FLAG_VALIDATE = 8
 
 D_QK, D_V, PAGE_SIZE = 576, 512, 64
 

@@ -32,11 +32,14 @@ struct DeviceInfo {
     bool ok = false;
 };
 
-// Properties of the current device (cached per device index).
+// Properties of the current device (cached per device index, under a lock: host threads may make their first calls
+// at the same time).
 bool current_device_info(DeviceInfo &info) {
     static DeviceInfo cache[64];
+    static std::mutex mu;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { set_error("cudaGetDevice failed"); return false; }
+    std::lock_guard<std::mutex> lock(mu);
     if (dev >= 0 && dev < 64 && cache[dev].ok) { info = cache[dev]; return true; }
     DeviceInfo d;
     d.device = dev;
@@ -248,8 +251,11 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     e = record_timing_event(0, stream);
     if (e == cudaSuccess)
         e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
-                        v.cost_start, v.worker_begin, v.split_list, v.worker_req, v.split_rec, v.status, stream);
+                        v.cost_start, v.worker_begin, v.split_list, v.worker_req, v.split_rec, v.status, vb == vbegin, stream);
     if (e == cudaSuccess) e = record_timing_event(1, stream);
+    // validation mode: the table entries the call will use, checked on the device before the decode kernel runs
+    if (e == cudaSuccess && (shape->flags & SPLASH_FLAG_VALIDATE) && !sparse && vb == vbegin)
+        e = launch_validate_pages(p, v.req_lo, v.req_hi, stream);
     if (e == cudaSuccess && sparse && !fused_sparse)
         e = launch_sparse_gather(B, sparse->max_selected, sparse->pages_per_request, sparse->pool656, sparse->num_pool_pages,
                                  sparse->block_table, sparse->table_stride, sparse->ctx_lens, sparse->sel, sparse->sel_stride,
@@ -446,6 +452,7 @@ const char *splash_status_string(int status) {
         case SPLASH_UNSUPPORTED_DEVICE: return "unsupported device";
         case SPLASH_CUDA_ERROR: return "CUDA error";
         case SPLASH_DEVICE_TIMEOUT: return "device wait timed out";
+        case SPLASH_BAD_PAGE_ID: return "block-table entry outside the pool";
         default: return "unknown status";
     }
 }

@@ -6,6 +6,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <mutex>
+
 #include "../../include/splash_mla.h"
 
 namespace splash {
@@ -195,14 +197,23 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-// Function attributes are per device: true the first time a launcher runs on the current device.
-inline bool first_use_on_device(bool (&seen)[64]) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
-    if (seen[dev]) return false;
-    seen[dev] = true;
-    return true;
-}
+// Per-device one-time set-up of a launcher (function attributes are per device).  The set-up runs under a lock and a
+// device counts as done only once it has succeeded, so a second host thread whose first call on a device comes at the
+// same time waits for the attribute to be in place instead of launching without it.
+struct DeviceOnce {
+    std::mutex mu;
+    bool done[64] = {};
+    template <typename F>
+    cudaError_t run(F &&setup) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return setup();
+        std::lock_guard<std::mutex> lock(mu);
+        if (done[dev]) return cudaSuccess;
+        const cudaError_t e = setup();
+        if (e == cudaSuccess) done[dev] = true;
+        return e;
+    }
+};
 
 // ---- host helpers (splash_api.cu) -----------------------------------------
 void set_error(const char *fmt, ...);
@@ -212,7 +223,8 @@ void count_launch(int n = 1);
 cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list, int32_t *worker_req, int4 *split_rec,
-                        int32_t *status, cudaStream_t stream);
+                        int32_t *status, bool reset_status, cudaStream_t stream);
+cudaError_t launch_validate_pages(const DecodeParams &p, const int32_t *req_lo, const int32_t *req_hi, cudaStream_t stream);
 cudaError_t launch_decode_sparse_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_sparse_gather(int B, int max_sel, int pages_per_request, const void *kv_pool, int num_pool_pages,
                                  const int32_t *block_table, int64_t table_stride, const int32_t *seq_lens,

@@ -71,7 +71,10 @@ decode_simt_kernel(const DecodeParams p) {
             const int t0 = page_idx * kPage;
             const int a = max(seg.lo, t0) - t0;
             const int b = min(seg.hi, t0 + kPage) - t0;
-            const int64_t page = p.block_table[(int64_t)seg.request * p.table_stride + page_idx];
+            int64_t page = p.block_table[(int64_t)seg.request * p.table_stride + page_idx];
+            // an id outside the pool is never dereferenced: the page reads as zeros, like a box outside a tensor map
+            const bool in_pool = page >= 0 && page < p.num_pool_pages;
+            if (!in_pool) page = 0;
 
             // ---- stage rows [a, b) of the page ------------------------------------
             if (KV_DTYPE == 0) {
@@ -80,7 +83,7 @@ decode_simt_kernel(const DecodeParams p) {
                 constexpr int kVecPerRow = kDQK / 8;   // 72
                 for (int idx = a * kVecPerRow + tid; idx < b * kVecPerRow; idx += kSimtThreads) {
                     int r = idx / kVecPerRow, c = idx % kVecPerRow;
-                    *reinterpret_cast<uint4 *>(&sm.rows[r][c * 8]) = src[idx];
+                    *reinterpret_cast<uint4 *>(&sm.rows[r][c * 8]) = in_pool ? src[idx] : make_uint4(0u, 0u, 0u, 0u);
                 }
             } else {
                 const uint4 *src = reinterpret_cast<const uint4 *>(
@@ -88,7 +91,7 @@ decode_simt_kernel(const DecodeParams p) {
                 constexpr int kVecPerRow = kDQK / 16;  // 36
                 for (int idx = a * kVecPerRow + tid; idx < b * kVecPerRow; idx += kSimtThreads) {
                     int r = idx / kVecPerRow, c = idx % kVecPerRow;
-                    uint4 v = src[idx];
+                    uint4 v = in_pool ? src[idx] : make_uint4(0u, 0u, 0u, 0u);
                     const __nv_fp8x2_storage_t *pairs = reinterpret_cast<const __nv_fp8x2_storage_t *>(&v);
                     uint32_t o[8];
 #pragma unroll
@@ -100,7 +103,7 @@ decode_simt_kernel(const DecodeParams p) {
                     dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                     dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
                 }
-                if (tid >= a && tid < b) sm.tok_scale[tid] = p.kv_scales[page * kPage + tid];
+                if (tid >= a && tid < b) sm.tok_scale[tid] = in_pool ? p.kv_scales[page * kPage + tid] : 1.0f;
             }
             __syncthreads();
 

@@ -710,12 +710,9 @@ cudaError_t launch_decode_sparse_pair(const DecodeParams &p, cudaStream_t stream
                      (uint64_t)p.B, (uint64_t)p.q_stride_head * 2, 128,
                      (uint64_t)(p.B > 1 ? p.q_stride_request : p.q_stride_head * p.H) * 2, (uint32_t)kN, 9))
         return cudaErrorInvalidValue;
-    static bool configured[64] = {};
-    cudaError_t e = cudaSuccess;
-    if (first_use_on_device(configured)) {
-        e = cudaFuncSetAttribute(decode_sparse_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return e;
-    }
+    static DeviceOnce once;
+    cudaError_t e = once.run([&] { return cudaFuncSetAttribute(decode_sparse_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes); });
+    if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.num_workers * 2)); cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;

@@ -623,12 +623,9 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
 template <int N>
 cudaError_t launch_n(const DecodeParams &p, const CUtensorMap &mkv, const CUtensorMap &mq, cudaStream_t stream) {
     const int smem = (int)Layout<N>::kBytes;
-    static bool configured[64] = {};      // (per device attribute; set again if it was lost to another device)
-    cudaError_t e = cudaSuccess;
-    if (first_use_on_device(configured)) {
-        e = cudaFuncSetAttribute(decode_umma_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-    }
+    static DeviceOnce once;
+    cudaError_t e = once.run([&] { return cudaFuncSetAttribute(decode_umma_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); });
+    if (e != cudaSuccess) return e;
     e = launch_dependent(decode_umma_kernel<N>, dim3((unsigned)(p.num_workers * p.num_groups)), dim3(kThreads), (size_t)smem,
                          stream, p, mkv, mq);
     count_launch();

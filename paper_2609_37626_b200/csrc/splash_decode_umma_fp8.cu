@@ -143,6 +143,10 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 if (lane == 0) {
                     ok = mbar_wait(ctx, bar(kBarKvEmpty + stage), ph ^ 1, kBarKvEmpty + stage);
                     mark(kv_it, 0);
+                    if (ok && !in_pool) {      // the page reads as zeros; give its tokens the scale 1
+                        float *sc1 = reinterpret_cast<float *>(smem + kOffScale + stage * kScaleBytes);
+                        for (int t = 0; t < kPage; ++t) sc1[t] = 1.0f;
+                    }
                     if (ok && !g.both) {
                         mbar_expect_tx(bar(kBarKvFull + stage), kStageBytes + (in_pool ? kScaleBytes : 0u));
                         tma_load_4d(sbase + kOffKv + stage * kStageBytes, &tmap_kv, bar(kBarKvFull + stage), 0, g.tok0, 0, page);
@@ -546,12 +550,9 @@ cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream) {
                      (uint64_t)(p.num_pool_pages > 0 ? p.num_pool_pages : 1), (uint64_t)kDQK, 64,
                      (uint64_t)kPage * kDQK, 64))
         return cudaErrorInvalidValue;
-    static bool configured[64] = {};
-    cudaError_t e = cudaSuccess;
-    if (first_use_on_device(configured)) {
-        e = cudaFuncSetAttribute(decode_umma_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return e;
-    }
+    static DeviceOnce once;
+    cudaError_t e = once.run([&] { return cudaFuncSetAttribute(decode_umma_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes); });
+    if (e != cudaSuccess) return e;
     e = launch_dependent(decode_umma_fp8_kernel, dim3((unsigned)(p.num_workers * p.num_groups)), dim3(kThreads),
                          (size_t)kSmemBytes, stream, p, mkv);
     count_launch();

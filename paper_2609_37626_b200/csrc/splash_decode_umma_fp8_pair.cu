@@ -201,6 +201,13 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                             // scale pages of both pages, for this CTA's softmax warps
                             const bool in_a = page_a >= 0 && page_a < p.num_pool_pages;
                             const bool in_b = g.has_b && page_b >= 0 && page_b < p.num_pool_pages;
+                            if (!in_a || (g.has_b && !in_b)) {     // a page outside the pool reads as zeros; give its tokens the scale 1
+                                float *sc1 = reinterpret_cast<float *>(smem + kOffScale + stage * 2 * kScaleBytes);
+                                for (int t = 0; t < kPage; ++t) {
+                                    if (!in_a) sc1[t] = 1.0f;
+                                    if (g.has_b && !in_b) sc1[kPage + t] = 1.0f;
+                                }
+                            }
                             mbar_expect_tx(bar(kBarScFull + stage), (in_a ? kScaleBytes : 0u) + (in_b ? kScaleBytes : 0u));
                             const uint32_t sdst = sbase + kOffScale + stage * 2 * kScaleBytes;
                             if (in_a) bulk_load(sdst, p.kv_scales + (int64_t)page_a * kPage, kScaleBytes, bar(kBarScFull + stage));
@@ -664,12 +671,9 @@ cudaError_t launch_decode_umma_fp8_pair(const DecodeParams &p, cudaStream_t stre
     const uint64_t h = (uint64_t)(p.head_end - p.head_begin);
     if (!make_store_map_3d(&mpart, p.partial_out, kDV, h, (uint64_t)2 * p.num_workers, (uint64_t)kDV * 4, h * kDV * 4, 32))
         return cudaErrorInvalidValue;
-    static bool configured[64] = {};
-    cudaError_t e = cudaSuccess;
-    if (first_use_on_device(configured)) {
-        e = cudaFuncSetAttribute(decode_umma_fp8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-        if (e != cudaSuccess) return e;
-    }
+    static DeviceOnce once;
+    cudaError_t e = once.run([&] { return cudaFuncSetAttribute(decode_umma_fp8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes); });
+    if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.num_workers * 2)); cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;

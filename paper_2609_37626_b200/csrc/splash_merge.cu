@@ -183,13 +183,14 @@ cudaError_t launch_split_combine(const DecodeParams &p, const int4 *split_rec, c
     // at most one request straddles each boundary between consecutive workers
     const int max_split = p.num_workers < p.B ? p.num_workers : p.B;
     dim3 grid((unsigned)((int64_t)(p.head_end - p.head_begin) * max_split));
-    static bool configured[64] = {};
-    if (first_use_on_device(configured)) {   // keep the decode kernel's shared-memory carve-out
+    static DeviceOnce once;
+    once.run([&] {   // keep the decode kernel's shared-memory carve-out (a preference: a failure is not an error)
         cudaFuncSetAttribute(split_combine_kernel<false, false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         cudaFuncSetAttribute(split_combine_kernel<true, false>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         cudaFuncSetAttribute(split_combine_kernel<false, true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         cudaFuncSetAttribute(split_combine_kernel<true, true>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    }
+        return cudaSuccess;
+    });
     // many requests per worker: every request is cut into a few pieces at most
     const bool lean = (int64_t)p.B * 4 >= p.num_workers;
     auto kernel = p.partial_f16 ? (lean ? split_combine_kernel<true, true> : split_combine_kernel<true, false>)

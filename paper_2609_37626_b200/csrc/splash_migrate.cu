@@ -72,12 +72,16 @@ static __device__ __align__(256) int32_t g_static_remap[kStaticMigrateMaxPageId]
 // Device address of g_static_remap on the current device.  In host code the array's
 // name only stands for the symbol; the address a kernel can use comes from
 // cudaGetSymbolAddress, looked up once per device with that device current.
+// The per-device cache is filled under a lock, so that two host threads making their first call on a device at the
+// same time do not race on it (both would store the same address, but the lock costs nothing next to a launch).
 cudaError_t static_remap_address(int32_t **ptr) {
     static int32_t *cache[64] = {nullptr};
+    static std::mutex mu;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
     if (cache[dev] == nullptr) {
         void *addr = nullptr;
         e = cudaGetSymbolAddress(&addr, g_static_remap);

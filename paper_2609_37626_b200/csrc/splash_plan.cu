@@ -21,7 +21,7 @@ constexpr int kPlanSmemRequests = 4096;
 constexpr int kPlanSmemWorkers = 512;
 
 __global__ void __launch_bounds__(kPlanThreads)
-plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ kv_begin,
+plan_kernel(int B, int W, int overhead, int len_cap, int reset_status, const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ kv_begin,
             const int32_t *__restrict__ kv_end, int32_t *tile_start,
             int32_t *__restrict__ req_lo, int32_t *__restrict__ req_hi,
             int32_t *__restrict__ req_wfirst, int32_t *__restrict__ req_wlast,
@@ -38,7 +38,9 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
     if (staged) { tile_start = s_tile; cost_start = s_cost; worker_begin = s_wbeg; }
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     grid_launch_dependents();     // the decode kernel may start its set-up now; it waits for this grid before reading the plan
-    if (tid < 16) status[tid] = 0;
+    // the status block is cleared by the first pass of a call only: a later pass (more than 128 (head, row) pairs)
+    // must not wipe what an earlier one recorded
+    if (reset_status && tid < 16) status[tid] = 0;
     if (tid == 0) { carry_tiles = 0; carry_cost = 0; tile_start[0] = 0; cost_start[0] = 0; n_split = 0; }
     __syncthreads();
 
@@ -129,18 +131,43 @@ plan_kernel(int B, int W, int overhead, int len_cap, const int32_t *__restrict__
     }
 }
 
+// Validation mode: every block-table entry of a page that intersects a request's effective range must name a page of
+// the pool.  One block per request (grid-stride), threads over its pages; the first offender found wins the status word.
+__global__ void __launch_bounds__(256)
+validate_pages_kernel(int B, int num_pool_pages, int table_stride, const int32_t *__restrict__ block_table,
+                      const int32_t *__restrict__ req_lo, const int32_t *__restrict__ req_hi, int32_t *status) {
+    for (int i = blockIdx.x; i < B; i += gridDim.x) {
+        const int lo = req_lo[i], hi = req_hi[i];
+        if (hi <= lo) continue;
+        for (int pg = lo / kPage + threadIdx.x; pg < (hi + kPage - 1) / kPage; pg += blockDim.x) {
+            const int id = block_table[(int64_t)i * table_stride + pg];
+            if (id < 0 || id >= num_pool_pages) {
+                if (atomicCAS(status, 0, (int)SPLASH_BAD_PAGE_ID) == 0) { status[1] = i; status[2] = pg; status[3] = id; }
+            }
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_validate_pages(const DecodeParams &p, const int32_t *req_lo, const int32_t *req_hi, cudaStream_t stream) {
+    const int grid = p.B < 1024 ? p.B : 1024;
+    validate_pages_kernel<<<grid, 256, 0, stream>>>(p.B, p.num_pool_pages, p.table_stride, p.block_table, req_lo, req_hi, p.status);
+    count_launch();
+    return cudaGetLastError();
+}
 
 cudaError_t launch_plan(const DecodeParams &p, const int32_t *kv_begin, const int32_t *kv_end,
                         int32_t *tile_start, int32_t *req_lo, int32_t *req_hi, int32_t *req_wfirst,
                         int32_t *req_wlast, int32_t *cost_start, int32_t *worker_begin, int32_t *split_list,
-                        int32_t *worker_req, int4 *split_rec, int32_t *status, cudaStream_t stream) {
+                        int32_t *worker_req, int4 *split_rec, int32_t *status, bool reset_status, cudaStream_t stream) {
     // same shared-memory carve-out as the decode kernel that follows: no reconfiguration between them
-    static bool configured[64] = {};
-    if (first_use_on_device(configured)) {
+    static DeviceOnce once;
+    once.run([&] {
         cudaFuncSetAttribute(plan_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
-    }
-    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.len_cap, p.seq_lens, kv_begin, kv_end, tile_start,
+        return cudaSuccess;     // a preference: a failure is not an error
+    });
+    plan_kernel<<<1, kPlanThreads, 0, stream>>>(p.B, p.num_workers, p.request_overhead_tiles, p.len_cap, reset_status ? 1 : 0, p.seq_lens, kv_begin, kv_end, tile_start,
                                                 req_lo, req_hi, req_wfirst, req_wlast, cost_start, worker_begin, split_list, worker_req, split_rec, status);
     count_launch();
     return cudaGetLastError();

@@ -1,5 +1,11 @@
-"""The split-KV plan the device writes, against a plain-Python restatement: it must
-cover every (request, tile) exactly once, in order, and depend only on lengths."""
+"""The split-KV plan the device writes.
+
+The plan is an integer step with many valid answers (any cut of the tile sequence into contiguous runs gives
+correct attention), so what PINS it are the partition properties checked at the end: effective ranges as
+defined, boundaries that start at 0, end at the tile total and never decrease, and every non-empty request's
+first / last worker containing its first / last tile -- i.e. every (request, tile) is covered exactly once, in
+order.  The equality with ``python_plan`` below is a regression check only: that function restates the
+kernel's own balancing rule and is no independent source of truth."""
 import numpy as np
 import pytest
 
