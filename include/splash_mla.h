@@ -264,6 +264,50 @@ SPLASH_API int splash_kv_page_migrate(const void *src_pool, const float *src_sca
 SPLASH_API size_t splash_kv_page_migrate_workspace_bytes(int32_t max_page_id);
 
 /*
+ * A decode call that carries a page migration with it: the overlapped transfer of a layout
+ * switch, in which one layer's state moves while another layer computes, so that about one
+ * layer's transfer stays exposed (Sec. 4.1 "Overlapped transfer", the exposed-cost equation of
+ * Sec. 4.2).  The effect is that of
+ *     splash_kv_page_migrate(job...)  and  splash_mla_decode(...)
+ * issued on `stream` in either order; the two must therefore be independent: the decode reads
+ * none of the job's destination pages and not the job's block table (the usual case: the job
+ * moves the pages of ANOTHER layer's cache; source pages may be shared, they are only read).
+ *
+ * How: slices of 65..128 (head, row) pairs run on CTA pairs in which the MMA-issuing warps of
+ * each pair's second CTA have nothing to do; those warps copy the job's pages (16-byte
+ * streaming loads and stores, byte-exact) while the rest of the kernel decodes, on SMs and
+ * HBM bandwidth the decode leaves unused.  The job's table rewrite (three small kernels) runs
+ * on `stream` before the decode.  Calls that do not run on the CTA-pair kernels (narrower
+ * slices, SPLASH_FLAG_SIMT / NO_PAIR, more than 128 (head, row) pairs) run the plain page-copy
+ * kernel after the decode instead: same results, no overlap.
+ *
+ * job == NULL or job->n == 0: exactly splash_mla_decode.  The job's fields are the arguments of
+ * splash_kv_page_migrate, validated the same way; on an error nothing has been launched.
+ */
+typedef struct splash_migrate_job {
+    uint32_t struct_size;                /* sizeof(splash_migrate_job) */
+    const void *src_pool; const float *src_scales;
+    void *dst_pool; float *dst_scales;
+    int64_t page_bytes;
+    const int32_t *src_page_ids, *dst_page_ids;
+    int64_t n;
+    int32_t src_id_base, dst_id_base, max_page_id;
+    int32_t *block_table;
+    int64_t num_table_entries;
+    void *workspace;
+    size_t workspace_bytes;
+} splash_migrate_job;
+
+SPLASH_API int splash_mla_decode_migrating(const splash_mla_shape *shape,
+                      const void *q, const void *kv_pool, const float *kv_scales,
+                      const int32_t *block_table, const int32_t *seq_lens,
+                      int32_t head_begin, int32_t head_end,
+                      const int32_t *kv_begin, const int32_t *kv_end,
+                      float *out, float *lse,
+                      void *workspace, size_t workspace_bytes, void *stream,
+                      const splash_migrate_job *job);
+
+/*
  * splash_kv_page_migrate without a workspace argument and without any allocation.
  * (The paper has no counterpart for this entry point; it exists for the library's
  * callers.)

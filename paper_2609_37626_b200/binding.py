@@ -61,6 +61,22 @@ class MlaShape(ctypes.Structure):
     ]
 
 
+class MigrateJob(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("src_pool", ctypes.c_void_p), ("src_scales", ctypes.c_void_p),
+        ("dst_pool", ctypes.c_void_p), ("dst_scales", ctypes.c_void_p),
+        ("page_bytes", ctypes.c_int64),
+        ("src_page_ids", ctypes.c_void_p), ("dst_page_ids", ctypes.c_void_p),
+        ("n", ctypes.c_int64),
+        ("src_id_base", ctypes.c_int32), ("dst_id_base", ctypes.c_int32), ("max_page_id", ctypes.c_int32),
+        ("block_table", ctypes.c_void_p),
+        ("num_table_entries", ctypes.c_int64),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t),
+    ]
+
+
 _lib = None
 
 
@@ -77,6 +93,9 @@ def load() -> ctypes.CDLL:
     vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
     lib.splash_mla_decode.restype = ctypes.c_int
     lib.splash_mla_decode.argtypes = [ctypes.POINTER(MlaShape), vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.splash_mla_decode_migrating.restype = ctypes.c_int
+    lib.splash_mla_decode_migrating.argtypes = [ctypes.POINTER(MlaShape), vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, sz, vp,
+                                                ctypes.POINTER(MigrateJob)]
     lib.splash_mla_decode_workspace_bytes.restype = sz
     lib.splash_mla_decode_workspace_bytes.argtypes = [ctypes.POINTER(MlaShape), i32, i32]
     lib.splash_mla_decode_sparse.restype = ctypes.c_int
@@ -174,8 +193,10 @@ def splash_mla_decode(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch
                       head_end: Optional[int] = None, kv_begin: Optional[torch.Tensor] = None,
                       kv_end: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
                       lse: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
-                      stream: Optional[torch.cuda.Stream] = None, flags: int = 0):
+                      stream: Optional[torch.cuda.Stream] = None, flags: int = 0, migrate_job=None):
     """Decode attention of one shard; see ``splash_mla_decode`` in include/splash_mla.h.
+    With ``migrate_job`` (from ``make_migrate_job``) the call is ``splash_mla_decode_migrating``: the job's pages
+    move while this call decodes.
 
     q [B][H][576] bf16; kv_pool [P][64][576] bf16, or uint8 / float8_e4m3fn with
     kv_scales [P][64] fp32; block_table [B][stride] int32; seq_lens, kv_begin, kv_end
@@ -199,12 +220,45 @@ def splash_mla_decode(q: torch.Tensor, kv_pool: torch.Tensor, block_table: torch
     if workspace is None:
         need = splash_mla_decode_workspace_bytes(shape, head_begin, head_end)
         workspace = _workspace(q.device, need, "decode")
+    if migrate_job is not None:
+        rc = lib.splash_mla_decode_migrating(ctypes.byref(shape), _ptr(q), _ptr(kv_pool), _ptr(kv_scales), _ptr(block_table),
+                                             _ptr(seq_lens), head_begin, head_end, _ptr(kv_begin), _ptr(kv_end),
+                                             _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                             _stream_ptr(stream), ctypes.byref(migrate_job[0]))
+        _check(rc)
+        return out, lse
     rc = lib.splash_mla_decode(ctypes.byref(shape), _ptr(q), _ptr(kv_pool), _ptr(kv_scales), _ptr(block_table),
                                _ptr(seq_lens), head_begin, head_end, _ptr(kv_begin), _ptr(kv_end),
                                _ptr(out), _ptr(lse), _ptr(workspace), workspace.numel() * workspace.element_size(),
                                _stream_ptr(stream))
     _check(rc)
     return out, lse
+
+
+def make_migrate_job(src_pool: torch.Tensor, dst_pool: torch.Tensor, src_page_ids: torch.Tensor,
+                     dst_page_ids: torch.Tensor, block_table: torch.Tensor, *,
+                     src_scales: Optional[torch.Tensor] = None, dst_scales: Optional[torch.Tensor] = None,
+                     src_id_base: int = 0, dst_id_base: int = 0, max_page_id: Optional[int] = None,
+                     workspace: Optional[torch.Tensor] = None):
+    """The arguments of ``splash_kv_page_migrate`` as a job for ``splash_mla_decode(..., migrate_job=...)``.
+    Returns (MigrateJob, tensors kept alive with it)."""
+    lib = load()
+    assert src_pool.is_contiguous() and dst_pool.is_contiguous() and block_table.is_contiguous()
+    assert src_page_ids.dtype == torch.int32 and dst_page_ids.dtype == torch.int32
+    if max_page_id is None:
+        max_page_id = max(src_id_base + src_pool.shape[0], dst_id_base + dst_pool.shape[0])
+    if workspace is None:
+        workspace = torch.empty(int(lib.splash_kv_page_migrate_workspace_bytes(max_page_id)), dtype=torch.uint8,
+                                device=src_pool.device)
+    job = MigrateJob(struct_size=ctypes.sizeof(MigrateJob), src_pool=src_pool.data_ptr(),
+                     src_scales=None if src_scales is None else src_scales.data_ptr(), dst_pool=dst_pool.data_ptr(),
+                     dst_scales=None if dst_scales is None else dst_scales.data_ptr(),
+                     page_bytes=src_pool.shape[1] * src_pool.shape[2] * src_pool.element_size(),
+                     src_page_ids=src_page_ids.data_ptr(), dst_page_ids=dst_page_ids.data_ptr(), n=src_page_ids.numel(),
+                     src_id_base=src_id_base, dst_id_base=dst_id_base, max_page_id=max_page_id,
+                     block_table=block_table.data_ptr(), num_table_entries=block_table.numel(),
+                     workspace=workspace.data_ptr(), workspace_bytes=workspace.numel())
+    return job, (src_pool, dst_pool, src_page_ids, dst_page_ids, block_table, src_scales, dst_scales, workspace)
 
 
 def splash_mla_decode_sparse_workspace_bytes(shape: MlaShape, max_selected: int, head_begin: int, head_end: int) -> int:

@@ -173,17 +173,68 @@ struct SparseStage {
     bool fused;        // one kernel gathers, dequantises and multiplies (CTA pairs); else gather kernel + dense kernels
 };
 
+// Argument checks shared by the page-migration entry points (the workspace variant, the job of a decode call).
+int check_migrate_args(const void *src_pool, const float *src_scales, const void *dst_pool, const float *dst_scales,
+                       int64_t page_bytes, const int32_t *src_page_ids, const int32_t *dst_page_ids, int64_t n,
+                       int32_t max_page_id, const int32_t *block_table, int64_t num_table_entries,
+                       const void *workspace, size_t workspace_bytes) {
+    if (n < 0 || num_table_entries < 0 || page_bytes <= 0 || page_bytes % 16 || max_page_id < 0) {
+        set_error("bad sizes (page_bytes must be a positive multiple of 16)"); return SPLASH_INVALID_ARG;
+    }
+    if (n == 0) return SPLASH_OK;   // nothing moves, the table keeps every entry
+    if (!src_pool || !dst_pool || !src_page_ids || !dst_page_ids) { set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG; }
+    if ((src_scales == nullptr) != (dst_scales == nullptr)) { set_error("give both scale pools or neither"); return SPLASH_INVALID_ARG; }
+    if (num_table_entries > 0 && (!block_table || !workspace)) { set_error("block_table / workspace is NULL"); return SPLASH_INVALID_ARG; }
+    if (!aligned(src_pool, 16) || !aligned(dst_pool, 16) || !aligned(src_scales, 16) || !aligned(dst_scales, 16) ||
+        !aligned(workspace, 16)) {
+        set_error("misaligned pointer (pools, scales, workspace: 16 B)"); return SPLASH_INVALID_ARG;
+    }
+    if (num_table_entries > 0 && workspace_bytes < splash_kv_page_migrate_workspace_bytes(max_page_id)) {
+        set_error("workspace too small"); return SPLASH_INVALID_ARG;
+    }
+    if (n > 0x7fffffffLL) { set_error("too many pages"); return SPLASH_INVALID_ARG; }
+    return SPLASH_OK;
+}
+
+int check_migrate_job(const splash_migrate_job *job) {
+    if (job->struct_size != sizeof(splash_migrate_job)) {
+        set_error("job.struct_size is %u, this library expects %zu", job->struct_size, sizeof(splash_migrate_job));
+        return SPLASH_INVALID_ARG;
+    }
+    return check_migrate_args(job->src_pool, job->src_scales, job->dst_pool, job->dst_scales, job->page_bytes, job->src_page_ids,
+                              job->dst_page_ids, job->n, job->max_page_id, job->block_table, job->num_table_entries,
+                              job->workspace, job->workspace_bytes);
+}
+
+cudaError_t run_migrate_job(const splash_migrate_job *job, bool do_table, bool do_copy, cudaStream_t stream) {
+    return launch_page_migrate(job->src_pool, job->src_scales, job->dst_pool, job->dst_scales, job->page_bytes, job->src_page_ids,
+                               job->dst_page_ids, job->n, job->src_id_base, job->dst_id_base, job->max_page_id, job->block_table,
+                               job->num_table_entries, static_cast<int32_t *>(job->workspace), do_table, do_copy, stream);
+}
+
 // One dense decode call: plan, decode kernel, combine.  With a sparse stage, seq_lens are the list counts, kv_pool
 // and block_table the dense cache and its table, and the gather kernel runs between the plan and the decode kernel.
 int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_pool, const float *kv_scales,
                  const int32_t *block_table, const int32_t *seq_lens, int32_t head_begin, int32_t head_end,
                  const int32_t *kv_begin, const int32_t *kv_end, float *out, float *lse,
-                 void *workspace, size_t workspace_bytes, void *stream_, const SparseStage *sparse) {
+                 void *workspace, size_t workspace_bytes, void *stream_, const SparseStage *sparse,
+                 const splash_migrate_job *job = nullptr) {
     g_launches = 0;
     int rc = check_shape(shape, head_begin, head_end);
     if (rc != SPLASH_OK) return rc;
+    if (job != nullptr) {
+        rc = check_migrate_job(job);
+        if (rc != SPLASH_OK) return rc;
+        if (job->n == 0) job = nullptr;
+    }
     const int B = shape->num_requests;
-    if (B == 0 || head_end == head_begin) return SPLASH_OK;   // idle rank: nothing to do
+    if (B == 0 || head_end == head_begin) {     // idle rank: no attention to compute; its pages still move
+        if (job != nullptr) {
+            cudaError_t e = run_migrate_job(job, true, true, static_cast<cudaStream_t>(stream_));
+            if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
+        }
+        return SPLASH_OK;
+    }
     if (!q || !kv_pool || !block_table || !seq_lens || !out || !lse || !workspace) {
         set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG;
     }
@@ -206,6 +257,10 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     const int vbegin = head_begin * R, vend = head_end * R;
     const int vstep = R > 1 ? kMaxHeads : vend - vbegin;
     cudaError_t e = cudaSuccess;
+    // a page-copy job: its table rewrite runs first; its page copy rides in the decode kernel if that is a CTA-pair
+    // kernel (one pass only), else runs as a kernel of its own after the decode
+    bool job_copy_pending = job != nullptr;
+    if (job != nullptr) e = run_migrate_job(job, true, false, static_cast<cudaStream_t>(stream_));
     for (int vb = vbegin; vb < vend && e == cudaSuccess; vb += vstep) {
     const int ve = vb + vstep < vend ? vb + vstep : vend;
     const int h = ve - vb;
@@ -247,6 +302,13 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
         p.request_overhead_tiles = kRequestOverheadTilesPair;
     // the bf16 CTA-pair kernel writes its partial outputs as f16
     p.partial_f16 = (pair && shape->kv_dtype == SPLASH_KV_BF16 && !fused_sparse) ? 1 : 0;
+    if (job_copy_pending && pair && !fused_sparse && vend - vbegin <= vstep) {
+        p.mig_src = static_cast<const uint4 *>(job->src_pool); p.mig_dst = static_cast<uint4 *>(job->dst_pool);
+        p.mig_src_scales = reinterpret_cast<const uint4 *>(job->src_scales); p.mig_dst_scales = reinterpret_cast<uint4 *>(job->dst_scales);
+        p.mig_src_ids = job->src_page_ids; p.mig_dst_ids = job->dst_page_ids;
+        p.mig_page_vecs = job->page_bytes / 16; p.mig_n = (int32_t)job->n;
+        job_copy_pending = false;
+    }
 
     e = record_timing_event(0, stream);
     if (e == cudaSuccess)
@@ -270,6 +332,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     if (e == cudaSuccess) e = record_timing_event(3, stream);
     if (e == cudaSuccess && g_timing) g_events_recorded = true;
     }
+    if (e == cudaSuccess && job_copy_pending) e = run_migrate_job(job, false, true, static_cast<cudaStream_t>(stream_));
     if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
     return SPLASH_OK;
 }
@@ -284,6 +347,14 @@ int splash_mla_decode(const splash_mla_shape *shape, const void *q, const void *
                       void *workspace, size_t workspace_bytes, void *stream_) {
     return decode_dense(shape, q, kv_pool, kv_scales, block_table, seq_lens, head_begin, head_end, kv_begin, kv_end, out, lse,
                         workspace, workspace_bytes, stream_, nullptr);
+}
+
+int splash_mla_decode_migrating(const splash_mla_shape *shape, const void *q, const void *kv_pool, const float *kv_scales,
+                                const int32_t *block_table, const int32_t *seq_lens, int32_t head_begin, int32_t head_end,
+                                const int32_t *kv_begin, const int32_t *kv_end, float *out, float *lse,
+                                void *workspace, size_t workspace_bytes, void *stream_, const splash_migrate_job *job) {
+    return decode_dense(shape, q, kv_pool, kv_scales, block_table, seq_lens, head_begin, head_end, kv_begin, kv_end, out, lse,
+                        workspace, workspace_bytes, stream_, nullptr, job);
 }
 
 namespace {
@@ -390,24 +461,12 @@ int splash_kv_page_migrate(const void *src_pool, const float *src_scales, void *
                            int32_t *block_table, int64_t num_table_entries,
                            void *workspace, size_t workspace_bytes, void *stream_) {
     g_launches = 0;
-    if (n < 0 || num_table_entries < 0 || page_bytes <= 0 || page_bytes % 16 || max_page_id < 0) {
-        set_error("bad sizes (page_bytes must be a positive multiple of 16)"); return SPLASH_INVALID_ARG;
-    }
-    if (n == 0) return SPLASH_OK;   // nothing moves, the table keeps every entry
-    if (!src_pool || !dst_pool || !src_page_ids || !dst_page_ids) { set_error("a required pointer is NULL"); return SPLASH_INVALID_ARG; }
-    if ((src_scales == nullptr) != (dst_scales == nullptr)) { set_error("give both scale pools or neither"); return SPLASH_INVALID_ARG; }
-    if (num_table_entries > 0 && (!block_table || !workspace)) { set_error("block_table / workspace is NULL"); return SPLASH_INVALID_ARG; }
-    if (!aligned(src_pool, 16) || !aligned(dst_pool, 16) || !aligned(src_scales, 16) || !aligned(dst_scales, 16) ||
-        !aligned(workspace, 16)) {
-        set_error("misaligned pointer (pools, scales, workspace: 16 B)"); return SPLASH_INVALID_ARG;
-    }
-    if (num_table_entries > 0 && workspace_bytes < splash_kv_page_migrate_workspace_bytes(max_page_id)) {
-        set_error("workspace too small"); return SPLASH_INVALID_ARG;
-    }
-    if (n > 0x7fffffffLL) { set_error("too many pages"); return SPLASH_INVALID_ARG; }
+    const int rc = check_migrate_args(src_pool, src_scales, dst_pool, dst_scales, page_bytes, src_page_ids, dst_page_ids, n,
+                                      max_page_id, block_table, num_table_entries, workspace, workspace_bytes);
+    if (rc != SPLASH_OK || n == 0) return rc;
     cudaError_t e = launch_page_migrate(src_pool, src_scales, dst_pool, dst_scales, page_bytes, src_page_ids,
                                         dst_page_ids, n, src_id_base, dst_id_base, max_page_id, block_table,
-                                        num_table_entries, static_cast<int32_t *>(workspace),
+                                        num_table_entries, static_cast<int32_t *>(workspace), true, true,
                                         static_cast<cudaStream_t>(stream_));
     if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
     return SPLASH_OK;
@@ -438,7 +497,7 @@ int splash_kv_page_migrate_static(const void *src_pool, const float *src_scales,
     cudaError_t e = static_remap_address(&remap);      // first call on a device looks the symbol up
     if (e != cudaSuccess) { set_error("cudaGetSymbolAddress failed: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
     e = launch_page_migrate(src_pool, src_scales, dst_pool, dst_scales, page_bytes, src_page_ids, dst_page_ids, n,
-                            src_id_base, dst_id_base, max_page_id, block_table, num_table_entries, remap,
+                            src_id_base, dst_id_base, max_page_id, block_table, num_table_entries, remap, true, true,
                             static_cast<cudaStream_t>(stream_));
     if (e != cudaSuccess) { set_error("CUDA error: %s", cudaGetErrorString(e)); return SPLASH_CUDA_ERROR; }
     return SPLASH_OK;

@@ -118,6 +118,14 @@ struct DecodeParams {
     const int32_t *sel, *ctx_lens;
     int64_t sel_stride;
     int32_t num_workers;
+    // optional page-copy job carried along by the CTA-pair kernels in warps that have nothing else to do (the issuer
+    // warps of each pair's second CTA): page mig_src_ids[j] of mig_src -> page mig_dst_ids[j] of mig_dst, j < mig_n,
+    // mig_page_vecs 16-byte vectors per page, with the pages' scale pages when the scale pointers are set
+    const uint4 *mig_src, *mig_src_scales;
+    uint4 *mig_dst, *mig_dst_scales;
+    const int32_t *mig_src_ids, *mig_dst_ids;
+    int64_t mig_page_vecs;
+    int32_t mig_n;
     int32_t request_overhead_tiles;   // per-request cost the plan adds to the tile count
     long long *trace;          // optional device buffer for pipeline timestamps (diagnostics), or NULL
 };
@@ -252,7 +260,7 @@ cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, v
                                 float *dst_scales, int64_t page_bytes, const int32_t *src_ids,
                                 const int32_t *dst_ids, int64_t n, int32_t src_base, int32_t dst_base,
                                 int32_t max_page_id, int32_t *block_table, int64_t num_entries,
-                                int32_t *remap, cudaStream_t stream);
+                                int32_t *remap, bool do_table, bool do_copy, cudaStream_t stream);
 
 cudaError_t static_remap_address(int32_t **ptr);
 

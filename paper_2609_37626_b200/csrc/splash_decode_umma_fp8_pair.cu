@@ -327,7 +327,10 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
             }
         }
     } else if (warp >= kWarpQk && warp < kWarpSoftmax) {
-        // the issuer warps of the peer CTA have nothing to do
+        // the issuer warps of the peer CTA have nothing to do for the attention itself: they carry the call's page-copy
+        // job, if it has one (a layer's pages on the move while this layer decodes)
+        if (p.mig_n > 0)
+            copy_pages_in_idle_warp(p, worker * (kQkWarps + kPvWarps) + (warp - kWarpQk), p.num_workers * (kQkWarps + kPvWarps), lane);
     } else if (warp >= kWarpConvert && warp < kWarpConvert + kConvertWarps) {
         // ===================================================== query converters (this CTA's 64 heads)
         const int ct = (warp - kWarpConvert) * 32 + lane;   // 0..127

@@ -297,7 +297,10 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
             }
         }
     } else if (warp >= kWarpQk && warp < kWarpSoftmax) {
-        // the issuer warps of the peer CTA have nothing to do
+        // the issuer warps of the peer CTA have nothing to do for the attention itself: they carry the call's page-copy
+        // job, if it has one (a layer's pages on the move while this layer decodes)
+        if (p.mig_n > 0)
+            copy_pages_in_idle_warp(p, worker * (kQkWarps + kPvWarps) + (warp - kWarpQk), p.num_workers * (kQkWarps + kPvWarps), lane);
     } else {
         // ===================================================== softmax + epilogue warps
         // S partial layout per CTA: TMEM lane L < 64 = head L, tokens of half-page 0 in 32 columns;

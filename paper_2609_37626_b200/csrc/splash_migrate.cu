@@ -96,9 +96,9 @@ cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, v
                                 float *dst_scales, int64_t page_bytes, const int32_t *src_ids,
                                 const int32_t *dst_ids, int64_t n, int32_t src_base, int32_t dst_base,
                                 int32_t max_page_id, int32_t *block_table, int64_t num_entries,
-                                int32_t *remap, cudaStream_t stream) {
+                                int32_t *remap, bool do_table, bool do_copy, cudaStream_t stream) {
     cudaError_t e;
-    if (num_entries > 0 && max_page_id > 0) {
+    if (do_table && num_entries > 0 && max_page_id > 0) {
         remap_fill_kernel<<<(max_page_id + 255) / 256, 256, 0, stream>>>(remap, max_page_id);
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
@@ -111,6 +111,7 @@ cudaError_t launch_page_migrate(const void *src_pool, const float *src_scales, v
         count_launch();
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
+    if (!do_copy) return cudaSuccess;
     dim3 grid((unsigned)n, kCopyCtasPerPage);
     page_copy_kernel<<<grid, kCopyThreads, 0, stream>>>(
         static_cast<const uint4 *>(src_pool), static_cast<uint4 *>(dst_pool),

@@ -92,6 +92,58 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     tmem_ld16(taddr + 16, *reinterpret_cast<float(*)[16]>(&v[16]));
 }
 
+// The page-copy job of a decode call (a layer's pages moving while another layer decodes), as carried by one warp:
+// copy warp cw of ncw takes pages cw, cw + ncw, ...  A page is copied in pieces of 4 KB (eight 16-byte loads per
+// lane); the loads of the next piece are issued before the stores of the current one, across page boundaries, so
+// that a warp always has 4 KB of loads in flight.  Streaming loads and stores: the bytes are not needed again soon.
+// (Pulling each page into L2 ahead of its loads made the copy slower and the decode beside it too.)  Byte-exact.  A
+// page that is not a multiple of 4 KB has its remainder copied 512 bytes at a time; scale pages ride along.
+__device__ __forceinline__ void copy_pages_in_idle_warp(const DecodeParams &p, int cw, int ncw, int lane) {
+    constexpr int kInFlight = 8, kPiece = kInFlight * 32;        // 16-byte vectors per piece
+    const int64_t vecs = p.mig_page_vecs;
+    const int pieces_per_page = (int)(vecs / kPiece);
+    const int my_pages = p.mig_n > cw ? (p.mig_n - cw + ncw - 1) / ncw : 0;
+    if (my_pages == 0) return;
+    auto page_src = [&](int k) { return p.mig_src + (int64_t)p.mig_src_ids[cw + (int64_t)k * ncw] * vecs; };
+    auto page_dst = [&](int k) { return p.mig_dst + (int64_t)p.mig_dst_ids[cw + (int64_t)k * ncw] * vecs; };
+    // what does not fit the 4 KB pieces: the tail of every page and the scale pages
+    for (int k = 0; k < my_pages; ++k) {
+        const int64_t j = cw + (int64_t)k * ncw;
+        for (int64_t c = (int64_t)pieces_per_page * kPiece + lane; c < vecs; c += 32) __stcs(page_dst(k) + c, __ldcs(page_src(k) + c));
+        if (p.mig_src_scales != nullptr && lane < kPage * 4 / 16)
+            __stcs(p.mig_dst_scales + (int64_t)p.mig_dst_ids[j] * (kPage * 4 / 16) + lane,
+                   __ldcs(p.mig_src_scales + (int64_t)p.mig_src_ids[j] * (kPage * 4 / 16) + lane));
+    }
+    if (pieces_per_page == 0) return;
+    const int64_t total = (int64_t)my_pages * pieces_per_page;
+    const uint4 *src = nullptr;
+    uint4 *dst_page = nullptr;
+    // loads piece `it` into v and returns where it goes
+    auto load_piece = [&](uint4 (&v)[kInFlight], int64_t it) -> uint4 * {
+        const int piece = (int)(it % pieces_per_page);
+        if (piece == 0) {
+            const int k = (int)(it / pieces_per_page);
+            src = page_src(k); dst_page = page_dst(k);
+        }
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) v[u] = __ldcs(src + (int64_t)piece * kPiece + u * 32 + lane);
+        return dst_page + (int64_t)piece * kPiece + lane;
+    };
+    auto store_piece = [&](const uint4 (&v)[kInFlight], uint4 *to) {
+#pragma unroll
+        for (int u = 0; u < kInFlight; ++u) __stcs(to + u * 32, v[u]);
+    };
+    uint4 va[kInFlight], vb[kInFlight];
+    uint4 *ta = load_piece(va, 0), *tb = nullptr;
+    for (int64_t it = 0; it < total; it += 2) {
+        if (it + 1 < total) tb = load_piece(vb, it + 1);
+        store_piece(va, ta);
+        if (it + 1 >= total) break;
+        if (it + 2 < total) ta = load_piece(va, it + 2);
+        store_piece(vb, tb);
+    }
+}
+
 // Page tiles of the two CTAs of a pair for one step, after the token shift.
 struct PairGeom { TileGeom a, b; bool has_b; };
 
