@@ -286,7 +286,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     p.softmax_scale = shape->softmax_scale;
     p.tile_start = v.tile_start; p.req_lo = v.req_lo; p.req_hi = v.req_hi; p.worker_begin = v.worker_begin;
     p.worker_req = v.worker_req;
-    p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out;
+    p.status = v.status; p.partial_lse = v.partial_lse; p.partial_out = v.partial_out; p.partial_scale = v.partial_scale;
     p.trace = g_trace;
     p.len_cap = sparse ? sparse->max_selected : -1;
     if (fused_sparse) {

@@ -36,6 +36,7 @@ constexpr int kRequestOverheadTilesFp8Pair = 14;   // CTA-pair kernel: tiles are
 //                         req_wlast[B], cost_start[B+1], worker_begin[W+1], split_list[W+1]
 //                         (status[8] = number of entries of split_list)
 // then (256-B aligned)    partial_lse [2W][h] fp32
+// then (256-B aligned)    partial_scale [2W][h] fp32 (f16 partial outputs only: the power of two a row was divided by)
 // then (256-B aligned)    partial_out [2W][h][512] fp32
 struct PlanView {
     int32_t *status;        // 16 ints
@@ -50,6 +51,7 @@ struct PlanView {
     int32_t *worker_req;    // [W+1] the request that holds a worker's first tile (what the kernels would bisect for)
     int4 *split_rec;        // [W+1] per entry of split_list: (request, first worker, last worker, first tile of the request)
     float *partial_lse;     // [2W][h]
+    float *partial_scale;   // [2W][h]
     float *partial_out;     // [2W][h][512]
     int32_t num_workers;    // W
     int32_t h;              // width of the head slice
@@ -76,6 +78,8 @@ inline __host__ PlanView make_plan_view(void *workspace, int B, int W, int h) {
     v.split_rec = reinterpret_cast<int4 *>(p + off); off += sizeof(int4) * (size_t)(W + 1);
     off = align_up(off, 256);
     v.partial_lse = reinterpret_cast<float *>(p + off); off += sizeof(float) * (size_t)2 * W * h;
+    off = align_up(off, 256);
+    v.partial_scale = reinterpret_cast<float *>(p + off); off += sizeof(float) * (size_t)2 * W * h;
     off = align_up(off, 256);
     v.partial_out = reinterpret_cast<float *>(p + off); off += sizeof(float) * (size_t)2 * W * h * kDV;
     v.num_workers = W;
@@ -110,8 +114,11 @@ struct DecodeParams {
     const int32_t *worker_req;   // request holding each worker's first tile, from the plan
     int32_t *status;
     float *partial_lse, *partial_out;
+    float *partial_scale;      // f16 partial outputs: row (slot, head) holds O * 2^k with 2^-k stored here
     int32_t partial_f16;       // 1: the partial outputs are f16 (same slot order, rows of 512 halves): half the bytes for the
-                               // decode kernel to write and the combine kernel to read; 11 significant bits of a normalised O
+                               // decode kernel to write and the combine kernel to read; 11 significant bits of a normalised O,
+                               // each row scaled by a power of two so that its largest entry sits just below f16's maximum
+                               // (exact, and no limit on the magnitude of the cache values)
     int32_t len_cap;           // >= 0: seq_lens holds list counts; one outside [0, len_cap] counts as 1 (sparse decode)
     // fused sparse decode: kv_pool holds 656-byte rows, block_table / num_pool_pages describe it, and request i
     // attends over the tokens sel[i * sel_stride + j], j < seq_lens[i], each below ctx_lens[i]

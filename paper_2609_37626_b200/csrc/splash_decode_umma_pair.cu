@@ -447,13 +447,63 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                 const int n = cf;
                 const int dv0 = 256 * n + 128 * g + 2 * (lane & 3);
                 const int nvalid = min(kN, p.head_end - head0);
+                // A partial piece is stored as f16.  So that neither large nor tiny cache values leave f16's range, every
+                // row is first multiplied by the power of two that puts its largest entry into [2^14, 2^15) -- exact --
+                // and the inverse goes to partial_scale beside the row's LSE for the combine kernel.  The row maximum
+                // takes one more pass over the accumulator: this thread's four rows over its 128 columns, the 4 lanes
+                // that share a row, then the 4 warps that hold the row's other columns (through the exchange buffer).
+                float up[2][2] = {{1.f, 1.f}, {1.f, 1.f}};        // 2^k of rows (half, A / B)
+                if (seg.slot >= 0) {
+                    float mx[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll 1
+                    for (int hc = 0; hc < 4; ++hc) {
+                        const int half = hc >> 1, c = hc & 1;
+                        float o[32];
+                        tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * q4 + 16 * half) << 16) + kColO + n * 128 + c * 64, o);
+                        tmem_wait_ld();
+                        float a = 0.f, b = 0.f;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            a = fmaxf(a, fmaxf(fabsf(o[4 * k]), fabsf(o[4 * k + 1])));
+                            b = fmaxf(b, fmaxf(fabsf(o[4 * k + 2]), fabsf(o[4 * k + 3])));
+                        }
+                        if (half == 0) { mx[0][0] = fmaxf(mx[0][0], a); mx[0][1] = fmaxf(mx[0][1], b); }
+                        else { mx[1][0] = fmaxf(mx[1][0], a); mx[1][1] = fmaxf(mx[1][1], b); }
+                    }
+#pragma unroll
+                    for (int half = 0; half < 2; ++half)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int row = 32 * (q4 & 1) + 16 * half + 8 * e + (lane >> 2);
+                            float v = mx[half][e] * l_s[row];
+                            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+                            v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+                            if ((lane & 3) == 0) xch[row * 4 + slot4] = v;
+                        }
+                    named_bar_sync_dyn<128>(2 + half_id);
+#pragma unroll
+                    for (int half = 0; half < 2; ++half)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int row = 32 * (q4 & 1) + 16 * half + 8 * e + (lane >> 2);
+                            const float4 x4 = *reinterpret_cast<const float4 *>(&xch[row * 4]);
+                            const float rmax = fmaxf(fmaxf(x4.x, x4.y), fmaxf(x4.z, x4.w));
+                            const int ex = (int)((__float_as_uint(rmax) >> 23) & 0xffu);
+                            int k = (ex == 0 || ex == 255) ? 0 : 14 - (ex - 127);      // zero / subnormal / non-finite rows stay as they are
+                            k = max(-100, min(100, k));
+                            up[half][e] = __uint_as_float((uint32_t)(127 + k) << 23);
+                            if (slot4 == 0 && (lane & 3) == 0 && row < nvalid)
+                                p.partial_scale[(int64_t)seg.slot * h + (head0 - p.head_begin) + row] = __uint_as_float((uint32_t)(127 - k) << 23);
+                        }
+                    named_bar_sync_dyn<128>(2 + half_id);            // the exchange buffer may be written again
+                }
 #pragma unroll 1
                 for (int hc = 0; hc < 4; ++hc) {
                     const int half = hc >> 1, c = hc & 1;
                     const int hA = 32 * (q4 & 1) + 16 * half + (lane >> 2), hB = hA + 8;
                     float o[32];
                     tmem_ld_16x256b_x8(tmem_base + ((uint32_t)(32 * q4 + 16 * half) << 16) + kColO + n * 128 + c * 64, o);
-                    const float iA = l_s[hA], iB = l_s[hB];
+                    const float iA = l_s[hA] * (half ? up[1][0] : up[0][0]), iB = l_s[hB] * (half ? up[1][1] : up[0][1]);
                     float *rowA = obase + (int64_t)hA * ostride + dv0 + c * 64, *rowB = obase + (int64_t)hB * ostride + dv0 + c * 64;
                     tmem_wait_ld();
                     if (seg.slot >= 0) {

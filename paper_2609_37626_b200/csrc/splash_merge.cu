@@ -64,6 +64,7 @@ template <bool kF16, bool kLean>
 __global__ void __launch_bounds__(kMergeThreads, kLean ? 16 : 8)
 split_combine_kernel(const DecodeParams p, const int4 *__restrict__ split_rec) {
     __shared__ float w_s[kMaxParts];
+    __shared__ float sc_s[kF16 ? kMaxParts : 1];      // f16 pieces: the power of two each row was divided by
     __shared__ int slot_s[kMaxParts];
     __shared__ float red_s[kMergeThreads / 32];
     const int h = p.head_end - p.head_begin;
@@ -92,9 +93,15 @@ split_combine_kernel(const DecodeParams p, const int4 *__restrict__ split_rec) {
         const int wb0 = p.worker_begin[w], wb1 = p.worker_begin[w + 1];
         const float L0 = p.partial_lse[(int64_t)(2 * w) * h + k];
         const float L1 = j == 0 ? p.partial_lse[(int64_t)(2 * w + 1) * h + k] : 0.f;
+        float S0 = 1.f, S1 = 1.f;
+        if constexpr (kF16) {
+            S0 = p.partial_scale[(int64_t)(2 * w) * h + k];
+            if (j == 0) S1 = p.partial_scale[(int64_t)(2 * w + 1) * h + k];
+        }
         const bool live = wb1 > wb0;
         const int slot = 2 * w + (rs <= wb0 ? 0 : 1);
         const float L = live ? ((slot & 1) ? L1 : L0) : -INFINITY;
+        if constexpr (kF16) sc_s[j] = (slot & 1) ? S1 : S0;
         slot_s[j] = slot;
         w_s[j] = L;
         m = fmaxf(m, L);
@@ -141,8 +148,9 @@ split_combine_kernel(const DecodeParams p, const int4 *__restrict__ split_rec) {
             raw[u] = load_part(slot_s[j + u]);
 #pragma unroll
         for (int u = 0; u < 16; ++u) {
-            const float wgt = w_s[j + u] * inv_z;
+            float wgt = w_s[j + u] * inv_z;
             if (wgt != 0.f) {          // a dead worker's slot holds stale bytes
+                if constexpr (kF16) wgt *= sc_s[j + u];
                 const float4 v = widen(raw[u]);
                 acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
                 acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
@@ -158,8 +166,9 @@ split_combine_kernel(const DecodeParams p, const int4 *__restrict__ split_rec) {
             if (j + u < nparts) raw[u] = load_part(slot_s[j + u]);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const float wgt = j + u < nparts ? w_s[j + u] * inv_z : 0.f;
+            float wgt = j + u < nparts ? w_s[j + u] * inv_z : 0.f;
             if (wgt != 0.f) {          // a dead worker's slot holds stale bytes
+                if constexpr (kF16) wgt *= sc_s[j + u];
                 const float4 v = widen(raw[u]);
                 acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
                 acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);

@@ -327,3 +327,22 @@ def test_random_shapes_ranges_and_slices(seed):
         compare(out, lse, *ref, kv_dtype=kv_dtype, rows=rows, what=f"seed {seed} flags {flags}")
         mask = np.ones(H, bool); mask[hb:he] = False
         assert np.all(out[:, mask] == 9.0) and np.all(lse[:, mask] == 9.0)
+
+
+@pytest.mark.parametrize("shift", [17, -20])
+@pytest.mark.parametrize("H", [128, 80])
+def test_split_requests_with_large_and_tiny_cache_values(H, shift):
+    """Requests cut into several pieces on the CTA-pair kernel, whose partial outputs travel as f16 rows: cache
+    values of magnitude 2^17 (beyond f16's largest number) and 2^-20 (inside its subnormal range), the queries
+    scaled the other way so that the logits stay those of N(0,1) data.  Every piece is stored relative to a
+    per-row power of two, so neither overflows nor loses bits."""
+    w = W.make_workload("magnitude", 930 + H, [6000, 300, 9000, 64], H=H)
+    f = np.float32(2.0 ** shift)
+    kv = W.bf16_bits_to_f32(w.kv_pool)
+    fin = np.isfinite(kv)
+    w.kv_pool[fin] = W.f32_to_bf16_bits(kv[fin] * f)                 # a power of two: exact in bf16; poison stays poison
+    w.q[...] = W.f32_to_bf16_bits(W.bf16_bits_to_f32(w.q) / f)
+    ref_o, ref_l = oracle_run(w)
+    out, lse = gpu_run(w)
+    assert np.isfinite(out).all()
+    compare(out / f, lse, ref_o / float(f), ref_l, kv_dtype=0, what=f"values x 2^{shift}")
