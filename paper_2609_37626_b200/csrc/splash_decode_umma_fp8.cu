@@ -296,9 +296,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const float e0 = __uint_as_float(w[k] << 16) * inv, e1 = __uint_as_float(w[k] & 0xffff0000u) * inv;
-                        hi[k] = to_e4m3x2(e0, e1);
-                        const float2 back = from_e4m3x2(hi[k]);
-                        lo[k] = to_e4m3x2(e0 - back.x, e1 - back.y);
+                        split_e4m3_e4m3_x2(e0, e1, hi[k], lo[k]);
                     }
                     const uint32_t d = (uint32_t)(part * 288 + v * 8);
                     const uint32_t off = (d >> 6) * kSlab + sw64((uint32_t)hd, d & 63);

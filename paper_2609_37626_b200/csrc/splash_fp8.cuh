@@ -56,6 +56,16 @@ __device__ __forceinline__ void split_e4m3_e5m2_x2(float lo, float hi, uint16_t 
     asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(res) : "r"(h2), "r"(back));
     asm("cvt.rn.satfinite.e5m2x2.f16x2 %0, %1;" : "=h"(rest) : "r"(res));
 }
+// Two floats -> (e4m3 pair, e4m3 pair of the residuals) in packed f16 arithmetic, for the query operands: the value
+// passes through f16 (11 significant bits against the 8 of the bf16 query it comes from), the residual is exact in f16.
+__device__ __forceinline__ void split_e4m3_e4m3_x2(float lo, float hi, uint16_t &main, uint16_t &rest) {
+    uint32_t h2, back, res;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h2) : "f"(hi), "f"(lo));
+    asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(main) : "r"(h2));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(main));
+    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(res) : "r"(h2), "r"(back));
+    asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(rest) : "r"(res));
+}
 __device__ __forceinline__ float fast_log2(float x) {
     float y;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
