@@ -288,6 +288,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 // (at most one tile ahead of the softmax: two S buffers).
                 int qk_i = does_qk ? 0 : ntiles, pv_i = 0;
                 unsigned long long idle_since = 0;
+                uint32_t idle_polls = 0;          // the wall clock is read once per 256 idle polls: reading it costs hundreds of cycles
                 while (pv_i < ntiles) {
                     bool progressed = false;
                     if ((qk_i > pv_i) && mbar_test_wait(bar(kBarPFull), (p_it + pv_i) & 1)) {
@@ -311,7 +312,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                             progressed = true;
                         }
                     }
-                    if (progressed) { idle_since = 0; continue; }
+                    if (progressed) { idle_since = 0; idle_polls = 0; continue; }
+                    if ((++idle_polls & 255u) != 0u) continue;
                     if (*ctx.abort_flag) { ok = false; break; }
                     const unsigned long long now = global_timer_ns();
                     if (idle_since == 0) idle_since = now;
