@@ -191,6 +191,23 @@ class GpuBench:
             times.append(a.elapsed_time(b))
         return np.array(times)
 
+    def timed_round_robin(self, fns, steps, warmup):
+        """Median milliseconds of each of several step functions, timed in turn within one loop."""
+        torch = self.torch
+        for _ in range(warmup):
+            for fn in fns:
+                self.flush_l2(); fn()
+        torch.cuda.synchronize()
+        times = [[] for _ in fns]
+        for _ in range(steps):
+            for k, fn in enumerate(fns):
+                self.flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); fn(); b.record()
+                b.synchronize()
+                times[k].append(a.elapsed_time(b))
+        return [np.median(t) for t in times]
+
     def decode_workload(self, w, steps, warmup, peaks, traffic_table, name):
         torch, binding = self.torch, self.binding
         dw = binding.DeviceWorkload(w, self.device)
@@ -561,11 +578,10 @@ class GpuBench:
                 migrate(None)
                 dw.decode(out=out, lse=lse)
 
-        t_dec = float(np.median(self.timed(decode_only, steps, warmup)))
-        t_mig = float(np.median(self.timed(migrate_only, steps, warmup)))
-        t_ser = float(np.median(self.timed(serial, steps, warmup)))
-        t_pipe = float(np.median(self.timed(carried, steps, warmup)))
-        t_two = float(np.median(self.timed(pipelined, steps, warmup)))
+        # the five sequences take turns inside one timing loop, so that the clock the power cap leaves (it sinks while
+        # the load lasts) is the same for all of them
+        t_dec, t_mig, t_ser, t_pipe, t_two = (float(x) for x in self.timed_round_robin(
+            [decode_only, migrate_only, serial, carried, pipelined], steps, warmup))
         per_layer = (t_ser - t_dec) / layers           # what one layer's migration costs when nothing hides it
         return {"layers": layers, "decode_only_ms": t_dec, "migrate_only_ms": t_mig, "serial_ms": t_ser,
                 "pipelined_ms": t_pipe, "exposed_ms": t_pipe - t_dec,

@@ -51,6 +51,7 @@ constexpr uint32_t kPeerBytes = 4 * kSlab;          // the peer page's chunks th
 constexpr uint32_t kScaleBytes = 256;
 constexpr int kStages = 3;
 constexpr int kPrefetchAhead = 1;                    // supertiles between the L2 prefetch of a page and its use (4: 1.5 % slower; none: 5 %)
+constexpr int kPrefetchAheadBusy = 4;                // the same while the call carries a page-copy job
 constexpr float kTau = 6.0f;
 constexpr float kLift = 2.75f;
 
@@ -215,7 +216,8 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
                             // A stage is held from its load until P.V has read it, about three supertiles, so the
                             // load of supertile s + 3 starts only when the issuers are about to need it: have its
                             // page in L2 by then.
-                            const int tf = ta + 2 * kPrefetchAhead + (int)rank;
+                            // (further ahead while a page-copy job shares the memory system: the loads then take longer)
+                            const int tf = ta + 2 * (p.mig_n > 0 ? kPrefetchAheadBusy : kPrefetchAhead) + (int)rank;
                             if (tf < seg.tile_end) {
                                 const int page_f = table[first_page + tf];
                                 if (page_f >= 0 && page_f < p.num_pool_pages) tma_prefetch_4d(&tmap_page, 0, 0, 0, page_f);

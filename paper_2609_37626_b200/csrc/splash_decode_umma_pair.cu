@@ -55,6 +55,7 @@ constexpr uint32_t kQBytes = 9 * kQSlab;            // 73,728
 constexpr uint32_t kPHalfBytes = kN * 64;           // P of one half-page: 64 heads x 32 tokens bf16
 constexpr int kStages = 4;
 constexpr int kPrefetchAhead = 1;                   // tiles between the L2 prefetch of a page and its use (4: 3 % slower; none: 4 %)
+constexpr int kPrefetchAheadBusy = 4;               // the same while the call carries a page-copy job
 constexpr float kTau = 8.0f;                        // O is rescaled only when a row maximum grows by more than 2^8
 
 enum BarrierId {
@@ -184,7 +185,8 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
                             // A stage is held from its load until P.V has read it, about three tiles, so the
                             // load of tile t + 3 starts only when the issuers are about to need it: have its
                             // half of the page in L2 by then.
-                            const int tf = tile + kPrefetchAhead;
+                            // (further ahead while a page-copy job shares the memory system: the loads then take longer)
+                            const int tf = tile + (p.mig_n > 0 ? kPrefetchAheadBusy : kPrefetchAhead);
                             if (tf < seg.tile_end) {
                                 const int page_f = table[first_page + tf];
                                 // this CTA's half of the page is 32 consecutive rows: one contiguous range
