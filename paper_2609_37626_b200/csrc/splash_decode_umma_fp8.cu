@@ -17,6 +17,7 @@
 // the bf16 kernel (fp8 MMAs run at twice the rate), which is why the roofline of this
 // workload is taken at the bf16 rate.
 #include "splash_fp8.cuh"
+#include "splash_pair.cuh"
 
 namespace splash {
 
@@ -135,6 +136,10 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                     entry = idx < seg.tile_end ? table[first_page + idx] : 0;
                 }
                 const int page = __shfl_sync(0xffffffffu, entry, rel & 31);
+                // the next page (when its table entry is among the 32 this warp holds): pulled into L2 now, so that its
+                // TMA load, which can only start when a stage comes free, finds it there
+                const int page_ahead = __shfl_sync(0xffffffffu, entry, (rel + 1) & 31);
+                const bool ahead_ok = (rel & 31) + 1 < 32 && tile + 1 < seg.tile_end;
                 const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + tile) * kPage);
                 const uint32_t stage = kv_it % kStages, ph = (kv_it / kStages) & 1;
                 // a page id outside the pool reads as zeros through the tensor map; its
@@ -153,6 +158,8 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                         if (in_pool)
                             bulk_load(sbase + kOffScale + stage * kScaleBytes, p.kv_scales + (int64_t)page * kPage,
                                       kScaleBytes, bar(kBarKvFull + stage));
+                        if (ahead_ok && page_ahead >= 0 && page_ahead < p.num_pool_pages)
+                            bulk_prefetch_l2(static_cast<const uint8_t *>(p.kv_pool) + (size_t)page_ahead * (kPage * kDQK), kStageBytes);
                         mark(kv_it, 1);
                     }
                 }
