@@ -291,7 +291,7 @@ class GpuBench:
                 "roofline": {"bound": "hbm" if t_hbm >= t_tensor else "tensor", "roofline_ms": max(t_hbm, t_tensor) * 1e3,
                              "frac": max(t_hbm, t_tensor) * 1e3 / p50, "of": "whole call, p50", "peak_source": peaks["source"],
                              "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
-                             "passes_over_the_cache": -(-h * R // 128)},
+                             "launch_chains": 1, "cta_pairs_per_kv_worker": -(-h * R // 128)},
                 "launches_per_step": binding.splash_last_launch_count()}
 
     def sparse_workload(self, seq_lens, H, steps, warmup, peaks, topk=2048):

@@ -139,8 +139,9 @@ typedef struct splash_mla_shape {
  *     q   (i, g, r, d) at q  [i*q_stride_request   + g*q_stride_head   + r*576 + d], q_stride_head   = R*576
  *     out (i, g, r, d) at out[i*out_stride_request + g*out_stride_head + r*512 + d], out_stride_head = R*512
  *     lse (i, g, r)    at lse[i*lse_stride_request + g*R + r]
- * 1 <= R <= 8.  A slice of more than 128 / R heads is served 128 (head, row) pairs at a
- * time, each pass reading the cache once.
+ * 1 <= R <= 8.  A slice of more than 128 / R heads runs as several CTA pairs per KV worker,
+ * 128 (head, row) pairs each, side by side on the same pages in one launch: the cache
+ * crosses HBM once (the other pairs' reads of a page hit L2).
  *
  *   q            bf16, 16-byte aligned
  *   kv_pool      [num_pool_pages][64][576] bf16 (73,728 B / page) or e4m3 bytes

@@ -96,14 +96,18 @@ int check_shape(const splash_mla_shape *s, int32_t head_begin, int32_t head_end)
 }
 
 // How one decode call is cut into CTAs.
-struct Tiling { int heads_per_group, num_groups, num_workers; };
+struct Tiling { int heads_per_group, num_groups, num_workers, pair_groups; };
 
 // h = width of the slice in (virtual) heads
 Tiling choose_tiling(const splash_mla_shape *s, int h, int sm_count, bool simt) {
     Tiling t;
-    if (!simt && s->q_rows > 1) {      // several query rows per request: always a CTA pair, whatever the width
+    t.pair_groups = 1;
+    if (!simt && s->q_rows > 1) {      // several query rows per request: always CTA pairs, whatever the width
+        // more than 128 (head, row) pairs: several pairs per KV worker, side by side on the same pages
         t.heads_per_group = 64; t.num_groups = 2;
-        t.num_workers = sm_count / 2 > 0 ? sm_count / 2 : 1;
+        t.pair_groups = (h + kMaxHeads - 1) / kMaxHeads;
+        const int w = (sm_count / 2) / t.pair_groups;
+        t.num_workers = w > 0 ? w : 1;
         return t;
     }
     if (simt) {
@@ -143,8 +147,7 @@ size_t splash_mla_decode_workspace_bytes(const splash_mla_shape *shape, int32_t 
     if (!current_device_info(dev)) return 0;
     // with R query rows per request the call runs over virtual heads, at most kMaxHeads of them at a time
     const int R = shape->q_rows > 1 ? (int)shape->q_rows : 1;
-    int h = (head_end - head_begin) * R;
-    if (R > 1 && h > kMaxHeads) h = kMaxHeads;
+    const int h = (head_end - head_begin) * R;
     if (h == 0 || shape->num_requests == 0) return 256;
     // the larger of the two kernels' needs, so one workspace serves both paths
     size_t need = 0;
@@ -252,10 +255,11 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     const bool simt = (shape->flags & SPLASH_FLAG_SIMT) != 0;
     // R query rows per request: the kernels see R * num_heads virtual heads (head g, row r -> g * R + r: the rows
     // of a head are dense, so a virtual head is 576 / 512 elements from the next) and mask causally by
-    // (virtual head mod R); a slice wider than 128 virtual heads is served 128 at a time.
+    // (virtual head mod R); a slice wider than 128 virtual heads runs as several CTA pairs per KV worker in ONE launch
+    // chain (the loop below has a single pass).
     const int R = shape->q_rows > 1 ? (int)shape->q_rows : 1;
     const int vbegin = head_begin * R, vend = head_end * R;
-    const int vstep = R > 1 ? kMaxHeads : vend - vbegin;
+    const int vstep = vend - vbegin;
     cudaError_t e = cudaSuccess;
     // a page-copy job: its table rewrite runs first; its page copy rides in the decode kernel if that is a CTA-pair
     // kernel (one pass only), else runs as a kernel of its own after the decode
@@ -266,7 +270,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     const int h = ve - vb;
     Tiling t = choose_tiling(shape, h, dev.sm_count, simt);
     const bool fused_sparse = sparse && sparse->fused && !simt;
-    if (fused_sparse) { t.heads_per_group = 64; t.num_groups = 2; t.num_workers = dev.sm_count / 2 > 0 ? dev.sm_count / 2 : 1; }
+    if (fused_sparse) { t.heads_per_group = 64; t.num_groups = 2; t.num_workers = dev.sm_count / 2 > 0 ? dev.sm_count / 2 : 1; t.pair_groups = 1; }
     PlanView v = make_plan_view(workspace, B, t.num_workers, h);
     if (workspace_bytes < v.bytes) {
         set_error("workspace has %zu bytes, %zu needed", workspace_bytes, v.bytes); return SPLASH_INVALID_ARG;
@@ -283,6 +287,7 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
     p.B = B; p.H = shape->num_heads * R; p.head_begin = vb; p.head_end = ve; p.q_rows = R;
     p.table_stride = shape->block_table_stride; p.num_pool_pages = shape->num_pool_pages;
     p.heads_per_group = t.heads_per_group; p.num_groups = t.num_groups; p.num_workers = t.num_workers;
+    p.pair_groups = t.pair_groups;
     p.softmax_scale = shape->softmax_scale;
     p.tile_start = v.tile_start; p.req_lo = v.req_lo; p.req_hi = v.req_hi; p.worker_begin = v.worker_begin;
     p.worker_req = v.worker_req;

@@ -108,6 +108,10 @@ struct DecodeParams {
                                // row r attends causally: tokens below seq_len - (R - 1 - r)
     int32_t heads_per_group;   // heads one CTA computes
     int32_t num_groups;        // head groups per KV worker
+    int32_t pair_groups;       // CTA-pair kernels: CTA pairs per KV worker (1; more when several query rows per request
+                               // make more than 128 (head, row) pairs: pair g of a worker takes pairs [128 g, 128 g + 128)
+                               // and the pairs of a worker stream the same pages side by side, so the second read of a
+                               // page hits L2 and the cache crosses HBM once)
     float softmax_scale;
     // plan (device pointers into the workspace)
     const int32_t *tile_start, *req_lo, *req_hi, *worker_begin;

@@ -103,8 +103,9 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
     const uint32_t sbase = smem_u32(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t rank = cluster_ctarank();             // 0 = leader: issues the MMAs
-    const int worker = blockIdx.x >> 1;
-    const int head0 = p.head_begin + (int)rank * kN;
+    const int pair_id = blockIdx.x >> 1;                // CTA pair: (KV worker, group of 128 heads)
+    const int worker = pair_id / p.pair_groups;
+    const int head0 = p.head_begin + (pair_id % p.pair_groups) * (2 * kN) + (int)rank * kN;
     const int h = p.head_end - p.head_begin;
 
     volatile uint32_t *misc = reinterpret_cast<volatile uint32_t *>(smem + kOffMisc);
@@ -302,7 +303,7 @@ decode_umma_pair_kernel(const DecodeParams p, const __grid_constant__ CUtensorMa
         // the issuer warps of the peer CTA have nothing to do for the attention itself: they carry the call's page-copy
         // job, if it has one (a layer's pages on the move while this layer decodes)
         if (p.mig_n > 0)
-            copy_pages_in_idle_warp(p, worker * (kQkWarps + kPvWarps) + (warp - kWarpQk), p.num_workers * (kQkWarps + kPvWarps), lane);
+            copy_pages_in_idle_warp(p, pair_id * (kQkWarps + kPvWarps) + (warp - kWarpQk), p.num_workers * p.pair_groups * (kQkWarps + kPvWarps), lane);
     } else {
         // ===================================================== softmax + epilogue warps
         // S partial layout per CTA: TMEM lane L < 64 = head L, tokens of half-page 0 in 32 columns;
@@ -586,7 +587,7 @@ cudaError_t launch_decode_umma_pair(const DecodeParams &p, cudaStream_t stream) 
     cudaError_t e = once.run([&] { return cudaFuncSetAttribute(decode_umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes); });
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(p.num_workers * 2)); cfg.blockDim = dim3(kThreads);
+    cfg.gridDim = dim3((unsigned)(p.num_workers * p.pair_groups * 2)); cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;
     cudaLaunchAttribute attr[1];      // (the cluster shape is part of the kernel's declaration)
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -68,6 +68,9 @@ def compare_rows(out, lse, ref_out, ref_lse, kv_dtype, hb, he, what):
 @pytest.mark.parametrize("R,H,lens", [
     (2, 16, [2, 63, 64, 65, 128, 129, 1000]), (4, 16, [3, 4, 64, 66, 67, 300, 4097]), (8, 16, [5, 8, 65, 70, 200]),
     (2, 64, [1, 64, 65, 777]), (3, 40, [130, 64, 2, 5000]), (2, 128, [66, 1500, 64]), (4, 128, [131, 12345]),
+    # more than 128 (head, row) pairs: several CTA pairs per KV worker in one launch (8 x 128 = 1,024 pairs in 8 groups;
+    # 3 x 100 = 300 pairs in 3 groups, the last one partly filled)
+    (8, 128, [300, 70, 2000]), (3, 100, [129, 3000, 7]),
 ])
 def test_rows_match_the_oracle(flags, kv_dtype, R, H, lens):
     w = W.make_workload("rows", 800 + R + H, lens, H=H, kv_dtype=kv_dtype)
