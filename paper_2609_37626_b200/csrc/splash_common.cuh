@@ -262,6 +262,7 @@ int simt_heads_per_group();
 void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *num_groups, int *num_workers);
 cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &shape, cudaStream_t stream);
 cudaError_t launch_decode_umma_fp8(const DecodeParams &p, cudaStream_t stream);
+cudaError_t launch_decode_umma_fp8_narrow(const DecodeParams &p, cudaStream_t stream);   // 16 / 32 heads per CTA
 cudaError_t launch_decode_umma_fp8_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_decode_umma_pair(const DecodeParams &p, cudaStream_t stream);
 cudaError_t launch_split_combine(const DecodeParams &p, const int4 *split_rec, cudaStream_t stream);

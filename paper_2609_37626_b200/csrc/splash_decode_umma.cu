@@ -644,8 +644,8 @@ cudaError_t launch_n(const DecodeParams &p, const CUtensorMap &mkv, const CUtens
 }  // namespace
 
 void umma_tiling(int kv_dtype, int h, int sm_count, int *heads_per_group, int *num_groups, int *num_workers) {
-    // e4m3 KV always runs 64-head groups (narrower slices pad their group with zero heads)
-    const int n = kv_dtype == SPLASH_KV_E4M3_TOKEN_SCALE ? 64 : (h <= 16 ? 16 : (h <= 32 ? 32 : 64));
+    (void)kv_dtype;       // both cache formats have 16-, 32- and 64-head kernels
+    const int n = h <= 16 ? 16 : (h <= 32 ? 32 : 64);
     *heads_per_group = n;
     *num_groups = (h + n - 1) / n;
     const int w = sm_count / *num_groups;
@@ -659,7 +659,7 @@ cudaError_t launch_decode_umma(const DecodeParams &p, const splash_mla_shape &sh
             const cudaError_t e = launch_decode_umma_fp8_pair(p, stream);
             if (e != cudaErrorNotSupported) return e;      // output rows not 16-byte aligned: no TMA stores
         }
-        return launch_decode_umma_fp8(p, stream);
+        return p.heads_per_group < 64 ? launch_decode_umma_fp8_narrow(p, stream) : launch_decode_umma_fp8(p, stream);
     }
     if (p.num_groups == 2 && p.heads_per_group == 64 && !(shape.flags & SPLASH_FLAG_NO_PAIR)) return launch_decode_umma_pair(p, stream);
     alignas(64) CUtensorMap mkv, mq;

@@ -169,6 +169,19 @@ def test_fp8_kv(flags, lens):
     compare(out, lse, *ref, kv_dtype=1, what="fp8")
 
 
+# Narrow e4m3 slices run with the tokens on the MMA's M: 16 or 32 heads per CTA.  Widths that fill a group, widths
+# that leave it ragged, a slice in the middle of a wider layer, a request that many workers split, many short ones.
+@pytest.mark.parametrize("H,hb,he,lens", [
+    (32, 0, 32, [1, 17, 64, 200]), (24, 0, 24, [1000, 3, 4097]), (128, 48, 80, [333, 64, 129, 2000]),
+    (128, 100, 109, [65, 5000]), (32, 0, 32, [30000]), (16, 0, 16, [130] * 300), (20, 3, 20, list(range(1, 300, 5))),
+])
+def test_fp8_narrow_head_slices(H, hb, he, lens):
+    w = W.make_workload("fp8n", 740 + H + he + len(lens), lens, H=H, head_begin=hb, head_end=he, kv_dtype=1)
+    ref = oracle_run(w)
+    out, lse = gpu_run(w)
+    compare(out, lse, *ref, kv_dtype=1, rows=[(i, g) for i in range(len(lens)) for g in range(hb, he)], what="fp8 narrow")
+
+
 def test_fp8_extreme_rows(flags):
     w = W.make_workload("fp8x", 710, [200], H=16, kv_dtype=1)
     p = w.block_table[0, 0]

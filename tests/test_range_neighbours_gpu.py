@@ -42,8 +42,8 @@ def test_bf16_ranges_with_poisoned_neighbours(H, flags):
     compare(out, lse, *ref, kv_dtype=0, what=f"bf16 H={H} flags={flags}")
 
 
-# e4m3: the 64-head kernel (narrow slices pad their group), the CTA-pair kernel, two independent CTAs, SIMT
-@pytest.mark.parametrize("H,flags", [(16, 0), (64, 0), (128, 0), (128, 2), (16, 1), (96, 0)])
+# e4m3: 16 / 32 / 64 heads per CTA (24 and 40 pad their group), the CTA-pair kernel, two independent CTAs, SIMT
+@pytest.mark.parametrize("H,flags", [(16, 0), (24, 0), (32, 0), (40, 0), (64, 0), (128, 0), (128, 2), (16, 1), (96, 0)])
 def test_e4m3_ranges_with_poisoned_neighbours(H, flags):
     import torch
     w, kb, ke = make(H, 1, 4200 + H + flags)
