@@ -48,8 +48,9 @@ enum BarrierId {
     kBarQsRead,                   // the softmax warps have picked up the request's query scales
     kBarSFull,                    // [2]
     kBarSEmpty = kBarSFull + 2,   // [2]
-    kBarPFull = kBarSEmpty + 2,
-    kBarOFull,
+    kBarPFull = kBarSEmpty + 2,   // [2]: one per P buffer (the softmax warps may run two tiles ahead of a P.V issuer; with
+                                  // a single barrier two phases could complete between two of its polls)
+    kBarOFull = kBarPFull + 2,
     kBarOEmpty,
     kNumBarriers
 };
@@ -97,7 +98,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
         mbar_init(bar(kBarQFull), kNumConvertWarps); mbar_init(bar(kBarQEmpty), kQkWarps);
         mbar_init(bar(kBarQsRead), kNumSoftmaxWarps);
         for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxWarps); }
-        mbar_init(bar(kBarPFull), kNumSoftmaxWarps);
+        for (int b = 0; b < 2; ++b) mbar_init(bar(kBarPFull + b), kNumSoftmaxWarps);
         mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxWarps);
         misc[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -232,7 +233,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 const int ntiles = seg.tile_end - seg.tile_begin;
                 for (int i = 0; ok && i < ntiles; ++i, ++kv) {
                     const uint32_t stage = kv % kStages;
-                    ok = mbar_wait(ctx, bar(kBarPFull), kv & 1, kBarPFull);
+                    ok = mbar_wait(ctx, bar(kBarPFull + (kv & 1)), (kv >> 1) & 1, kBarPFull + (kv & 1));
                     if (ok && i == 0) ok = mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty);
                     if (!ok) break;
                     if (pj == 0) mark(kv, 6);
@@ -471,7 +472,7 @@ decode_umma_fp8_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap
                 tcgen05_fence_before();
                 if (st == 0) mark(s_it, 5);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPFull));
+                if (lane == 0) mbar_arrive(bar(kBarPFull + (s_it & 1)));
                 ++s_it;
             }
             // ---- row sums: the 4 threads of a row, then the two token halves

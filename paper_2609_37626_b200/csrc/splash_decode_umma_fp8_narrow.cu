@@ -4,24 +4,35 @@
 // softmax work; here the problem is transposed ("tokens on M"), as in the bf16 kernel's narrow
 // path, so that a 16-head slice costs 16-wide MMAs:
 //
-//     S^T [64 tokens x N heads]  = K_tile [64 x 576]   * (q_hi + q_lo)^T [576 x N]     (M = 64, K = 32)
-//     O^T [512 dv    x N heads] += V_tile^T [512 x 64] * (P_hi + P_lo)^T [64 x N]      (4 x M = 128)
+//     S^T [64 tokens x 2N]       = K_tile [64 x 576]   * [q_hi | q_lo]^T [576 x 2N]    (M = 64, K = 32)
+//     O^T [512 dv    x 2N]      += V_tile^T [512 x 64] * [P_hi | 16 P_lo]^T [64 x 2N]  (4 x M = 128)
 //
 // The cache bytes go to the tensor cores as stored (kind::f8f6f4); V is the first 512 columns of the
 // very K rows in shared memory, read as an MN-major operand.  The two bf16-precision operands are
 // split into two 8-bit terms each, exactly as in the 64-head kernel: q = qs_h (hi + lo) with one
-// scale per head (e4m3 + e4m3, rebuilt per request by converter warps one request ahead), and
-// P = hi + lo (e4m3 + e5m2) with the token scale folded into the weight in the log domain,
+// scale per head (e4m3 + e4m3, rebuilt per request by converter warps one request ahead; the two
+// terms sit side by side as 2N rows of one B operand and the softmax warps add the two halves of
+// S^T), and P = hi + lo with the token scale folded into the weight in the log domain,
 //     y = (q . codes) * qs_h * scale_t * softmax_scale * log2(e) + log2(scale_t),   P = 2^(y - m + 4.75),
-// the row sum adding P / scale_t.  With the tokens on the TMEM lanes the token scale is one
-// number per thread.  A page is 36,864 bytes and the query operands are small, so five stages
-// fit: the loop is a ring of dependent latencies and its period is the ring divided by the stages.
+// the row sum adding P / scale_t.  Here the two terms of P are 2N columns of ONE B operand too, so that the
+// V tile -- the operand whose read from shared memory sets the pace of these narrow MMAs -- is read once
+// per tile instead of twice; O^T then has a hi and a lo half that the epilogue adds, which lets the lo
+// term carry its own scale: it is stored as e4m3 of 16 x the residual (three significant bits, never out
+// of range since an e4m3 residual is at most 2^-4 of the value) and the epilogue adds lo / 16.  With the tokens on the TMEM lanes the token scale is one
+// number per thread, and a thread's weights for its token are N adjacent bytes of an MN-major
+// P^T: one 16-byte store per 16 heads.  A page is 36,864 bytes and the query operands are small,
+// so five stages fit: the loop is a ring of dependent latencies and its period is the ring divided
+// by the stages.
 //
-// Warp roles (352 threads): TMA producer (pages + scale pages, next page pulled into L2), 4 MMA
-// issuers (one S^T partial accumulator and one dv block each, ready-driven), 4 softmax / epilogue
-// warps (per-head maxima and sums by a warp-shuffle reduce-scatter plus a small exchange), 2 query
-// converter warps.  Every wait is bounded; on expiry the CTA records SPLASH_DEVICE_TIMEOUT and leaves
-// in order.
+// The softmax warps keep one reference maximum per head and move it only when a logit exceeds it by
+// more than 2^4 (the headroom that e4m3's range leaves above the lift): whether any does is one
+// barrier-wide OR per tile, and only then do they reduce the maxima across tokens, move the
+// references and rescale O^T.  Row sums stay per thread until the request ends.
+//
+// Warp roles (352 threads): TMA producer (pages + scale pages, next page pulled into L2), 2 QK^T
+// issuers (one partial accumulator of S^T each), 2 P.V issuers (two dv blocks each), 4 softmax /
+// epilogue warps, 2 query converter warps.  Every wait is bounded; on expiry the CTA records
+// SPLASH_DEVICE_TIMEOUT and leaves in order.
 #include "splash_fp8.cuh"
 #include "splash_pair.cuh"
 
@@ -31,11 +42,13 @@ namespace {
 
 using namespace umma;
 
-constexpr int kMmaWarps = 4;
+constexpr int kQkWarps = 2;                        // = partial accumulators of S^T
+constexpr int kPvWarps = 2;                        // each owns two of the four dv blocks of O^T
 constexpr int kNumSoftmaxWarps = 4;
 constexpr int kNumConvertWarps = 2;
-constexpr int kWarpMma = 1;
-constexpr int kWarpSoftmax = kWarpMma + kMmaWarps;          // 5: TMEM lane quadrant = warp & 3
+constexpr int kWarpQk = 1;
+constexpr int kWarpPv = kWarpQk + kQkWarps;
+constexpr int kWarpSoftmax = kWarpPv + kPvWarps;            // 5: TMEM lane quadrant = warp & 3
 constexpr int kWarpConvert = kWarpSoftmax + kNumSoftmaxWarps;
 constexpr int kThreads = (kWarpConvert + kNumConvertWarps) * 32;   // 11 warps = 352 threads
 constexpr int kChunks = 9;                         // 576 / 64-element (64 B) chunks
@@ -54,39 +67,44 @@ enum BarrierId {
     kBarQsRead,                        // the softmax warps have picked up the request's query scales
     kBarSFull,                         // [2]
     kBarSEmpty = kBarSFull + 2,        // [2]
-    kBarPFull = kBarSEmpty + 2,
-    kBarOFull,
+    kBarPFull = kBarSEmpty + 2,        // [2]: one per P buffer.  With a single barrier the softmax warps, which may run two
+                                       // tiles ahead of a P.V issuer, could complete two phases between two of its polls
+    kBarOFull = kBarPFull + 2,
     kBarOEmpty,
     kNumBarriers
 };
 
 template <int N>
 struct Layout {
-    static constexpr uint32_t kQSlab = N * 64;                 // one chunk of the query operand: N heads x 64 B
-    static constexpr uint32_t kQBytes = kChunks * kQSlab;      // one term (hi or lo)
-    static constexpr uint32_t kPBytes = N * 64;                // one term of P^T: N heads x 64 tokens, one byte each
+    static constexpr uint32_t kQSlab = 2 * N * 64;             // one chunk of the query operand: (N hi rows, N lo rows) x 64 B
+    static constexpr uint32_t kQBytes = kChunks * kQSlab;
+    static constexpr uint32_t kPBytes = 2 * N * 64;            // P^T: [2N / 16 groups: hi, then lo][64 tokens][16 heads], one byte each
     static constexpr uint32_t kOffKv = 0;
-    static constexpr uint32_t kOffQHi = kOffKv + kStages * kStageBytes;
-    static constexpr uint32_t kOffQLo = kOffQHi + kQBytes;
-    static constexpr uint32_t kOffPHi = kOffQLo + kQBytes;
-    static constexpr uint32_t kOffPLo = kOffPHi + kPBytes;
-    static constexpr uint32_t kOffScale = kOffPLo + kPBytes;   // float [kStages][64]
+    static constexpr uint32_t kOffQ = kOffKv + kStages * kStageBytes;
+    static constexpr uint32_t kOffP = kOffQ + kQBytes;         // double buffered (tile parity)
+    static constexpr uint32_t kOffScale = kOffP + 2 * kPBytes; // float [kStages][64]
     static constexpr uint32_t kOffQs = kOffScale + kStages * kScaleBytes;   // float [4][N] query scales, by segment & 3
     static constexpr uint32_t kOffRed = kOffQs + 4 * N * 4;    // float [N][4]
-    static constexpr uint32_t kOffM = kOffRed + N * 16;        // float [N] running max, log2 domain
+    static constexpr uint32_t kOffM = kOffRed + N * 16;        // float [N] reference maxima, log2 domain
     static constexpr uint32_t kOffAlpha = kOffM + N * 4;       // float [N]
     static constexpr uint32_t kOffL = kOffAlpha + N * 4;       // float [N]
     static constexpr uint32_t kOffBar = kOffL + N * 4;
-    static constexpr uint32_t kOffMisc = (kOffBar + kNumBarriers * 8 + 15) / 16 * 16;   // u32: tmem base, abort, rescale flags
+    static constexpr uint32_t kOffMisc = (kOffBar + kNumBarriers * 8 + 15) / 16 * 16;   // u32: tmem base, abort
     static constexpr uint32_t kBytes = kOffMisc + 16;
-    static constexpr int kAcc = 4;                             // partial accumulators of S^T = issuers that take part in QK^T
-    static constexpr int kSBufs = 2;
-    static constexpr uint32_t kColO = 0;                       // 4 dv blocks x N columns
-    static constexpr uint32_t kColS = 4 * N;                   // kSBufs x kAcc x N columns
-    static_assert(kColS + kSBufs * kAcc * N <= 512, "tensor memory overflow");
+    static constexpr uint32_t kColO = 0;                       // 4 dv blocks x (N hi, N lo) columns
+    static constexpr uint32_t kColS = 8 * N;                   // 2 buffers x kQkWarps partials x (N hi, N lo) columns
+    static_assert(kColS + 2 * kQkWarps * 2 * N <= 512, "tensor memory overflow");
     static_assert(kBytes <= 232448, "shared memory overflow");
-    static_assert(kOffQHi % 1024 == 0 && kQSlab % 512 == 0 && kOffPHi % 512 == 0 && kPBytes % 512 == 0, "swizzle atoms need aligned windows");
+    static_assert(kOffQ % 1024 == 0 && kQSlab % 512 == 0 && kOffP % 128 == 0, "operands need aligned windows");
 };
+
+// Shared-memory matrix descriptor without swizzle (layout type 0), for the MN-major P^T: 16 heads of one token
+// are 16 adjacent bytes, eight tokens make a 128-byte core matrix, `k_group_bytes` leads from one group of eight
+// tokens to the next and `mn_group_bytes` from one group of 16 heads to the next.
+__device__ __forceinline__ uint64_t make_desc_mn_plain(uint32_t saddr, uint32_t k_group_bytes, uint32_t mn_group_bytes) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((k_group_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((mn_group_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
 
 // Reduce-scatter over the 32 lanes of a warp (see the bf16 kernel): on return lane L holds, in v[0 .. max(1, N/32)),
 // the reduction over all lanes of the entries it owns (N = 32: head L; N = 16: head L >> 1, both lanes of a pair).
@@ -140,13 +158,13 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
         return;
     }
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kMmaWarps); }
-        mbar_init(bar(kBarQFull), kNumConvertWarps); mbar_init(bar(kBarQEmpty), L::kAcc);
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kPvWarps); }
+        mbar_init(bar(kBarQFull), kNumConvertWarps); mbar_init(bar(kBarQEmpty), kQkWarps);
         mbar_init(bar(kBarQsRead), kNumSoftmaxWarps);
-        for (int b = 0; b < L::kSBufs; ++b) { mbar_init(bar(kBarSFull + b), L::kAcc); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxWarps); }
-        mbar_init(bar(kBarPFull), kNumSoftmaxWarps);
-        mbar_init(bar(kBarOFull), kMmaWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxWarps);
-        misc[1] = 0; misc[2] = 0; misc[3] = 0;
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxWarps); }
+        for (int b = 0; b < 2; ++b) mbar_init(bar(kBarPFull + b), kNumSoftmaxWarps);
+        mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxWarps);
+        misc[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
@@ -228,96 +246,73 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 ++kv_it;
             }
         }
-    } else if (warp >= kWarpMma && warp < kWarpMma + kMmaWarps) {
-        // ===================================================== MMA issuers
+    } else if (warp < kWarpPv) {
+        // ===================================================== QK^T issuers: S^T = K [q hi | q lo]^T
         if (lane == 0) {
-            const int mw = warp - kWarpMma;          // issuer index: S^T accumulator mw, dv block mw
-            constexpr uint32_t kIdescQK = make_idesc_e4m3(64, N, 0);
-            // the low-order term of P is e5m2 (the B operand here)
-            constexpr uint32_t kIdescPV = make_idesc_e4m3(128, N, 1), kIdescPVLo = make_idesc_e4m3(128, N, 1, 1);
-            uint32_t kv_it = 0, s_it = 0, p_it = 0, seg_it = 0;
+            const int a = warp - kWarpQk;            // partial accumulator a
+            constexpr uint32_t kIdescQK = make_idesc_e4m3(64, 2 * N, 0);
+            uint32_t kv = 0, seg_it = 0;
             bool ok = true;
-            // This issuer's share of S^T for the tile with global index kv: steps idx = mw, mw + 4, ... of the
-            // 36 (18 K = 32 steps x (q hi, q lo)), into partial accumulator mw.
-            auto issue_qk = [&](uint32_t kv, uint32_t sidx) {
-                const uint32_t stage = kv % kStages, b = sidx % L::kSBufs;
-                if (mw == 0) mark(kv, 2);
-                tcgen05_fence_after();
-                const uint32_t k0 = sbase + L::kOffKv + stage * kStageBytes;
-                const uint32_t d = tmem_base + L::kColS + (b * L::kAcc + mw) * N;
-#pragma unroll
-                for (int t = 0; t < 36 / L::kAcc; ++t) {
-                    const int idx = t * L::kAcc + mw, hl = idx / 18, ks = idx % 18, c = ks >> 1, k = ks & 1;
-                    const uint32_t q0 = sbase + (hl ? L::kOffQLo : L::kOffQHi);
-                    uint64_t dk = make_desc_sw64(k0 + c * kSlab + k * 32, 16, 512);          // A: 64 tokens x 32
-                    uint64_t dq = make_desc_sw64(q0 + c * L::kQSlab + k * 32, 16, 512);      // B: N heads x 32
-                    umma_e4m3(d, dk, dq, kIdescQK, t != 0);
-                }
-                umma_commit(bar(kBarSFull + b));
-                if (mw == 0) mark(kv, 3);
-            };
-            // O^T block mw += V^T block mw (128 dv x 64 tokens) * (P hi + P lo)^T: 2 K = 32 steps x 2 terms
-            auto issue_pv = [&](uint32_t stage, bool first_tile) {
-                tcgen05_fence_after();
-                const uint32_t v0 = sbase + L::kOffKv + stage * kStageBytes + (2 * mw) * kSlab;
-#pragma unroll
-                for (int hl = 0; hl < 2; ++hl) {
-#pragma unroll
-                    for (int k = 0; k < 2; ++k) {
-                        // A: two 64-element chunks (LBO apart) x 32 tokens (SBO per 8 tokens), MN-major
-                        uint64_t da = make_desc_sw64(v0 + k * 2048, kSlab, 512);
-                        uint64_t db = make_desc_sw64(sbase + (hl ? L::kOffPLo : L::kOffPHi) + k * 32, 16, 512);
-                        umma_e4m3(tmem_base + L::kColO + mw * N, da, db, hl ? kIdescPVLo : kIdescPV, (!first_tile) || (hl | k) != 0);
-                    }
-                }
-            };
             while (ok && it.next(p, seg)) {
                 const int ntiles = seg.tile_end - seg.tile_begin;
                 ok = mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
-                if (!ok) break;
-                // Issue whatever is ready: P.V of tile pv_i (frees a stage) or QK^T of tile qk_i (at most two tiles
-                // ahead of the softmax: two S buffers).
-                int qk_i = 0, pv_i = 0;
-                unsigned long long idle_since = 0;
-                uint32_t idle_polls = 0;
-                while (pv_i < ntiles) {
-                    bool progressed = false;
-                    if ((qk_i > pv_i) && mbar_test_wait(bar(kBarPFull), (p_it + pv_i) & 1)) {
-                        if (pv_i == 0 && !mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty)) { ok = false; break; }
-                        if (mw == 0) mark(kv_it + pv_i, 6);
-                        const uint32_t stage = (kv_it + pv_i) % kStages;
-                        issue_pv(stage, pv_i == 0);
-                        umma_commit(bar(kBarKvEmpty + stage));   // P.V done: stage free, P buffers free, O^T updated
-                        if (pv_i + 1 == ntiles) umma_commit(bar(kBarOFull));
-                        if (mw == 0) mark(kv_it + pv_i, 7);
-                        ++pv_i;
-                        progressed = true;
+                for (int i = 0; ok && i < ntiles; ++i, ++kv) {
+                    const uint32_t stage = kv % kStages, b = kv & 1;
+                    ok = mbar_wait(ctx, bar(kBarKvFull + stage), (kv / kStages) & 1, kBarKvFull + stage) &&
+                         mbar_wait(ctx, bar(kBarSEmpty + b), ((kv >> 1) & 1) ^ 1, kBarSEmpty + b);
+                    if (!ok) break;
+                    if (a == 0) mark(kv, 2);
+                    tcgen05_fence_after();
+                    const uint32_t k0 = sbase + L::kOffKv + stage * kStageBytes;
+                    const uint32_t d = tmem_base + L::kColS + (b * kQkWarps + a) * (2 * N);
+                    // 18 K = 32 steps per tile; this issuer takes every second
+#pragma unroll
+                    for (int t = 0; t < 18 / kQkWarps; ++t) {
+                        const int ks = t * kQkWarps + a, c = ks >> 1, k = ks & 1;
+                        uint64_t dk = make_desc_sw64(k0 + c * kSlab + k * 32, 16, 512);                      // A: 64 tokens x 32
+                        uint64_t dq = make_desc_sw64(sbase + L::kOffQ + c * L::kQSlab + k * 32, 16, 512);    // B: 2N rows x 32
+                        umma_e4m3(d, dk, dq, kIdescQK, t != 0);
                     }
-                    if (qk_i < ntiles && qk_i < pv_i + 2) {
-                        const uint32_t kv = kv_it + qk_i, sidx = s_it + qk_i;
-                        if (mbar_test_wait(bar(kBarKvFull + kv % kStages), (kv / kStages) & 1) &&
-                            mbar_test_wait(bar(kBarSEmpty + sidx % L::kSBufs), ((sidx / L::kSBufs) & 1) ^ 1)) {
-                            issue_qk(kv, sidx);
-                            ++qk_i;
-                            if (qk_i == ntiles) umma_commit(bar(kBarQEmpty));
-                            progressed = true;
-                        }
-                    }
-                    if (progressed) { idle_since = 0; idle_polls = 0; continue; }
-                    if ((++idle_polls & 255u) != 0u) continue;
-                    if (*ctx.abort_flag) { ok = false; break; }
-                    const unsigned long long now = global_timer_ns();
-                    if (idle_since == 0) idle_since = now;
-                    else if (now - idle_since > kWaitLimitNs) {
-                        *ctx.abort_flag = 1;
-                        if (atomicCAS(ctx.status, 0, (int)SPLASH_DEVICE_TIMEOUT) == 0) {
-                            ctx.status[1] = (int)blockIdx.x; ctx.status[2] = 100 + (qk_i > pv_i ? kBarPFull : kBarKvFull);
-                            ctx.status[3] = pv_i;
-                        }
-                        ok = false; break;
-                    }
+                    umma_commit(bar(kBarSFull + b));
+                    if (a == 0) mark(kv, 3);
                 }
-                kv_it += ntiles; s_it += ntiles; p_it += ntiles;
+                if (ok) umma_commit(bar(kBarQEmpty));
+                ++seg_it;
+            }
+        }
+    } else if (warp < kWarpSoftmax) {
+        // ===================================================== P.V issuers: [O^T hi | O^T lo] += V^T [P hi | 16 P lo]^T
+        if (lane == 0) {
+            const int pj = warp - kWarpPv;           // dv blocks 2 pj and 2 pj + 1
+            constexpr uint32_t kIdescPV = make_idesc_e4m3(128, 2 * N, 1, 0, 1);
+            uint32_t kv = 0, seg_it = 0;
+            bool ok = true;
+            while (ok && it.next(p, seg)) {
+                const int ntiles = seg.tile_end - seg.tile_begin;
+                for (int i = 0; ok && i < ntiles; ++i, ++kv) {
+                    const uint32_t stage = kv % kStages;
+                    ok = mbar_wait(ctx, bar(kBarPFull + (kv & 1)), (kv >> 1) & 1, kBarPFull + (kv & 1));
+                    if (ok && i == 0) ok = mbar_wait(ctx, bar(kBarOEmpty), (seg_it & 1) ^ 1, kBarOEmpty);
+                    if (!ok) break;
+                    if (pj == 0) mark(kv, 6);
+                    tcgen05_fence_after();
+                    const uint32_t v0 = sbase + L::kOffKv + stage * kStageBytes;
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+#pragma unroll
+                        for (int jj = 0; jj < 2; ++jj) {
+                            const int j = 2 * pj + jj;
+                            // A: two 64-element chunks (LBO apart) x 32 tokens (SBO per 8 tokens), MN-major
+                            uint64_t da = make_desc_sw64(v0 + (2 * j) * kSlab + k * 2048, kSlab, 512);
+                            // B: 32 tokens (four groups of eight, 128 B apart) x 2N columns (groups of 16, 1024 B apart)
+                            uint64_t db = make_desc_mn_plain(sbase + L::kOffP + (kv & 1) * L::kPBytes + k * 512, 128, 1024);
+                            umma_e4m3(tmem_base + L::kColO + j * (2 * N), da, db, kIdescPV, (i != 0) || k != 0);
+                        }
+                    }
+                    umma_commit(bar(kBarKvEmpty + stage));   // P.V done: stage free, P buffers free, O^T updated
+                    if (i + 1 == ntiles) umma_commit(bar(kBarOFull));
+                    if (pj == 0) mark(kv, 7);
+                }
                 ++seg_it;
             }
         }
@@ -370,10 +365,11 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                     split_e4m3_e4m3_x2(e0, e1, hi[k], lo[k]);
                 }
                 const uint32_t d = (uint32_t)(part * (kVecs * 8) + v * 8);
+                // the lo rows follow the N hi rows of the chunk (N is a multiple of 8: same swizzle phase)
                 const uint32_t off = (d >> 6) * L::kQSlab + sw64((uint32_t)hd, d & 63);
-                *reinterpret_cast<uint2 *>(smem + L::kOffQHi + off) =
+                *reinterpret_cast<uint2 *>(smem + L::kOffQ + off) =
                     make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
-                *reinterpret_cast<uint2 *>(smem + L::kOffQLo + off) =
+                *reinterpret_cast<uint2 *>(smem + L::kOffQ + N * 64 + off) =
                     make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
             }
             fence_proxy_async();
@@ -412,81 +408,114 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarQsRead));
             if (st < N) m_s[st] = -INFINITY;
-            float l_own = 0.f;            // running sum of the head this lane owns (this warp's 16 tokens)
+            float l[N];                   // running sums of P / scale_t over this thread's tokens, one per head
+#pragma unroll
+            for (int n = 0; n < N; ++n) l[n] = 0.f;
             softmax_bar_sync();
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;
             for (int i = 0; i < ntiles; ++i) {
                 const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + seg.tile_begin + i) * kPage);
                 const bool valid = lane < 16 && row >= g.r_lo && row < g.r_hi;
-                const uint32_t b = s_it % L::kSBufs, stage = s_it % kStages;
-                ok &= mbar_wait(ctx, bar(kBarSFull + b), (s_it / L::kSBufs) & 1, kBarSFull + b);
+                const uint32_t b = s_it & 1, stage = s_it % kStages;
+                ok &= mbar_wait(ctx, bar(kBarSFull + b), (s_it >> 1) & 1, kBarSFull + b);
                 if (st == 0) mark(s_it, 4);
                 // the scale page rode on the stage's own barrier, long complete by now
                 ok &= mbar_wait(ctx, bar(kBarKvFull + stage), (s_it / kStages) & 1, kBarKvFull + stage);
                 tcgen05_fence_after();
                 float s[N];
                 {
-                    const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (L::kAcc * N);
+                    // S^T = the sum of four N-column pieces: (partial 0, partial 1) x (q hi, q lo)
+                    float t0[N], t1[N];
+                    const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (2 * kQkWarps * N);
 #pragma unroll
-                    for (int c = 0; c < N / 16; ++c)
+                    for (int c = 0; c < N / 16; ++c) {
                         tmem_ld16(sb + c * 16, *reinterpret_cast<float(*)[16]>(&s[c * 16]));
-#pragma unroll
-                    for (int a = 1; a < L::kAcc; ++a) {
-                        float part[N];
-#pragma unroll
-                        for (int c = 0; c < N / 16; ++c)
-                            tmem_ld16(sb + a * N + c * 16, *reinterpret_cast<float(*)[16]>(&part[c * 16]));
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int n = 0; n < N; ++n) s[n] += part[n];
+                        tmem_ld16(sb + N + c * 16, *reinterpret_cast<float(*)[16]>(&t0[c * 16]));
                     }
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int n = 0; n < N; ++n) s[n] += t0[n];
+#pragma unroll
+                    for (int c = 0; c < N / 16; ++c) {
+                        tmem_ld16(sb + 2 * N + c * 16, *reinterpret_cast<float(*)[16]>(&t0[c * 16]));
+                        tmem_ld16(sb + 3 * N + c * 16, *reinterpret_cast<float(*)[16]>(&t1[c * 16]));
+                    }
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int n = 0; n < N; ++n) s[n] += t0[n] + t1[n];
                 }
-                tmem_wait_ld();
                 tcgen05_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarSEmpty + b));
                 // this thread's token: its scale, log2 of it for the weight, its reciprocal for the row sums
                 const float ts = valid ? scale_s[stage * 64 + g.tok0 + row] : 1.0f;
                 const float lg = fast_log2(ts), rts = fast_rcp(ts), tsl = ts * scale_log2;
-                float mx[N];
+                bool exceeds = false;     // some logit of this token lies more than kTau above its head's reference
 #pragma unroll
-                for (int n = 0; n < N; ++n) {
-                    s[n] = valid ? fmaf(s[n] * qs_s[n], tsl, lg) : -INFINITY;      // log2-domain logit + log2(token scale)
-                    mx[n] = s[n];
-                }
-                ReduceScatter<N, 16, true>::run(mx, lane);
-                if (N >= 32 || (lane & 1) == 0) red[owned_head<N>(lane) * 4 + sw] = mx[0];
-                if (st == 0) misc[2 + (i & 1)] = 0;      // this tile's "some maximum grew" flag
-                softmax_bar_sync();
-                if (st < N) {
-                    float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
-                    float mt = fmaxf(fmaxf(r4.x, r4.y), fmaxf(r4.z, r4.w));
-                    float m_old = m_s[st];
-                    float al = 1.f;
-                    if (mt > m_old + kTau) {        // also taken when m_old = -inf
-                        al = (m_old == -INFINITY) ? 0.f : fast_exp2(m_old - mt);
-                        m_s[st] = mt;
-                        misc[2 + (i & 1)] = 1;
+                for (int n4 = 0; n4 < N; n4 += 4) {
+                    const float4 q4v = *reinterpret_cast<const float4 *>(&qs_s[n4]);
+                    const float4 m4 = *reinterpret_cast<const float4 *>(&m_s[n4]);
+                    const float qv[4] = {q4v.x, q4v.y, q4v.z, q4v.w}, mv[4] = {m4.x, m4.y, m4.z, m4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float y = valid ? fmaf(s[n4 + e] * qv[e], tsl, lg) : -INFINITY;   // log2-domain logit + log2(token scale)
+                        s[n4 + e] = y;
+                        exceeds |= y > mv[e] + kTau;
                     }
-                    alpha_s[st] = al;
                 }
-                softmax_bar_sync();
-                const bool rescale = misc[2 + (i & 1)] != 0;
-                if (rescale) l_own *= alpha_s[owned_head<N>(lane)];
+                const bool grew = softmax_bar_or(exceeds);
+                if (grew) {
+                    // the rare path (the first tile of a request, then a handful of times): per-head maxima over the
+                    // tile's tokens, new references for the heads that grew, their rescale factors
+                    float mx[N];
 #pragma unroll
-                for (int n = 0; n < N; ++n) { s[n] = fast_exp2(s[n] - m_s[n] + kLift); mx[n] = s[n] * rts; }
-                ReduceScatter<N, 16, false>::run(mx, lane);      // per-head sums of P / scale_t over this warp's tokens
-                l_own += mx[0];
-                // P.V of the previous tile must be done with the P buffers and with O^T
-                if (s_it > 0) {
-                    const uint32_t prev = s_it - 1;
+                    for (int n = 0; n < N; ++n) mx[n] = s[n];
+                    ReduceScatter<N, 16, true>::run(mx, lane);
+                    if (N >= 32 || (lane & 1) == 0) red[owned_head<N>(lane) * 4 + sw] = mx[0];
+                    softmax_bar_sync();
+                    if (st < N) {
+                        float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
+                        float mt = fmaxf(fmaxf(r4.x, r4.y), fmaxf(r4.z, r4.w));
+                        float m_old = m_s[st];
+                        float al = 1.f;
+                        if (mt > m_old + kTau) {        // also taken when m_old = -inf
+                            al = (m_old == -INFINITY) ? 0.f : fast_exp2(m_old - mt);
+                            m_s[st] = mt;
+                        }
+                        alpha_s[st] = al;
+                    }
+                    softmax_bar_sync();
+#pragma unroll
+                    for (int n = 0; n < N; ++n) l[n] *= alpha_s[n];
+                }
+                uint32_t phi[N / 4], plo[N / 4];      // four heads' bytes per word
+#pragma unroll
+                for (int n4 = 0; n4 < N; n4 += 4) {
+                    const float4 m4 = *reinterpret_cast<const float4 *>(&m_s[n4]);
+                    const float w0 = fast_exp2(s[n4 + 0] - m4.x + kLift), w1 = fast_exp2(s[n4 + 1] - m4.y + kLift);
+                    const float w2 = fast_exp2(s[n4 + 2] - m4.z + kLift), w3 = fast_exp2(s[n4 + 3] - m4.w + kLift);
+                    l[n4 + 0] = fmaf(w0, rts, l[n4 + 0]); l[n4 + 1] = fmaf(w1, rts, l[n4 + 1]);
+                    l[n4 + 2] = fmaf(w2, rts, l[n4 + 2]); l[n4 + 3] = fmaf(w3, rts, l[n4 + 3]);
+                    // hi = the e4m3 value nearest to the weight, lo = 16 x what is left, e4m3 again
+                    uint16_t h01, l01, h23, l23;
+                    split_e4m3_e4m3x16_x2(w0, w1, h01, l01);
+                    split_e4m3_e4m3x16_x2(w2, w3, h23, l23);
+                    phi[n4 / 4] = (uint32_t)h01 | ((uint32_t)h23 << 16);
+                    plo[n4 / 4] = (uint32_t)l01 | ((uint32_t)l23 << 16);
+                }
+                // the P.V that read this P buffer (two tiles back) must be done; a rescale of O^T also needs the
+                // previous tile's P.V
+                if (s_it > 1) {
+                    const uint32_t prev = s_it - 2;
                     ok &= mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
                 }
-                tcgen05_fence_after();
-                if (rescale && i > 0) {
+                if (grew && i > 0) {
+                    const uint32_t prev = s_it - 1;
+                    ok &= mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
+                    tcgen05_fence_after();
 #pragma unroll 1
-                    for (int c = 0; c < 4 * N / 16; ++c) {
+                    for (int c = 0; c < 8 * N / 16; ++c) {
                         float o[16];
                         const uint32_t addr = tmem_base + lane_addr + L::kColO + c * 16;
                         tmem_ld16(addr, o);
@@ -498,27 +527,25 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                     tmem_wait_st();
                 }
                 if (lane < 16) {
-                    // P^T hi / lo as K-major, 64-byte-swizzled B operands: row = head, byte = token.
-                    // hi = the e4m3 value nearest to the weight, lo = what is left, kept as e5m2.
-                    uint8_t *ph = smem + L::kOffPHi, *pl = smem + L::kOffPLo;
+                    // P^T hi / lo, MN-major: the 16 heads of a group are the 16 bytes of this token's row
+                    uint8_t *ph = smem + L::kOffP + (s_it & 1) * L::kPBytes + row * 16;
+                    uint8_t *pl = ph + (N / 16) * 1024;
 #pragma unroll
-                    for (int n = 0; n < N; n += 2) {
-                        uint16_t hi2, lo2;
-                        split_e4m3_e5m2_x2(s[n], s[n + 1], hi2, lo2);
-                        const uint32_t off = sw64((uint32_t)n, (uint32_t)row);     // head n + 1: same swizzle phase, 64 B on
-                        ph[off] = (uint8_t)(hi2 & 0xffu); ph[off + 64] = (uint8_t)(hi2 >> 8);
-                        pl[off] = (uint8_t)(lo2 & 0xffu); pl[off + 64] = (uint8_t)(lo2 >> 8);
+                    for (int gq = 0; gq < N / 16; ++gq) {
+                        *reinterpret_cast<uint4 *>(ph + gq * 1024) = make_uint4(phi[4 * gq], phi[4 * gq + 1], phi[4 * gq + 2], phi[4 * gq + 3]);
+                        *reinterpret_cast<uint4 *>(pl + gq * 1024) = make_uint4(plo[4 * gq], plo[4 * gq + 1], plo[4 * gq + 2], plo[4 * gq + 3]);
                     }
                 }
                 fence_proxy_async();
                 tcgen05_fence_before();
                 if (st == 0) mark(s_it, 5);
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(kBarPFull));
+                if (lane == 0) mbar_arrive(bar(kBarPFull + (s_it & 1)));
                 ++s_it;
             }
-            // ---- row sums over all four warps' partial sums
-            if (N >= 32 || (lane & 1) == 0) red[owned_head<N>(lane) * 4 + sw] = l_own;
+            // ---- row sums: over the 16 tokens of a warp, then over the four warps
+            ReduceScatter<N, 16, false>::run(l, lane);
+            if (N >= 32 || (lane & 1) == 0) red[owned_head<N>(lane) * 4 + sw] = l[0];
             softmax_bar_sync();
             if (st < N) {
                 float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
@@ -550,13 +577,14 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 const int dv = 128 * j + 32 * q4 + lane;
 #pragma unroll
                 for (int c = 0; c < N / 16; ++c) {
-                    float o[16];
-                    tmem_ld16(tmem_base + lane_addr + L::kColO + j * N + c * 16, o);
+                    float o[16], o_lo[16];
+                    tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + c * 16, o);
+                    tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + N + c * 16, o_lo);
                     tmem_wait_ld();
 #pragma unroll
                     for (int k = 0; k < 16; ++k) {
                         const int n = c * 16 + k;
-                        if (n < nvalid) obase[(int64_t)n * ostride + dv] = o[k] * l_s[n];
+                        if (n < nvalid) obase[(int64_t)n * ostride + dv] = fmaf(o_lo[k], 0.0625f, o[k]) * l_s[n];
                     }
                 }
             }

@@ -66,6 +66,18 @@ __device__ __forceinline__ void split_e4m3_e4m3_x2(float lo, float hi, uint16_t 
     asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(res) : "r"(h2), "r"(back));
     asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(rest) : "r"(res));
 }
+// Two floats -> (e4m3 pair, e4m3 pair of 16 x the residuals): the residual of an e4m3 rounding is at most 2^-4 of
+// the value, so 16 x residual fits the format whenever the value does, and keeps three significant bits.  For kernels
+// that accumulate the two terms separately and add them as hi + lo / 16.
+__device__ __forceinline__ void split_e4m3_e4m3x16_x2(float lo, float hi, uint16_t &main, uint16_t &rest) {
+    uint32_t h2, back, res;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h2) : "f"(hi), "f"(lo));
+    asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(main) : "r"(h2));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(back) : "h"(main));
+    asm("sub.rn.f16x2 %0, %1, %2;" : "=r"(res) : "r"(h2), "r"(back));
+    asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(res) : "r"(res), "r"(0x4C004C00u));     // x 16
+    asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(rest) : "r"(res));
+}
 __device__ __forceinline__ float fast_log2(float x) {
     float y;
     asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

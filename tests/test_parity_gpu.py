@@ -76,6 +76,22 @@ def test_request_counts_and_skewed_lengths(flags, B):
     compare(out, lse, *ref, kv_dtype=0, what=f"B={B}")
 
 
+# Every KV worker gets several requests of dozens of tiles each: the pipelines reach their steady state (all stages, both
+# S and P buffers in flight, the softmax warps as far ahead of the P.V issuers as the barriers allow) and cross request
+# boundaries in it.  One case per kernel family; sampled outputs against the oracle, the device status word clean.
+@pytest.mark.parametrize("kv_dtype,H,flags", [(1, 16, 0), (1, 32, 0), (1, 64, 0), (1, 128, 0), (1, 128, 2),
+                                              (0, 16, 0), (0, 32, 0), (0, 64, 0), (0, 128, 0), (0, 128, 2)])
+def test_long_segments_several_per_worker(kv_dtype, H, flags):
+    rng = np.random.default_rng(4000 + H + kv_dtype)
+    lens = rng.integers(2500, 4500, size=150)
+    w = W.make_workload("steady", 380 + H + kv_dtype, lens, H=H, kv_dtype=kv_dtype)
+    out, lse = gpu_run(w, flags=flags)
+    pairs = np.array(sorted({(int(rng.integers(0, len(lens))), int(rng.integers(0, H))) for _ in range(120)}), np.int32)
+    ref_o, ref_l = oracle_run(w, pairs=pairs)
+    compare(out, lse, ref_o, ref_l, kv_dtype=kv_dtype, rows=[tuple(p) for p in pairs], what=f"steady H={H} dtype={kv_dtype}")
+    assert np.isfinite(out).all() and np.isfinite(lse).all()
+
+
 def test_more_requests_than_the_plan_stages_in_shared_memory():
     # 4,500 short requests (the plan kernel keeps its prefix arrays in shared memory up to 4,096): sampled outputs
     # against the oracle, every output finite, empty requests zero
