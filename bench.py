@@ -244,7 +244,8 @@ class GpuBench:
         if hs > 64:     # slices of more than 64 heads run on CTA pairs
             kernel = "decode_umma_fp8_pair_kernel" if fp8 else "decode_umma_pair_kernel"
         else:
-            kernel = "decode_umma_fp8_kernel" if fp8 else "decode_umma_kernel<%d>" % (16 if hs <= 16 else 32 if hs <= 32 else 64)
+            n = 16 if hs <= 16 else 32 if hs <= 32 else 64
+            kernel = ("decode_umma_fp8_narrow_kernel<%d>" % n if n < 64 else "decode_umma_fp8_kernel") if fp8 else "decode_umma_kernel<%d>" % n
         # the stricter reading: the whole call against the nominal peaks of the part (fp8 MMA rate for e4m3 KV)
         nom_tensor = NOMINAL_PEAKS["fp8_tflops"] if fp8 else NOMINAL_PEAKS["bf16_tflops"]
         tn_hbm, tn_tensor = alg_bytes / (NOMINAL_PEAKS["hbm_gbs"] * 1e9), alg_flops / (nom_tensor * 1e12)
@@ -293,6 +294,41 @@ class GpuBench:
                              "algorithmic_bytes": alg_bytes, "algorithmic_flops": alg_flops,
                              "launch_chains": 1, "cta_pairs_per_kv_worker": -(-h * R // 128)},
                 "launches_per_step": binding.splash_last_launch_count()}
+
+    def slice_workload(self, w, dw, out, lse, head_begin, head_end, steps, warmup, peaks):
+        """A TP rank's share of workload `w`: the same cache and requests, heads [head_begin, head_end) only."""
+        import copy
+        torch, binding = self.torch, self.binding
+        ws = copy.copy(w)
+        ws.head_begin, ws.head_end = head_begin, head_end
+        step = lambda: dw.decode(out=out, lse=lse, head_begin=head_begin, head_end=head_end)
+        ms = self.timed(step, steps, warmup)
+        launches = binding.splash_last_launch_count()
+        binding.splash_set_kernel_timing(True)
+        kt = []
+        for _ in range(steps):
+            self.flush_l2(); step()
+            kt.append(binding.splash_get_kernel_timing())
+        binding.splash_set_kernel_timing(False)
+        kt = np.array(kt)
+        rc, detail = binding.splash_workspace_status(binding.decode_workspace(torch.device(self.device)))
+        if rc != 0:
+            raise RuntimeError(f"device status {rc} {detail}")
+        dec_ms, p50 = float(kt[:, 1].mean()), float(np.median(ms))
+        alg_bytes = ws.algorithmic_bytes()
+        t_hbm = alg_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        hs = head_end - head_begin
+        n = 16 if hs <= 16 else 32 if hs <= 32 else 64
+        kernel = ("decode_umma_fp8_narrow_kernel<%d>" % n if n < 64 else "decode_umma_fp8_kernel") if w.kv_dtype == 1 \
+            else "decode_umma_kernel<%d>" % n
+        return {"ms_per_step": float(ms.mean()), "ms_p50": p50, "ms_p95": float(np.percentile(ms, 95)),
+                "tokens_per_s": w.B / (ms.mean() * 1e-3), "launches_per_step": launches, "heads": hs,
+                "requests": w.B, "tokens": w.total_tokens(),
+                "roofline": {"bound": "hbm", "achieved": alg_bytes / (dec_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                             "unit": "GB/s", "frac": t_hbm / dec_ms, "frac_whole_call": t_hbm / p50, "traffic": None,
+                             "kernel": kernel, "kernel_ms": dec_ms, "plan_ms": float(kt[:, 0].mean()),
+                             "combine_ms": float(kt[:, 2].mean()), "algorithmic_bytes": alg_bytes,
+                             "roofline_ms": t_hbm, "peak_source": peaks["source"]}}
 
     def sparse_workload(self, seq_lens, H, steps, warmup, peaks, topk=2048):
         """Sparse decode: every request attends over the (at most) topk tokens of a seeded list, cache rows in the
@@ -755,7 +791,8 @@ def main():
             steps2 = max(5, args.steps // 2)
             if idx == 5:
                 try:
-                    extra["c5"] = {"page_migrate": gb.migrate_workload(w, dw, steps2, args.warmup, peaks),
+                    extra["c5"] = {"tp8_slice": gb.slice_workload(w, dw, out, lse, 32, 48, steps2, args.warmup, peaks),
+                                   "page_migrate": gb.migrate_workload(w, dw, steps2, args.warmup, peaks),
                                    "migrate_under_decode": gb.overlap_workload(w, dw, steps2, args.warmup)}
                 except Exception as exc:  # report, do not hide
                     extra["c5"] = {"error": repr(exc)}
@@ -776,6 +813,8 @@ def main():
                         del dwx
                         r["cp"] = gb.cp_workload(wx, steps2, args.warmup)
                     if name == "c5":
+                        # a TP-8 rank's share of the same step: 16 of the 128 heads over the same e4m3 cache
+                        r["tp8_slice"] = gb.slice_workload(wx, dwx, ox, lx, 32, 48, steps2, args.warmup, peaks)
                         r["page_migrate"] = gb.migrate_workload(wx, dwx, steps2, args.warmup, peaks)
                         r["migrate_under_decode"] = gb.overlap_workload(wx, dwx, steps2, args.warmup)
                     extra[name] = r

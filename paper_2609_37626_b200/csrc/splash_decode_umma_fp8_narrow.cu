@@ -20,9 +20,8 @@
 // term carry its own scale: it is stored as e4m3 of 16 x the residual (three significant bits, never out
 // of range since an e4m3 residual is at most 2^-4 of the value) and the epilogue adds lo / 16.  With the tokens on the TMEM lanes the token scale is one
 // number per thread, and a thread's weights for its token are N adjacent bytes of an MN-major
-// P^T: one 16-byte store per 16 heads.  A page is 36,864 bytes and the query operands are small,
-// so five stages fit: the loop is a ring of dependent latencies and its period is the ring divided
-// by the stages.
+// P^T.  A page is 36,864 bytes and the query operands are small, so five stages fit (four with 32
+// heads): the loop is a ring of dependent latencies and its period is the ring divided by the stages.
 //
 // The softmax warps keep one reference maximum per head and move it only when a logit exceeds it by
 // more than 2^4 (the headroom that e4m3's range leaves above the lift): whether any does is one
@@ -31,7 +30,7 @@
 //
 // Warp roles (352 threads): TMA producer (pages + scale pages, next page pulled into L2), 2 QK^T
 // issuers (one partial accumulator of S^T each), 2 P.V issuers (two dv blocks each), 4 softmax /
-// epilogue warps, 2 query converter warps.  Every wait is bounded; on expiry the CTA records
+// epilogue warps, 2 query converter warps (a request ahead: the query operands are double buffered).  Every wait is bounded; on expiry the CTA records
 // SPLASH_DEVICE_TIMEOUT and leaves in order.
 #include "splash_fp8.cuh"
 #include "splash_pair.cuh"
@@ -45,27 +44,25 @@ using namespace umma;
 constexpr int kQkWarps = 2;                        // = partial accumulators of S^T
 constexpr int kPvWarps = 2;                        // each owns two of the four dv blocks of O^T
 constexpr int kNumSoftmaxWarps = 4;
-constexpr int kNumConvertWarps = 2;
 constexpr int kWarpQk = 1;
 constexpr int kWarpPv = kWarpQk + kQkWarps;
 constexpr int kWarpSoftmax = kWarpPv + kPvWarps;            // 5: TMEM lane quadrant = warp & 3
 constexpr int kWarpConvert = kWarpSoftmax + kNumSoftmaxWarps;
-constexpr int kThreads = (kWarpConvert + kNumConvertWarps) * 32;   // 11 warps = 352 threads
 constexpr int kChunks = 9;                         // 576 / 64-element (64 B) chunks
 constexpr uint32_t kSlab = 64 * 64;                // one chunk of one page: 64 tokens x 64 B
 constexpr uint32_t kStageBytes = kChunks * kSlab;  // 36,864
 constexpr uint32_t kScaleBytes = 256;              // 64 fp32 token scales of a page
-constexpr int kStages = 5;
+constexpr int kMaxStages = 5;
 constexpr float kTau = 4.0f;                       // lazy rescale threshold, log2 units
 constexpr float kLift = 4.75f;                     // weights are stored as 2^(y - m + kLift) <= 2^8.75 = 431 < 448
 
 enum BarrierId {
-    kBarKvFull = 0,                    // [kStages]
-    kBarKvEmpty = kBarKvFull + kStages,
-    kBarQFull = kBarKvEmpty + kStages,
-    kBarQEmpty,
-    kBarQsRead,                        // the softmax warps have picked up the request's query scales
-    kBarSFull,                         // [2]
+    kBarKvFull = 0,                    // [stages]
+    kBarKvEmpty = kBarKvFull + kMaxStages,
+    kBarQFull = kBarKvEmpty + kMaxStages,   // [2]: one per query operand buffer
+    kBarQEmpty = kBarQFull + 2,        // [2]: the QK^T issuers are done with the buffer AND the softmax warps with the request
+                                       // (they stage its output tile there)
+    kBarSFull = kBarQEmpty + 2,        // [2]
     kBarSEmpty = kBarSFull + 2,        // [2]
     kBarPFull = kBarSEmpty + 2,        // [2]: one per P buffer.  With a single barrier the softmax warps, which may run two
                                        // tiles ahead of a P.V issuer, could complete two phases between two of its polls
@@ -76,12 +73,15 @@ enum BarrierId {
 
 template <int N>
 struct Layout {
+    static constexpr int kStages = N == 16 ? 5 : 4;
+    static constexpr int kNumConvertWarps = 2;                 // four threads per head, 16 heads per pass
+    static constexpr int kThreads = (kWarpConvert + kNumConvertWarps) * 32;   // 11 warps = 352 threads
     static constexpr uint32_t kQSlab = 2 * N * 64;             // one chunk of the query operand: (N hi rows, N lo rows) x 64 B
-    static constexpr uint32_t kQBytes = kChunks * kQSlab;
+    static constexpr uint32_t kQBytes = kChunks * kQSlab;      // one buffer; there are two (request parity)
     static constexpr uint32_t kPBytes = 2 * N * 64;            // P^T: [2N / 16 groups: hi, then lo][64 tokens][16 heads], one byte each
     static constexpr uint32_t kOffKv = 0;
     static constexpr uint32_t kOffQ = kOffKv + kStages * kStageBytes;
-    static constexpr uint32_t kOffP = kOffQ + kQBytes;         // double buffered (tile parity)
+    static constexpr uint32_t kOffP = kOffQ + 2 * kQBytes;     // double buffered (tile parity)
     static constexpr uint32_t kOffScale = kOffP + 2 * kPBytes; // float [kStages][64]
     static constexpr uint32_t kOffQs = kOffScale + kStages * kScaleBytes;   // float [4][N] query scales, by segment & 3
     static constexpr uint32_t kOffRed = kOffQs + 4 * N * 4;    // float [N][4]
@@ -106,41 +106,20 @@ __device__ __forceinline__ uint64_t make_desc_mn_plain(uint32_t saddr, uint32_t 
            ((uint64_t)((mn_group_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
 }
 
-// Reduce-scatter over the 32 lanes of a warp (see the bf16 kernel): on return lane L holds, in v[0 .. max(1, N/32)),
-// the reduction over all lanes of the entries it owns (N = 32: head L; N = 16: head L >> 1, both lanes of a pair).
-template <int CNT, int MASK, bool IS_MAX>
-struct ReduceScatter {
-    template <int N>
-    static __device__ __forceinline__ void run(float (&v)[N], int lane) {
-        if constexpr (MASK >= 1) {
-            if constexpr (CNT > 1) {
-                constexpr int kHalf = CNT / 2;
-                const bool upper = (lane & MASK) != 0;
-#pragma unroll
-                for (int i = 0; i < kHalf; ++i) {
-                    float keep = upper ? v[i + kHalf] : v[i];
-                    float send = upper ? v[i] : v[i + kHalf];
-                    float recv = __shfl_xor_sync(0xffffffffu, send, MASK);
-                    v[i] = IS_MAX ? fmaxf(keep, recv) : keep + recv;
-                }
-                ReduceScatter<kHalf, MASK / 2, IS_MAX>::run(v, lane);
-            } else {
-                float recv = __shfl_xor_sync(0xffffffffu, v[0], MASK);
-                v[0] = IS_MAX ? fmaxf(v[0], recv) : v[0] + recv;
-                ReduceScatter<1, MASK / 2, IS_MAX>::run(v, lane);
-            }
-        }
-    }
-};
-
+// N columns of 16 TMEM lanes in the accumulator fragment layout: v[4k + e] = (lane T/4, column 8k + 2(T%4) + e),
+// v[4k + 2 + e] = (lane T/4 + 8, the same column), k < N / 8, e < 2.
 template <int N>
-__device__ __forceinline__ int owned_head(int lane) { return N >= 32 ? lane : lane >> 1; }
+__device__ __forceinline__ void tmem_ld_frag(uint32_t taddr, float (&v)[N / 2]) {
+    if constexpr (N == 16) tmem_ld_16x256b_x2(taddr, v);
+    else tmem_ld_16x256b_x4(taddr, v);
+}
 
 // ---------------------------------------------------------------- the kernel
 template <int N>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(Layout<N>::kThreads, 1)
 decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmap_kv) {
     using L = Layout<N>;
+    constexpr int kStages = L::kStages, kThreads = L::kThreads;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -159,8 +138,7 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
     }
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), kPvWarps); }
-        mbar_init(bar(kBarQFull), kNumConvertWarps); mbar_init(bar(kBarQEmpty), kQkWarps);
-        mbar_init(bar(kBarQsRead), kNumSoftmaxWarps);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarQFull + b), L::kNumConvertWarps); mbar_init(bar(kBarQEmpty + b), kQkWarps + kNumSoftmaxWarps); }
         for (int b = 0; b < 2; ++b) { mbar_init(bar(kBarSFull + b), kQkWarps); mbar_init(bar(kBarSEmpty + b), kNumSoftmaxWarps); }
         for (int b = 0; b < 2; ++b) mbar_init(bar(kBarPFull + b), kNumSoftmaxWarps);
         mbar_init(bar(kBarOFull), kPvWarps); mbar_init(bar(kBarOEmpty), kNumSoftmaxWarps);
@@ -255,7 +233,8 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
             bool ok = true;
             while (ok && it.next(p, seg)) {
                 const int ntiles = seg.tile_end - seg.tile_begin;
-                ok = mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
+                const uint32_t qb = seg_it & 1;
+                ok = mbar_wait(ctx, bar(kBarQFull + qb), (seg_it >> 1) & 1, kBarQFull + qb);
                 for (int i = 0; ok && i < ntiles; ++i, ++kv) {
                     const uint32_t stage = kv % kStages, b = kv & 1;
                     ok = mbar_wait(ctx, bar(kBarKvFull + stage), (kv / kStages) & 1, kBarKvFull + stage) &&
@@ -270,13 +249,13 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                     for (int t = 0; t < 18 / kQkWarps; ++t) {
                         const int ks = t * kQkWarps + a, c = ks >> 1, k = ks & 1;
                         uint64_t dk = make_desc_sw64(k0 + c * kSlab + k * 32, 16, 512);                      // A: 64 tokens x 32
-                        uint64_t dq = make_desc_sw64(sbase + L::kOffQ + c * L::kQSlab + k * 32, 16, 512);    // B: 2N rows x 32
+                        uint64_t dq = make_desc_sw64(sbase + L::kOffQ + qb * L::kQBytes + c * L::kQSlab + k * 32, 16, 512);    // B: 2N rows x 32
                         umma_e4m3(d, dk, dq, kIdescQK, t != 0);
                     }
                     umma_commit(bar(kBarSFull + b));
                     if (a == 0) mark(kv, 3);
                 }
-                if (ok) umma_commit(bar(kBarQEmpty));
+                if (ok) umma_commit(bar(kBarQEmpty + qb));
                 ++seg_it;
             }
         }
@@ -318,69 +297,84 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
         }
     } else if (warp >= kWarpConvert) {
         // ===================================================== query converters
-        // bf16 query rows -> e4m3 hi + lo operands with one scale per head, 64 / N threads per head.  They run a
-        // segment ahead of the softmax warps: the operands of the next request are rebuilt as soon as the last
-        // QK^T of the current one has been issued and retired.
-        constexpr int kPerHead = 64 / N;               // threads per head: 4 (N = 16) or 2 (N = 32)
-        constexpr int kVecs = 72 / kPerHead;           // 8-element vectors per thread
-        const int ct = (warp - kWarpConvert) * 32 + lane;   // 0..63
+        // bf16 query rows -> e4m3 hi + lo operands with one scale per head, four threads per head.  The operands are
+        // double buffered, so the converters work a whole request ahead: the row is read once, into registers, and
+        // the latency of those loads (several microseconds while the cache streams at full rate) stays off the
+        // path from one request's last tile to the next one's first.
+        constexpr int kVecs = 18;                      // 8-element vectors per thread: a quarter of a row
+        const int ct = (warp - kWarpConvert) * 32 + lane;   // 0..63: head ct / 4 of a pass, quarter ct % 4
         float *qs_s = reinterpret_cast<float *>(smem + L::kOffQs);
         uint32_t seg_it = 0;
         bool ok = true;
         while (ok && it.next(p, seg)) {
-            ok = mbar_wait(ctx, bar(kBarQEmpty), (seg_it & 1) ^ 1, kBarQEmpty);
-            if (!ok) break;
-            const int hd = ct / kPerHead, part = ct % kPerHead;
-            const int gh = head0 + hd;
-            const bool live = gh < p.head_end;
-            const uint4 *src = reinterpret_cast<const uint4 *>(
-                static_cast<const __nv_bfloat16 *>(p.q) + (int64_t)seg.request * p.q_stride_request +
-                (int64_t)(live ? gh : p.head_begin) * p.q_stride_head + part * (kVecs * 8));
-            float amax = 0.f;
-            if (live) {
-#pragma unroll 6
+            const uint32_t qb = seg_it & 1;
+            uint8_t *qdst = smem + L::kOffQ + qb * L::kQBytes;
+            const int part = ct & 3;
+            {
+                // the rows of the request after this one: into L2 now, so that their loads, a request from now, are short
+                SegmentIter peek = it;
+                Segment nxt;
+                if (peek.next(p, nxt)) {
+                    const char *row0 = reinterpret_cast<const char *>(static_cast<const __nv_bfloat16 *>(p.q) +
+                                       (int64_t)nxt.request * p.q_stride_request + (int64_t)head0 * p.q_stride_head);
+                    const int64_t bytes = (int64_t)min(N, p.head_end - head0) * p.q_stride_head * 2;
+                    for (int64_t o = (int64_t)ct * 128; o < bytes; o += 64 * 128)
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(row0 + o));
+                }
+            }
+#pragma unroll 1
+            for (int pass = 0; pass < N / 16; ++pass) {
+                const int hd = pass * 16 + (ct >> 2);
+                const int gh = head0 + hd;
+                const bool live = gh < p.head_end;
+                const uint4 *src = reinterpret_cast<const uint4 *>(
+                    static_cast<const __nv_bfloat16 *>(p.q) + (int64_t)seg.request * p.q_stride_request +
+                    (int64_t)(live ? gh : p.head_begin) * p.q_stride_head + part * (kVecs * 8));
+                uint4 x[kVecs];
+#pragma unroll
+                for (int v = 0; v < kVecs; ++v) x[v] = live ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
+                float amax = 0.f;
+#pragma unroll
                 for (int v = 0; v < kVecs; ++v) {
-                    uint4 x = __ldg(src + v);
-                    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+                    const uint32_t w[4] = {x[v].x, x[v].y, x[v].z, x[v].w};
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         amax = fmaxf(amax, fabsf(__uint_as_float(w[k] << 16)));
                         amax = fmaxf(amax, fabsf(__uint_as_float(w[k] & 0xffff0000u)));
                     }
                 }
-            }
-#pragma unroll
-            for (int mk = 1; mk < kPerHead; mk <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, mk));
-            const float qs = amax > 0.f ? amax * (1.0f / 448.0f) : 1.0f;
-            const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
-            if (part == 0) qs_s[(seg_it & 3) * N + hd] = qs;
-#pragma unroll 2
-            for (int v = 0; v < kVecs; ++v) {
-                uint4 x = live ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
-                const uint32_t w[4] = {x.x, x.y, x.z, x.w};
-                uint16_t hi[4], lo[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const float e0 = __uint_as_float(w[k] << 16) * inv, e1 = __uint_as_float(w[k] & 0xffff0000u) * inv;
-                    split_e4m3_e4m3_x2(e0, e1, hi[k], lo[k]);
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+                const float qs = amax > 0.f ? amax * (1.0f / 448.0f) : 1.0f;
+                const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
+                if (pass == 0) {
+                    // this buffer's previous request (two back): its QK^T retired, its softmax under way
+                    ok = mbar_wait(ctx, bar(kBarQEmpty + qb), ((seg_it >> 1) & 1) ^ 1, kBarQEmpty + qb);
+                    if (!ok) break;
                 }
-                const uint32_t d = (uint32_t)(part * (kVecs * 8) + v * 8);
-                // the lo rows follow the N hi rows of the chunk (N is a multiple of 8: same swizzle phase)
-                const uint32_t off = (d >> 6) * L::kQSlab + sw64((uint32_t)hd, d & 63);
-                *reinterpret_cast<uint2 *>(smem + L::kOffQ + off) =
-                    make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
-                *reinterpret_cast<uint2 *>(smem + L::kOffQ + N * 64 + off) =
-                    make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
+                if (part == 0) qs_s[(seg_it & 3) * N + hd] = qs;
+#pragma unroll
+                for (int v = 0; v < kVecs; ++v) {
+                    const uint32_t w[4] = {x[v].x, x[v].y, x[v].z, x[v].w};
+                    uint16_t hi[4], lo[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float e0 = __uint_as_float(w[k] << 16) * inv, e1 = __uint_as_float(w[k] & 0xffff0000u) * inv;
+                        split_e4m3_e4m3_x2(e0, e1, hi[k], lo[k]);
+                    }
+                    const uint32_t d = (uint32_t)(part * (kVecs * 8) + v * 8);
+                    // the lo rows follow the N hi rows of the chunk (N is a multiple of 8: same swizzle phase)
+                    const uint32_t off = (d >> 6) * L::kQSlab + sw64((uint32_t)hd, d & 63);
+                    *reinterpret_cast<uint2 *>(qdst + off) =
+                        make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
+                    *reinterpret_cast<uint2 *>(qdst + N * 64 + off) =
+                        make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
+                }
             }
+            if (!ok) break;
             fence_proxy_async();
             __syncwarp();
-            // The softmax warps wait on QFull by phase parity, so QFull must never complete two phases ahead of
-            // them: hold this request's arrival until they have entered the previous one.
-            if (lane == 0) {
-                if (seg_it > 0) ok = mbar_wait(ctx, bar(kBarQsRead), (seg_it - 1) & 1, kBarQsRead);
-                mbar_arrive(bar(kBarQFull));
-            }
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (lane == 0) mbar_arrive(bar(kBarQFull + qb));
             ++seg_it;
         }
     } else {
@@ -388,7 +382,12 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
         const int q4 = warp & 3;                       // TMEM lane quadrant of this warp
         const int sw = warp - kWarpSoftmax;            // softmax warp 0..3
         const int st = sw * 32 + lane;                 // 0..127
-        const int row = 16 * q4 + lane;                // token row of the S^T tile (lanes < 16)
+        // S^T comes out of tensor memory in the accumulator fragment layout, which spreads the 16 lanes that an
+        // M = 64 tile has per quadrant over all 32 threads: this thread holds tokens rA and rB = rA + 8 and, of each
+        // group of eight heads, heads 2 tq and 2 tq + 1.
+        const int rA = 16 * q4 + (lane >> 2), rB = rA + 8;
+        const int tq = lane & 3;
+        constexpr int kR = N / 8;                      // groups of eight heads
         const uint32_t lane_addr = (uint32_t)(32 * q4) << 16;
         float *red = reinterpret_cast<float *>(smem + L::kOffRed);
         float *m_s = reinterpret_cast<float *>(smem + L::kOffM);
@@ -403,76 +402,74 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
         bool ok = true;
         while (it.next(p, seg)) {
             // the converter warps have written this segment's query operands and scales
-            ok &= mbar_wait(ctx, bar(kBarQFull), seg_it & 1, kBarQFull);
+            ok &= mbar_wait(ctx, bar(kBarQFull + (seg_it & 1)), (seg_it >> 1) & 1, kBarQFull + (seg_it & 1));
             const float *qs_s = qs_all + (seg_it & 3) * N;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarQsRead));
             if (st < N) m_s[st] = -INFINITY;
-            float l[N];                   // running sums of P / scale_t over this thread's tokens, one per head
+            float l[2 * kR];              // sums of P / scale_t over this thread's tokens: heads 8k + 2 tq + e at [2k + e]
 #pragma unroll
-            for (int n = 0; n < N; ++n) l[n] = 0.f;
+            for (int n = 0; n < 2 * kR; ++n) l[n] = 0.f;
             softmax_bar_sync();
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;
             for (int i = 0; i < ntiles; ++i) {
                 const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + seg.tile_begin + i) * kPage);
-                const bool valid = lane < 16 && row >= g.r_lo && row < g.r_hi;
+                const bool vA = rA >= g.r_lo && rA < g.r_hi, vB = rB >= g.r_lo && rB < g.r_hi;
                 const uint32_t b = s_it & 1, stage = s_it % kStages;
                 ok &= mbar_wait(ctx, bar(kBarSFull + b), (s_it >> 1) & 1, kBarSFull + b);
                 if (st == 0) mark(s_it, 4);
                 // the scale page rode on the stage's own barrier, long complete by now
                 ok &= mbar_wait(ctx, bar(kBarKvFull + stage), (s_it / kStages) & 1, kBarKvFull + stage);
                 tcgen05_fence_after();
-                float s[N];
+                float s[4 * kR];
                 {
                     // S^T = the sum of four N-column pieces: (partial 0, partial 1) x (q hi, q lo)
-                    float t0[N], t1[N];
+                    float t0[4 * kR], t1[4 * kR], t2[4 * kR];
                     const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (2 * kQkWarps * N);
-#pragma unroll
-                    for (int c = 0; c < N / 16; ++c) {
-                        tmem_ld16(sb + c * 16, *reinterpret_cast<float(*)[16]>(&s[c * 16]));
-                        tmem_ld16(sb + N + c * 16, *reinterpret_cast<float(*)[16]>(&t0[c * 16]));
-                    }
+                    tmem_ld_frag<N>(sb, s);
+                    tmem_ld_frag<N>(sb + N, t0);
+                    tmem_ld_frag<N>(sb + 2 * N, t1);
+                    tmem_ld_frag<N>(sb + 3 * N, t2);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int n = 0; n < N; ++n) s[n] += t0[n];
-#pragma unroll
-                    for (int c = 0; c < N / 16; ++c) {
-                        tmem_ld16(sb + 2 * N + c * 16, *reinterpret_cast<float(*)[16]>(&t0[c * 16]));
-                        tmem_ld16(sb + 3 * N + c * 16, *reinterpret_cast<float(*)[16]>(&t1[c * 16]));
-                    }
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int n = 0; n < N; ++n) s[n] += t0[n] + t1[n];
+                    for (int n = 0; n < 4 * kR; ++n) s[n] = (s[n] + t0[n]) + (t1[n] + t2[n]);
                 }
                 tcgen05_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarSEmpty + b));
-                // this thread's token: its scale, log2 of it for the weight, its reciprocal for the row sums
-                const float ts = valid ? scale_s[stage * 64 + g.tok0 + row] : 1.0f;
-                const float lg = fast_log2(ts), rts = fast_rcp(ts), tsl = ts * scale_log2;
-                bool exceeds = false;     // some logit of this token lies more than kTau above its head's reference
+                // this thread's tokens: their scales, log2 of them for the weights, reciprocals for the row sums
+                const float tsA = vA ? scale_s[stage * 64 + g.tok0 + rA] : 1.0f, tsB = vB ? scale_s[stage * 64 + g.tok0 + rB] : 1.0f;
+                const float lgA = fast_log2(tsA), lgB = fast_log2(tsB), rtsA = fast_rcp(tsA), rtsB = fast_rcp(tsB);
+                const float tslA = tsA * scale_log2, tslB = tsB * scale_log2;
+                bool exceeds = false;     // some logit of these tokens lies more than kTau above its head's reference
 #pragma unroll
-                for (int n4 = 0; n4 < N; n4 += 4) {
-                    const float4 q4v = *reinterpret_cast<const float4 *>(&qs_s[n4]);
-                    const float4 m4 = *reinterpret_cast<const float4 *>(&m_s[n4]);
-                    const float qv[4] = {q4v.x, q4v.y, q4v.z, q4v.w}, mv[4] = {m4.x, m4.y, m4.z, m4.w};
+                for (int k = 0; k < kR; ++k) {
+                    const float2 q2 = *reinterpret_cast<const float2 *>(&qs_s[8 * k + 2 * tq]);
+                    const float2 m2 = *reinterpret_cast<const float2 *>(&m_s[8 * k + 2 * tq]);
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float y = valid ? fmaf(s[n4 + e] * qv[e], tsl, lg) : -INFINITY;   // log2-domain logit + log2(token scale)
-                        s[n4 + e] = y;
-                        exceeds |= y > mv[e] + kTau;
+                    for (int e = 0; e < 2; ++e) {
+                        const float qv = e ? q2.y : q2.x, lim = (e ? m2.y : m2.x) + kTau;
+                        // log2-domain logit + log2(token scale)
+                        const float yA = vA ? fmaf(s[4 * k + e] * qv, tslA, lgA) : -INFINITY;
+                        const float yB = vB ? fmaf(s[4 * k + 2 + e] * qv, tslB, lgB) : -INFINITY;
+                        s[4 * k + e] = yA; s[4 * k + 2 + e] = yB;
+                        exceeds |= (yA > lim) | (yB > lim);
                     }
                 }
                 const bool grew = softmax_bar_or(exceeds);
                 if (grew) {
                     // the rare path (the first tile of a request, then a handful of times): per-head maxima over the
                     // tile's tokens, new references for the heads that grew, their rescale factors
-                    float mx[N];
 #pragma unroll
-                    for (int n = 0; n < N; ++n) mx[n] = s[n];
-                    ReduceScatter<N, 16, true>::run(mx, lane);
-                    if (N >= 32 || (lane & 1) == 0) red[owned_head<N>(lane) * 4 + sw] = mx[0];
+                    for (int k = 0; k < kR; ++k) {
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            float mx = fmaxf(s[4 * k + e], s[4 * k + 2 + e]);
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                            if (lane < 4) red[(8 * k + 2 * tq + e) * 4 + sw] = mx;
+                        }
+                    }
                     softmax_bar_sync();
                     if (st < N) {
                         float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
@@ -487,22 +484,23 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                     }
                     softmax_bar_sync();
 #pragma unroll
-                    for (int n = 0; n < N; ++n) l[n] *= alpha_s[n];
+                    for (int k = 0; k < kR; ++k) {
+                        const float2 a2 = *reinterpret_cast<const float2 *>(&alpha_s[8 * k + 2 * tq]);
+                        l[2 * k] *= a2.x; l[2 * k + 1] *= a2.y;
+                    }
                 }
-                uint32_t phi[N / 4], plo[N / 4];      // four heads' bytes per word
+                uint16_t hiA[kR], loA[kR], hiB[kR], loB[kR];      // two adjacent heads per 16-bit word
 #pragma unroll
-                for (int n4 = 0; n4 < N; n4 += 4) {
-                    const float4 m4 = *reinterpret_cast<const float4 *>(&m_s[n4]);
-                    const float w0 = fast_exp2(s[n4 + 0] - m4.x + kLift), w1 = fast_exp2(s[n4 + 1] - m4.y + kLift);
-                    const float w2 = fast_exp2(s[n4 + 2] - m4.z + kLift), w3 = fast_exp2(s[n4 + 3] - m4.w + kLift);
-                    l[n4 + 0] = fmaf(w0, rts, l[n4 + 0]); l[n4 + 1] = fmaf(w1, rts, l[n4 + 1]);
-                    l[n4 + 2] = fmaf(w2, rts, l[n4 + 2]); l[n4 + 3] = fmaf(w3, rts, l[n4 + 3]);
+                for (int k = 0; k < kR; ++k) {
+                    const float2 m2 = *reinterpret_cast<const float2 *>(&m_s[8 * k + 2 * tq]);
+                    const float o0 = kLift - m2.x, o1 = kLift - m2.y;
+                    const float a0 = fast_exp2(s[4 * k + 0] + o0), a1 = fast_exp2(s[4 * k + 1] + o1);
+                    const float b0 = fast_exp2(s[4 * k + 2] + o0), b1 = fast_exp2(s[4 * k + 3] + o1);
+                    l[2 * k] = fmaf(a0, rtsA, fmaf(b0, rtsB, l[2 * k]));
+                    l[2 * k + 1] = fmaf(a1, rtsA, fmaf(b1, rtsB, l[2 * k + 1]));
                     // hi = the e4m3 value nearest to the weight, lo = 16 x what is left, e4m3 again
-                    uint16_t h01, l01, h23, l23;
-                    split_e4m3_e4m3x16_x2(w0, w1, h01, l01);
-                    split_e4m3_e4m3x16_x2(w2, w3, h23, l23);
-                    phi[n4 / 4] = (uint32_t)h01 | ((uint32_t)h23 << 16);
-                    plo[n4 / 4] = (uint32_t)l01 | ((uint32_t)l23 << 16);
+                    split_e4m3_e4m3x16_x2(a0, a1, hiA[k], loA[k]);
+                    split_e4m3_e4m3x16_x2(b0, b1, hiB[k], loB[k]);
                 }
                 // the P.V that read this P buffer (two tiles back) must be done; a rescale of O^T also needs the
                 // previous tile's P.V
@@ -526,14 +524,15 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                     }
                     tmem_wait_st();
                 }
-                if (lane < 16) {
-                    // P^T hi / lo, MN-major: the 16 heads of a group are the 16 bytes of this token's row
-                    uint8_t *ph = smem + L::kOffP + (s_it & 1) * L::kPBytes + row * 16;
-                    uint8_t *pl = ph + (N / 16) * 1024;
+                {
+                    // P^T hi / lo, MN-major: the 16 heads of a group are the 16 bytes of a token's row; groups of 16
+                    // heads are 1024 B apart, the lo groups follow the hi groups
+                    uint8_t *pa = smem + L::kOffP + (s_it & 1) * L::kPBytes + rA * 16 + 2 * tq;
 #pragma unroll
-                    for (int gq = 0; gq < N / 16; ++gq) {
-                        *reinterpret_cast<uint4 *>(ph + gq * 1024) = make_uint4(phi[4 * gq], phi[4 * gq + 1], phi[4 * gq + 2], phi[4 * gq + 3]);
-                        *reinterpret_cast<uint4 *>(pl + gq * 1024) = make_uint4(plo[4 * gq], plo[4 * gq + 1], plo[4 * gq + 2], plo[4 * gq + 3]);
+                    for (int k = 0; k < kR; ++k) {
+                        uint8_t *ph = pa + (k >> 1) * 1024 + (k & 1) * 8, *pl = ph + (N / 16) * 1024;
+                        *reinterpret_cast<uint16_t *>(ph) = hiA[k]; *reinterpret_cast<uint16_t *>(ph + 8 * 16) = hiB[k];
+                        *reinterpret_cast<uint16_t *>(pl) = loA[k]; *reinterpret_cast<uint16_t *>(pl + 8 * 16) = loB[k];
                     }
                 }
                 fence_proxy_async();
@@ -543,9 +542,15 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 if (lane == 0) mbar_arrive(bar(kBarPFull + (s_it & 1)));
                 ++s_it;
             }
-            // ---- row sums: over the 16 tokens of a warp, then over the four warps
-            ReduceScatter<N, 16, false>::run(l, lane);
-            if (N >= 32 || (lane & 1) == 0) red[owned_head<N>(lane) * 4 + sw] = l[0];
+            // ---- row sums: over the 16 tokens of a warp (the eight threads with this tq), then over the four warps
+#pragma unroll
+            for (int n = 0; n < 2 * kR; ++n) {
+                float v = l[n];
+                v += __shfl_xor_sync(0xffffffffu, v, 4);
+                v += __shfl_xor_sync(0xffffffffu, v, 8);
+                v += __shfl_xor_sync(0xffffffffu, v, 16);
+                if (lane < 4) red[(8 * (n >> 1) + 2 * tq + (n & 1)) * 4 + sw] = v;
+            }
             softmax_bar_sync();
             if (st < N) {
                 float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
@@ -572,27 +577,67 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 ostride = kDV;
             }
             const int nvalid = min(N, p.head_end - head0);
+            if (((reinterpret_cast<uintptr_t>(obase) | (uintptr_t)(ostride * 4)) & 15) == 0) {
+                // Through shared memory and the bulk-copy engine: plain stores of this tile (one 128-byte line per warp
+                // instruction, 64 of them per thread) take ~6,000 cycles while the cache streams, 2.5 times this.  The
+                // finished request's query operands are dead by now and serve as the staging buffer, [N heads][256 dv]
+                // floats, filled and drained twice.
+                float *stg = reinterpret_cast<float *>(smem + L::kOffQ + (seg_it & 1) * L::kQBytes);
+                static_assert(N * 256 * 4 <= (int)L::kQBytes, "the staging tile must fit a query operand buffer");
 #pragma unroll 1
-            for (int j = 0; j < 4; ++j) {
-                const int dv = 128 * j + 32 * q4 + lane;
+                for (int half = 0; half < 2; ++half) {
 #pragma unroll
-                for (int c = 0; c < N / 16; ++c) {
-                    float o[16], o_lo[16];
-                    tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + c * 16, o);
-                    tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + N + c * 16, o_lo);
-                    tmem_wait_ld();
+                    for (int jj = 0; jj < 2; ++jj) {
+                        const int j = 2 * half + jj;
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const int n = c * 16 + k;
-                        if (n < nvalid) obase[(int64_t)n * ostride + dv] = fmaf(o_lo[k], 0.0625f, o[k]) * l_s[n];
+                        for (int c = 0; c < N / 16; ++c) {
+                            float o[16], o_lo[16];
+                            tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + c * 16, o);
+                            tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + N + c * 16, o_lo);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) {
+                                const int n = c * 16 + k;
+                                stg[n * 256 + jj * 128 + 32 * q4 + lane] = fmaf(o_lo[k], 0.0625f, o[k]) * l_s[n];
+                            }
+                        }
+                    }
+                    fence_proxy_async();
+                    softmax_bar_sync();
+                    if (st < nvalid) {
+                        bulk_store(obase + (int64_t)st * ostride + half * 256, smem_u32(stg + st * 256), 1024);
+                        bulk_commit_group();
+                        bulk_wait_group_read();          // the row has left shared memory
+                    }
+                    softmax_bar_sync();
+                }
+            } else {
+#pragma unroll 1
+                for (int j = 0; j < 4; ++j) {
+                    const int dv = 128 * j + 32 * q4 + lane;
+#pragma unroll
+                    for (int c = 0; c < N / 16; ++c) {
+                        float o[16], o_lo[16];
+                        tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + c * 16, o);
+                        tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + N + c * 16, o_lo);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            const int n = c * 16 + k;
+                            if (n < nvalid) obase[(int64_t)n * ostride + dv] = fmaf(o_lo[k], 0.0625f, o[k]) * l_s[n];
+                        }
                     }
                 }
             }
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarOEmpty));
+            if (lane == 0) {
+                mbar_arrive(bar(kBarOEmpty));
+                mbar_arrive(bar(kBarQEmpty + (seg_it & 1)));      // the converters may rebuild this operand buffer
+            }
             ++seg_it;
         }
+        bulk_wait_group();        // this thread's output rows have reached global memory
     }
 
     fill_empty_requests(p, worker, head0, N, tid, kThreads);
@@ -619,7 +664,7 @@ cudaError_t launch_n(const DecodeParams &p, const CUtensorMap &mkv, cudaStream_t
     static DeviceOnce once;
     cudaError_t e = once.run([&] { return cudaFuncSetAttribute(decode_umma_fp8_narrow_kernel<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem); });
     if (e != cudaSuccess) return e;
-    e = launch_dependent(decode_umma_fp8_narrow_kernel<N>, dim3((unsigned)(p.num_workers * p.num_groups)), dim3(kThreads),
+    e = launch_dependent(decode_umma_fp8_narrow_kernel<N>, dim3((unsigned)(p.num_workers * p.num_groups)), dim3(Layout<N>::kThreads),
                          (size_t)smem, stream, p, mkv);
     count_launch();
     return e;
