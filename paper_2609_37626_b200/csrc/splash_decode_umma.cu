@@ -71,7 +71,11 @@ struct Layout {
     static constexpr uint32_t kOffKv = 0;
     static constexpr uint32_t kOffQ = kOffKv + kStages * kStageBytes;
     static constexpr uint32_t kOffP = kOffQ + kQBytes;
-    static constexpr uint32_t kOffRed = kOffP + kPBytes;     // float [N][4]
+    // output staging for the narrow groups, [N heads][256 dv] floats: the finished tile leaves through the bulk-copy engine
+    // (64-head groups have no shared memory left for it and store from registers)
+    static constexpr uint32_t kOutBytes = N < 64 ? N * 1024 : 0;
+    static constexpr uint32_t kOffOut = kOffP + kPBytes;
+    static constexpr uint32_t kOffRed = kOffOut + kOutBytes; // float [N][4]
     static constexpr uint32_t kOffM = kOffRed + N * 16;      // float [N] running max, log2 domain
     static constexpr uint32_t kOffAlpha = kOffM + N * 4;     // float [N]
     static constexpr uint32_t kOffL = kOffAlpha + N * 4;     // float [N]
@@ -589,18 +593,55 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 ostride = kDV;
             }
             const int nvalid = min(N, p.head_end - head0);
+            bool staged = false;
+            if constexpr (N < 64) {
+                if (((reinterpret_cast<uintptr_t>(obase) | (uintptr_t)(ostride * 4)) & 15) == 0) {
+                    // Through shared memory and the bulk-copy engine: plain stores of this tile (one 128-byte line per
+                    // warp instruction, 64 of them per thread) take ~6,000 cycles while the cache streams, 2.5 times this.
+                    staged = true;
+                    float *stg = reinterpret_cast<float *>(smem + L::kOffOut);
 #pragma unroll 1
-            for (int j = 0; j < 4; ++j) {
-                const int dv = 128 * j + 32 * q4 + lane;
+                    for (int half = 0; half < 2; ++half) {
 #pragma unroll
-                for (int c = 0; c < N / 16; ++c) {
-                    float o[16];
-                    tmem_ld16(tmem_base + lane_addr + L::kColO + j * N + c * 16, o);
-                    tmem_wait_ld();
+                        for (int jj = 0; jj < 2; ++jj) {
+                            const int j = 2 * half + jj;
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const int n = c * 16 + k;
-                        if (n < nvalid) obase[(int64_t)n * ostride + dv] = o[k] * l_s[n];
+                            for (int c = 0; c < N / 16; ++c) {
+                                float o[16];
+                                tmem_ld16(tmem_base + lane_addr + L::kColO + j * N + c * 16, o);
+                                tmem_wait_ld();
+#pragma unroll
+                                for (int k = 0; k < 16; ++k) {
+                                    const int n = c * 16 + k;
+                                    stg[n * 256 + jj * 128 + 32 * q4 + lane] = o[k] * l_s[n];
+                                }
+                            }
+                        }
+                        fence_proxy_async();
+                        softmax_bar_sync();
+                        if (st < nvalid) {
+                            bulk_store(obase + (int64_t)st * ostride + half * 256, smem_u32(stg + st * 256), 1024);
+                            bulk_commit_group();
+                            bulk_wait_group_read();          // the row has left shared memory
+                        }
+                        softmax_bar_sync();
+                    }
+                }
+            }
+            if (!staged) {
+#pragma unroll 1
+                for (int j = 0; j < 4; ++j) {
+                    const int dv = 128 * j + 32 * q4 + lane;
+#pragma unroll
+                    for (int c = 0; c < N / 16; ++c) {
+                        float o[16];
+                        tmem_ld16(tmem_base + lane_addr + L::kColO + j * N + c * 16, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            const int n = c * 16 + k;
+                            if (n < nvalid) obase[(int64_t)n * ostride + dv] = o[k] * l_s[n];
+                        }
                     }
                 }
             }
@@ -609,6 +650,7 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             if (lane == 0) mbar_arrive(bar(kBarOEmpty));
             ++seg_it;
         }
+        bulk_wait_group();        // this thread's output rows have reached global memory
     }
 
     fill_empty_requests(p, worker, head0, N, tid, kThreads);

@@ -13,7 +13,7 @@
 // scale per head (e4m3 + e4m3, rebuilt per request by converter warps one request ahead; the two
 // terms sit side by side as 2N rows of one B operand and the softmax warps add the two halves of
 // S^T), and P = hi + lo with the token scale folded into the weight in the log domain,
-//     y = (q . codes) * qs_h * scale_t * softmax_scale * log2(e) + log2(scale_t),   P = 2^(y - m + 4.75),
+//     y = (q . codes) * qs_h * scale_t * softmax_scale * log2(e) + log2(scale_t),   P = 2^(y - m + 2.75),
 // the row sum adding P / scale_t.  Here the two terms of P are 2N columns of ONE B operand too, so that the
 // V tile -- the operand whose read from shared memory sets the pace of these narrow MMAs -- is read once
 // per tile instead of twice; O^T then has a hi and a lo half that the epilogue adds, which lets the lo
@@ -24,13 +24,13 @@
 // heads): the loop is a ring of dependent latencies and its period is the ring divided by the stages.
 //
 // The softmax warps keep one reference maximum per head and move it only when a logit exceeds it by
-// more than 2^4 (the headroom that e4m3's range leaves above the lift): whether any does is one
+// more than 2^6 (the headroom that e4m3's range leaves above the lift): whether any does is one
 // barrier-wide OR per tile, and only then do they reduce the maxima across tokens, move the
 // references and rescale O^T.  Row sums stay per thread until the request ends.
 //
-// Warp roles (352 threads): TMA producer (pages + scale pages, next page pulled into L2), 2 QK^T
-// issuers (one partial accumulator of S^T each), 2 P.V issuers (two dv blocks each), 4 softmax /
-// epilogue warps, 2 query converter warps (a request ahead: the query operands are double buffered).  Every wait is bounded; on expiry the CTA records
+// Warp roles (352 threads, 480 with 32 heads): TMA producer (pages + scale pages, next page pulled into L2), 2 QK^T
+// issuers (one partial accumulator of S^T each), 2 P.V issuers (two dv blocks each), N / 4 softmax /
+// epilogue warps (one per TMEM lane quadrant and group of 16 heads), 2 query converter warps (a request ahead: the query operands are double buffered).  Every wait is bounded; on expiry the CTA records
 // SPLASH_DEVICE_TIMEOUT and leaves in order.
 #include "splash_fp8.cuh"
 #include "splash_pair.cuh"
@@ -43,18 +43,19 @@ using namespace umma;
 
 constexpr int kQkWarps = 2;                        // = partial accumulators of S^T
 constexpr int kPvWarps = 2;                        // each owns two of the four dv blocks of O^T
-constexpr int kNumSoftmaxWarps = 4;
 constexpr int kWarpQk = 1;
 constexpr int kWarpPv = kWarpQk + kQkWarps;
 constexpr int kWarpSoftmax = kWarpPv + kPvWarps;            // 5: TMEM lane quadrant = warp & 3
-constexpr int kWarpConvert = kWarpSoftmax + kNumSoftmaxWarps;
 constexpr int kChunks = 9;                         // 576 / 64-element (64 B) chunks
 constexpr uint32_t kSlab = 64 * 64;                // one chunk of one page: 64 tokens x 64 B
 constexpr uint32_t kStageBytes = kChunks * kSlab;  // 36,864
 constexpr uint32_t kScaleBytes = 256;              // 64 fp32 token scales of a page
 constexpr int kMaxStages = 5;
-constexpr float kTau = 4.0f;                       // lazy rescale threshold, log2 units
-constexpr float kLift = 4.75f;                     // weights are stored as 2^(y - m + kLift) <= 2^8.75 = 431 < 448
+// A reference maximum moves when a logit exceeds it by more than kTau (log2 units); every move costs the tile a pass
+// over O^T behind the previous tile's P.V, and with 16 or 32 heads per CTA the moves of all heads add up (kTau = 4:
+// every third tile early in a request).  Weights are stored as 2^(y - m + kLift) <= 2^8.75 = 431 < 448.
+constexpr float kTau = 6.0f;
+constexpr float kLift = 2.75f;
 
 enum BarrierId {
     kBarKvFull = 0,                    // [stages]
@@ -74,8 +75,11 @@ enum BarrierId {
 template <int N>
 struct Layout {
     static constexpr int kStages = N == 16 ? 5 : 4;
+    static constexpr int kSoftmaxWarps = N / 4;                // one per TMEM lane quadrant and group of 16 heads
+    static constexpr int kSoftmaxThreads = 32 * kSoftmaxWarps;
+    static constexpr int kWarpConvert = kWarpSoftmax + kSoftmaxWarps;
     static constexpr int kNumConvertWarps = 2;                 // four threads per head, 16 heads per pass
-    static constexpr int kThreads = (kWarpConvert + kNumConvertWarps) * 32;   // 11 warps = 352 threads
+    static constexpr int kThreads = (kWarpConvert + kNumConvertWarps) * 32;   // 352 (N = 16) or 480 (N = 32)
     static constexpr uint32_t kQSlab = 2 * N * 64;             // one chunk of the query operand: (N hi rows, N lo rows) x 64 B
     static constexpr uint32_t kQBytes = kChunks * kQSlab;      // one buffer; there are two (request parity)
     static constexpr uint32_t kPBytes = 2 * N * 64;            // P^T: [2N / 16 groups: hi, then lo][64 tokens][16 heads], one byte each
@@ -119,7 +123,8 @@ template <int N>
 __global__ void __launch_bounds__(Layout<N>::kThreads, 1)
 decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tmap_kv) {
     using L = Layout<N>;
-    constexpr int kStages = L::kStages, kThreads = L::kThreads;
+    constexpr int kStages = L::kStages, kThreads = L::kThreads, kNumSoftmaxWarps = L::kSoftmaxWarps, kWarpConvert = L::kWarpConvert;
+    constexpr int kSoftmaxThreads = L::kSoftmaxThreads;
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t sbase = smem_u32(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -330,17 +335,23 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 const uint4 *src = reinterpret_cast<const uint4 *>(
                     static_cast<const __nv_bfloat16 *>(p.q) + (int64_t)seg.request * p.q_stride_request +
                     (int64_t)(live ? gh : p.head_begin) * p.q_stride_head + part * (kVecs * 8));
-                uint4 x[kVecs];
-#pragma unroll
-                for (int v = 0; v < kVecs; ++v) x[v] = live ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
+                // 16 heads keep the quarter row in registers between the two passes; with 32 heads (480 threads, 128
+                // registers each) it is read again, nine vectors at a time, from the cache it has just come into
+                constexpr int kBatch = N == 16 ? kVecs : kVecs / 2;
+                uint4 x[kBatch];
                 float amax = 0.f;
+#pragma unroll 1
+                for (int v0 = 0; v0 < kVecs; v0 += kBatch) {
 #pragma unroll
-                for (int v = 0; v < kVecs; ++v) {
-                    const uint32_t w[4] = {x[v].x, x[v].y, x[v].z, x[v].w};
+                    for (int v = 0; v < kBatch; ++v) x[v] = live ? __ldg(src + v0 + v) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        amax = fmaxf(amax, fabsf(__uint_as_float(w[k] << 16)));
-                        amax = fmaxf(amax, fabsf(__uint_as_float(w[k] & 0xffff0000u)));
+                    for (int v = 0; v < kBatch; ++v) {
+                        const uint32_t w[4] = {x[v].x, x[v].y, x[v].z, x[v].w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            amax = fmaxf(amax, fabsf(__uint_as_float(w[k] << 16)));
+                            amax = fmaxf(amax, fabsf(__uint_as_float(w[k] & 0xffff0000u)));
+                        }
                     }
                 }
                 amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
@@ -348,27 +359,34 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 const float qs = amax > 0.f ? amax * (1.0f / 448.0f) : 1.0f;
                 const float inv = amax > 0.f ? 448.0f / amax : 1.0f;
                 if (pass == 0) {
-                    // this buffer's previous request (two back): its QK^T retired, its softmax under way
+                    // this buffer's previous request (two back): its QK^T retired, its output tile staged and gone
                     ok = mbar_wait(ctx, bar(kBarQEmpty + qb), ((seg_it >> 1) & 1) ^ 1, kBarQEmpty + qb);
                     if (!ok) break;
                 }
                 if (part == 0) qs_s[(seg_it & 3) * N + hd] = qs;
+#pragma unroll 1
+                for (int v0 = 0; v0 < kVecs; v0 += kBatch) {
+                    if (kBatch < kVecs) {
 #pragma unroll
-                for (int v = 0; v < kVecs; ++v) {
-                    const uint32_t w[4] = {x[v].x, x[v].y, x[v].z, x[v].w};
-                    uint16_t hi[4], lo[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const float e0 = __uint_as_float(w[k] << 16) * inv, e1 = __uint_as_float(w[k] & 0xffff0000u) * inv;
-                        split_e4m3_e4m3_x2(e0, e1, hi[k], lo[k]);
+                        for (int v = 0; v < kBatch; ++v) x[v] = live ? __ldg(src + v0 + v) : make_uint4(0u, 0u, 0u, 0u);
                     }
-                    const uint32_t d = (uint32_t)(part * (kVecs * 8) + v * 8);
-                    // the lo rows follow the N hi rows of the chunk (N is a multiple of 8: same swizzle phase)
-                    const uint32_t off = (d >> 6) * L::kQSlab + sw64((uint32_t)hd, d & 63);
-                    *reinterpret_cast<uint2 *>(qdst + off) =
-                        make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
-                    *reinterpret_cast<uint2 *>(qdst + N * 64 + off) =
-                        make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
+#pragma unroll
+                    for (int v = 0; v < kBatch; ++v) {
+                        const uint32_t w[4] = {x[v].x, x[v].y, x[v].z, x[v].w};
+                        uint16_t hi[4], lo[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float e0 = __uint_as_float(w[k] << 16) * inv, e1 = __uint_as_float(w[k] & 0xffff0000u) * inv;
+                            split_e4m3_e4m3_x2(e0, e1, hi[k], lo[k]);
+                        }
+                        const uint32_t d = (uint32_t)(part * (kVecs * 8) + (v0 + v) * 8);
+                        // the lo rows follow the N hi rows of the chunk (N is a multiple of 8: same swizzle phase)
+                        const uint32_t off = (d >> 6) * L::kQSlab + sw64((uint32_t)hd, d & 63);
+                        *reinterpret_cast<uint2 *>(qdst + off) =
+                            make_uint2((uint32_t)hi[0] | ((uint32_t)hi[1] << 16), (uint32_t)hi[2] | ((uint32_t)hi[3] << 16));
+                        *reinterpret_cast<uint2 *>(qdst + N * 64 + off) =
+                            make_uint2((uint32_t)lo[0] | ((uint32_t)lo[1] << 16), (uint32_t)lo[2] | ((uint32_t)lo[3] << 16));
+                    }
                 }
             }
             if (!ok) break;
@@ -380,14 +398,16 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
     } else {
         // ===================================================== softmax + epilogue warps
         const int q4 = warp & 3;                       // TMEM lane quadrant of this warp
-        const int sw = warp - kWarpSoftmax;            // softmax warp 0..3
-        const int st = sw * 32 + lane;                 // 0..127
+        const int sw = warp - kWarpSoftmax;            // softmax warp
+        const int wq = sw & 3;                         // its slot in the per-head exchange of four
+        const int h0 = 16 * (sw >> 2);                 // its group of 16 heads
+        const int st = sw * 32 + lane;                 // 0 .. 8N
         // S^T comes out of tensor memory in the accumulator fragment layout, which spreads the 16 lanes that an
         // M = 64 tile has per quadrant over all 32 threads: this thread holds tokens rA and rB = rA + 8 and, of each
-        // group of eight heads, heads 2 tq and 2 tq + 1.
+        // group of eight heads (its warp has two), heads 2 tq and 2 tq + 1.
         const int rA = 16 * q4 + (lane >> 2), rB = rA + 8;
         const int tq = lane & 3;
-        constexpr int kR = N / 8;                      // groups of eight heads
+        constexpr int kR = 2;                          // groups of eight heads per warp
         const uint32_t lane_addr = (uint32_t)(32 * q4) << 16;
         float *red = reinterpret_cast<float *>(smem + L::kOffRed);
         float *m_s = reinterpret_cast<float *>(smem + L::kOffM);
@@ -408,7 +428,7 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
             float l[2 * kR];              // sums of P / scale_t over this thread's tokens: heads 8k + 2 tq + e at [2k + e]
 #pragma unroll
             for (int n = 0; n < 2 * kR; ++n) l[n] = 0.f;
-            softmax_bar_sync();
+            named_bar_sync<1, kSoftmaxThreads>();
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;
             for (int i = 0; i < ntiles; ++i) {
@@ -424,11 +444,11 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 {
                     // S^T = the sum of four N-column pieces: (partial 0, partial 1) x (q hi, q lo)
                     float t0[4 * kR], t1[4 * kR], t2[4 * kR];
-                    const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (2 * kQkWarps * N);
-                    tmem_ld_frag<N>(sb, s);
-                    tmem_ld_frag<N>(sb + N, t0);
-                    tmem_ld_frag<N>(sb + 2 * N, t1);
-                    tmem_ld_frag<N>(sb + 3 * N, t2);
+                    const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (2 * kQkWarps * N) + h0;
+                    tmem_ld_16x256b_x2(sb, s);
+                    tmem_ld_16x256b_x2(sb + N, t0);
+                    tmem_ld_16x256b_x2(sb + 2 * N, t1);
+                    tmem_ld_16x256b_x2(sb + 3 * N, t2);
                     tmem_wait_ld();
 #pragma unroll
                     for (int n = 0; n < 4 * kR; ++n) s[n] = (s[n] + t0[n]) + (t1[n] + t2[n]);
@@ -443,8 +463,8 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 bool exceeds = false;     // some logit of these tokens lies more than kTau above its head's reference
 #pragma unroll
                 for (int k = 0; k < kR; ++k) {
-                    const float2 q2 = *reinterpret_cast<const float2 *>(&qs_s[8 * k + 2 * tq]);
-                    const float2 m2 = *reinterpret_cast<const float2 *>(&m_s[8 * k + 2 * tq]);
+                    const float2 q2 = *reinterpret_cast<const float2 *>(&qs_s[h0 + 8 * k + 2 * tq]);
+                    const float2 m2 = *reinterpret_cast<const float2 *>(&m_s[h0 + 8 * k + 2 * tq]);
 #pragma unroll
                     for (int e = 0; e < 2; ++e) {
                         const float qv = e ? q2.y : q2.x, lim = (e ? m2.y : m2.x) + kTau;
@@ -455,7 +475,7 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                         exceeds |= (yA > lim) | (yB > lim);
                     }
                 }
-                const bool grew = softmax_bar_or(exceeds);
+                const bool grew = named_bar_or<1, kSoftmaxThreads>(exceeds);
                 if (grew) {
                     // the rare path (the first tile of a request, then a handful of times): per-head maxima over the
                     // tile's tokens, new references for the heads that grew, their rescale factors
@@ -467,10 +487,10 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
                             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
                             mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-                            if (lane < 4) red[(8 * k + 2 * tq + e) * 4 + sw] = mx;
+                            if (lane < 4) red[(h0 + 8 * k + 2 * tq + e) * 4 + wq] = mx;
                         }
                     }
-                    softmax_bar_sync();
+                    named_bar_sync<1, kSoftmaxThreads>();
                     if (st < N) {
                         float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
                         float mt = fmaxf(fmaxf(r4.x, r4.y), fmaxf(r4.z, r4.w));
@@ -482,17 +502,17 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                         }
                         alpha_s[st] = al;
                     }
-                    softmax_bar_sync();
+                    named_bar_sync<1, kSoftmaxThreads>();
 #pragma unroll
                     for (int k = 0; k < kR; ++k) {
-                        const float2 a2 = *reinterpret_cast<const float2 *>(&alpha_s[8 * k + 2 * tq]);
+                        const float2 a2 = *reinterpret_cast<const float2 *>(&alpha_s[h0 + 8 * k + 2 * tq]);
                         l[2 * k] *= a2.x; l[2 * k + 1] *= a2.y;
                     }
                 }
                 uint16_t hiA[kR], loA[kR], hiB[kR], loB[kR];      // two adjacent heads per 16-bit word
 #pragma unroll
                 for (int k = 0; k < kR; ++k) {
-                    const float2 m2 = *reinterpret_cast<const float2 *>(&m_s[8 * k + 2 * tq]);
+                    const float2 m2 = *reinterpret_cast<const float2 *>(&m_s[h0 + 8 * k + 2 * tq]);
                     const float o0 = kLift - m2.x, o1 = kLift - m2.y;
                     const float a0 = fast_exp2(s[4 * k + 0] + o0), a1 = fast_exp2(s[4 * k + 1] + o1);
                     const float b0 = fast_exp2(s[4 * k + 2] + o0), b1 = fast_exp2(s[4 * k + 3] + o1);
@@ -513,7 +533,7 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                     ok &= mbar_wait(ctx, bar(kBarKvEmpty + prev % kStages), (prev / kStages) & 1, kBarKvEmpty + prev % kStages);
                     tcgen05_fence_after();
 #pragma unroll 1
-                    for (int c = 0; c < 8 * N / 16; ++c) {
+                    for (int c = sw >> 2; c < 8 * N / 16; c += N / 16) {      // the warps of a quadrant share its columns
                         float o[16];
                         const uint32_t addr = tmem_base + lane_addr + L::kColO + c * 16;
                         tmem_ld16(addr, o);
@@ -530,7 +550,7 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                     uint8_t *pa = smem + L::kOffP + (s_it & 1) * L::kPBytes + rA * 16 + 2 * tq;
 #pragma unroll
                     for (int k = 0; k < kR; ++k) {
-                        uint8_t *ph = pa + (k >> 1) * 1024 + (k & 1) * 8, *pl = ph + (N / 16) * 1024;
+                        uint8_t *ph = pa + (h0 >> 4) * 1024 + k * 8, *pl = ph + (N / 16) * 1024;
                         *reinterpret_cast<uint16_t *>(ph) = hiA[k]; *reinterpret_cast<uint16_t *>(ph + 8 * 16) = hiB[k];
                         *reinterpret_cast<uint16_t *>(pl) = loA[k]; *reinterpret_cast<uint16_t *>(pl + 8 * 16) = loB[k];
                     }
@@ -549,9 +569,9 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                 v += __shfl_xor_sync(0xffffffffu, v, 4);
                 v += __shfl_xor_sync(0xffffffffu, v, 8);
                 v += __shfl_xor_sync(0xffffffffu, v, 16);
-                if (lane < 4) red[(8 * (n >> 1) + 2 * tq + (n & 1)) * 4 + sw] = v;
+                if (lane < 4) red[(h0 + 8 * (n >> 1) + 2 * tq + (n & 1)) * 4 + wq] = v;
             }
-            softmax_bar_sync();
+            named_bar_sync<1, kSoftmaxThreads>();
             if (st < N) {
                 float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
                 float l = (r4.x + r4.y) + (r4.z + r4.w);
@@ -563,7 +583,7 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                     else p.partial_lse[(int64_t)seg.slot * h + (gh - p.head_begin)] = lse;
                 }
             }
-            softmax_bar_sync();
+            named_bar_sync<1, kSoftmaxThreads>();
             // ---- epilogue: O^T block j holds dv = 128 j + TMEM lane, one column per head
             ok &= mbar_wait(ctx, bar(kBarOFull), seg_it & 1, kBarOFull);
             tcgen05_fence_after();
@@ -589,8 +609,8 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
 #pragma unroll
                     for (int jj = 0; jj < 2; ++jj) {
                         const int j = 2 * half + jj;
-#pragma unroll
-                        for (int c = 0; c < N / 16; ++c) {
+                        {
+                            const int c = sw >> 2;        // this warp's 16 heads of the block
                             float o[16], o_lo[16];
                             tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + c * 16, o);
                             tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + N + c * 16, o_lo);
@@ -603,20 +623,20 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
                         }
                     }
                     fence_proxy_async();
-                    softmax_bar_sync();
+                    named_bar_sync<1, kSoftmaxThreads>();
                     if (st < nvalid) {
                         bulk_store(obase + (int64_t)st * ostride + half * 256, smem_u32(stg + st * 256), 1024);
                         bulk_commit_group();
                         bulk_wait_group_read();          // the row has left shared memory
                     }
-                    softmax_bar_sync();
+                    named_bar_sync<1, kSoftmaxThreads>();
                 }
             } else {
 #pragma unroll 1
                 for (int j = 0; j < 4; ++j) {
                     const int dv = 128 * j + 32 * q4 + lane;
-#pragma unroll
-                    for (int c = 0; c < N / 16; ++c) {
+                    {
+                        const int c = sw >> 2;
                         float o[16], o_lo[16];
                         tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + c * 16, o);
                         tmem_ld16(tmem_base + lane_addr + L::kColO + j * (2 * N) + N + c * 16, o_lo);
