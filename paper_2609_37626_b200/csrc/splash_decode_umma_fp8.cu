@@ -8,11 +8,11 @@
 // are each split into two e4m3 terms that accumulate into the same fp32 accumulator:
 //
 //   q_h   = qs_h * (hi + lo),  qs_h = max|q_h| / 448, hi = e4m3(q/qs), lo = e4m3(q/qs - hi)
-//   P_ht  = u_hi + u_lo,       u = 2^(y - m + 4) with y = log2-domain logit + log2(scale_t)
+//   P_ht  = u_hi + u_lo,       u = 2^(y - m + 2.75) with y = log2-domain logit + log2(scale_t)
 //
 // i.e. the per-token scale is folded into the softmax weight in the log domain, so the
-// weights of a tile are automatically normalised (u <= 2^8 with the lazy-rescale threshold
-// of 2^4) and sit in e4m3's normal range; the row sum adds u / scale_t = 2^(x - m + 4).
+// weights of a tile are automatically normalised (u <= 2^8.75 with the lazy-rescale threshold
+// of 2^6) and sit in e4m3's range; the row sum adds u / scale_t = 2^(x - m + 2.75).
 // Four e4m3 products per bf16-precision product pair cost the tensor pipe the same time as
 // the bf16 kernel (fp8 MMAs run at twice the rate), which is why the roofline of this
 // workload is taken at the bf16 rate.
@@ -37,8 +37,11 @@ constexpr uint32_t kSlab = 64 * 64;                // one chunk of one page: 64 
 constexpr uint32_t kStageBytes = kChunks * kSlab;  // 36,864
 constexpr uint32_t kScaleBytes = 256;              // 64 fp32 token scales of a page
 constexpr int kStages = 3;
-constexpr float kTau = 4.0f;                       // lazy rescale threshold, log2 units
-constexpr float kLift = 4.75f;                     // weights are stored as 2^(y - m + kLift) <= 2^8.75 = 431 < 448
+// lazy rescale threshold, log2 units: with 64 heads per CTA every move of any head's reference costs the tile a pass over
+// O^T (at 2^4 the long-context and the many-request timings were 7-9 % slower); weights are stored as
+// 2^(y - m + kLift) <= 2^8.75 = 431 < 448
+constexpr float kTau = 6.0f;
+constexpr float kLift = 2.75f;
 
 enum BarrierId {
     kBarKvFull = 0,
