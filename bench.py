@@ -295,7 +295,7 @@ class GpuBench:
                              "launch_chains": 1, "cta_pairs_per_kv_worker": -(-h * R // 128)},
                 "launches_per_step": binding.splash_last_launch_count()}
 
-    def slice_workload(self, w, dw, out, lse, head_begin, head_end, steps, warmup, peaks):
+    def slice_workload(self, w, dw, out, lse, head_begin, head_end, steps, warmup, peaks, traffic=None):
         """A TP rank's share of workload `w`: the same cache and requests, heads [head_begin, head_end) only."""
         import copy
         torch, binding = self.torch, self.binding
@@ -325,7 +325,7 @@ class GpuBench:
                 "tokens_per_s": w.B / (ms.mean() * 1e-3), "launches_per_step": launches, "heads": hs,
                 "requests": w.B, "tokens": w.total_tokens(),
                 "roofline": {"bound": "hbm", "achieved": alg_bytes / (dec_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                             "unit": "GB/s", "frac": t_hbm / dec_ms, "frac_whole_call": t_hbm / p50, "traffic": None,
+                             "unit": "GB/s", "frac": t_hbm / dec_ms, "frac_whole_call": t_hbm / p50, "traffic": traffic,
                              "kernel": kernel, "kernel_ms": dec_ms, "plan_ms": float(kt[:, 0].mean()),
                              "combine_ms": float(kt[:, 2].mean()), "algorithmic_bytes": alg_bytes,
                              "roofline_ms": t_hbm, "peak_source": peaks["source"]}}
@@ -692,6 +692,8 @@ def main():
     ap.add_argument("--only-main", action="store_true", help="skip the other configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sparse-only", action="store_true", help="print only the sparse-decode workload's numbers")
+    ap.add_argument("--head-slice", default=None, metavar="BEGIN:END",
+                    help="time a TP rank's share of the workload: the same cache and requests, heads [BEGIN, END) only")
     ap.add_argument("--stub-step", action="store_true",
                     help="CPU test of the launcher and the rank plumbing: gloo, a host stand-in for the step, no measurement")
     args = ap.parse_args()
@@ -739,6 +741,13 @@ def main():
         w = W.make_workload(w.name, W.BASE_SEED + idx + 100 * rank, w.seq_lens, H=w.H, head_begin=w.head_begin,
                             head_end=w.head_end, kv_dtype=w.kv_dtype)
     gen_s = time.time() - t_gen
+    traffic_key = args.workload
+    if args.head_slice:
+        hb, he = (int(x) for x in args.head_slice.split(":"))
+        if not (0 <= hb < he <= w.H):
+            raise SystemExit("--head-slice must lie inside the workload's %d heads" % w.H)
+        w.head_begin, w.head_end = hb, he
+        traffic_key = "%s_heads%d" % (args.workload, he - hb)
 
     if args.sparse_only:
         w2 = W.config(2)
@@ -751,7 +760,7 @@ def main():
     if not stub:
         torch.cuda.synchronize()
         sampler.start()
-    main_res, dw, out, lse = gb.decode_workload(w, args.steps, args.warmup, peaks, traffic, args.workload)
+    main_res, dw, out, lse = gb.decode_workload(w, args.steps, args.warmup, peaks, traffic, traffic_key)
     if stub:
         if world > 1:
             dist.barrier()
@@ -791,7 +800,7 @@ def main():
             steps2 = max(5, args.steps // 2)
             if idx == 5:
                 try:
-                    extra["c5"] = {"tp8_slice": gb.slice_workload(w, dw, out, lse, 32, 48, steps2, args.warmup, peaks),
+                    extra["c5"] = {"tp8_slice": gb.slice_workload(w, dw, out, lse, 32, 48, steps2, args.warmup, peaks, traffic.get("c5_heads16")),
                                    "page_migrate": gb.migrate_workload(w, dw, steps2, args.warmup, peaks),
                                    "migrate_under_decode": gb.overlap_workload(w, dw, steps2, args.warmup)}
                 except Exception as exc:  # report, do not hide
@@ -814,7 +823,7 @@ def main():
                         r["cp"] = gb.cp_workload(wx, steps2, args.warmup)
                     if name == "c5":
                         # a TP-8 rank's share of the same step: 16 of the 128 heads over the same e4m3 cache
-                        r["tp8_slice"] = gb.slice_workload(wx, dwx, ox, lx, 32, 48, steps2, args.warmup, peaks)
+                        r["tp8_slice"] = gb.slice_workload(wx, dwx, ox, lx, 32, 48, steps2, args.warmup, peaks, traffic.get("c5_heads16"))
                         r["page_migrate"] = gb.migrate_workload(wx, dwx, steps2, args.warmup, peaks)
                         r["migrate_under_decode"] = gb.overlap_workload(wx, dwx, steps2, args.warmup)
                     extra[name] = r
