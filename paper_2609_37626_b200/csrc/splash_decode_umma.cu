@@ -100,40 +100,6 @@ struct Layout {
     static_assert(kOffQ % 1024 == 0 && kOffP % 1024 == 0 && (N * 128) % 1024 == 0, "swizzle atoms need 1024-byte alignment");
 };
 
-// Reduce-scatter over the 32 lanes of a warp: on return lane L holds, in v[0 .. max(1, N/32)),
-// the reduction over all lanes of the entries it owns (N = 64: heads 2L, 2L+1; N = 32: head L;
-// N = 16: head L >> 1, both lanes of a pair holding it).
-template <int CNT, int MASK, bool IS_MAX>
-struct ReduceScatter {
-    template <int N>
-    static __device__ __forceinline__ void run(float (&v)[N], int lane) {
-        if constexpr (MASK >= 1) {
-            if constexpr (CNT > 1) {
-                constexpr int kHalf = CNT / 2;
-                const bool upper = (lane & MASK) != 0;
-#pragma unroll
-                for (int i = 0; i < kHalf; ++i) {
-                    float keep = upper ? v[i + kHalf] : v[i];
-                    float send = upper ? v[i] : v[i + kHalf];
-                    float recv = __shfl_xor_sync(0xffffffffu, send, MASK);
-                    v[i] = IS_MAX ? fmaxf(keep, recv) : keep + recv;
-                }
-                ReduceScatter<kHalf, MASK / 2, IS_MAX>::run(v, lane);
-            } else {
-                float recv = __shfl_xor_sync(0xffffffffu, v[0], MASK);
-                v[0] = IS_MAX ? fmaxf(v[0], recv) : v[0] + recv;
-                ReduceScatter<1, MASK / 2, IS_MAX>::run(v, lane);
-            }
-        }
-    }
-};
-
-template <int N>
-__device__ __forceinline__ int owned_head(int lane, int i) {
-    if (N >= 32) return lane * (N / 32) + i;
-    return lane >> 1;     // N == 16
-}
-
 // ---------------------------------------------------------------- the kernel
 template <int N>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -246,7 +212,8 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             const int mw = warp - 1;                 // issuer index: S^T accumulator mw, dv block mw
             const bool does_qk = mw < L::kAcc;
             constexpr uint32_t kIdescQK = L::kHeadsOnM ? make_idesc(64, 64, 0, 0) : make_idesc(64, N, 0, 0);
-            constexpr uint32_t kIdescPV = make_idesc(128, N, 1, 0);
+            // P^T is K-major (swizzled) when the softmax has the heads on M, MN-major (plain) when it has the tokens on M
+            constexpr uint32_t kIdescPV = make_idesc(128, N, 1, L::kHeadsOnM ? 0 : 1);
             uint32_t kv_it = 0, s_it = 0, p_it = 0, seg_it = 0;
             bool ok = true;
             // This issuer's share of S^T for the tile with global index kv: the K = 16 steps
@@ -278,7 +245,9 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                 for (int k = 0; k < 4; ++k) {
                     // A: two 64-element chunks (LBO apart) x 16 tokens (SBO per 8 tokens), MN-major
                     uint64_t da = make_desc(v0 + k * 2048, kSlabBytes, 1024);
-                    uint64_t db = make_desc(p0 + k * 32, 16, 1024);
+                    // B: 16 tokens x N heads.  K-major: 32 B into the swizzled rows; MN-major: two groups of eight tokens
+                    // (128 B apart) x groups of eight heads (1,024 B apart)
+                    uint64_t db = L::kHeadsOnM ? make_desc(p0 + k * 32, 16, 1024) : make_desc_mn_plain(p0 + k * 256, 128, 1024);
                     umma_bf16(tmem_base + L::kColO + mw * N, da, db, kIdescPV, (!first_tile) || k != 0);
                 }
             };
@@ -339,14 +308,12 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
         const int q4 = warp & 3;                       // TMEM lane quadrant of this warp
         const int sw = warp - 1 - kMmaWarps;           // softmax warp 0..3
         const int st = sw * 32 + lane;                 // 0..127
-        const int row = 16 * q4 + lane;                // token row of the S^T tile (lanes < 16)
         const uint32_t lane_addr = (uint32_t)(32 * q4) << 16;
         float *red = reinterpret_cast<float *>(smem + L::kOffRed);
         float *m_s = reinterpret_cast<float *>(smem + L::kOffM);
         float *alpha_s = reinterpret_cast<float *>(smem + L::kOffAlpha);
         float *l_s = reinterpret_cast<float *>(smem + L::kOffL);
         const float scale_log2 = p.softmax_scale * kLog2e;
-        constexpr int kOwn = N >= 32 ? N / 32 : 1;
         uint32_t s_it = 0, p_it = 0, seg_it = 0;
         // A failed (timed-out) wait only clears `ok`: the role keeps walking its tiles so that every thread still
         // meets the named barriers -- once the CTA aborts, waits return at once.
@@ -356,15 +323,16 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             // heads-on-M: this thread's two heads (reference maxima; partial row sums over its tokens)
             const int hA = 16 * q4 + (lane >> 2);
             float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;
-            float l_own[kOwn];            // running sums of the heads this lane owns (this warp's 16 tokens)
+            // tokens on M: sums over this thread's two tokens, heads 8k + 2 tq + e at [2k + e]
+            constexpr int kR = L::kHeadsOnM ? 1 : N / 8;
+            float l_tk[2 * kR];
 #pragma unroll
-            for (int k = 0; k < kOwn; ++k) l_own[k] = 0.f;
+            for (int k = 0; k < 2 * kR; ++k) l_tk[k] = 0.f;
             softmax_bar_sync();
             const int first_page = seg.lo / kPage;
             const int ntiles = seg.tile_end - seg.tile_begin;
             for (int i = 0; i < ntiles; ++i) {
                 const TileGeom g = tile_geom(seg.lo, seg.hi, (first_page + seg.tile_begin + i) * kPage);
-                const bool valid = lane < 16 && row >= g.r_lo && row < g.r_hi;
                 const uint32_t b = s_it % L::kSBufs;
                 ok &= mbar_wait(ctx, bar(kBarSFull + b), (s_it / L::kSBufs) & 1, kBarSFull + b);
                 if (st == 0) mark(s_it, 4);
@@ -452,60 +420,85 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                     }
                 }
                 } else {
-                float s[N];
+                // ---- tokens on M.  S^T [64 tokens x N heads] sits in 16 lanes per TMEM quadrant; the fragment load
+                // spreads them over all 32 threads: this thread holds tokens rA = 16 q4 + lane/4 and rB = rA + 8 and,
+                // of each group of eight heads, heads 2 tq and 2 tq + 1.
+                const int rA = 16 * q4 + (lane >> 2), rB = rA + 8, tq = lane & 3;
+                const bool vA = rA >= g.r_lo && rA < g.r_hi, vB = rB >= g.r_lo && rB < g.r_hi;
+                float s[4 * kR];
                 {
+                    float t0[4 * kR], t1[4 * kR], t2[4 * kR];
                     const uint32_t sb = tmem_base + lane_addr + L::kColS + b * (L::kAcc * N);
+                    tmem_ld_frag<N>(sb, s);
+                    tmem_ld_frag<N>(sb + N, t0);
+                    tmem_ld_frag<N>(sb + 2 * N, t1);
+                    tmem_ld_frag<N>(sb + 3 * N, t2);
+                    tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < N / 16; ++c)
-                        tmem_ld16(sb + c * 16, *reinterpret_cast<float(*)[16]>(&s[c * 16]));
-#pragma unroll
-                    for (int a = 1; a < L::kAcc; ++a) {
-                        float part[N];
-#pragma unroll
-                        for (int c = 0; c < N / 16; ++c)
-                            tmem_ld16(sb + a * N + c * 16, *reinterpret_cast<float(*)[16]>(&part[c * 16]));
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int n = 0; n < N; ++n) s[n] += part[n];
-                    }
+                    for (int n = 0; n < 4 * kR; ++n) s[n] = (s[n] + t0[n]) + (t1[n] + t2[n]);
+                    static_assert(L::kAcc == 4, "four partial accumulators are summed here");
                 }
-                tmem_wait_ld();
                 tcgen05_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar(kBarSEmpty + b));
-                float mx[N];
+                // One reference maximum per head, moved only when a logit exceeds it by more than the threshold: whether
+                // any does is one barrier-wide OR; the common tile needs no reduction over tokens at all.
+                bool exceeds = false;
 #pragma unroll
-                for (int n = 0; n < N; ++n) { s[n] = valid ? s[n] * scale_log2 : -INFINITY; mx[n] = s[n]; }
-                ReduceScatter<N, 16, true>::run(mx, lane);
-                if (N >= 32 || (lane & 1) == 0) {
+                for (int k = 0; k < kR; ++k) {
+                    const float2 m2 = *reinterpret_cast<const float2 *>(&m_s[8 * k + 2 * tq]);
 #pragma unroll
-                    for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + sw] = mx[k];
-                }
-                if (st == 0) misc[2 + (i & 1)] = 0;      // this tile's "some maximum grew" flag
-                softmax_bar_sync();
-                if (st < N) {
-                    float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
-                    float mt = fmaxf(fmaxf(r4.x, r4.y), fmaxf(r4.z, r4.w));
-                    float m_old = m_s[st];
-                    float al = 1.f;
-                    if (mt > m_old + kRescaleThreshold) {        // also taken when m_old = -inf
-                        al = (m_old == -INFINITY) ? 0.f : fast_exp2(m_old - mt);
-                        m_s[st] = mt;
-                        misc[2 + (i & 1)] = 1;
+                    for (int e = 0; e < 2; ++e) {
+                        const float lim = (e ? m2.y : m2.x) + kRescaleThreshold;
+                        const float yA = vA ? s[4 * k + e] * scale_log2 : -INFINITY;
+                        const float yB = vB ? s[4 * k + 2 + e] * scale_log2 : -INFINITY;
+                        s[4 * k + e] = yA; s[4 * k + 2 + e] = yB;
+                        exceeds |= (yA > lim) | (yB > lim);
                     }
-                    alpha_s[st] = al;
                 }
-                softmax_bar_sync();
-                const bool rescale = misc[2 + (i & 1)] != 0;
+                const bool rescale = softmax_bar_or(exceeds);
                 if (rescale) {
+                    // the rare path (the first tile of a request, then a handful of times): per-head maxima over the
+                    // tile's tokens, new references for the heads that grew, their rescale factors
 #pragma unroll
-                    for (int k = 0; k < kOwn; ++k) l_own[k] *= alpha_s[owned_head<N>(lane, k)];
+                    for (int k = 0; k < kR; ++k) {
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            float mx = fmaxf(s[4 * k + e], s[4 * k + 2 + e]);
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                            if (lane < 4) red[(8 * k + 2 * tq + e) * 4 + sw] = mx;
+                        }
+                    }
+                    softmax_bar_sync();
+                    if (st < N) {
+                        float4 r4 = *reinterpret_cast<const float4 *>(&red[st * 4]);
+                        float mt = fmaxf(fmaxf(r4.x, r4.y), fmaxf(r4.z, r4.w));
+                        float m_old = m_s[st];
+                        float al = 1.f;
+                        if (mt > m_old + kRescaleThreshold) {        // also taken when m_old = -inf
+                            al = (m_old == -INFINITY) ? 0.f : fast_exp2(m_old - mt);
+                            m_s[st] = mt;
+                        }
+                        alpha_s[st] = al;
+                    }
+                    softmax_bar_sync();
+#pragma unroll
+                    for (int k = 0; k < kR; ++k) {
+                        const float2 a2 = *reinterpret_cast<const float2 *>(&alpha_s[8 * k + 2 * tq]);
+                        l_tk[2 * k] *= a2.x; l_tk[2 * k + 1] *= a2.y;
+                    }
                 }
+                uint32_t pA[kR], pB[kR];          // two adjacent heads per word
 #pragma unroll
-                for (int n = 0; n < N; ++n) { s[n] = fast_exp2(s[n] - m_s[n]); mx[n] = s[n]; }
-                ReduceScatter<N, 16, false>::run(mx, lane);      // per-head sums over this warp's tokens
-#pragma unroll
-                for (int k = 0; k < kOwn; ++k) l_own[k] += mx[k];
+                for (int k = 0; k < kR; ++k) {
+                    const float2 m2 = *reinterpret_cast<const float2 *>(&m_s[8 * k + 2 * tq]);
+                    const float a0 = fast_exp2(s[4 * k + 0] - m2.x), a1 = fast_exp2(s[4 * k + 1] - m2.y);
+                    const float b0 = fast_exp2(s[4 * k + 2] - m2.x), b1 = fast_exp2(s[4 * k + 3] - m2.y);
+                    l_tk[2 * k] += a0 + b0; l_tk[2 * k + 1] += a1 + b1;
+                    pA[k] = pack_bf16x2(a0, a1); pB[k] = pack_bf16x2(b0, b1);
+                }
                 // P.V of the previous tile must be done with the P buffer and with O^T
                 if (s_it > 0) {
                     const uint32_t prev = s_it - 1;
@@ -525,14 +518,14 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                     }
                     tmem_wait_st();
                 }
-                if (lane < 16) {
-                    // P^T as the K-major, 128-byte-swizzled B operand: row = head, 64 tokens per row
-                    uint8_t *pb = smem + L::kOffP;
-                    const uint32_t chunk = (uint32_t)row >> 3, within = ((uint32_t)row & 7) * 2;
+                {
+                    // P^T as the MN-major B operand: eight heads of a token are 16 adjacent bytes, groups of eight heads
+                    // 1,024 B apart
+                    uint8_t *pa = smem + L::kOffP + rA * 16 + tq * 4;
 #pragma unroll
-                    for (int n = 0; n < N; ++n) {
-                        __nv_bfloat16 v = __float2bfloat16_rn(s[n]);
-                        *reinterpret_cast<__nv_bfloat16 *>(pb + n * 128 + ((chunk ^ (uint32_t)(n & 7)) << 4) + within) = v;
+                    for (int k = 0; k < kR; ++k) {
+                        *reinterpret_cast<uint32_t *>(pa + k * 1024) = pA[k];
+                        *reinterpret_cast<uint32_t *>(pa + k * 1024 + 8 * 16) = pB[k];
                     }
                 }
                 }
@@ -561,10 +554,15 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
                     }
                 }
             } else {
-                // ---- row sums over all 128 lanes' partial sums
-                if (N >= 32 || (lane & 1) == 0) {
+                // ---- row sums: over the 16 tokens of a warp (the eight threads with this tq), then over the four warps
+                const int tq = lane & 3;
 #pragma unroll
-                    for (int k = 0; k < kOwn; ++k) red[owned_head<N>(lane, k) * 4 + sw] = l_own[k];
+                for (int n = 0; n < 2 * kR; ++n) {
+                    float v = l_tk[n];
+                    v += __shfl_xor_sync(0xffffffffu, v, 4);
+                    v += __shfl_xor_sync(0xffffffffu, v, 8);
+                    v += __shfl_xor_sync(0xffffffffu, v, 16);
+                    if (lane < 4) red[(8 * (n >> 1) + 2 * tq + (n & 1)) * 4 + sw] = v;
                 }
                 softmax_bar_sync();
                 if (st < N) {

@@ -102,22 +102,6 @@ struct Layout {
     static_assert(kOffQ % 1024 == 0 && kQSlab % 512 == 0 && kOffP % 128 == 0, "operands need aligned windows");
 };
 
-// Shared-memory matrix descriptor without swizzle (layout type 0), for the MN-major P^T: 16 heads of one token
-// are 16 adjacent bytes, eight tokens make a 128-byte core matrix, `k_group_bytes` leads from one group of eight
-// tokens to the next and `mn_group_bytes` from one group of 16 heads to the next.
-__device__ __forceinline__ uint64_t make_desc_mn_plain(uint32_t saddr, uint32_t k_group_bytes, uint32_t mn_group_bytes) {
-    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((k_group_bytes >> 4) & 0x3FFFu) << 16) |
-           ((uint64_t)((mn_group_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
-}
-
-// N columns of 16 TMEM lanes in the accumulator fragment layout: v[4k + e] = (lane T/4, column 8k + 2(T%4) + e),
-// v[4k + 2 + e] = (lane T/4 + 8, the same column), k < N / 8, e < 2.
-template <int N>
-__device__ __forceinline__ void tmem_ld_frag(uint32_t taddr, float (&v)[N / 2]) {
-    if constexpr (N == 16) tmem_ld_16x256b_x2(taddr, v);
-    else tmem_ld_16x256b_x4(taddr, v);
-}
-
 // ---------------------------------------------------------------- the kernel
 template <int N>
 __global__ void __launch_bounds__(Layout<N>::kThreads, 1)

@@ -248,6 +248,22 @@ __device__ __forceinline__ uint64_t make_desc_sw64(uint32_t saddr, uint32_t lbo_
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (4ull << 61);
 }
 
+// Shared-memory matrix descriptor without swizzle (layout type 0) for an MN-major operand, used for P^T with the tokens
+// on K: 16 bytes of one token (16 heads of 8 bits, 8 heads of 16) are adjacent, eight tokens make a 128-byte core matrix,
+// `k_group_bytes` leads from one group of eight tokens to the next and `mn_group_bytes` from one group of heads to the next.
+__device__ __forceinline__ uint64_t make_desc_mn_plain(uint32_t saddr, uint32_t k_group_bytes, uint32_t mn_group_bytes) {
+    return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)((k_group_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((mn_group_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46);
+}
+
+// N columns of 16 TMEM lanes in the accumulator fragment layout: v[4k + e] = (lane T/4, column 8k + 2(T%4) + e),
+// v[4k + 2 + e] = (lane T/4 + 8, the same column), k < N / 8, e < 2.
+template <int N>
+__device__ __forceinline__ void tmem_ld_frag(uint32_t taddr, float (&v)[N / 2]) {
+    if constexpr (N == 16) tmem_ld_16x256b_x2(taddr, v);
+    else tmem_ld_16x256b_x4(taddr, v);
+}
+
 // byte offset of (row, byte column) inside a [rows][64 B] slab in the 64-byte swizzle
 __device__ __forceinline__ uint32_t sw64(uint32_t row, uint32_t col_byte) {
     return row * 64 + ((((col_byte >> 4) ^ (row >> 1)) & 3) << 4) + (col_byte & 15);
