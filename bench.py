@@ -173,9 +173,14 @@ class GpuBench:
         self.torch, self.binding, self.device = torch, binding, device
         binding.load()
         self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        self.flush_read_buf = torch.ones(256 << 20, dtype=torch.uint8, device=device)
 
     def flush_l2(self):
+        # Write a buffer larger than L2, then read another one: the write alone leaves 126 MB of DIRTY lines behind, and
+        # the timed kernel would pay for their write-back while it streams (c3: 115.7 us against 103.4 us; the same
+        # 103 us with no flush at all, the inputs being larger than L2, and 106 us under ncu, which invalidates).
         self.flush_buf.fill_(1)
+        self.flush_read_buf.view(self.torch.int64).sum()
 
     def timed(self, fn, steps, warmup):
         torch = self.torch
@@ -222,8 +227,14 @@ class GpuBench:
         for _ in range(steps):
             self.flush_l2(); step()
             kt.append(binding.splash_get_kernel_timing())
+        # the same with the flush's dirty lines left in L2 (write only): reported beside the main figure
+        kd = []
+        for _ in range(max(3, steps // 4)):
+            self.flush_buf.fill_(1); step()
+            kd.append(binding.splash_get_kernel_timing())
         binding.splash_set_kernel_timing(False)
         kt = np.array(kt)
+        dirty_ms = float(np.array(kd)[:, 1].mean())
         ws = binding.decode_workspace(torch.device(self.device))
         rc, detail = binding.splash_workspace_status(ws)
         if rc != 0:
@@ -261,6 +272,8 @@ class GpuBench:
                      "achieved_gbs": alg_bytes / (dec_ms * 1e-3) / 1e9,
                      "achieved_tflops": alg_flops / (dec_ms * 1e-3) / 1e12,
                      "plan_ms": float(kt[:, 0].mean()), "combine_ms": float(kt[:, 2].mean()),
+                     "after_write_only_flush": {"kernel_ms": dirty_ms, "frac": max(t_hbm, t_tensor) * 1e3 / dirty_ms,
+                                                "what": "L2 left full of the flush's dirty lines: the kernel also pays for their write-back"},
                      "note": ("e4m3 KV: 'frac' takes the tensor peak at the bf16 rate (two 8-bit terms per operand); "
                               "'nominal' takes the fp8 rate, under which this workload is HBM-bound") if fp8 else None})
         res = {"ms_per_step": float(ms.mean()), "ms_p50": float(np.median(ms)), "ms_p95": float(np.percentile(ms, 95)),
@@ -862,7 +875,7 @@ def main():
             "config": {"workload": W.CONFIG_NAMES[idx - 1] if not stub else "stub", "requests_per_gpu": w.B,
                        "heads": w.head_end - w.head_begin,
                        "tokens_per_gpu": w.total_tokens(), "kv_dtype": "bf16" if w.kv_dtype == 0 else "e4m3+token scale",
-                       "page_size": 64, "l2": "256 MiB flush write between steps; KV larger than L2",
+                       "page_size": 64, "l2": "between steps: 256 MiB flush write, then a 256 MiB read that evicts the flush's dirty lines; KV larger than L2",
                        "parallelism": f"dp{world} (request slices, no collective)"},
             "ms_p50": main_res["ms_p50"], "ms_p95": main_res["ms_p95"],
             "tokens_per_s_78_layers": value / 78,
