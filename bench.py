@@ -308,6 +308,35 @@ class GpuBench:
                              "launch_chains": 1, "cta_pairs_per_kv_worker": -(-h * R // 128)},
                 "launches_per_step": binding.splash_last_launch_count()}
 
+    def layer_loop(self, w, dw, out, lse, steps, warmup, layers=8):
+        """One decode step of a model: the same batch through `layers` layers.  The first layer's call plans, the
+        others take its partition again (SPLASH_FLAG_REUSE_PLAN); L2 flushed before every layer, as the GEMMs between
+        two attention layers would leave it."""
+        torch, binding = self.torch, self.binding
+        def step(reuse):
+            times = []
+            for k in range(layers):
+                self.flush_l2()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); dw.decode(out=out, lse=lse, flags=binding.SPLASH_FLAG_REUSE_PLAN if (reuse and k > 0) else 0); b.record()
+                times.append((a, b))
+            torch.cuda.synchronize()
+            return [a.elapsed_time(b) for a, b in times]
+        for _ in range(max(1, warmup // 2)):
+            step(True); step(False)
+        first, rest, plain = [], [], []
+        for _ in range(max(2, steps // 4)):
+            t = step(True); first.append(t[0]); rest.extend(t[1:])
+            plain.extend(step(False))
+        rc, detail = binding.splash_workspace_status(binding.decode_workspace(torch.device(self.device)))
+        if rc != 0:
+            raise RuntimeError(f"device status {rc} {detail}")
+        per_layer = (float(np.median(first)) + (layers - 1) * float(np.median(rest))) / layers
+        return {"layers": layers, "ms_first_layer": float(np.median(first)), "ms_other_layers": float(np.median(rest)),
+                "ms_every_layer_planning": float(np.median(plain)), "ms_per_layer": per_layer,
+                "tokens_per_s_per_layer": w.B / (per_layer * 1e-3),
+                "how": "layer 0 plans, layers 1.. pass SPLASH_FLAG_REUSE_PLAN (the partition depends on lengths, ranges and shape only)"}
+
     def slice_workload(self, w, dw, out, lse, head_begin, head_end, steps, warmup, peaks, traffic=None):
         """A TP rank's share of workload `w`: the same cache and requests, heads [head_begin, head_end) only."""
         import copy
@@ -813,7 +842,8 @@ def main():
             steps2 = max(5, args.steps // 2)
             if idx == 5:
                 try:
-                    extra["c5"] = {"tp8_slice": gb.slice_workload(w, dw, out, lse, 32, 48, steps2, args.warmup, peaks, traffic.get("c5_heads16")),
+                    extra["c5"] = {"layer_loop": gb.layer_loop(w, dw, out, lse, steps2, args.warmup),
+                                   "tp8_slice": gb.slice_workload(w, dw, out, lse, 32, 48, steps2, args.warmup, peaks, traffic.get("c5_heads16")),
                                    "page_migrate": gb.migrate_workload(w, dw, steps2, args.warmup, peaks),
                                    "migrate_under_decode": gb.overlap_workload(w, dw, steps2, args.warmup)}
                 except Exception as exc:  # report, do not hide
@@ -831,6 +861,7 @@ def main():
                     r, dwx, ox, lx = gb.decode_workload(wx, args.steps, args.warmup, peaks, traffic, name)
                     if name in ("c3", "c5"):
                         targets[name] = r["roofline"]["frac"]
+                    r["layer_loop"] = gb.layer_loop(wx, dwx, ox, lx, steps2, args.warmup)
                     if name == "c4":
                         del dwx
                         r["cp"] = gb.cp_workload(wx, steps2, args.warmup)

@@ -88,7 +88,17 @@ enum {
      * the first bad one in the workspace status word: splash_workspace_status() then returns SPLASH_BAD_PAGE_ID with
      * detail = (request, page index within the request, the id found).  With or without the flag an id outside the
      * pool is never dereferenced (the page reads as zeros); the flag makes the mistake visible. */
-    SPLASH_FLAG_VALIDATE = 8u
+    SPLASH_FLAG_VALIDATE = 8u,
+    /* splash_mla_decode / splash_mla_decode_migrating only: the work partition of the previous call on this workspace is
+     * taken again and the plan kernel is not launched.  The partition (App. B's linear-in-context cost: page tiles, not
+     * requests, spread evenly over the CTAs) is a function of seq_lens, kv_begin / kv_end, the width head_end - head_begin,
+     * the shape (num_requests, q_rows, kv_dtype, the other flag bits) and the device only -- not of q, the cache, the
+     * scales or the block table -- and a decode step runs the same batch through every layer of the model: the first
+     * layer's call plans, the others pass this bit.  The caller asserts that those arguments are what they were in the
+     * last call WITHOUT this bit on the same workspace (nothing checks it; a different batch would be cut along the old
+     * batch's boundaries and give wrong results, within bounds).  The error words of the status block are cleared as in
+     * any call.  Ignored by the sparse entry point and together with SPLASH_FLAG_VALIDATE (which needs the plan's pass). */
+    SPLASH_FLAG_REUSE_PLAN = 16u
 };
 
 /*

@@ -29,6 +29,7 @@ SPLASH_FLAG_SIMT = 1
 SPLASH_FLAG_NO_PAIR = 2
 SPLASH_FLAG_SPARSE_FUSED = 4
 SPLASH_FLAG_VALIDATE = 8
+SPLASH_FLAG_REUSE_PLAN = 16
 
 D_QK, D_V, PAGE_SIZE = 576, 512, 64
 

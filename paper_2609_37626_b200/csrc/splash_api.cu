@@ -315,10 +315,18 @@ int decode_dense(const splash_mla_shape *shape, const void *q, const void *kv_po
         job_copy_pending = false;
     }
 
+    // the previous call's partition taken again (the same batch in the next layer): no plan kernel, only the error words
+    // of the status block are cleared (word 8, the number of split requests, belongs to the plan)
+    const bool reuse_plan = (shape->flags & SPLASH_FLAG_REUSE_PLAN) && !(shape->flags & SPLASH_FLAG_VALIDATE) && !sparse;
     e = record_timing_event(0, stream);
-    if (e == cudaSuccess)
-        e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
-                        v.cost_start, v.worker_begin, v.split_list, v.worker_req, v.split_rec, v.status, vb == vbegin, stream);
+    if (e == cudaSuccess) {
+        if (reuse_plan) {
+            if (vb == vbegin) e = cudaMemsetAsync(v.status, 0, 8 * sizeof(int32_t), stream);
+        } else {
+            e = launch_plan(p, kv_begin, kv_end, v.tile_start, v.req_lo, v.req_hi, v.req_wfirst, v.req_wlast,
+                            v.cost_start, v.worker_begin, v.split_list, v.worker_req, v.split_rec, v.status, vb == vbegin, stream);
+        }
+    }
     if (e == cudaSuccess) e = record_timing_event(1, stream);
     // validation mode: the table entries the call will use, checked on the device before the decode kernel runs
     if (e == cudaSuccess && (shape->flags & SPLASH_FLAG_VALIDATE) && !sparse && vb == vbegin)
