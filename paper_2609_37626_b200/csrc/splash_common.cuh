@@ -185,15 +185,26 @@ struct SegmentIter {
 // for its own heads.  Called by all threads of the CTA once its segments are done.
 __device__ __forceinline__ void fill_empty_requests(const DecodeParams &p, int worker, int head0, int heads_per_group,
                                                     int tid, int nthreads) {
+    // The plan's arrays are a launch old and have left the caches: a loop over this worker's requests that looks at one
+    // request per iteration is a chain of round trips to DRAM at the very end of the CTA (seven on the rollout workload).
+    // Instead every lane looks at a request of its own -- one round trip -- and the warp then zeroes what it found.
     const int nheads = min(heads_per_group, p.head_end - head0);
-    for (int i = worker; i < p.B; i += p.num_workers) {
-        if (p.tile_start[i + 1] != p.tile_start[i]) continue;
-        for (int idx = tid; idx < nheads * (kDV / 4); idx += nthreads) {
-            const int hh = idx / (kDV / 4), c = idx % (kDV / 4);
-            reinterpret_cast<float4 *>(p.out + (int64_t)i * p.out_stride_request + (int64_t)(head0 + hh) * p.out_stride_head)[c] =
-                make_float4(0.f, 0.f, 0.f, 0.f);
+    const int lane = tid & 31, wid = tid >> 5, nwarps = nthreads >> 5;
+    for (int64_t j0 = (int64_t)wid * 32; worker + j0 * p.num_workers < p.B; j0 += (int64_t)nwarps * 32) {
+        const int64_t mine = worker + (j0 + lane) * p.num_workers;
+        const bool empty = mine < p.B && p.tile_start[mine + 1] == p.tile_start[mine];
+        unsigned found = __ballot_sync(0xffffffffu, empty);
+        while (found) {
+            const int src = __ffs(found) - 1;
+            found &= found - 1;
+            const int64_t i = worker + (j0 + src) * p.num_workers;
+            for (int idx = lane; idx < nheads * (kDV / 4); idx += 32) {
+                const int hh = idx / (kDV / 4), c = idx % (kDV / 4);
+                reinterpret_cast<float4 *>(p.out + i * p.out_stride_request + (int64_t)(head0 + hh) * p.out_stride_head)[c] =
+                    make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            for (int hh = lane; hh < nheads; hh += 32) p.lse[i * p.lse_stride_request + head0 + hh] = -INFINITY;
         }
-        for (int hh = tid; hh < nheads; hh += nthreads) p.lse[(int64_t)i * p.lse_stride_request + head0 + hh] = -INFINITY;
     }
 }
 

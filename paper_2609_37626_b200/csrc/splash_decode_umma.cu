@@ -648,7 +648,6 @@ decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap tma
             if (lane == 0) mbar_arrive(bar(kBarOEmpty));
             ++seg_it;
         }
-        bulk_wait_group();        // this thread's output rows have reached global memory
     }
 
     fill_empty_requests(p, worker, head0, N, tid, kThreads);

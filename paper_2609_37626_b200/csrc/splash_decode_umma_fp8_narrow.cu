@@ -641,7 +641,6 @@ decode_umma_fp8_narrow_kernel(const DecodeParams p, const __grid_constant__ CUte
             }
             ++seg_it;
         }
-        bulk_wait_group();        // this thread's output rows have reached global memory
     }
 
     fill_empty_requests(p, worker, head0, N, tid, kThreads);

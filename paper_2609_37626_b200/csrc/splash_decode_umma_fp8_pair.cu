@@ -631,7 +631,6 @@ decode_umma_fp8_pair_kernel(const DecodeParams p, const __grid_constant__ CUtens
             if (lane == 0) arrive_on_leader(kBarOEmpty);
             ++seg_it;
         }
-        if (lane == 0) bulk_wait_group();                 // this warp's output stores have completed
     }
 
     fill_empty_requests(p, worker, head0, kN, tid, kThreads);
