@@ -128,3 +128,29 @@ def test_c5_rollout_fp8_and_page_migration_full_size():
     dw.kv_scales[torch.from_numpy(src).long().cuda()] = float("nan")
     out2, lse2 = gpu_run(w, dw=dw)
     assert np.array_equal(out, out2) and np.array_equal(lse, lse2)
+
+
+def test_c5_tp8_share_full_size():
+    """A TP-8 rank's 16 heads of the rollout workload, as bench.py times it (heads [32, 48) of the same cache and
+    requests): one head of every request and all 16 heads of the 8 longest and 8 shortest against the oracle; nothing
+    written outside the slice; the eight shares side by side equal the 128-head call within twice the tolerance."""
+    import torch
+    from paper_2609_37626_b200 import binding
+    w = W.config(5)
+    dw = binding.DeviceWorkload(w)
+    out, lse = gpu_run(w, dw=dw, sentinel=3.0, head_begin=32, head_end=48)
+    rng = np.random.default_rng(58)
+    order = np.argsort(w.seq_lens, kind="stable")
+    pairs = {(i, int(rng.integers(32, 48))) for i in range(w.B)}
+    pairs |= {(int(i), g) for i in list(order[:8]) + list(order[-8:]) for g in range(32, 48)}
+    check_sampled(w, out, lse, sorted(pairs), "c5 heads [32, 48)", head_begin=32, head_end=48)
+    assert np.all(out[:, :32] == 3.0) and np.all(out[:, 48:] == 3.0) and np.all(lse[:, :32] == 3.0) and np.all(lse[:, 48:] == 3.0)
+    assert np.isfinite(out[:, 32:48]).all() and np.isfinite(lse[:, 32:48]).all()
+    cat_o = torch.zeros((w.B, 128, 512), dtype=torch.float32, device="cuda")
+    cat_l = torch.zeros((w.B, 128), dtype=torch.float32, device="cuda")
+    for hb in range(0, 128, 16):
+        dw.decode(out=cat_o, lse=cat_l, head_begin=hb, head_end=hb + 16)
+    full_o, full_l = dw.decode()
+    torch.cuda.synchronize()
+    assert (cat_o - full_o).abs().max().item() <= 1e-1 and (cat_l - full_l).abs().max().item() <= 1e-2
+    assert np.array_equal(cat_o[:, 32:48].cpu().numpy(), out[:, 32:48])       # the same launch twice: the same bits
