@@ -29,7 +29,7 @@ constexpr int kRequestOverheadTilesDefault = 4;
 constexpr int kRequestOverheadTilesFp8 = 6;        // also right for the 16- / 32-head e4m3 kernel: a TP-8 share of the rollout
                                                    // workload takes 237 / 232 / 228 / 224 / 227 / 232 / 239 us with 2 / 3 / 4 / 6 / 8 / 10 / 14
 constexpr int kRequestOverheadTilesPair = 5;       // bf16 CTA-pair kernel (a segment costs 7,500 cycles, a tile 1,650)
-constexpr int kRequestOverheadTilesFp8Pair = 14;   // CTA-pair kernel: tiles are cheaper, the per-request work is not
+constexpr int kRequestOverheadTilesFp8Pair = 13;   // CTA-pair kernel: tiles are cheaper, the per-request work is not
 
 // ---- workspace layout ------------------------------------------------------
 // [0, 64)                 status block (int32 x 16): [0] status, [1..3] detail

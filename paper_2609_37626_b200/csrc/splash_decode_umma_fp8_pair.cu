@@ -52,8 +52,8 @@ constexpr uint32_t kScaleBytes = 256;
 constexpr int kStages = 3;
 constexpr int kPrefetchAhead = 1;                    // supertiles between the L2 prefetch of a page and its use (4: 1.5 % slower; none: 5 %)
 constexpr int kPrefetchAheadBusy = 4;                // the same while the call carries a page-copy job
-constexpr float kTau = 6.0f;
-constexpr float kLift = 2.75f;
+constexpr float kTau = 7.0f;                          // (6 / 2.75: 0.3 % slower on the rollout workload, 4 / 4.75 more)
+constexpr float kLift = 1.75f;
 
 enum BarrierId {
     kBarKFull = 0,                        // [3] leader: both CTAs' pages landed (tx bytes of both)
